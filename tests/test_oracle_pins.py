@@ -1,0 +1,357 @@
+"""Pins for the fp64 oracle: closed forms, brute force, invariants, limits that reduce to a
+library routine, finite differences.  Each test is chosen so that a plausible mistake in the
+oracle (dropped term, wrong sign or index, transposed operand) makes it fail.  CPU only."""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import spa_oracle as O
+from oracle.brute_force import block_fwd_bruteforce
+from spa_workloads import get_config, make_inputs, scaled_config
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def tiny_problem(seed=0, B=3, N=12, C=8, H=2, keep=0.5):
+    rng = np.random.default_rng(seed)
+    x = rng.normal(size=(B, N, C))
+    w_g = rng.normal(size=C) / np.sqrt(C)
+    b_g = float(np.quantile(x @ w_g, 1 - keep) * -1.0)
+    W_qkv = rng.normal(size=(3 * C, C)) / np.sqrt(C)
+    b_qkv = rng.normal(size=3 * C) * 0.1
+    W_o = rng.normal(size=(C, C)) / np.sqrt(C)
+    b_o = rng.normal(size=C) * 0.1
+    return dict(x=x, w_g=w_g, b_g=b_g, tau=0.0, W_qkv=W_qkv, b_qkv=b_qkv, W_o=W_o, b_o=b_o, H=H)
+
+
+# ------------------------------------------------------------------ gate + select
+def test_gate_closed_form_along_w():
+    rng = np.random.default_rng(1)
+    C = 16
+    w = rng.normal(size=C)
+    u = w / np.linalg.norm(w)
+    k = np.array([[-2.0, 0.0, 0.5, 3.0]])
+    x = k[:, :, None] * u[None, None, :]
+    s = O.gate(x, w, 0.25)
+    np.testing.assert_allclose(s, k * np.linalg.norm(w) + 0.25, rtol=0, atol=1e-13)
+
+
+def test_gate_exact_rational_on_integers():
+    rng = np.random.default_rng(2)
+    x = rng.integers(-5, 6, size=(4, 4, 8))
+    w = rng.integers(-3, 4, size=8)
+    s = O.gate(x.astype(float), w.astype(float), 2.0)
+    for b in range(4):
+        for n in range(4):
+            exact = Fraction(2) + sum(Fraction(int(w[c])) * int(x[b, n, c]) for c in range(8))
+            assert Fraction(float(s[b, n])) == exact
+
+
+def test_gate_max_with_upscale_scores():
+    x = np.zeros((1, 3, 2))
+    s = O.gate(x, np.ones(2), 0.5, s_up=np.array([[-1.0, 0.5, 2.0]]))
+    np.testing.assert_array_equal(s, [[0.5, 0.5, 2.0]])
+
+
+def test_select_is_strict_threshold():
+    m = O.select(np.array([[-1.0, 0.0, 1e-9, 2.0]]), 0.0)
+    np.testing.assert_array_equal(m, [[False, False, True, True]])
+
+
+def test_mask_matches_generator_blobs_where_noise_is_small():
+    cfg = get_config(1)
+    inp = make_inputs(cfg)
+    s = O.gate(inp.x, inp.w_g, inp.b_g)
+    m = O.select(s, inp.tau)
+    u = inp.w_g / np.linalg.norm(inp.w_g)
+    along = inp.x @ u - cfg.offset * inp.blob_mask       # noise coordinate along the gate direction
+    calm = np.abs(along) < 0.45 * cfg.offset
+    assert calm.mean() > 0.7
+    np.testing.assert_array_equal(m[calm], inp.blob_mask[calm])
+
+
+def test_margin_of_generated_inputs():
+    for i in (1, 2):
+        inp = make_inputs(get_config(i))
+        s = O.gate(inp.x, inp.w_g, inp.b_g)
+        assert np.abs(s - inp.tau).min() >= 1e-3
+
+
+# ------------------------------------------------------------------ packing indices
+def test_pack_indices_invariants_and_pushback():
+    rng = np.random.default_rng(3)
+    B, N = 5, 17
+    mask = rng.random((B, N)) < 0.4
+    mask[2] = False                       # an image with nothing selected
+    cu, idx, inv = O.pack_indices(mask)
+    assert cu.dtype == np.int32 and idx.dtype == np.int32 and inv.dtype == np.int32
+    assert cu[0] == 0 and cu[-1] == mask.sum() == idx.size
+    assert np.all(np.diff(idx) > 0)
+    ref = []                              # brute force: push back in scan order
+    for b in range(B):
+        for n in range(N):
+            if mask[b, n]:
+                ref.append(b * N + n)
+    np.testing.assert_array_equal(idx, ref)
+    for i, t in enumerate(idx):
+        b = t // N
+        assert cu[b] <= i < cu[b + 1]
+        assert inv[t] == i
+    assert np.all(inv[~mask.reshape(-1)] == -1)
+    assert cu[3] == cu[2]
+
+
+def test_pack_unpack_identity_bitwise():
+    rng = np.random.default_rng(4)
+    x = rng.normal(size=(3, 10, 4))
+    mask = rng.random((3, 10)) < 0.5
+    _, idx, _ = O.pack_indices(mask)
+    xp = O.pack_rows(x, idx)
+    assert np.array_equal(xp, x.reshape(-1, 4)[mask.reshape(-1)])
+    y = O.unpack_scatter(xp, x, idx)
+    assert np.array_equal(y, x)
+    z = rng.normal(size=xp.shape)
+    y = O.unpack_scatter(z, x, idx)
+    assert np.array_equal(y.reshape(-1, 4)[~mask.reshape(-1)], x.reshape(-1, 4)[~mask.reshape(-1)])
+    assert np.array_equal(y.reshape(-1, 4)[mask.reshape(-1)], z)
+    yr = O.unpack_scatter(z, x, idx, residual=True)
+    assert np.array_equal(yr.reshape(-1, 4)[mask.reshape(-1)], xp + z)
+
+
+def test_gate_scale_is_sigmoid_times_row():
+    x = np.ones((1, 2, 3))
+    xp = O.pack_rows(x, np.array([0, 1]), s=np.array([[0.0, np.log(3.0)]]), gate_scale=True)
+    np.testing.assert_allclose(xp, [[0.5] * 3, [0.75] * 3], atol=1e-15)
+
+
+# ------------------------------------------------------------------ attention
+def test_block_matches_bruteforce():
+    for seed, keep in ((0, 0.5), (1, 0.25), (2, 0.9)):
+        p = tiny_problem(seed=seed, keep=keep)
+        fwd = O.block_fwd(**p)
+        y_bf = block_fwd_bruteforce(**p)
+        assert 0 < fwd["idx"].size < p["x"].shape[0] * p["x"].shape[1]
+        np.testing.assert_allclose(fwd["y"], y_bf, rtol=0, atol=1e-12)
+    p = tiny_problem(seed=5)
+    np.testing.assert_allclose(O.block_fwd(**p, residual=True)["y"],
+                               block_fwd_bruteforce(**p, residual=True), rtol=0, atol=1e-12)
+
+
+def test_per_image_equals_masked_dense_and_rows_sum_to_one():
+    p = tiny_problem(seed=7, B=4, N=9)
+    fwd = O.block_fwd(**p)
+    ao2 = O.attention_fwd_masked_dense(fwd["qkv"], fwd["cu_seqlens"], p["H"])
+    np.testing.assert_allclose(fwd["ao"], ao2, rtol=0, atol=1e-12)
+    _, _, probs = O.attention_fwd(fwd["qkv"], fwd["cu_seqlens"], p["H"], return_probs=True)
+    assert probs
+    for _, _, P in probs:
+        np.testing.assert_allclose(P.sum(axis=1), 1.0, atol=1e-14)
+        assert np.all(P >= 0)
+
+
+def _dense_mha_torch(x, W_qkv, b_qkv, W_o, b_o, H):
+    xt = torch.tensor(x, dtype=torch.float64)
+    B, N, C = xt.shape
+    qkv = torch.nn.functional.linear(xt, torch.tensor(W_qkv), torch.tensor(b_qkv))
+    q, k, v = qkv.split(C, dim=-1)
+    sh = lambda t: t.reshape(B, N, H, C // H).transpose(1, 2)
+    o = torch.nn.functional.scaled_dot_product_attention(sh(q), sh(k), sh(v))
+    o = o.transpose(1, 2).reshape(B, N, C)
+    return torch.nn.functional.linear(o, torch.tensor(W_o), torch.tensor(b_o))
+
+
+def test_all_selected_limit_is_dense_mha():
+    p = tiny_problem(seed=8, B=2, N=11, C=12, H=3)
+    p["tau"] = -np.inf
+    fwd = O.block_fwd(**p)
+    assert fwd["mask"].all()
+    ref = _dense_mha_torch(p["x"], p["W_qkv"], p["b_qkv"], p["W_o"], p["b_o"], p["H"]).numpy()
+    np.testing.assert_allclose(fwd["y"], ref, rtol=0, atol=1e-12)
+
+
+def test_lse_against_library_logsumexp():
+    from scipy.special import logsumexp
+    p = tiny_problem(seed=9)
+    fwd = O.block_fwd(**p)
+    C, H = p["x"].shape[2], p["H"]
+    d = C // H
+    cu = fwd["cu_seqlens"]
+    for b in range(len(cu) - 1):
+        lo, hi = cu[b], cu[b + 1]
+        for h in range(H):
+            q = fwd["qkv"][lo:hi, h * d:(h + 1) * d]
+            k = fwd["qkv"][lo:hi, C + h * d:C + (h + 1) * d]
+            np.testing.assert_allclose(fwd["lse"][h, lo:hi], logsumexp(q @ k.T / np.sqrt(d), axis=1),
+                                       atol=1e-13)
+
+
+def test_zero_query_weights_give_segment_mean_of_v():
+    p = tiny_problem(seed=10)
+    C = p["x"].shape[2]
+    p["W_qkv"][:C] = 0.0
+    p["b_qkv"][:C] = 0.0
+    fwd = O.block_fwd(**p)
+    cu = fwd["cu_seqlens"]
+    v = fwd["qkv"][:, 2 * C:]
+    for b in range(len(cu) - 1):
+        lo, hi = cu[b], cu[b + 1]
+        if hi > lo:
+            np.testing.assert_allclose(fwd["ao"][lo:hi], np.tile(v[lo:hi].mean(0), (hi - lo, 1)), atol=1e-13)
+
+
+def test_equal_values_pass_through_attention():
+    rng = np.random.default_rng(11)
+    C, H = 8, 2
+    qkv = rng.normal(size=(7, 3 * C))
+    qkv[:, 2 * C:] = rng.normal(size=C)[None, :]
+    ao, _ = O.attention_fwd(qkv, np.array([0, 3, 7]), H)
+    np.testing.assert_allclose(ao, qkv[:, 2 * C:], atol=1e-14)
+
+
+def test_single_token_segment():
+    rng = np.random.default_rng(12)
+    C, H = 8, 2
+    d = C // H
+    qkv = rng.normal(size=(3, 3 * C))
+    ao, lse = O.attention_fwd(qkv, np.array([0, 1, 2, 3]), H)
+    np.testing.assert_allclose(ao, qkv[:, 2 * C:], atol=1e-15)
+    for h in range(H):
+        s11 = (qkv[:, h * d:(h + 1) * d] * qkv[:, C + h * d:C + (h + 1) * d]).sum(1) / np.sqrt(d)
+        np.testing.assert_allclose(lse[h], s11, atol=1e-14)
+
+
+def test_permutation_equivariance_and_image_independence():
+    p = tiny_problem(seed=13, B=3, N=10)
+    y0 = O.block_fwd(**p)["y"]
+    perm = np.random.default_rng(0).permutation(10)
+    p2 = dict(p)
+    p2["x"] = p["x"].copy()
+    p2["x"][1] = p["x"][1][perm]
+    y1 = O.block_fwd(**p2)["y"]
+    np.testing.assert_allclose(y1[1], y0[1][perm], atol=1e-12)
+    assert np.array_equal(y1[0], y0[0]) and np.array_equal(y1[2], y0[2])
+    p3 = dict(p)
+    p3["x"] = p["x"].copy()
+    p3["x"][2] = np.random.default_rng(1).normal(size=p["x"][2].shape)
+    y2 = O.block_fwd(**p3)["y"]
+    assert np.array_equal(y2[0], y0[0]) and np.array_equal(y2[1], y0[1])
+
+
+def test_none_selected_limit():
+    p = tiny_problem(seed=14)
+    p["tau"] = np.inf
+    fwd = O.block_fwd(**p)
+    assert fwd["idx"].size == 0 and fwd["cu_seqlens"][-1] == 0
+    assert np.array_equal(fwd["y"], p["x"])
+    dY = np.random.default_rng(2).normal(size=p["x"].shape)
+    bwd = O.block_bwd(fwd, dY, p["x"], p["W_qkv"], p["W_o"], p["H"])
+    assert np.array_equal(bwd["dX"], dY)
+    assert not bwd["dW_qkv"].any() and not bwd["dW_o"].any()
+
+
+def test_container_cuts():
+    p = tiny_problem(seed=15, B=2, N=12, keep=0.8)
+    fwd = O.block_fwd(**p)
+    big = O.block_fwd(**p, container_len=10_000)
+    np.testing.assert_allclose(big["y"], fwd["y"], atol=0)
+    one = O.block_fwd(**p, container_len=1)
+    np.testing.assert_allclose(one["ao"], one["qkv"][:, 2 * p["x"].shape[2]:], atol=1e-15)
+    cuts = O.container_cuts(np.array([0, 5, 5, 12], np.int32), 4)
+    np.testing.assert_array_equal(cuts, [0, 4, 5, 8, 12])
+
+
+# ------------------------------------------------------------------ backward
+def _loss(p, G, residual=False):
+    return float((O.block_fwd(**p, residual=residual)["y"] * G).sum())
+
+
+@pytest.mark.parametrize("residual", [False, True])
+def test_backward_against_central_differences(residual):
+    p = tiny_problem(seed=20, B=2, N=7, C=6, H=2, keep=0.6)
+    rng = np.random.default_rng(21)
+    G = rng.normal(size=p["x"].shape)
+    fwd = O.block_fwd(**p, residual=residual)
+    assert 2 < fwd["idx"].size < 14
+    bwd = O.block_bwd(fwd, G, p["x"], p["W_qkv"], p["W_o"], p["H"], residual=residual)
+    h = 1e-6
+    for name, grad in (("x", bwd["dX"]), ("W_qkv", bwd["dW_qkv"]), ("b_qkv", bwd["db_qkv"]),
+                       ("W_o", bwd["dW_o"]), ("b_o", bwd["db_o"])):
+        base = p[name]
+        num = np.zeros_like(base)
+        it = np.nditer(base, flags=["multi_index"])
+        for _ in it:
+            i = it.multi_index
+            pp = dict(p); a = base.copy(); a[i] += h; pp[name] = a
+            pm = dict(p); c = base.copy(); c[i] -= h; pm[name] = c
+            num[i] = (_loss(pp, G, residual) - _loss(pm, G, residual)) / (2 * h)
+        denom = max(np.abs(num).max(), 1e-12)
+        assert np.abs(num - grad).max() / denom <= 1e-6, name
+
+
+def test_backward_unselected_rows_and_key_shift_invariance():
+    p = tiny_problem(seed=22, B=3, N=9)
+    fwd = O.block_fwd(**p)
+    dY = np.random.default_rng(23).normal(size=p["x"].shape)
+    bwd = O.block_bwd(fwd, dY, p["x"], p["W_qkv"], p["W_o"], p["H"])
+    unsel = ~fwd["mask"].reshape(-1)
+    C = p["x"].shape[2]
+    assert np.array_equal(bwd["dX"].reshape(-1, C)[unsel], dY.reshape(-1, C)[unsel])
+    # softmax ignores a shift common to all keys of a segment, so dK sums to zero there
+    cu = fwd["cu_seqlens"]
+    dk = bwd["dqkv"][:, C:2 * C]
+    for b in range(len(cu) - 1):
+        if cu[b + 1] > cu[b]:
+            np.testing.assert_allclose(dk[cu[b]:cu[b + 1]].sum(0), 0.0, atol=1e-12)
+
+
+def test_all_selected_backward_is_dense_mha_backward():
+    p = tiny_problem(seed=24, B=2, N=6, C=8, H=2)
+    p["tau"] = -np.inf
+    fwd = O.block_fwd(**p)
+    G = np.random.default_rng(25).normal(size=p["x"].shape)
+    bwd = O.block_bwd(fwd, G, p["x"], p["W_qkv"], p["W_o"], p["H"])
+    t = {k: torch.tensor(p[k], dtype=torch.float64, requires_grad=True)
+         for k in ("x", "W_qkv", "b_qkv", "W_o", "b_o")}
+    B, N, C = p["x"].shape
+    H = p["H"]
+    qkv = t["x"] @ t["W_qkv"].T + t["b_qkv"]
+    q, k, v = qkv.split(C, dim=-1)
+    sh = lambda a: a.reshape(B, N, H, C // H).transpose(1, 2)
+    att = torch.softmax(sh(q) @ sh(k).transpose(-1, -2) / (C // H) ** 0.5, dim=-1) @ sh(v)
+    y = att.transpose(1, 2).reshape(B, N, C) @ t["W_o"].T + t["b_o"]
+    (y * torch.tensor(G)).sum().backward()
+    for name, key in (("x", "dX"), ("W_qkv", "dW_qkv"), ("b_qkv", "db_qkv"), ("W_o", "dW_o"), ("b_o", "db_o")):
+        np.testing.assert_allclose(bwd[key], t[name].grad.numpy(), rtol=0, atol=1e-11)
+
+
+# ------------------------------------------------------------------ complexity model
+def _golden_rows():
+    rows = []
+    with open(os.path.join(GOLDEN, "eq7_eq9_macs.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                eq, *nums = line.split()
+                rows.append((eq, *map(int, nums)))
+    return rows
+
+
+def test_mac_count_against_eq7_and_eq9():
+    for eq, B, N, C, Bp, L, macs in _golden_rows():
+        if eq == "eq7":    # everything selected, one segment per image: plain MSA
+            m = O.mac_count(B, N, C, np.arange(B + 1) * N)
+            assert m["qkv"] + m["attn"] + m["proj"] == macs
+        else:              # containers of length L: the packed terms of Eq. 9 plus the gate term
+            m = O.mac_count(B, N, C, np.arange(Bp + 1) * L)
+            assert m["qkv"] + m["attn"] == Bp * (3 * L * C * C + 2 * L * L * C)
+            assert m["gate"] + B * N * C * C + m["qkv"] + m["attn"] == macs
+
+
+def test_full_config_shapes_run():
+    cfg = scaled_config(get_config(2), B=4)
+    inp = make_inputs(cfg)
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
+    frac = fwd["mask"].mean(axis=1)
+    assert np.all(np.abs(frac - inp.keep_target) < 0.08)
