@@ -1,0 +1,171 @@
+/*
+ * spa.h - C boundary of the Select-and-Pack-Attention (SPA) block library for NVIDIA B200 (sm_100a).
+ *
+ * One SPA block (Ren et al., "Context-Aware Token Selection and Packing for Enhanced Vision
+ * Transformer", Sec. 3.2): a linear gate scores every token (Eq. 4); tokens whose logit exceeds a
+ * threshold are selected (deterministic form of Eq. 6); the selections of all images are packed
+ * into one dense buffer ("Token Packing"); QKV projection, self-attention restricted to tokens of
+ * the same image, and the output projection run on the packed buffer; results are scattered back
+ * and unselected tokens pass through unchanged.
+ *
+ * Conventions shared by every call
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned, unless a
+ *     parameter is explicitly documented as a host pointer.  The library never allocates or
+ *     frees device memory; scratch comes from the caller-provided `workspace`
+ *     (spa_workspace_bytes() bytes, 256-byte aligned).
+ *   - `stream` is a cudaStream_t passed as void*.  Calls validate their arguments on the host
+ *     and return a negative spa_status synchronously; otherwise they enqueue work on `stream`
+ *     and return SPA_OK without synchronising.
+ *   - Conditions only the device can see (more selected tokens than `capacity`, a bounded wait
+ *     that ran out) are recorded in the int32 `d_status` word (first error wins; the caller zeroes
+ *     it) and the kernels finish cleanly.  `d_status` may be NULL.
+ *   - Storage dtype T is float (SPA_F32) or bfloat16 (SPA_BF16); accumulation is always fp32.
+ *     C*sizeof(T) and (C/H)*sizeof(T) must be multiples of 16 bytes; C/H must be 32 or 64.
+ *   - Packed buffers have `capacity` rows allocated (capacity <= B*N); only the first
+ *     N_p = cu_seqlens[B] rows are defined.  N_p lives on the device: no call reads it back.
+ *   - Layouts are row-major with the last index contiguous: x[B][N][C], x_packed[capacity][C],
+ *     qkv[capacity][3C] with column = which*C + h*(C/H) + e (which = 0,1,2 for q,k,v),
+ *     attn_out[capacity][C] with column = h*(C/H) + e, lse[H][capacity], weights W[out][in].
+ */
+#ifndef SPA_H_
+#define SPA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPA_OK = 0,
+  SPA_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, misaligned pointer          */
+  SPA_ERR_UNSUPPORTED = -2, /* dtype, head dimension or row size the kernels do not cover   */
+  SPA_ERR_CAPACITY = -3,    /* device: more selected tokens than `capacity`                 */
+  SPA_ERR_CUDA = -4,        /* a CUDA runtime call failed (see spa_last_cuda_error)         */
+  SPA_ERR_TIMEOUT = -5      /* device: a bounded wait expired                               */
+} spa_status;
+
+typedef enum { SPA_F32 = 0, SPA_BF16 = 1 } spa_dtype;
+
+enum {
+  SPA_FLAG_RESIDUAL = 1,  /* selected rows: y = x + z instead of y = z                     */
+  SPA_FLAG_INPLACE = 2,   /* spa_unpack_scatter: y aliases x, only selected rows written   */
+  SPA_FLAG_GATE_SCALE = 4,/* Eq. 5: packed rows are scaled by sigmoid(score)               */
+  SPA_FLAG_SIMT_ONLY = 8  /* bf16 only: run the fp32-FMA kernels instead of the tensor-core ones */
+};
+
+typedef struct spa_params {
+  int32_t B;          /* images in the batch                                             */
+  int32_t N;          /* tokens per image                                                */
+  int32_t C;          /* channels                                                        */
+  int32_t H;          /* attention heads; head dimension d = C / H                       */
+  int32_t dtype;      /* spa_dtype of x, weights, packed buffers                         */
+  int32_t flags;      /* SPA_FLAG_* bits                                                 */
+  int32_t capacity;   /* rows allocated in packed buffers, 1 <= capacity <= B*N          */
+  float tau;          /* selection threshold on the gate logit                           */
+  float softmax_scale;/* 0 selects 1/sqrt(d)                                             */
+} spa_params;
+
+/* Bytes of scratch the calls below that take `workspace` need for these parameters. */
+size_t spa_workspace_bytes(const spa_params* p);
+
+/* Gate and hard selection (Sec. 3.2, Eq. 4 and the thresholded form of Eq. 6).
+ *   scores[b*N+n] = b_g + sum_c w_g[c] * x[b][n][c];  if s_up != NULL, scores = max(scores, s_up).
+ *   mask[b*N+n]   = scores > tau ? 1 : 0   (strict).
+ * x: T[B][N][C]; w_g: T[C]; b_g: host scalar; s_up: float[B*N] or NULL;
+ * scores: float[B*N] out; mask: uint8[B*N] out. */
+int spa_gate(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up,
+             float* scores, uint8_t* mask, void* stream);
+
+/* Token packing (Sec. 3.2 "Token Packing"): stable compaction of the selected tokens, images in
+ * batch order and tokens in raster order.
+ *   cu_seqlens[0] = 0, cu_seqlens[b+1] = cu_seqlens[b] + popcount(mask[b][:]);
+ *   idx[i] = flat position b*N+n of packed row i (ascending);  inv[b*N+n] = i or -1;
+ *   x_packed[i][:] = x[idx[i]][:]   (times sigmoid(scores[idx[i]]) under SPA_FLAG_GATE_SCALE).
+ * mask: uint8[B*N] (non-zero = selected); scores: float[B*N], only read under GATE_SCALE, else
+ * may be NULL; x_packed: T[capacity][C] out; idx: int32[capacity] out; inv: int32[B*N] out or
+ * NULL; cu_seqlens: int32[B+1] out.  If more than `capacity` tokens are selected the surplus rows
+ * are dropped, cu_seqlens still holds the true counts and SPA_ERR_CAPACITY is recorded in d_status;
+ * every later call clamps N_p to capacity.  B*N must not exceed 2^20. */
+int spa_select_pack(const spa_params* p, const void* x, const uint8_t* mask, const float* scores,
+                    void* x_packed, int32_t* idx, int32_t* inv, int32_t* cu_seqlens,
+                    int32_t* d_status, void* stream);
+
+/* QKV projection on the packed tokens (the 3LC^2 term of Eq. 9):
+ *   qkv[i][j] = b_qkv[j] + sum_c W_qkv[j][c] * x_packed[i][c],  i < N_p, j < 3C.
+ * W_qkv: T[3C][C]; b_qkv: T[3C] or NULL; qkv: T[capacity][3C] out. */
+int spa_packed_qkv(const spa_params* p, const void* x_packed, const void* W_qkv, const void* b_qkv,
+                   const int32_t* cu_seqlens, void* qkv, int32_t* d_status, void* stream);
+
+/* Multi-head self-attention in which a packed token attends only to tokens of its own segment
+ * (Sec. 3.2: the attention mask keeps tokens from attending to other images; the 2L^2C term).
+ * For segment s = [seg_offsets[s], seg_offsets[s+1]) and head h, over rows i, j of the segment:
+ *   S_ij = scale * q_i . k_j;  P = softmax_j(S);  attn_out_i = sum_j P_ij v_j;
+ *   lse[h][i] = log sum_j exp(S_ij).
+ * seg_offsets: int32[n_seg+1], ascending, seg_offsets[0] = 0; pass cu_seqlens and B for the
+ * default same-image mask.  N_p = seg_offsets[n_seg].  attn_out: T[capacity][C]; lse: float[H][capacity]. */
+int spa_packed_attention_fwd(const spa_params* p, const void* qkv, const int32_t* seg_offsets,
+                             int32_t n_seg, void* attn_out, float* lse, int32_t* d_status,
+                             void* stream);
+
+/* Gradient of spa_packed_attention_fwd with respect to qkv (the paper trains through the block,
+ * Sec. 1; it gives no derivation, this is the standard softmax-attention gradient):
+ *   D_i = sum_e d_attn_out_ie * attn_out_ie;  P_ij = exp(S_ij - lse_i);
+ *   dV_j = sum_i P_ij dO_i;  dS_ij = P_ij (dO_i . v_j - D_i);
+ *   dQ_i = scale * sum_j dS_ij k_j;  dK_j = scale * sum_i dS_ij q_i.
+ * dqkv: T[capacity][3C] out, same column layout as qkv.  workspace: scratch, may be NULL when
+ * spa_workspace_bytes() is 0. */
+int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* attn_out,
+                             const float* lse, const void* d_attn_out, const int32_t* seg_offsets,
+                             int32_t n_seg, void* dqkv, void* workspace, int32_t* d_status,
+                             void* stream);
+
+/* Output projection on the packed tokens:  z[i][j] = b_o[j] + sum_c W_o[j][c] * a[i][c].
+ * a: T[capacity][C]; W_o: T[C][C]; b_o: T[C] or NULL; z: T[capacity][C] out. */
+int spa_packed_proj(const spa_params* p, const void* a, const void* W_o, const void* b_o,
+                    const int32_t* cu_seqlens, void* z, int32_t* d_status, void* stream);
+
+/* Unpack: y[b][n][:] = z_packed[inv[b*N+n]][:] for selected tokens, x[b][n][:] otherwise
+ * (Sec. 3.2: negative tokens are passed on unchanged).  SPA_FLAG_RESIDUAL adds x on selected rows.
+ * Out of place (y != x) every row of y is written; under SPA_FLAG_INPLACE y must equal x and only
+ * the selected rows are written. */
+int spa_unpack_scatter(const spa_params* p, const void* z_packed, const void* x, const int32_t* idx,
+                       const int32_t* inv, const int32_t* cu_seqlens, void* y, int32_t* d_status,
+                       void* stream);
+
+/* Transpose of spa_unpack_scatter:  dz_packed[i][:] = dY[idx[i]][:];  dX[t][:] = dY[t][:] for
+ * unselected tokens t.  Selected rows of dX are left for spa_select_pack_bwd.  dX may equal dY
+ * (nothing is copied for unselected rows then) or be NULL. */
+int spa_unpack_scatter_bwd(const spa_params* p, const void* dY, const int32_t* idx,
+                           const int32_t* inv, const int32_t* cu_seqlens, void* dz_packed, void* dX,
+                           void* stream);
+
+/* Transpose of the pack gather:  dX[idx[i]][:] = dx_packed[i][:]  (+ dY[idx[i]][:] under
+ * SPA_FLAG_RESIDUAL; dY may be NULL otherwise). */
+int spa_select_pack_bwd(const spa_params* p, const void* dx_packed, const void* dY,
+                        const int32_t* idx, const int32_t* cu_seqlens, void* dX, void* stream);
+
+/* Gradients of a packed linear layer out = a W^T + b with W: T[n_out][n_in]:
+ *   da[i][:] = dout[i][:] W           (T[capacity][n_in], may be NULL)
+ *   dW = dout^T a                     (float[n_out][n_in], may be NULL)
+ *   db[j] = sum_i dout[i][j]          (float[n_out], may be NULL)
+ * Sums over packed rows run in a fixed order: results are bitwise reproducible.
+ * n_in and n_out must be multiples of 16 bytes / sizeof(T). */
+int spa_packed_linear_bwd(const spa_params* p, const void* a, const void* W, const void* dout,
+                          int32_t n_in, int32_t n_out, const int32_t* cu_seqlens, void* da,
+                          float* dW, float* db, void* workspace, int32_t* d_status, void* stream);
+
+/* Blocking read of the device status word: synchronises `stream` and returns its value. */
+int spa_read_status(const int32_t* d_status, void* stream);
+
+/* Static text for a spa_status value. */
+const char* spa_status_string(int status);
+
+/* Text of the last CUDA error a call of this library met on the calling thread ("" if none). */
+const char* spa_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPA_H_ */

@@ -1,0 +1,165 @@
+"""ctypes binding of libspa.so: the same names as include/spa.h, argument marshalling only.
+
+Every function takes torch tensors that already live on the GPU (PyTorch is used for device
+memory and streams, nothing else), checks nothing but presence, and raises SpaError when the
+library returns a negative status.  There is no fallback: if the library is missing or no CUDA
+device is present, calling into it raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspa.so")
+
+SPA_OK, SPA_ERR_INVALID_ARG, SPA_ERR_UNSUPPORTED, SPA_ERR_CAPACITY, SPA_ERR_CUDA, SPA_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+SPA_F32, SPA_BF16 = 0, 1
+SPA_FLAG_RESIDUAL, SPA_FLAG_INPLACE, SPA_FLAG_GATE_SCALE, SPA_FLAG_SIMT_ONLY = 1, 2, 4, 8
+
+EXPORTS = (
+    "spa_workspace_bytes", "spa_gate", "spa_select_pack", "spa_packed_qkv", "spa_packed_attention_fwd",
+    "spa_packed_attention_bwd", "spa_packed_proj", "spa_unpack_scatter", "spa_unpack_scatter_bwd",
+    "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
+    "spa_last_cuda_error",
+)
+
+
+class SpaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().spa_status_string(status).decode()
+        if status == SPA_ERR_CUDA:
+            msg += ": " + lib().spa_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+class SpaParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("C", C.c_int32), ("H", C.c_int32), ("dtype", C.c_int32),
+                ("flags", C.c_int32), ("capacity", C.c_int32), ("tau", C.c_float), ("softmax_scale", C.c_float)]
+
+
+def make_params(B, N, Cc, H, dtype, capacity=None, flags=0, tau=0.0, softmax_scale=0.0) -> SpaParams:
+    dt = {"f32": SPA_F32, "bf16": SPA_BF16, torch.float32: SPA_F32, torch.bfloat16: SPA_BF16}.get(dtype, dtype)
+    return SpaParams(B, N, Cc, H, dt, flags, capacity if capacity is not None else max(B * N, 1), tau, softmax_scale)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library.  Raises if it has not been built (run `python -m paper_2410_23608_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with paper_2410_23608_b200.build.build()")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, f32 = C.c_void_p, C.c_int32, C.c_float
+        pp = C.POINTER(SpaParams)
+        L.spa_workspace_bytes.restype = C.c_size_t
+        L.spa_workspace_bytes.argtypes = [pp]
+        L.spa_gate.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp]
+        L.spa_select_pack.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_packed_qkv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_packed_attention_fwd.argtypes = [pp, vp, vp, i32, vp, vp, vp, vp]
+        L.spa_packed_attention_bwd.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        L.spa_packed_proj.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_unpack_scatter.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_unpack_scatter_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_select_pack_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp]
+        L.spa_packed_linear_bwd.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_read_status.argtypes = [vp, vp]
+        for name in EXPORTS:
+            if name not in ("spa_workspace_bytes", "spa_status_string", "spa_last_cuda_error"):
+                getattr(L, name).restype = C.c_int
+        L.spa_status_string.restype = C.c_char_p
+        L.spa_status_string.argtypes = [C.c_int]
+        L.spa_last_cuda_error.restype = C.c_char_p
+        L.spa_last_cuda_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("the SPA library takes device tensors only")
+    if not t.is_contiguous():
+        raise ValueError("tensors must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc < 0:
+        raise SpaError(rc, where)
+
+
+def spa_workspace_bytes(p: SpaParams) -> int:
+    return int(lib().spa_workspace_bytes(C.byref(p)))
+
+
+def spa_gate(p, x, w_g, b_g, s_up, scores, mask, stream=None):
+    _check(lib().spa_gate(C.byref(p), _ptr(x), _ptr(w_g), float(b_g), _ptr(s_up), _ptr(scores), _ptr(mask),
+                          _stream(stream)), "spa_gate")
+
+
+def spa_select_pack(p, x, mask, scores, x_packed, idx, inv, cu_seqlens, d_status=None, stream=None):
+    _check(lib().spa_select_pack(C.byref(p), _ptr(x), _ptr(mask), _ptr(scores), _ptr(x_packed), _ptr(idx), _ptr(inv),
+                                 _ptr(cu_seqlens), _ptr(d_status), _stream(stream)), "spa_select_pack")
+
+
+def spa_packed_qkv(p, x_packed, W_qkv, b_qkv, cu_seqlens, qkv, d_status=None, stream=None):
+    _check(lib().spa_packed_qkv(C.byref(p), _ptr(x_packed), _ptr(W_qkv), _ptr(b_qkv), _ptr(cu_seqlens), _ptr(qkv),
+                                _ptr(d_status), _stream(stream)), "spa_packed_qkv")
+
+
+def spa_packed_attention_fwd(p, qkv, seg_offsets, n_seg, attn_out, lse, d_status=None, stream=None):
+    _check(lib().spa_packed_attention_fwd(C.byref(p), _ptr(qkv), _ptr(seg_offsets), int(n_seg), _ptr(attn_out),
+                                          _ptr(lse), _ptr(d_status), _stream(stream)), "spa_packed_attention_fwd")
+
+
+def spa_packed_attention_bwd(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace=None,
+                             d_status=None, stream=None):
+    _check(lib().spa_packed_attention_bwd(C.byref(p), _ptr(qkv), _ptr(attn_out), _ptr(lse), _ptr(d_attn_out),
+                                          _ptr(seg_offsets), int(n_seg), _ptr(dqkv), _ptr(workspace), _ptr(d_status),
+                                          _stream(stream)), "spa_packed_attention_bwd")
+
+
+def spa_packed_proj(p, a, W_o, b_o, cu_seqlens, z, d_status=None, stream=None):
+    _check(lib().spa_packed_proj(C.byref(p), _ptr(a), _ptr(W_o), _ptr(b_o), _ptr(cu_seqlens), _ptr(z),
+                                 _ptr(d_status), _stream(stream)), "spa_packed_proj")
+
+
+def spa_unpack_scatter(p, z_packed, x, idx, inv, cu_seqlens, y, d_status=None, stream=None):
+    _check(lib().spa_unpack_scatter(C.byref(p), _ptr(z_packed), _ptr(x), _ptr(idx), _ptr(inv), _ptr(cu_seqlens),
+                                    _ptr(y), _ptr(d_status), _stream(stream)), "spa_unpack_scatter")
+
+
+def spa_unpack_scatter_bwd(p, dY, idx, inv, cu_seqlens, dz_packed, dX, stream=None):
+    _check(lib().spa_unpack_scatter_bwd(C.byref(p), _ptr(dY), _ptr(idx), _ptr(inv), _ptr(cu_seqlens),
+                                        _ptr(dz_packed), _ptr(dX), _stream(stream)), "spa_unpack_scatter_bwd")
+
+
+def spa_select_pack_bwd(p, dx_packed, dY, idx, cu_seqlens, dX, stream=None):
+    _check(lib().spa_select_pack_bwd(C.byref(p), _ptr(dx_packed), _ptr(dY), _ptr(idx), _ptr(cu_seqlens), _ptr(dX),
+                                     _stream(stream)), "spa_select_pack_bwd")
+
+
+def spa_packed_linear_bwd(p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, workspace=None, d_status=None,
+                          stream=None):
+    _check(lib().spa_packed_linear_bwd(C.byref(p), _ptr(a), _ptr(W), _ptr(dout), int(n_in), int(n_out),
+                                       _ptr(cu_seqlens), _ptr(da), _ptr(dW), _ptr(db), _ptr(workspace),
+                                       _ptr(d_status), _stream(stream)), "spa_packed_linear_bwd")
+
+
+def spa_read_status(d_status, stream=None) -> int:
+    return int(lib().spa_read_status(_ptr(d_status), _stream(stream)))

@@ -1,0 +1,207 @@
+// C boundary: argument validation and dispatch to the kernels.  Nothing here computes.
+#include <stdio.h>
+#include <string.h>
+
+#include "spa_common.cuh"
+#include "spa_tc.cuh"
+
+namespace spa {
+
+static thread_local char g_cuda_error[256] = "";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_params(const spa_params* p) {
+  if (p == nullptr) return SPA_ERR_INVALID_ARG;
+  if (p->B < 0 || p->N <= 0 || p->C <= 0 || p->H <= 0) return SPA_ERR_INVALID_ARG;
+  if ((long long)p->B * p->N > (1LL << 20)) return SPA_ERR_UNSUPPORTED;
+  if (p->capacity < 1 || (long long)p->capacity > (long long)(p->B > 0 ? p->B : 1) * p->N) return SPA_ERR_INVALID_ARG;
+  if (p->dtype != SPA_F32 && p->dtype != SPA_BF16) return SPA_ERR_UNSUPPORTED;
+  if (p->C % p->H != 0) return SPA_ERR_INVALID_ARG;
+  const int es = p->dtype == SPA_F32 ? 4 : 2;
+  if ((p->C * es) % 16 != 0 || p->C > 8192) return SPA_ERR_UNSUPPORTED;
+  return SPA_OK;
+}
+
+int check_heads(const spa_params* p) {
+  const int d = p->C / p->H;
+  return (d == 32 || d == 64) ? SPA_OK : SPA_ERR_UNSUPPORTED;
+}
+
+// bf16 problems run on the tensor-core kernels unless the caller asks for the fp32-FMA ones
+inline bool use_tc(const spa_params* p) { return p->dtype == SPA_BF16 && !(p->flags & SPA_FLAG_SIMT_ONLY); }
+
+#define SPA_REQUIRE(cond, code) do { if (!(cond)) return (code); } while (0)
+#define SPA_PTR(ptr) SPA_REQUIRE((ptr) != nullptr && aligned16(ptr), SPA_ERR_INVALID_ARG)
+#define SPA_OPT_PTR(ptr) SPA_REQUIRE((ptr) == nullptr || aligned16(ptr), SPA_ERR_INVALID_ARG)
+
+}  // namespace
+}  // namespace spa
+
+using namespace spa;
+
+extern "C" {
+
+size_t spa_workspace_bytes(const spa_params* p) {
+  if (check_params(p) != SPA_OK) return 0;
+  return tc_workspace_bytes(*p);
+}
+
+int spa_gate(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up, float* scores,
+             uint8_t* mask, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(w_g); SPA_PTR(scores); SPA_PTR(mask); SPA_OPT_PTR(s_up);
+  return launch_gate(*p, x, w_g, b_g, s_up, scores, mask, (cudaStream_t)stream);
+}
+
+int spa_select_pack(const spa_params* p, const void* x, const uint8_t* mask, const float* scores, void* x_packed,
+                    int32_t* idx, int32_t* inv, int32_t* cu_seqlens, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(mask); SPA_PTR(x_packed); SPA_PTR(idx); SPA_PTR(cu_seqlens); SPA_OPT_PTR(inv);
+  if (p->flags & SPA_FLAG_GATE_SCALE) SPA_PTR(scores);
+  if (p->B == 0) {
+    cudaError_t e = cudaMemsetAsync(cu_seqlens, 0, sizeof(int32_t), (cudaStream_t)stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "spa_select_pack"); return SPA_ERR_CUDA; }
+    return SPA_OK;
+  }
+  return launch_select_pack(*p, x, mask, scores, x_packed, idx, inv, cu_seqlens, d_status, (cudaStream_t)stream);
+}
+
+int spa_packed_qkv(const spa_params* p, const void* x_packed, const void* W_qkv, const void* b_qkv,
+                   const int32_t* cu_seqlens, void* qkv, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x_packed); SPA_PTR(W_qkv); SPA_PTR(cu_seqlens); SPA_PTR(qkv); SPA_OPT_PTR(b_qkv);
+  if (use_tc(p) && tc_linear_supported(p->C, 3 * p->C))
+    return launch_linear_fwd_tc(*p, x_packed, W_qkv, b_qkv, p->C, 3 * p->C, cu_seqlens, qkv, d_status,
+                                (cudaStream_t)stream);
+  return launch_linear_fwd_simt(*p, x_packed, W_qkv, b_qkv, p->C, 3 * p->C, cu_seqlens, qkv, (cudaStream_t)stream);
+}
+
+int spa_packed_proj(const spa_params* p, const void* a, const void* W_o, const void* b_o, const int32_t* cu_seqlens,
+                    void* z, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(a); SPA_PTR(W_o); SPA_PTR(cu_seqlens); SPA_PTR(z); SPA_OPT_PTR(b_o);
+  if (use_tc(p) && tc_linear_supported(p->C, p->C))
+    return launch_linear_fwd_tc(*p, a, W_o, b_o, p->C, p->C, cu_seqlens, z, d_status, (cudaStream_t)stream);
+  return launch_linear_fwd_simt(*p, a, W_o, b_o, p->C, p->C, cu_seqlens, z, (cudaStream_t)stream);
+}
+
+int spa_packed_attention_fwd(const spa_params* p, const void* qkv, const int32_t* seg_offsets, int32_t n_seg,
+                             void* attn_out, float* lse, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  rc = check_heads(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(qkv); SPA_PTR(seg_offsets); SPA_PTR(attn_out); SPA_PTR(lse);
+  SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
+  if (use_tc(p) && tc_attention_fwd_supported(*p))
+    return launch_attention_fwd_tc(*p, qkv, seg_offsets, n_seg, attn_out, lse, d_status, (cudaStream_t)stream);
+  return launch_attention_fwd_simt(*p, qkv, seg_offsets, n_seg, attn_out, lse, (cudaStream_t)stream);
+}
+
+int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
+                             const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg, void* dqkv,
+                             void* workspace, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  rc = check_heads(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(qkv); SPA_PTR(attn_out); SPA_PTR(lse); SPA_PTR(d_attn_out); SPA_PTR(seg_offsets); SPA_PTR(dqkv);
+  SPA_OPT_PTR(workspace);
+  SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
+  if (use_tc(p) && tc_attention_bwd_supported(*p) && workspace != nullptr)
+    return launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace, d_status,
+                                   (cudaStream_t)stream);
+  return launch_attention_bwd_simt(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv,
+                                   (cudaStream_t)stream);
+}
+
+int spa_unpack_scatter(const spa_params* p, const void* z_packed, const void* x, const int32_t* idx,
+                       const int32_t* inv, const int32_t* cu_seqlens, void* y, int32_t* d_status, void* stream) {
+  (void)d_status;
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(z_packed); SPA_PTR(cu_seqlens); SPA_PTR(y);
+  if (p->flags & SPA_FLAG_INPLACE) {
+    SPA_PTR(idx);
+    SPA_REQUIRE(x == nullptr || x == y, SPA_ERR_INVALID_ARG);
+    x = y;
+  } else {
+    SPA_PTR(x); SPA_PTR(inv);
+    SPA_REQUIRE(x != y, SPA_ERR_INVALID_ARG);
+  }
+  if (p->B == 0) return SPA_OK;
+  return launch_unpack_scatter(*p, z_packed, x, idx, inv, cu_seqlens, y, (cudaStream_t)stream);
+}
+
+int spa_unpack_scatter_bwd(const spa_params* p, const void* dY, const int32_t* idx, const int32_t* inv,
+                           const int32_t* cu_seqlens, void* dz_packed, void* dX, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dY); SPA_PTR(inv); SPA_PTR(cu_seqlens); SPA_PTR(dz_packed); SPA_OPT_PTR(dX);
+  if (p->B == 0) return SPA_OK;
+  return launch_unpack_scatter_bwd(*p, dY, idx, inv, cu_seqlens, dz_packed, dX, (cudaStream_t)stream);
+}
+
+int spa_select_pack_bwd(const spa_params* p, const void* dx_packed, const void* dY, const int32_t* idx,
+                        const int32_t* cu_seqlens, void* dX, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dx_packed); SPA_PTR(idx); SPA_PTR(cu_seqlens); SPA_PTR(dX);
+  if (p->flags & SPA_FLAG_RESIDUAL) SPA_PTR(dY);
+  if (p->B == 0) return SPA_OK;
+  return launch_select_pack_bwd(*p, dx_packed, dY, idx, cu_seqlens, dX, (cudaStream_t)stream);
+}
+
+int spa_packed_linear_bwd(const spa_params* p, const void* a, const void* W, const void* dout, int32_t n_in,
+                          int32_t n_out, const int32_t* cu_seqlens, void* da, float* dW, float* db, void* workspace,
+                          int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dout); SPA_PTR(cu_seqlens);
+  SPA_OPT_PTR(da); SPA_OPT_PTR(dW); SPA_OPT_PTR(db); SPA_OPT_PTR(workspace);
+  if (da != nullptr) SPA_PTR(W);
+  if (dW != nullptr) SPA_PTR(a);
+  SPA_REQUIRE(n_in > 0 && n_out > 0, SPA_ERR_INVALID_ARG);
+  const int es = p->dtype == SPA_F32 ? 4 : 2;
+  SPA_REQUIRE((n_in * es) % 16 == 0 && (n_out * es) % 16 == 0, SPA_ERR_UNSUPPORTED);
+  if (use_tc(p) && tc_linear_supported(n_in, n_out) && workspace != nullptr)
+    return launch_linear_bwd_tc(*p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, workspace, d_status,
+                                (cudaStream_t)stream);
+  return launch_linear_bwd_simt(*p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, (cudaStream_t)stream);
+}
+
+int spa_read_status(const int32_t* d_status, void* stream) {
+  if (d_status == nullptr) return SPA_ERR_INVALID_ARG;
+  int32_t v = 0;
+  cudaError_t e = cudaMemcpyAsync(&v, d_status, sizeof(v), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error(e, "spa_read_status"); return SPA_ERR_CUDA; }
+  return v;
+}
+
+const char* spa_status_string(int status) {
+  switch (status) {
+    case SPA_OK: return "ok";
+    case SPA_ERR_INVALID_ARG: return "invalid argument";
+    case SPA_ERR_UNSUPPORTED: return "unsupported dtype, head dimension or size";
+    case SPA_ERR_CAPACITY: return "more selected tokens than the packed capacity";
+    case SPA_ERR_CUDA: return "CUDA runtime error";
+    case SPA_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+const char* spa_last_cuda_error(void) { return g_cuda_error; }
+
+}  // extern "C"

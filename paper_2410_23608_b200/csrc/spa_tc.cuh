@@ -1,0 +1,25 @@
+// Tensor-core (tcgen05 / TMEM / TMA) kernels for bf16 problems: entry points used by the dispatcher.
+#pragma once
+
+#include "spa_common.cuh"
+
+namespace spa {
+
+size_t tc_workspace_bytes(const spa_params& p);
+
+bool tc_linear_supported(int n_in, int n_out);
+int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
+                         const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st);
+int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
+                         const int32_t* cu, void* da, float* dW, float* db, void* workspace, int32_t* d_status,
+                         cudaStream_t st);
+
+bool tc_attention_fwd_supported(const spa_params& p);
+int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
+                            int32_t* d_status, cudaStream_t st);
+bool tc_attention_bwd_supported(const spa_params& p);
+int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
+                            const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
+                            cudaStream_t st);
+
+}  // namespace spa
