@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of one SPA block (forward + backward) on synthetic data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl ours|reference]
+
+A step is one pass of the whole block over one batch: gate, select/pack, QKV, segment-masked
+attention, output projection, unpack, then the backward pass.  The metric is selected tokens per
+second (N_p of the batch / step time), whole job over all GPUs.  At N > 1 every rank runs the same
+independent replica on its own GPU (images are independent; the block has no exchange step).
+
+Timing: CUDA events on the launching stream, max over ranks, several buffer sets rotated so the
+working set exceeds L2.  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "selected_tokens_per_sec_spa_block_fwd_bwd"
+UNIT = "tokens/s"
+L2_BYTES = 126e6
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            m = json.load(f)
+        return dict(hbm=float(m["hbm_gbs"]), tensor=float(m["bf16_tflops"]), source="measured")
+    return dict(hbm=6650.0, tensor=1590.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- work model
+def work_model(cfg, cu):
+    """Algorithmic bytes and FLOPs of every call for the realised selection (FLOPs = 2 x MACs)."""
+    n = np.diff(np.asarray(cu, np.int64))
+    Np, S2 = int(n.sum()), int((n * n).sum())
+    B, N, C, H, es = cfg.B, cfg.N, cfg.C, cfg.H, cfg.elem_size
+    BN = B * N
+    w = {}
+    w["gate"] = dict(bytes=BN * C * es + 5 * BN, flops=2 * BN * C)
+    w["select_pack"] = dict(bytes=BN + 2 * Np * C * es + 4 * Np + 4 * BN, flops=0)
+    w["qkv"] = dict(bytes=(Np * C + 3 * C * C + 3 * Np * C) * es, flops=2 * Np * C * 3 * C)
+    w["attn_fwd"] = dict(bytes=4 * Np * C * es + 4 * H * Np, flops=4 * C * S2)
+    w["proj"] = dict(bytes=(2 * Np * C + C * C) * es, flops=2 * Np * C * C)
+    w["unpack"] = dict(bytes=2 * BN * C * es + 4 * BN, flops=0)
+    w["unpack_bwd"] = dict(bytes=2 * BN * C * es + 4 * BN, flops=0)
+    w["proj_bwd"] = dict(bytes=(3 * Np * C + C * C) * es + 4 * C * C, flops=4 * Np * C * C)
+    w["attn_bwd"] = dict(bytes=(3 + 1 + 1 + 3) * Np * C * es + 4 * H * Np, flops=10 * C * S2)
+    w["qkv_bwd"] = dict(bytes=(Np * C + 3 * Np * C + Np * C + 3 * C * C) * es + 12 * C * C, flops=12 * Np * C * C)
+    w["pack_bwd"] = dict(bytes=2 * Np * C * es + 4 * Np, flops=0)
+    return w, Np, S2
+
+
+def call_sequence(L, blk, d, b_g):
+    """The block as (name, thunk) pairs, one per C-ABI call, in execution order."""
+    p, C = blk.p, blk.C
+    return [
+        ("gate", lambda: L.spa_gate(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask)),
+        ("select_pack", lambda: L.spa_select_pack(p, d["x"], blk.mask, blk.scores, blk.xp, blk.idx, blk.inv, blk.cu,
+                                                  blk.status)),
+        ("qkv", lambda: L.spa_packed_qkv(p, blk.xp, d["W_qkv"], d["b_qkv"], blk.cu, blk.qkv, blk.status)),
+        ("attn_fwd", lambda: L.spa_packed_attention_fwd(p, blk.qkv, blk.cu, blk.B, blk.ao, blk.lse, blk.status)),
+        ("proj", lambda: L.spa_packed_proj(p, blk.ao, d["W_o"], d["b_o"], blk.cu, blk.z, blk.status)),
+        ("unpack", lambda: L.spa_unpack_scatter(p, blk.z, d["x"], blk.idx, blk.inv, blk.cu, blk.y, blk.status)),
+        ("unpack_bwd", lambda: L.spa_unpack_scatter_bwd(p, d["dY"], blk.idx, blk.inv, blk.cu, blk.dz, blk.dX)),
+        ("proj_bwd", lambda: L.spa_packed_linear_bwd(p, blk.ao, d["W_o"], blk.dz, C, C, blk.cu, blk.dao, blk.dW_o,
+                                                     blk.db_o, blk.workspace, blk.status)),
+        ("attn_bwd", lambda: L.spa_packed_attention_bwd(p, blk.qkv, blk.ao, blk.lse, blk.dao, blk.cu, blk.B, blk.dqkv,
+                                                        blk.workspace, blk.status)),
+        ("qkv_bwd", lambda: L.spa_packed_linear_bwd(p, blk.xp, d["W_qkv"], blk.dqkv, C, 3 * C, blk.cu, blk.dxp,
+                                                    blk.dW_qkv, blk.db_qkv, blk.workspace, blk.status)),
+        ("pack_bwd", lambda: L.spa_select_pack_bwd(p, blk.dxp, d["dY"], blk.idx, blk.cu, blk.dX)),
+    ]
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.strip().splitlines():
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ----------------------------------------------------------------------------- oracle timing
+def oracle_step(O, inp, cfg):
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
+    O.block_bwd(fwd, inp.dY, inp.x, inp.W_qkv, inp.W_o, cfg.H)
+    return int(fwd["cu_seqlens"][-1])
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(inp, cfg, budget_s=12.0, max_reps=20, min_reps=1):
+    from oracle import spa_oracle as O
+    Np = oracle_step(O, inp, cfg)  # untimed first pass (page-in)
+    times = []
+    t_end = time.perf_counter() + budget_s
+    while len(times) < min_reps or (time.perf_counter() < t_end and len(times) < max_reps):
+        t0 = time.perf_counter()
+        oracle_step(O, inp, cfg)
+        times.append(time.perf_counter() - t0)
+    return Np, times
+
+
+def run_reference(args):
+    """The reference arm: the fp64 oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from spa_workloads import get_config, make_inputs
+    from oracle import spa_oracle as O
+    cfg = get_config(args.config)
+    inp = make_inputs(cfg)
+    Np = 0
+    for _ in range(args.warmup):
+        Np = oracle_step(O, inp, cfg)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        Np = oracle_step(O, inp, cfg)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    val = Np / dt
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "C": cfg.C, "H": cfg.H, "selected_tokens": Np},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"whole {cfg.name} batch, forward+backward, {args.steps} timed repetitions"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (default 2, ViT-S/16-like bf16)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 200 and args.warmup == 20:
+            args.steps, args.warmup = 5, 1
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2410_23608_b200 import build as spa_build
+    from paper_2410_23608_b200 import binding as L
+    from paper_2410_23608_b200.block import SpaBlock
+    from spa_workloads import get_config, make_inputs, scaled_config
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SPA library has no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        spa_build.build()
+    if world > 1:
+        dist.barrier()
+    L.lib()
+    args.warmup = max(args.warmup, 3)
+
+    cfg = get_config(args.config)
+    # rotating buffer sets: inputs, outputs and every intermediate differ from step to step
+    per_set = (4 * cfg.B * cfg.N * cfg.C + 12 * cfg.B * cfg.N * cfg.C) * cfg.elem_size
+    n_sets = args.sets if args.sets > 0 else max(2, int(np.ceil(2.5 * L2_BYTES / per_set)))
+    names = ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")
+    sets, inps = [], []
+    for s in range(n_sets):
+        inp = make_inputs(scaled_config(cfg, seed=cfg.seed + 1000 * s)) if s < 2 else inps[s % 2]
+        inps.append(inp)
+        d = {n: inp.torch(n, "cuda") for n in names}
+        blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau)
+        sets.append((inp, d, blk, call_sequence(L, blk, d, inp.b_g)))
+
+    def step(i):
+        for _, fn in sets[i % n_sets][3]:
+            fn()
+
+    stream = torch.cuda.current_stream()
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    Np_sets = [int(b.cu[-1].item()) for _, _, b, _ in sets]
+    assert all(b.read_status() == 0 for _, _, b, _ in sets)
+    tokens_per_step = float(np.mean([Np_sets[i % n_sets] for i in range(args.steps)]))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing of exactly K steps
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    n0 = L.spa_launch_count()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    launches = L.spa_launch_count() - n0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- end to end: pinned host inputs in, results out, every step
+    hx = [inp.torch("x").pin_memory() for inp in inps[:2]]
+    hdy = [inp.torch("dY").pin_memory() for inp in inps[:2]]
+    hy = torch.empty_like(hx[0]).pin_memory()
+    hdx = torch.empty_like(hx[0]).pin_memory()
+
+    def e2e_step(i):
+        inp, d, blk, seq = sets[i % n_sets]
+        d["x"].copy_(hx[i % 2], non_blocking=True)
+        d["dY"].copy_(hdy[i % 2], non_blocking=True)
+        for _, fn in seq:
+            fn()
+        hy.copy_(blk.y, non_blocking=True)
+        hdx.copy_(blk.dX, non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        e2e_step(i)
+    e1.record(stream)
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item()) / args.steps
+    bytes_io = cfg.B * cfg.N * cfg.C * cfg.elem_size
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-call device times (CUDA events between calls, same rotation), for the roofline
+    n_calls = len(sets[0][3])
+    reps = min(args.steps, 100)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_calls + 1)] for _ in range(reps)]
+    torch.cuda.synchronize()
+    for r in range(reps):
+        seq = sets[r % n_sets][3]
+        evs[r][0].record(stream)
+        for c, (_, fn) in enumerate(seq):
+            fn()
+            evs[r][c + 1].record(stream)
+    torch.cuda.synchronize()
+    call_ms = {}
+    for c, (name, _) in enumerate(sets[0][3]):
+        call_ms[name] = float(np.mean([evs[r][c].elapsed_time(evs[r][c + 1]) for r in range(reps)]))
+    pk = peaks()
+    work, Np0, S2 = work_model(cfg, sets[0][2].cu.cpu().numpy())
+    per_call = {}
+    for name, ms_c in call_ms.items():
+        wk = work[name]
+        t_b = wk["bytes"] / (pk["hbm"] * 1e9)
+        t_f = wk["flops"] / (pk["tensor"] * 1e12)
+        bound = "tensor" if (t_f > t_b and cfg.dtype == "bf16") else "hbm"
+        ach = wk["flops"] / (ms_c * 1e-3) / 1e12 if bound == "tensor" else wk["bytes"] / (ms_c * 1e-3) / 1e9
+        per_call[name] = dict(us=round(ms_c * 1e3, 2), bound=bound, achieved=round(ach, 2),
+                              frac=round(ach / pk[bound], 4))
+    top = max(call_ms, key=call_ms.get)
+    tr = per_call[top]
+    roofline = {"kernel": top, "bound": tr["bound"], "achieved": tr["achieved"], "peak": pk[tr["bound"]],
+                "unit": "TFLOP/s" if tr["bound"] == "tensor" else "GB/s", "frac": tr["frac"], "traffic": None,
+                "peak_source": pk["source"], "us_per_launch": tr["us"]}
+
+    # ---- forward-only time (same rotation), reported beside the headline
+    e0.record(stream)
+    for i in range(reps):
+        for _, fn in sets[i % n_sets][3][:6]:
+            fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    fwd_ms = e0.elapsed_time(e1) / reps
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        Np_o, times = time_oracle(inps[0], cfg)
+        cpu = {"value": Np_o / float(np.mean(times)), "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"whole {cfg.name} batch, forward+backward, {len(times)} repetitions "
+                         f"({sum(times):.1f} s of CPU work)"}
+
+    useful_flops = sum(work[k]["flops"] for k in work)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "C": cfg.C, "H": cfg.H,
+                   "selected_tokens": Np_sets[0], "sum_nb_squared": S2, "pass": "forward+backward",
+                   "l2_policy": f"{n_sets} rotating buffer sets, {per_set * n_sets / 1e6:.0f} MB > L2",
+                   "replicas": world},
+        "e2e": {"value": world * tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": 2 * bytes_io, "d2h_bytes_per_step": 2 * bytes_io},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "forward_only": {"ms_per_step": fwd_ms, "value": Np_sets[0] / (fwd_ms * 1e-3), "unit": UNIT},
+        "useful_tflops": useful_flops / (ms_per_step * 1e-3) / 1e12,
+        "per_call": per_call,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

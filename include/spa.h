@@ -165,6 +165,10 @@ const char* spa_status_string(int status);
 /* Text of the last CUDA error a call of this library met on the calling thread ("" if none). */
 const char* spa_last_cuda_error(void);
 
+/* Number of kernels this library has enqueued in this process so far (host-side tally, all
+ * threads; used to report launches per step). */
+unsigned long long spa_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

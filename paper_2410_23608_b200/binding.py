@@ -24,7 +24,7 @@ EXPORTS = (
     "spa_workspace_bytes", "spa_gate", "spa_select_pack", "spa_packed_qkv", "spa_packed_attention_fwd",
     "spa_packed_attention_bwd", "spa_packed_proj", "spa_unpack_scatter", "spa_unpack_scatter_bwd",
     "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
-    "spa_last_cuda_error",
+    "spa_last_cuda_error", "spa_launch_count",
 )
 
 
@@ -73,12 +73,14 @@ def lib() -> C.CDLL:
         L.spa_packed_linear_bwd.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
-            if name not in ("spa_workspace_bytes", "spa_status_string", "spa_last_cuda_error"):
+            if name not in ("spa_workspace_bytes", "spa_status_string", "spa_last_cuda_error", "spa_launch_count"):
                 getattr(L, name).restype = C.c_int
         L.spa_status_string.restype = C.c_char_p
         L.spa_status_string.argtypes = [C.c_int]
         L.spa_last_cuda_error.restype = C.c_char_p
         L.spa_last_cuda_error.argtypes = []
+        L.spa_launch_count.restype = C.c_ulonglong
+        L.spa_launch_count.argtypes = []
         _lib = L
     return _lib
 
@@ -163,3 +165,7 @@ def spa_packed_linear_bwd(p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, wo
 
 def spa_read_status(d_status, stream=None) -> int:
     return int(lib().spa_read_status(_ptr(d_status), _stream(stream)))
+
+
+def spa_launch_count() -> int:
+    return int(lib().spa_launch_count())

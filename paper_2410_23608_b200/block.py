@@ -1,0 +1,96 @@
+"""One SPA block as a sequence of library calls.
+
+`SpaBlock` owns the device buffers of one block (allocated once through PyTorch) and issues the
+C-ABI calls in order on the current stream.  It computes nothing itself: every step runs in the
+CUDA library.  Nothing here synchronises; N_p stays on the device.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as L
+
+
+class SpaBlock:
+    """Buffers + call sequence for gate -> select/pack -> QKV -> attention -> projection -> unpack
+    (paper Sec. 3.2) and the matching backward pass."""
+
+    def __init__(self, B: int, N: int, C: int, H: int, dtype: str, tau: float = 0.0, flags: int = 0,
+                 capacity: Optional[int] = None, backward: bool = True, device: str = "cuda"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("SpaBlock needs a CUDA device; there is no CPU path")
+        L.lib()
+        self.B, self.N, self.C, self.H = B, N, C, H
+        self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
+        cap = capacity if capacity is not None else max(B * N, 1)
+        self.p = L.make_params(B, N, C, H, dtype, cap, flags, tau)
+        self.cap = cap
+        dev = torch.device(device)
+        T = self.tdtype
+        e = lambda *s, dt=T: torch.empty(*s, dtype=dt, device=dev)
+        self.scores = e(max(B * N, 1), dt=torch.float32)
+        self.mask = e(max(B * N, 1), dt=torch.uint8)
+        self.cu = torch.zeros(B + 1, dtype=torch.int32, device=dev)
+        self.idx = e(cap, dt=torch.int32)
+        self.inv = e(max(B * N, 1), dt=torch.int32)
+        self.xp = e(cap, C)
+        self.qkv = e(cap, 3 * C)
+        self.ao = e(cap, C)
+        self.lse = e(H, cap, dt=torch.float32)
+        self.z = e(cap, C)
+        self.y = e(B, N, C)
+        self.status = torch.zeros(4, dtype=torch.int32, device=dev)
+        ws = L.spa_workspace_bytes(self.p)
+        self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if ws > 0 else None
+        if backward:
+            self.dz = e(cap, C)
+            self.dao = e(cap, C)
+            self.dqkv = e(cap, 3 * C)
+            self.dxp = e(cap, C)
+            self.dX = e(B, N, C)
+            self.dW_qkv = e(3 * C, C, dt=torch.float32)
+            self.db_qkv = e(3 * C, dt=torch.float32)
+            self.dW_o = e(C, C, dt=torch.float32)
+            self.db_o = e(C, dt=torch.float32)
+        self._saved = None
+
+    # ------------------------------------------------------------------ forward
+    def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None):
+        p = self.p
+        y = self.y if y is None else y
+        L.spa_gate(p, x, w_g, b_g, s_up, self.scores, self.mask)
+        L.spa_select_pack(p, x, self.mask, self.scores, self.xp, self.idx, self.inv, self.cu, self.status)
+        L.spa_packed_qkv(p, self.xp, W_qkv, b_qkv, self.cu, self.qkv, self.status)
+        L.spa_packed_attention_fwd(p, self.qkv, self.cu, self.B, self.ao, self.lse, self.status)
+        L.spa_packed_proj(p, self.ao, W_o, b_o, self.cu, self.z, self.status)
+        if p.flags & L.SPA_FLAG_INPLACE:
+            L.spa_unpack_scatter(p, self.z, None, self.idx, self.inv, self.cu, x, self.status)
+            y = x
+        else:
+            L.spa_unpack_scatter(p, self.z, x, self.idx, self.inv, self.cu, y, self.status)
+        self._saved = (W_qkv, W_o)
+        return y
+
+    # ------------------------------------------------------------------ backward
+    def backward(self, dY, dX=None):
+        """Gradients for the last forward(): returns dX; parameter gradients land in dW_qkv, db_qkv,
+        dW_o, db_o (fp32).  No gradient reaches the gate (hard threshold)."""
+        p = self.p
+        W_qkv, W_o = self._saved
+        dX = self.dX if dX is None else dX
+        C = self.C
+        L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
+        L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
+                                self.workspace, self.status)
+        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self.cu, self.B, self.dqkv,
+                                   self.workspace, self.status)
+        L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv, self.db_qkv,
+                                self.workspace, self.status)
+        L.spa_select_pack_bwd(p, self.dxp, dY, self.idx, self.cu, dX)
+        return dX
+
+    def read_status(self) -> int:
+        """Blocking: the device status word (0 = ok)."""
+        return L.spa_read_status(self.status)

@@ -2,6 +2,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "spa_common.cuh"
 #include "spa_tc.cuh"
 
@@ -12,6 +14,9 @@ static thread_local char g_cuda_error[256] = "";
 void set_cuda_error(cudaError_t e, const char* where) {
   snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
 }
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 namespace {
 
@@ -203,5 +208,7 @@ const char* spa_status_string(int status) {
 }
 
 const char* spa_last_cuda_error(void) { return g_cuda_error; }
+
+unsigned long long spa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

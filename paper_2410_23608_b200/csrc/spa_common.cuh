@@ -87,10 +87,12 @@ __device__ __forceinline__ int find_segment(const int32_t* __restrict__ offsets,
 
 // ---- host side -------------------------------------------------------------------------------
 void set_cuda_error(cudaError_t e, const char* where);
+void count_launch();  // one more kernel of this library was enqueued (host-side tally)
 #define SPA_CUDA_CHECK_LAUNCH(where)                                   \
   do {                                                                 \
     cudaError_t e__ = cudaGetLastError();                              \
     if (e__ != cudaSuccess) { ::spa::set_cuda_error(e__, where); return SPA_ERR_CUDA; } \
+    ::spa::count_launch();                                             \
   } while (0)
 
 // launchers implemented per .cu file; every one enqueues on `st` and returns a spa_status

@@ -1,0 +1,195 @@
+"""GPU edge cases of the SPA library against the oracle: empty and single-token segments, nothing or
+everything selected, ragged sizes, exact and insufficient capacity, the optional inputs and flags."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spa_oracle as O
+from spa_workloads import get_config, make_inputs, scaled_config
+from tests.gpu_util import TOL, assert_close, dev, host, round_to
+
+pytestmark = pytest.mark.gpu
+
+
+def L():
+    from paper_2410_23608_b200 import binding
+    return binding
+
+
+def block(B, N, C, H, dtype, **kw):
+    from paper_2410_23608_b200.block import SpaBlock
+    return SpaBlock(B, N, C, H, dtype, **kw)
+
+
+def random_problem(B, N, C, H, dtype, counts, seed=0):
+    """x, weights and a mask with exactly counts[b] selected tokens in image b."""
+    rng = np.random.default_rng(seed)
+    x = round_to(rng.normal(size=(B, N, C)), dtype)
+    mask = np.zeros((B, N), bool)
+    for b, c in enumerate(counts):
+        mask[b, rng.choice(N, size=c, replace=False)] = True
+    W_qkv = round_to(rng.normal(size=(3 * C, C)) / np.sqrt(C), dtype)
+    b_qkv = round_to(rng.normal(size=3 * C) * 0.02, dtype)
+    W_o = round_to(rng.normal(size=(C, C)) / np.sqrt(C), dtype)
+    b_o = round_to(rng.normal(size=C) * 0.02, dtype)
+    dY = round_to(rng.normal(size=(B, N, C)), dtype)
+    return x, mask, W_qkv, b_qkv, W_o, b_o, dY
+
+
+@pytest.mark.parametrize("dtype,C,H,xflags", [("f32", 96, 3, 0), ("bf16", 128, 2, 0), ("bf16", 128, 4, 0),
+                                               ("bf16", 128, 2, 8)])
+def test_ragged_segments_from_a_given_mask(dtype, C, H, xflags):
+    counts = [0, 1, 2, 63, 64, 65, 130, 0, 197, 7, 0]
+    B, N = len(counts), 197
+    x, mask, W_qkv, b_qkv, W_o, b_o, dY = random_problem(B, N, C, H, dtype, counts)
+    lib = L()
+    blk = block(B, N, C, H, dtype, flags=xflags)
+    p = blk.p
+    xd = dev(x, dtype)
+    blk.mask.copy_(torch.from_numpy(mask.reshape(-1).astype(np.uint8)))
+    lib.spa_select_pack(p, xd, blk.mask, None, blk.xp, blk.idx, blk.inv, blk.cu, blk.status)
+    cu, idx, inv = O.pack_indices(mask)
+    Np = int(cu[-1])
+    assert np.array_equal(blk.cu.cpu().numpy(), cu)
+    assert np.array_equal(blk.idx.cpu().numpy()[:Np], idx)
+    assert np.array_equal(blk.inv.cpu().numpy(), inv)
+    xp = O.pack_rows(x, idx)
+    assert np.array_equal(host(blk.xp)[:Np], xp)
+    Wq, bq, Wo, bo = (dev(a, dtype) for a in (W_qkv, b_qkv, W_o, b_o))
+    lib.spa_packed_qkv(p, blk.xp, Wq, bq, blk.cu, blk.qkv, blk.status)
+    lib.spa_packed_attention_fwd(p, blk.qkv, blk.cu, B, blk.ao, blk.lse, blk.status)
+    lib.spa_packed_proj(p, blk.ao, Wo, bo, blk.cu, blk.z, blk.status)
+    lib.spa_unpack_scatter(p, blk.z, xd, blk.idx, blk.inv, blk.cu, blk.y, blk.status)
+    qkv = O.linear(xp, W_qkv, b_qkv)
+    ao, lse = O.attention_fwd(qkv, cu, H)
+    z = O.linear(ao, W_o, b_o)
+    y = O.unpack_scatter(z, x, idx)
+    assert_close(host(blk.ao)[:Np], ao, dtype, "attn_out")
+    assert np.abs(host(blk.lse)[:, :Np] - lse).max() <= TOL[dtype]["lse"]
+    assert_close(host(blk.y), y, dtype, "y")
+    # single-token segment: attention returns v
+    one = int(cu[1])
+    assert_close(host(blk.ao)[one], host(blk.qkv)[one, 2 * C:], dtype, "n_b = 1")
+    # backward through the same chain
+    blk._saved = (Wq, Wo)
+    dX = blk.backward(dev(dY, dtype))
+    fwd = dict(idx=idx, ao=ao, qkv=qkv, lse=lse, xp=xp, seg=cu)
+    bwd = O.block_bwd(fwd, dY, x, W_qkv, W_o, H)
+    assert_close(host(blk.dqkv)[:Np], bwd["dqkv"], dtype, "dqkv", scale_max_abs=True)
+    assert_close(host(dX), bwd["dX"], dtype, "dX", scale_max_abs=True)
+    assert_close(host(blk.dW_qkv), bwd["dW_qkv"], dtype, "dW_qkv", scale_max_abs=True)
+    assert_close(host(blk.db_o), bwd["db_o"], dtype, "db_o", scale_max_abs=True)
+    assert blk.read_status() == 0
+
+
+@pytest.mark.parametrize("ci", [1, 2])
+def test_none_selected_and_all_selected(ci):
+    cfg = scaled_config(get_config(ci), B=3)
+    inp = make_inputs(cfg)
+    d = {n: dev(getattr(inp, n), cfg.dtype) for n in ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")}
+    # nothing selected: y == x and dX == dY bit for bit, parameter gradients are zero
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=float("inf"))
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    dX = blk.backward(d["dY"])
+    assert torch.equal(y, d["x"]) and torch.equal(dX, d["dY"])
+    assert not blk.cu.any() and not blk.mask.any() and bool((blk.inv == -1).all())
+    assert not blk.dW_qkv.any() and not blk.dW_o.any() and not blk.db_qkv.any() and not blk.db_o.any()
+    # everything selected: ordinary dense multi-head attention
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=float("-inf"))
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    dX = blk.backward(d["dY"])
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, -np.inf, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
+    bwd = O.block_bwd(fwd, inp.dY, inp.x, inp.W_qkv, inp.W_o, cfg.H)
+    assert np.array_equal(blk.cu.cpu().numpy(), np.arange(cfg.B + 1) * cfg.N)
+    assert_close(host(y), fwd["y"], cfg.dtype, "y")
+    assert_close(host(dX), bwd["dX"], cfg.dtype, "dX", scale_max_abs=True)
+    assert blk.read_status() == 0
+
+
+def test_capacity_exact_and_too_small():
+    cfg = scaled_config(get_config(2), B=5)
+    inp = make_inputs(cfg)
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
+    Np = int(fwd["cu_seqlens"][-1])
+    d = {n: dev(getattr(inp, n), cfg.dtype) for n in ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")}
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, capacity=Np)
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    blk.backward(d["dY"])
+    assert blk.read_status() == 0
+    assert_close(host(y), fwd["y"], cfg.dtype, "y")
+    # too small: an error status, no fault, counts still true, the rows that fit are right
+    small = Np - 37
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, capacity=small)
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    blk.backward(d["dY"])
+    torch.cuda.synchronize()
+    assert blk.read_status() == L().SPA_ERR_CAPACITY
+    assert np.array_equal(blk.cu.cpu().numpy(), fwd["cu_seqlens"])
+    assert np.array_equal(blk.idx.cpu().numpy(), fwd["idx"][:small])
+    assert np.array_equal(host(blk.xp), fwd["xp"][:small])
+    assert torch.isfinite(y.float()).all()
+
+
+def test_upscale_scores_gate_scale_and_containers():
+    lib = L()
+    cfg = scaled_config(get_config(2), B=4)
+    inp = make_inputs(cfg)
+    rng = np.random.default_rng(5)
+    s_up = rng.normal(size=(cfg.B, cfg.N)).astype(np.float32) * 3
+    s = O.gate(inp.x, inp.w_g, inp.b_g, s_up)
+    keep = np.abs(s - inp.tau) > 1e-3          # only compare decisions away from the threshold
+    mask = O.select(s, inp.tau)
+    d = {n: dev(getattr(inp, n), cfg.dtype) for n in ("x", "w_g", "W_qkv", "b_qkv")}
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, flags=lib.SPA_FLAG_GATE_SCALE)
+    p = blk.p
+    lib.spa_gate(p, d["x"], d["w_g"], inp.b_g, torch.from_numpy(s_up.reshape(-1)).cuda(), blk.scores, blk.mask)
+    assert np.abs(host(blk.scores) - s.reshape(-1)).max() <= 1e-4
+    got_mask = blk.mask.cpu().numpy().astype(bool).reshape(cfg.B, cfg.N)
+    assert np.array_equal(got_mask[keep], mask[keep])
+    # Eq. 5: packed rows scaled by sigmoid(score)
+    lib.spa_select_pack(p, d["x"], blk.mask, blk.scores, blk.xp, blk.idx, blk.inv, blk.cu, blk.status)
+    cu, idx, inv = O.pack_indices(got_mask)
+    xp = O.pack_rows(inp.x, idx, host(blk.scores).reshape(cfg.B, cfg.N), gate_scale=True)
+    assert np.array_equal(blk.idx.cpu().numpy()[:idx.size], idx)
+    assert_close(host(blk.xp)[:idx.size], xp, cfg.dtype, "gated rows")
+    # containers of length 49: attention limited to same image and same container
+    lib.spa_packed_qkv(p, blk.xp, d["W_qkv"], d["b_qkv"], blk.cu, blk.qkv, blk.status)
+    cuts = O.container_cuts(cu, 49)
+    seg = torch.from_numpy(cuts).cuda()
+    lib.spa_packed_attention_fwd(p, blk.qkv, seg, len(cuts) - 1, blk.ao, blk.lse, blk.status)
+    qkv = host(blk.qkv)[:idx.size]
+    ao, lse = O.attention_fwd(qkv, cuts, cfg.H)
+    assert_close(host(blk.ao)[:idx.size], ao, cfg.dtype, "container attention")
+    dao = round_to(rng.normal(size=ao.shape), cfg.dtype)
+    dao_d = torch.zeros_like(blk.ao)
+    dao_d[:idx.size] = dev(dao, cfg.dtype)
+    dqkv = torch.empty_like(blk.qkv)
+    lib.spa_packed_attention_bwd(p, blk.qkv, blk.ao, blk.lse, dao_d, seg, len(cuts) - 1, dqkv, blk.workspace,
+                                 blk.status)
+    ref = O.attention_bwd(qkv, host(blk.ao)[:idx.size], host(blk.lse)[:, :idx.size], dao, cuts, cfg.H)
+    assert_close(host(dqkv)[:idx.size], ref, cfg.dtype, "container attention bwd", scale_max_abs=True)
+    assert blk.read_status() == 0
+
+
+def test_invalid_arguments_are_rejected_on_the_host():
+    lib = L()
+    x = torch.zeros(2, 16, 64, device="cuda")
+    sc = torch.zeros(32, device="cuda")
+    mk = torch.zeros(32, dtype=torch.uint8, device="cuda")
+    w = torch.zeros(64, device="cuda")
+    with pytest.raises(lib.SpaError) as e:
+        lib.spa_gate(lib.make_params(2, 16, 64, 3, "f32"), x, w, 0.0, None, sc, mk)      # C % H != 0
+    assert e.value.status == lib.SPA_ERR_INVALID_ARG
+    with pytest.raises(lib.SpaError) as e:
+        lib.spa_gate(lib.make_params(2, 16, 64, 2, "f32"), x, None, 0.0, None, sc, mk)   # null pointer
+    assert e.value.status == lib.SPA_ERR_INVALID_ARG
+    with pytest.raises(lib.SpaError) as e:
+        lib.spa_gate(lib.make_params(2, 16, 64, 2, "f32"), x.view(-1)[1:], w, 0.0, None, sc, mk)  # misaligned
+    assert e.value.status == lib.SPA_ERR_INVALID_ARG
+    p = lib.make_params(2, 16, 64, 4, "f32")                                               # d = 16
+    with pytest.raises(lib.SpaError) as e:
+        lib.spa_packed_attention_fwd(p, x, torch.zeros(3, dtype=torch.int32, device="cuda"), 2, x, sc)
+    assert e.value.status == lib.SPA_ERR_UNSUPPORTED
+    with pytest.raises(lib.SpaError) as e:
+        lib.spa_gate(lib.make_params(2, 16, 64, 2, "f32", capacity=33), x, w, 0.0, None, sc, mk)  # capacity > B*N
+    assert e.value.status == lib.SPA_ERR_INVALID_ARG

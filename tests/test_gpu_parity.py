@@ -1,0 +1,172 @@
+"""GPU parity: the CUDA library, called through its C boundary, against the fp64 oracle on the same
+seeded inputs.  Integer and index outputs must match bit for bit; floating point within the stated
+tolerances (fp32: max-abs 1e-4; bf16: max-abs 3e-2 and relative RMS 1e-2)."""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import spa_oracle as O
+from spa_workloads import get_config, make_inputs, scaled_config
+from tests.gpu_util import TOL, assert_close, dev, host, round_to
+
+pytestmark = pytest.mark.gpu
+
+
+@functools.lru_cache(maxsize=None)
+def problem(i, residual=False):
+    cfg = get_config(i)
+    inp = make_inputs(cfg)
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H,
+                      residual=residual)
+    bwd = O.block_bwd(fwd, inp.dY, inp.x, inp.W_qkv, inp.W_o, cfg.H, residual=residual)
+    return cfg, inp, fwd, bwd
+
+
+def device_inputs(cfg, inp):
+    names = ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")
+    return {n: dev(getattr(inp, n), cfg.dtype) for n in names}
+
+
+def make_block(cfg, flags=0, capacity=None, tau=None):
+    from paper_2410_23608_b200.block import SpaBlock
+    return SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau if tau is None else tau, flags=flags,
+                    capacity=capacity)
+
+
+def check_indices(blk, fwd):
+    Np = int(fwd["cu_seqlens"][-1])
+    assert np.array_equal(blk.mask.cpu().numpy().astype(bool), fwd["mask"].reshape(-1))
+    assert np.array_equal(blk.cu.cpu().numpy(), fwd["cu_seqlens"])
+    assert np.array_equal(blk.idx.cpu().numpy()[:Np], fwd["idx"])
+    assert np.array_equal(blk.inv.cpu().numpy(), fwd["inv"])
+    return Np
+
+
+VARIANTS = [(1, 0), (2, 0), (2, 8), (3, 0), (3, 8), (4, 0), (5, 0), (5, 8)]  # (config, extra flags); 8 = fp32-FMA kernels
+
+
+@pytest.mark.parametrize("ci,xflags", VARIANTS)
+def test_block_forward_backward_end_to_end(ci, xflags):
+    cfg, inp, fwd, bwd = problem(ci)
+    d = device_inputs(cfg, inp)
+    blk = make_block(cfg, flags=xflags)
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    dX = blk.backward(d["dY"])
+    torch.cuda.synchronize()
+    assert blk.read_status() == 0
+    dt = cfg.dtype
+    Np = check_indices(blk, fwd)
+    assert np.abs(host(blk.scores) - fwd["scores"].reshape(-1)).max() <= TOL[dt]["score"]
+    assert np.array_equal(host(blk.xp)[:Np], fwd["xp"])            # a pure row gather: exact
+    assert_close(host(blk.qkv)[:Np], fwd["qkv"], dt, "qkv")
+    assert_close(host(blk.ao)[:Np], fwd["ao"], dt, "attn_out")
+    assert np.abs(host(blk.lse)[:, :Np] - fwd["lse"]).max() <= TOL[dt]["lse"]
+    assert_close(host(blk.z)[:Np], fwd["z"], dt, "z")
+    yh = host(y)
+    assert_close(yh, fwd["y"], dt, "y")
+    unsel = ~fwd["mask"]
+    assert np.array_equal(yh[unsel], inp.x[unsel])                 # pass-through rows: bitwise
+    # backward
+    assert np.array_equal(host(blk.dz)[:Np], bwd["dz"])
+    assert_close(host(blk.dao)[:Np], bwd["dao"], dt, "d_attn_out", scale_max_abs=True)
+    assert_close(host(blk.dqkv)[:Np], bwd["dqkv"], dt, "dqkv", scale_max_abs=True)
+    assert_close(host(blk.dxp)[:Np], bwd["dxp"], dt, "dx_packed", scale_max_abs=True)
+    dXh = host(dX)
+    assert_close(dXh, bwd["dX"], dt, "dX", scale_max_abs=True)
+    assert np.array_equal(dXh[unsel], inp.dY[unsel])
+    for name in ("dW_qkv", "db_qkv", "dW_o", "db_o"):
+        assert_close(host(getattr(blk, name)), bwd[name], dt, name, scale_max_abs=True)
+
+
+@pytest.mark.parametrize("ci,xflags", VARIANTS)
+def test_each_call_on_oracle_upstream(ci, xflags):
+    """Every call is fed the oracle's own upstream tensors (rounded to the storage dtype), so an error
+    cannot hide behind, or be blamed on, an earlier step."""
+    from paper_2410_23608_b200 import binding as L
+    cfg, inp, fwd, bwd = problem(ci)
+    dt = cfg.dtype
+    d = device_inputs(cfg, inp)
+    blk = make_block(cfg, flags=xflags)
+    p = blk.p
+    Np = int(fwd["cu_seqlens"][-1])
+    cap = blk.cap
+    cu = torch.from_numpy(fwd["cu_seqlens"]).cuda()
+    H, C = cfg.H, cfg.C
+
+    def padded(a, cols):
+        buf = np.zeros((cap, cols))
+        buf[:Np] = a
+        return buf
+
+    # QKV on the oracle's packed rows (exact copies of x rows)
+    xp = dev(padded(fwd["xp"], C), dt)
+    L.spa_packed_qkv(p, xp, d["W_qkv"], d["b_qkv"], cu, blk.qkv, blk.status)
+    assert_close(host(blk.qkv)[:Np], fwd["qkv"], dt, "qkv")
+    # attention on the oracle's qkv, rounded
+    qkv_r = round_to(fwd["qkv"], dt)
+    ao_ref, lse_ref = O.attention_fwd(qkv_r, fwd["cu_seqlens"], H)
+    qkv = dev(padded(qkv_r, 3 * C), dt)
+    L.spa_packed_attention_fwd(p, qkv, cu, cfg.B, blk.ao, blk.lse, blk.status)
+    assert_close(host(blk.ao)[:Np], ao_ref, dt, "attn_out")
+    assert np.abs(host(blk.lse)[:, :Np] - lse_ref).max() <= TOL[dt]["lse"]
+    # projection
+    ao_r = round_to(ao_ref, dt)
+    L.spa_packed_proj(p, dev(padded(ao_r, C), dt), d["W_o"], d["b_o"], cu, blk.z, blk.status)
+    assert_close(host(blk.z)[:Np], O.linear(ao_r, inp.W_o, inp.b_o), dt, "z")
+    # attention backward on rounded oracle tensors
+    dao_r = round_to(bwd["dao"], dt)
+    lse_t = torch.zeros(H, cap, dtype=torch.float32, device="cuda")
+    lse_t[:, :Np] = torch.from_numpy(lse_ref).float().cuda()
+    dqkv_ref = O.attention_bwd(qkv_r, ao_r, lse_t[:, :Np].double().cpu().numpy(), dao_r, fwd["cu_seqlens"], H)
+    L.spa_packed_attention_bwd(p, qkv, dev(padded(ao_r, C), dt), lse_t, dev(padded(dao_r, C), dt), cu, cfg.B,
+                               blk.dqkv, blk.workspace, blk.status)
+    assert_close(host(blk.dqkv)[:Np], dqkv_ref, dt, "dqkv", scale_max_abs=True)
+    # linear backward (QKV layer) on rounded oracle tensors
+    dqkv_r = round_to(bwd["dqkv"], dt)
+    da_ref, dW_ref, db_ref = O.linear_bwd(fwd["xp"], inp.W_qkv, dqkv_r)
+    L.spa_packed_linear_bwd(p, xp, d["W_qkv"], dev(padded(dqkv_r, 3 * C), dt), C, 3 * C, cu, blk.dxp, blk.dW_qkv,
+                            blk.db_qkv, blk.workspace, blk.status)
+    assert_close(host(blk.dxp)[:Np], da_ref, dt, "dx_packed", scale_max_abs=True)
+    assert_close(host(blk.dW_qkv), dW_ref, dt, "dW_qkv", scale_max_abs=True)
+    assert_close(host(blk.db_qkv), db_ref, dt, "db_qkv", scale_max_abs=True)
+    torch.cuda.synchronize()
+    assert blk.read_status() == 0
+
+
+@pytest.mark.parametrize("ci", [1, 2])
+@pytest.mark.parametrize("flags", [1, 2, 3])   # residual, in-place, both
+def test_residual_and_inplace_flags(ci, flags):
+    residual = bool(flags & 1)
+    cfg, inp, fwd, bwd = problem(ci, residual)
+    d = device_inputs(cfg, inp)
+    blk = make_block(cfg, flags=flags)
+    x = d["x"].clone()
+    y = blk.forward(x, d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    if flags & 2:
+        assert y.data_ptr() == x.data_ptr()
+    assert_close(host(y), fwd["y"], cfg.dtype, "y")
+    unsel = ~fwd["mask"]
+    assert np.array_equal(host(y)[unsel], inp.x[unsel])
+    dX = blk.backward(d["dY"])
+    assert_close(host(dX), bwd["dX"], cfg.dtype, "dX", scale_max_abs=True)
+    # dX aliasing dY: only the selected rows are rewritten
+    dY2 = d["dY"].clone()
+    dX2 = blk.backward(dY2, dX=dY2)
+    assert torch.equal(dX2, dX)
+    assert blk.read_status() == 0
+
+
+def test_run_to_run_determinism():
+    cfg, inp, fwd, bwd = problem(2)
+    d = device_inputs(cfg, inp)
+    outs = []
+    for _ in range(2):
+        blk = make_block(cfg)
+        y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+        dX = blk.backward(d["dY"])
+        Np = int(fwd["cu_seqlens"][-1])
+        outs.append([t.clone() for t in (y, dX, blk.dW_qkv, blk.db_qkv, blk.dW_o, blk.db_o, blk.dqkv[:Np])])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)

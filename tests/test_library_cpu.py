@@ -1,0 +1,55 @@
+"""CPU-side checks of the C boundary: the library builds, loads, exports every symbol that
+include/spa.h declares, and rejects bad arguments on the host before touching a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2410_23608_b200 import build, binding
+    build.build()
+    return binding
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "spa.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(spa_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert "spa_gate" in names and "spa_packed_attention_bwd" in names and len(names) >= 14
+    cdll = ctypes.CDLL(lib.LIB_PATH)
+    for n in names:
+        assert hasattr(cdll, n), n
+    assert set(lib.EXPORTS) == set(names)
+
+
+def test_status_strings(lib):
+    L = lib.lib()
+    assert L.spa_status_string(0) == b"ok"
+    for code in (-1, -2, -3, -4, -5):
+        assert L.spa_status_string(code) not in (b"ok", b"unknown status")
+    assert L.spa_status_string(-99) == b"unknown status"
+
+
+def test_host_side_validation_needs_no_gpu(lib):
+    L = lib.lib()
+    p = lib.make_params(2, 16, 64, 2, "f32")
+    assert L.spa_gate(ctypes.byref(p), None, None, 0.0, None, None, None, None) == lib.SPA_ERR_INVALID_ARG
+    assert L.spa_gate(None, None, None, 0.0, None, None, None, None) == lib.SPA_ERR_INVALID_ARG
+    bad = lib.make_params(2, 16, 60, 2, "bf16")     # 120-byte rows: not a multiple of 16
+    assert L.spa_gate(ctypes.byref(bad), None, None, 0.0, None, None, None, None) == lib.SPA_ERR_UNSUPPORTED
+    big = lib.make_params(4096, 4096, 64, 2, "bf16")
+    assert L.spa_workspace_bytes(ctypes.byref(big)) == 0     # B*N beyond the supported 2^20
+    assert L.spa_launch_count() >= 0
+
+
+def test_params_struct_layout_matches_header(lib):
+    assert ctypes.sizeof(lib.SpaParams) == 36
