@@ -6,8 +6,11 @@ from spa_workloads import bf16_round
 
 TOL = {
     # max-abs, relative RMS (None = not checked) per storage dtype
-    "f32": dict(max_abs=1e-4, rel_rms=None, lse=1e-5, score=1e-4),
-    "bf16": dict(max_abs=3e-2, rel_rms=1e-2, lse=1e-3, score=1e-4),
+    # lse: bound when the attention call reads the same qkv bits as the oracle; lse_chain: bound in an
+    # end-to-end chain, where the device qkv carries one storage rounding the oracle's does not
+    # (|dS| <= scale * sum_e |dq_e k_e + q_e dk_e| with relative steps of 2^-9 in bf16).
+    "f32": dict(max_abs=1e-4, rel_rms=None, lse=1e-5, lse_chain=1e-5, score=1e-4),
+    "bf16": dict(max_abs=3e-2, rel_rms=1e-2, lse=1e-3, lse_chain=3e-2, score=1e-4),
 }
 
 

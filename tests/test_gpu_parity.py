@@ -62,7 +62,7 @@ def test_block_forward_backward_end_to_end(ci, xflags):
     assert np.array_equal(host(blk.xp)[:Np], fwd["xp"])            # a pure row gather: exact
     assert_close(host(blk.qkv)[:Np], fwd["qkv"], dt, "qkv")
     assert_close(host(blk.ao)[:Np], fwd["ao"], dt, "attn_out")
-    assert np.abs(host(blk.lse)[:, :Np] - fwd["lse"]).max() <= TOL[dt]["lse"]
+    assert np.abs(host(blk.lse)[:, :Np] - fwd["lse"]).max() <= TOL[dt]["lse_chain"]
     assert_close(host(blk.z)[:Np], fwd["z"], dt, "z")
     yh = host(y)
     assert_close(yh, fwd["y"], dt, "y")
