@@ -55,7 +55,8 @@ extern "C" {
 
 size_t spa_workspace_bytes(const spa_params* p) {
   if (check_params(p) != SPA_OK) return 0;
-  return tc_workspace_bytes(*p);
+  const size_t a = tc_linear_workspace_bytes(*p), b = tc_attention_workspace_bytes(*p);
+  return a > b ? a : b;
 }
 
 int spa_gate(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up, float* scores,
@@ -85,9 +86,11 @@ int spa_packed_qkv(const spa_params* p, const void* x_packed, const void* W_qkv,
   int rc = check_params(p);
   if (rc != SPA_OK) return rc;
   SPA_PTR(x_packed); SPA_PTR(W_qkv); SPA_PTR(cu_seqlens); SPA_PTR(qkv); SPA_OPT_PTR(b_qkv);
-  if (use_tc(p) && tc_linear_supported(p->C, 3 * p->C))
-    return launch_linear_fwd_tc(*p, x_packed, W_qkv, b_qkv, p->C, 3 * p->C, cu_seqlens, qkv, d_status,
-                                (cudaStream_t)stream);
+  if (use_tc(p) && tc_linear_supported(p->C, 3 * p->C)) {
+    rc = launch_linear_fwd_tc(*p, x_packed, W_qkv, b_qkv, p->C, 3 * p->C, cu_seqlens, qkv, d_status,
+                              (cudaStream_t)stream);
+    if (rc != SPA_ERR_UNSUPPORTED) return rc;  // geometry the TMA path cannot describe: fp32-FMA kernels
+  }
   return launch_linear_fwd_simt(*p, x_packed, W_qkv, b_qkv, p->C, 3 * p->C, cu_seqlens, qkv, (cudaStream_t)stream);
 }
 
@@ -96,8 +99,10 @@ int spa_packed_proj(const spa_params* p, const void* a, const void* W_o, const v
   int rc = check_params(p);
   if (rc != SPA_OK) return rc;
   SPA_PTR(a); SPA_PTR(W_o); SPA_PTR(cu_seqlens); SPA_PTR(z); SPA_OPT_PTR(b_o);
-  if (use_tc(p) && tc_linear_supported(p->C, p->C))
-    return launch_linear_fwd_tc(*p, a, W_o, b_o, p->C, p->C, cu_seqlens, z, d_status, (cudaStream_t)stream);
+  if (use_tc(p) && tc_linear_supported(p->C, p->C)) {
+    rc = launch_linear_fwd_tc(*p, a, W_o, b_o, p->C, p->C, cu_seqlens, z, d_status, (cudaStream_t)stream);
+    if (rc != SPA_ERR_UNSUPPORTED) return rc;
+  }
   return launch_linear_fwd_simt(*p, a, W_o, b_o, p->C, p->C, cu_seqlens, z, (cudaStream_t)stream);
 }
 
@@ -180,9 +185,11 @@ int spa_packed_linear_bwd(const spa_params* p, const void* a, const void* W, con
   SPA_REQUIRE(n_in > 0 && n_out > 0, SPA_ERR_INVALID_ARG);
   const int es = p->dtype == SPA_F32 ? 4 : 2;
   SPA_REQUIRE((n_in * es) % 16 == 0 && (n_out * es) % 16 == 0, SPA_ERR_UNSUPPORTED);
-  if (use_tc(p) && tc_linear_supported(n_in, n_out) && workspace != nullptr)
-    return launch_linear_bwd_tc(*p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, workspace, d_status,
-                                (cudaStream_t)stream);
+  if (use_tc(p) && tc_linear_supported(n_in, n_out) && workspace != nullptr) {
+    rc = launch_linear_bwd_tc(*p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, workspace, d_status,
+                              (cudaStream_t)stream);
+    if (rc != SPA_ERR_UNSUPPORTED) return rc;
+  }
   return launch_linear_bwd_simt(*p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, (cudaStream_t)stream);
 }
 

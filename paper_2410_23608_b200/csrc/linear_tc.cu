@@ -1,0 +1,420 @@
+// bf16 linear layers on the packed tokens as tcgen05 GEMMs: QKV / output projection (the 3LC^2 and
+// NC^2 terms of Eq. 9), their input gradients and their weight gradients.
+//
+// One kernel, three operand arrangements.  D[128 x BN] tiles accumulate in TMEM (fp32); operands
+// are staged by TMA into 128-byte-swizzled shared memory through a ring of kStages buffers; one
+// thread issues tcgen05.mma, one thread issues TMA, four warps drain TMEM and store.
+//   forward   out = a W^T      A = a    (K-major),  B = W   (K-major),  M = packed rows (device)
+//   dgrad     da  = dout W     A = dout (K-major),  B = W   (MN-major), M = packed rows (device)
+//   wgrad     dW  = dout^T a   A = dout (MN-major), B = a   (MN-major), K = packed rows (device)
+// The packed row count N_p lives on the device: grids are sized for `capacity` rows and CTAs
+// beyond N_p exit at once.  wgrad splits K = N_p across CTAs; each split writes an fp32 partial to
+// the workspace and a second kernel adds the partials in a fixed order (no float atomics, bitwise
+// reproducible).  Rows of the last K block that lie beyond N_p are zeroed in shared memory before
+// the MMA reads them, so unspecified rows of the packed buffers never reach a sum.
+#include <mutex>
+#include <string>
+#include <unordered_map>
+
+#include "sm100_ptx.cuh"
+#include "spa_tc.cuh"
+
+namespace spa {
+
+// ------------------------------------------------------------------------------ tensor maps
+namespace {
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = []() -> EncodeFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeFn>(p);
+  }();
+  return fn;
+}
+
+std::mutex g_tm_mutex;
+std::unordered_map<std::string, CUtensorMap> g_tm_cache;
+}  // namespace
+
+bool make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t rows, uint64_t row_stride_bytes,
+                       uint32_t box_inner, uint32_t box_rows) {
+  struct Key { const void* b; uint64_t i, r, s; uint32_t bi, br; } key{base, inner, rows, row_stride_bytes, box_inner, box_rows};
+  std::string k(reinterpret_cast<const char*>(&key), sizeof(key));
+  std::lock_guard<std::mutex> lock(g_tm_mutex);
+  auto it = g_tm_cache.find(k);
+  if (it != g_tm_cache.end()) { *out = it->second; return true; }
+  EncodeFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {row_stride_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (g_tm_cache.size() > 4096) g_tm_cache.clear();
+  g_tm_cache.emplace(std::move(k), *out);
+  return true;
+}
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kStages = 3;
+constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kABytes = BM * BK * 2;
+
+template <int BN> __host__ __device__ constexpr int stage_bytes() { return kABytes + BN * BK * 2; }
+template <int BN> __host__ __device__ constexpr int gemm_smem_bytes() { return kStages * stage_bytes<BN>() + 1024 + 128; }
+
+template <typename OutT> struct OutStore;
+template <> struct OutStore<__nv_bfloat16> {
+  // 8 consecutive columns as one 16-byte store
+  __device__ static __forceinline__ void store8(__nv_bfloat16* dst, const float* v) {
+    *reinterpret_cast<uint4*>(dst) = Vec16<__nv_bfloat16>::from_float(v);
+  }
+};
+template <> struct OutStore<float> {
+  __device__ static __forceinline__ void store8(float* dst, const float* v) {
+    reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+};
+
+// dyn_which: 1 = M is the device-side packed row count, 2 = K is.
+template <int BN, bool kAMn, bool kBMn, typename OutT>
+__global__ void __launch_bounds__(kGemmThreads)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
+               long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
+               int dyn_which, int k_per_split, int32_t* d_status) {
+  constexpr int kStage = stage_bytes<BN>();
+  constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
+  {
+    const int rows = packed_rows(cu, n_seg, capacity);
+    if (dyn_which == 1) M = rows; else if (dyn_which == 2) K = rows;
+  }
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int k_begin = blockIdx.z * k_per_split;
+  int k_end = k_begin + k_per_split;
+  if (k_end > K) k_end = K;
+  if (m0 >= M || k_begin >= k_end) return;
+  const int nkb = (k_end - k_begin + BK - 1) / BK;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kStages * kStage;  // full[kStages], empty[kStages], tmem_full
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kStages * kStage + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStages * kStage + 68);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  const uint32_t tmem_full_bar = bar_base + 8u * (2 * kStages);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
+    ptx::mbar_init(tmem_full_bar, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), BN);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int issued = 0;
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % kStages;
+        if (kb >= kStages && !ptx::mbar_wait(empty_bar(s), ((kb / kStages) - 1) & 1)) {
+          record_status(d_status, SPA_ERR_TIMEOUT);
+          *abort_flag = 1;
+          break;
+        }
+        if (*abort_flag) break;
+        const uint32_t a_dst = smem_base + s * kStage, b_dst = a_dst + kABytes;
+        const int k0 = k_begin + kb * BK;
+        ptx::mbar_expect_tx(full_bar(s), kStage);
+        if (!kAMn) {
+          ptx::tma_load_2d(a_dst, &tmA, full_bar(s), k0, m0);
+        } else {
+#pragma unroll
+          for (int j = 0; j < BM / 64; ++j) ptx::tma_load_2d(a_dst + j * (BK * 128), &tmA, full_bar(s), m0 + 64 * j, k0);
+        }
+        if (!kBMn) {
+          ptx::tma_load_2d(b_dst, &tmB, full_bar(s), k0, n0);
+        } else {
+#pragma unroll
+          for (int j = 0; j < BN / 64; ++j) ptx::tma_load_2d(b_dst + j * (BK * 128), &tmB, full_bar(s), n0 + 64 * j, k0);
+        }
+        issued = kb + 1;
+      }
+      if (*abort_flag) {  // let our own copies land before the CTA's shared memory goes away
+        for (int kb = issued > kStages ? issued - kStages : 0; kb < issued; ++kb)
+          ptx::mbar_wait(full_bar(kb % kStages), (kb / kStages) & 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    bool issued_any = false;
+    for (int kb = 0; kb < nkb; ++kb) {
+      const int s = kb % kStages;
+      if (*abort_flag) break;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(full_bar(s), (kb / kStages) & 1))) {
+        if (lane == 0) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+        break;
+      }
+      const uint32_t a_src = smem_base + s * kStage, b_src = a_src + kABytes;
+      const int k_valid = k_end - (k_begin + kb * BK);
+      if ((kAMn || kBMn) && k_valid < BK) {
+        // K rows beyond the end of the reduction: zero them (a K row is one 128-byte line per 64-wide box)
+        const int n_lines = BK - k_valid;
+        if (kAMn)
+          for (int j = 0; j < BM / 64; ++j)
+            for (int c = lane; c < n_lines * 8; c += 32)
+              *reinterpret_cast<uint4*>(smem_al + s * kStage + j * (BK * 128) + (k_valid + c / 8) * 128 + (c % 8) * 16) =
+                  make_uint4(0, 0, 0, 0);
+        if (kBMn)
+          for (int j = 0; j < BN / 64; ++j)
+            for (int c = lane; c < n_lines * 8; c += 32)
+              *reinterpret_cast<uint4*>(smem_al + s * kStage + kABytes + j * (BK * 128) + (k_valid + c / 8) * 128 +
+                                        (c % 8) * 16) = make_uint4(0, 0, 0, 0);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+      }
+      ptx::tc_fence_after_sync();
+      if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k) {
+          const uint64_t adesc = kAMn ? ptx::smem_desc_sw128(a_src + k * 2048, BK * 128, 1024)
+                                      : ptx::smem_desc_sw128(a_src + k * 32, 16, 1024);
+          const uint64_t bdesc = kBMn ? ptx::smem_desc_sw128(b_src + k * 2048, BK * 128, 1024)
+                                      : ptx::smem_desc_sw128(b_src + k * 32, 16, 1024);
+          ptx::mma_bf16(tmem_base, adesc, bdesc, kIdesc, (kb | k) != 0 ? 1u : 0u);
+        }
+        ptx::mma_commit(empty_bar(s));
+      }
+      issued_any = true;
+      __syncwarp();
+    }
+    if (lane == 0 && issued_any) ptx::mma_commit(tmem_full_bar);
+    if (*abort_flag && issued_any) ptx::mbar_wait(tmem_full_bar, 0);  // drain before TMEM is freed
+  } else {
+    // ------------------------------------------------------------------ epilogue: TMEM -> registers -> global
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    if (__all_sync(0xffffffffu, ptx::mbar_wait(tmem_full_bar, 0) && !*abort_flag)) {
+      ptx::tc_fence_after_sync();
+      const int row = m0 + q * 32 + lane;
+      OutT* orow = out + (long long)blockIdx.z * split_stride + (long long)row * ldo;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, r);
+        ptx::tmem_ld_wait();
+        if (row < M) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int col = n0 + c * 32 + g * 8;
+            if (col < N) {
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]);
+              if (bias != nullptr) {
+                float b[8];
+                Vec16<__nv_bfloat16>::to_float(__ldg(reinterpret_cast<const uint4*>(bias + col)), b);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[e] += b[e];
+              }
+              OutStore<OutT>::store8(orow + col, v);
+            }
+          }
+        }
+      }
+    } else if (lane == 0) {
+      record_status(d_status, SPA_ERR_TIMEOUT);
+    }
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, BN);
+  }
+}
+
+// ---- wgrad helpers --------------------------------------------------------------------------------
+// Partial column sums of dout over the rows of one K split: part[z][col].
+__global__ void __launch_bounds__(256)
+colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const int32_t* __restrict__ cu, int n_seg,
+                      int capacity, int k_per_split, float* __restrict__ part) {
+  const int rows = packed_rows(cu, n_seg, capacity);
+  const int r_begin = blockIdx.y * k_per_split;
+  int r_end = r_begin + k_per_split;
+  if (r_end > rows) r_end = rows;
+  __shared__ float red[32][65];
+  const int cg = threadIdx.x & 7, rl = threadIdx.x >> 3;  // 8 column groups of 8, 32 row lanes
+  const int col = blockIdx.x * 64 + cg * 8;
+  float acc[8] = {};
+  if (col < n_out)
+    for (int i = r_begin + rl; i < r_end; i += 32) {
+      float f[8];
+      Vec16<__nv_bfloat16>::to_float(ld_nc16(dout + (long long)i * n_out + col), f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+    }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) red[rl][cg * 8 + e] = acc[e];
+  __syncthreads();
+  if (threadIdx.x < 64) {
+    const int c = blockIdx.x * 64 + threadIdx.x;
+    if (c < n_out) {
+      float s = 0.f;
+#pragma unroll
+      for (int r = 0; r < 32; ++r) s += red[r][threadIdx.x];
+      part[(long long)blockIdx.y * n_out + c] = s;
+    }
+  }
+}
+
+// out[e] = sum over the splits that hold rows (in split order) of part[s][e]; zero if there are none.
+__global__ void __launch_bounds__(256)
+split_reduce_kernel(const float* __restrict__ part, long long n, long long split_stride, int k_per_split,
+                    const int32_t* __restrict__ cu, int n_seg, int capacity, float* __restrict__ out) {
+  const int rows = packed_rows(cu, n_seg, capacity);
+  const int valid = (rows + k_per_split - 1) / k_per_split;
+  const long long n4 = n >> 2;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int z = 0; z < valid; ++z) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(part + (long long)z * split_stride) + i);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    reinterpret_cast<float4*>(out)[i] = s;
+  }
+}
+
+struct SplitPlan { int splits, k_per_split; };
+
+// K = packed rows is cut into equal spans (multiples of BK) so that tiles x splits fills the GPU.
+SplitPlan plan_splits(int capacity, int n_in, int n_out) {
+  const int tiles = ((n_out + BM - 1) / BM) * ((n_in + 127) / 128);
+  int splits = (2 * kNumSMs + tiles - 1) / tiles;
+  const int max_by_rows = (capacity + BK - 1) / BK;
+  if (splits > max_by_rows) splits = max_by_rows;
+  if (splits > 32) splits = 32;
+  if (splits < 1) splits = 1;
+  int kps = (capacity + splits - 1) / splits;
+  kps = ((kps + BK - 1) / BK) * BK;
+  splits = (capacity + kps - 1) / kps;
+  return {splits, kps};
+}
+
+size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
+  const SplitPlan sp = plan_splits(capacity, n_in, n_out);
+  size_t w = (size_t)sp.splits * n_out * n_in * sizeof(float);
+  w = (w + 255) & ~(size_t)255;
+  return w + (size_t)sp.splits * n_out * sizeof(float) + 256;
+}
+
+template <int BN, bool kAMn, bool kBMn, typename OutT>
+int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloat16* bias, OutT* out, long long ldo,
+                long long split_stride, int M, int N, int K, const int32_t* cu, int n_seg, int capacity, int dyn_which,
+                int k_per_split, int splits, int32_t* d_status, cudaStream_t st, const char* what) {
+  auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT>;
+  static bool attr_set = false;  // per instantiation
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes<BN>());
+    if (e != cudaSuccess) { set_cuda_error(e, what); return SPA_ERR_CUDA; }
+    attr_set = true;
+  }
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, splits);
+  kern<<<grid, kGemmThreads, gemm_smem_bytes<BN>(), st>>>(tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu, n_seg,
+                                                         capacity, dyn_which, k_per_split, d_status);
+  SPA_CUDA_CHECK_LAUNCH(what);
+  return SPA_OK;
+}
+
+}  // namespace
+
+bool tc_linear_supported(int n_in, int n_out) {
+  return n_in % 8 == 0 && n_out % 8 == 0 && n_in >= 64 && n_out >= 64 && encode_fn() != nullptr;
+}
+
+size_t tc_linear_workspace_bytes(const spa_params& p) {
+  if (p.dtype != SPA_BF16 || !tc_linear_supported(p.C, 3 * p.C)) return 0;
+  const size_t a = wgrad_workspace_bytes(p.capacity, p.C, 3 * p.C);
+  const size_t b = wgrad_workspace_bytes(p.capacity, p.C, p.C);
+  return a > b ? a : b;
+}
+
+int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
+                         const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st) {
+  CUtensorMap tmA, tmB;
+  if (!make_tmap_bf16_2d(&tmA, a, n_in, p.capacity, (uint64_t)n_in * 2, BK, BM) ||
+      !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, BK, 128))
+    return SPA_ERR_UNSUPPORTED;
+  return launch_gemm<128, false, false, __nv_bfloat16>(tmA, tmB, (const __nv_bfloat16*)bias, (__nv_bfloat16*)out, n_out,
+                                                       0, p.capacity, n_out, n_in, cu, p.B, p.capacity, 1, n_in, 1,
+                                                       d_status, st, "gemm_tc_kernel(fwd)");
+}
+
+int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
+                         const int32_t* cu, void* da, float* dW, float* db, void* workspace, int32_t* d_status,
+                         cudaStream_t st) {
+  CUtensorMap tmA, tmB, tmA2, tmB2;
+  if (da != nullptr && (!make_tmap_bf16_2d(&tmA, dout, n_out, p.capacity, (uint64_t)n_out * 2, BK, BM) ||
+                        !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, 64, BK)))
+    return SPA_ERR_UNSUPPORTED;
+  if (dW != nullptr && (!make_tmap_bf16_2d(&tmA2, dout, n_out, p.capacity, (uint64_t)n_out * 2, 64, BK) ||
+                        !make_tmap_bf16_2d(&tmB2, a, n_in, p.capacity, (uint64_t)n_in * 2, 64, BK)))
+    return SPA_ERR_UNSUPPORTED;
+  if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
+    int rc = launch_gemm<128, false, true, __nv_bfloat16>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0, p.capacity,
+                                                          n_in, n_out, cu, p.B, p.capacity, 1, n_out, 1, d_status, st,
+                                                          "gemm_tc_kernel(dgrad)");
+    if (rc != SPA_OK) return rc;
+  }
+  if (dW == nullptr && db == nullptr) return SPA_OK;
+  const SplitPlan sp = plan_splits(p.capacity, n_in, n_out);
+  float* part_w = reinterpret_cast<float*>(workspace);
+  size_t off = ((size_t)sp.splits * n_out * n_in * sizeof(float) + 255) & ~(size_t)255;
+  float* part_b = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + off);
+  if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]
+    int rc = launch_gemm<128, true, true, float>(tmA2, tmB2, nullptr, part_w, n_in, (long long)n_out * n_in, n_out, n_in,
+                                                 p.capacity, cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits,
+                                                 d_status, st, "gemm_tc_kernel(wgrad)");
+    if (rc != SPA_OK) return rc;
+    const long long n = (long long)n_out * n_in;
+    int grid = (int)((n / 4 + 255) / 256);
+    if (grid > kNumSMs * 8) grid = kNumSMs * 8;
+    split_reduce_kernel<<<grid, 256, 0, st>>>(part_w, n, n, sp.k_per_split, cu, p.B, p.capacity, dW);
+    SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(dW)");
+  }
+  if (db != nullptr) {
+    dim3 grid((n_out + 63) / 64, sp.splits);
+    colsum_partial_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity, sp.k_per_split,
+                                                part_b);
+    SPA_CUDA_CHECK_LAUNCH("colsum_partial_kernel");
+    split_reduce_kernel<<<(n_out / 4 + 255) / 256, 256, 0, st>>>(part_b, n_out, n_out, sp.k_per_split, cu, p.B,
+                                                                 p.capacity, db);
+    SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
+  }
+  return SPA_OK;
+}
+
+}  // namespace spa

@@ -5,7 +5,8 @@
 
 namespace spa {
 
-size_t tc_workspace_bytes(const spa_params& p);
+size_t tc_linear_workspace_bytes(const spa_params& p);
+size_t tc_attention_workspace_bytes(const spa_params& p);
 
 bool tc_linear_supported(int n_in, int n_out);
 int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,

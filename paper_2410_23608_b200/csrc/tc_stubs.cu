@@ -4,12 +4,7 @@
 
 namespace spa {
 
-size_t tc_workspace_bytes(const spa_params&) { return 0; }
-bool tc_linear_supported(int, int) { return false; }
-int launch_linear_fwd_tc(const spa_params&, const void*, const void*, const void*, int, int, const int32_t*, void*,
-                         int32_t*, cudaStream_t) { return SPA_ERR_UNSUPPORTED; }
-int launch_linear_bwd_tc(const spa_params&, const void*, const void*, const void*, int, int, const int32_t*, void*,
-                         float*, float*, void*, int32_t*, cudaStream_t) { return SPA_ERR_UNSUPPORTED; }
+size_t tc_attention_workspace_bytes(const spa_params&) { return 0; }
 bool tc_attention_fwd_supported(const spa_params&) { return false; }
 int launch_attention_fwd_tc(const spa_params&, const void*, const int32_t*, int, void*, float*, int32_t*,
                             cudaStream_t) { return SPA_ERR_UNSUPPORTED; }
