@@ -56,9 +56,11 @@ def work_model(cfg, cu):
     w["proj"] = dict(bytes=(2 * Np * C + C * C) * es, flops=2 * Np * C * C)
     w["unpack"] = dict(bytes=2 * BN * C * es + 4 * BN, flops=0)
     w["unpack_bwd"] = dict(bytes=2 * BN * C * es + 4 * BN, flops=0)
-    w["proj_bwd"] = dict(bytes=(3 * Np * C + C * C) * es + 4 * C * C, flops=4 * Np * C * C)
     w["attn_bwd"] = dict(bytes=(3 + 1 + 1 + 3) * Np * C * es + 4 * H * Np, flops=10 * C * S2)
-    w["qkv_bwd"] = dict(bytes=(Np * C + 3 * Np * C + Np * C + 3 * C * C) * es + 12 * C * C, flops=12 * Np * C * C)
+    for name, n_out in (("proj_bwd", C), ("qkv_bwd", 3 * C)):
+        w[name + ".da"] = dict(bytes=(Np * n_out + n_out * C + Np * C) * es, flops=2 * Np * C * n_out)
+        w[name + ".dW"] = dict(bytes=(Np * n_out + Np * C) * es + 4 * n_out * C, flops=2 * Np * C * n_out)
+        w[name + ".db"] = dict(bytes=Np * n_out * es + 4 * n_out, flops=Np * n_out)
     w["pack_bwd"] = dict(bytes=2 * Np * C * es + 4 * Np, flops=0)
     return w, Np, S2
 
@@ -85,6 +87,26 @@ def call_sequence(L, blk, d, b_g):
     ]
 
 
+def timing_units(L, blk, d, b_g):
+    """The calls again, with the linear-layer gradients split into their three products, so that
+    each timed unit is one kernel (dW: the split-K GEMM plus its fixed-order reduction)."""
+    p, C = blk.p, blk.C
+    units = [(n, f) for n, f in call_sequence(L, blk, d, b_g) if n not in ("proj_bwd", "qkv_bwd")]
+
+    def lin(a, W, dout, n_out, da, dW, db):
+        return lambda: L.spa_packed_linear_bwd(p, a, W, dout, C, n_out, blk.cu, da, dW, db, blk.workspace, blk.status)
+
+    units += [
+        ("proj_bwd.da", lin(blk.ao, d["W_o"], blk.dz, C, blk.dao, None, None)),
+        ("proj_bwd.dW", lin(blk.ao, d["W_o"], blk.dz, C, None, blk.dW_o, None)),
+        ("proj_bwd.db", lin(blk.ao, d["W_o"], blk.dz, C, None, None, blk.db_o)),
+        ("qkv_bwd.da", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, blk.dxp, None, None)),
+        ("qkv_bwd.dW", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, blk.dW_qkv, None)),
+        ("qkv_bwd.db", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, None, blk.db_qkv)),
+    ]
+    return units
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -94,7 +116,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -189,15 +211,15 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--config", type=int, default=2, help="workload 1..5 (default 2, ViT-S/16-like bf16)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.steps == 200 and args.warmup == 20:
+        if args.steps == 2000 and args.warmup == 50:
             args.steps, args.warmup = 5, 1
         return run_reference(args)
 
@@ -225,8 +247,10 @@ def main():
 
     cfg = get_config(args.config)
     # rotating buffer sets: inputs, outputs and every intermediate differ from step to step
-    per_set = (4 * cfg.B * cfg.N * cfg.C + 12 * cfg.B * cfg.N * cfg.C) * cfg.elem_size
-    n_sets = args.sets if args.sets > 0 else max(2, int(np.ceil(2.5 * L2_BYTES / per_set)))
+    # enough sets that even the smallest single tensor a call streams (x) exceeds L2 over one rotation
+    x_bytes = cfg.B * cfg.N * cfg.C * cfg.elem_size
+    per_set = 16 * x_bytes
+    n_sets = args.sets if args.sets > 0 else min(24, max(3, int(np.ceil(1.3 * L2_BYTES / x_bytes))))
     names = ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")
     sets, inps = [], []
     for s in range(n_sets):
@@ -236,11 +260,26 @@ def main():
         blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau)
         sets.append((inp, d, blk, call_sequence(L, blk, d, inp.b_g)))
 
-    def step(i):
-        for _, fn in sets[i % n_sets][3]:
-            fn()
+    def capture(fns):
+        """One CUDA graph holding the given library calls in order; returns (graph, kernels launched)."""
+        g = torch.cuda.CUDAGraph()
+        n_before = L.spa_launch_count()
+        with torch.cuda.graph(g):
+            for fn in fns:
+                fn()
+        return g, L.spa_launch_count() - n_before
 
     stream = torch.cuda.current_stream()
+    for s_ in range(n_sets):           # eager pass: first-use set-up (attributes, tensor maps) outside capture
+        for _, fn in sets[s_][3]:
+            fn()
+    torch.cuda.synchronize()
+    step_graphs = [capture([fn for _, fn in sets[s_][3]]) for s_ in range(n_sets)]
+    launches_per_step = step_graphs[0][1]
+
+    def step(i):
+        step_graphs[i % n_sets][0].replay()
+
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
@@ -257,13 +296,12 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    n0 = L.spa_launch_count()
     e0.record(stream)
     for i in range(args.steps):
         step(i)
     e1.record(stream)
     barrier()
-    launches = L.spa_launch_count() - n0
+    launches = launches_per_step * args.steps
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else None
     t = torch.tensor([ms], dtype=torch.float64, device="cuda")
@@ -283,8 +321,7 @@ def main():
         inp, d, blk, seq = sets[i % n_sets]
         d["x"].copy_(hx[i % 2], non_blocking=True)
         d["dY"].copy_(hdy[i % 2], non_blocking=True)
-        for _, fn in seq:
-            fn()
+        step(i)
         hy.copy_(blk.y, non_blocking=True)
         hdx.copy_(blk.dX, non_blocking=True)
 
@@ -307,21 +344,23 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- per-call device times (CUDA events between calls, same rotation), for the roofline
-    n_calls = len(sets[0][3])
-    reps = min(args.steps, 100)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_calls + 1)] for _ in range(reps)]
-    torch.cuda.synchronize()
-    for r in range(reps):
-        seq = sets[r % n_sets][3]
-        evs[r][0].record(stream)
-        for c, (_, fn) in enumerate(seq):
-            fn()
-            evs[r][c + 1].record(stream)
-    torch.cuda.synchronize()
-    call_ms = {}
-    for c, (name, _) in enumerate(sets[0][3]):
-        call_ms[name] = float(np.mean([evs[r][c].elapsed_time(evs[r][c + 1]) for r in range(reps)]))
+    # ---- per-kernel device times: each unit captured alone, once per buffer set, and replayed
+    reps = max(3, min(50, args.steps))
+    unit_names = [n for n, _ in timing_units(L, sets[0][2], sets[0][1], sets[0][0].b_g)]
+    per_set_units = [dict(timing_units(L, blk, d, inp.b_g)) for inp, d, blk, _ in sets]
+    call_ms, unit_launches = {}, {}
+    for name in unit_names:
+        g, n_l = capture([u[name] for u in per_set_units])
+        for _ in range(2):
+            g.replay()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        call_ms[name] = e0.elapsed_time(e1) / (reps * n_sets)
+        unit_launches[name] = n_l // n_sets
     pk = peaks()
     work, Np0, S2 = work_model(cfg, sets[0][2].cu.cpu().numpy())
     per_call = {}
@@ -332,7 +371,7 @@ def main():
         bound = "tensor" if (t_f > t_b and cfg.dtype == "bf16") else "hbm"
         ach = wk["flops"] / (ms_c * 1e-3) / 1e12 if bound == "tensor" else wk["bytes"] / (ms_c * 1e-3) / 1e9
         per_call[name] = dict(us=round(ms_c * 1e3, 2), bound=bound, achieved=round(ach, 2),
-                              frac=round(ach / pk[bound], 4))
+                              frac=round(ach / pk[bound], 4), kernels=unit_launches[name])
     top = max(call_ms, key=call_ms.get)
     tr = per_call[top]
     roofline = {"kernel": top, "bound": tr["bound"], "achieved": tr["achieved"], "peak": pk[tr["bound"]],
@@ -340,13 +379,16 @@ def main():
                 "peak_source": pk["source"], "us_per_launch": tr["us"]}
 
     # ---- forward-only time (same rotation), reported beside the headline
+    fwd_graphs = [capture([fn for _, fn in sets[s_][3][:6]])[0] for s_ in range(n_sets)]
+    for i in range(n_sets):
+        fwd_graphs[i].replay()
+    torch.cuda.synchronize()
     e0.record(stream)
-    for i in range(reps):
-        for _, fn in sets[i % n_sets][3][:6]:
-            fn()
+    for i in range(reps * n_sets):
+        fwd_graphs[i % n_sets].replay()
     e1.record(stream)
     torch.cuda.synchronize()
-    fwd_ms = e0.elapsed_time(e1) / reps
+    fwd_ms = e0.elapsed_time(e1) / (reps * n_sets)
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -362,7 +404,8 @@ def main():
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "C": cfg.C, "H": cfg.H,
                    "selected_tokens": Np_sets[0], "sum_nb_squared": S2, "pass": "forward+backward",
-                   "l2_policy": f"{n_sets} rotating buffer sets, {per_set * n_sets / 1e6:.0f} MB > L2",
+                   "l2_policy": f"{n_sets} rotating buffer sets (x alone {x_bytes * n_sets / 1e6:.0f} MB > L2)",
+                   "launch": "one CUDA graph per step",
                    "replicas": world},
         "e2e": {"value": world * tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 2 * bytes_io, "d2h_bytes_per_step": 2 * bytes_io},
