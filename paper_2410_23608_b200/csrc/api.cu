@@ -114,8 +114,10 @@ int spa_packed_attention_fwd(const spa_params* p, const void* qkv, const int32_t
   if (rc != SPA_OK) return rc;
   SPA_PTR(qkv); SPA_PTR(seg_offsets); SPA_PTR(attn_out); SPA_PTR(lse);
   SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
-  if (use_tc(p) && tc_attention_fwd_supported(*p))
-    return launch_attention_fwd_tc(*p, qkv, seg_offsets, n_seg, attn_out, lse, d_status, (cudaStream_t)stream);
+  if (use_tc(p) && tc_attention_fwd_supported(*p)) {
+    rc = launch_attention_fwd_tc(*p, qkv, seg_offsets, n_seg, attn_out, lse, d_status, (cudaStream_t)stream);
+    if (rc != SPA_ERR_UNSUPPORTED) return rc;
+  }
   return launch_attention_fwd_simt(*p, qkv, seg_offsets, n_seg, attn_out, lse, (cudaStream_t)stream);
 }
 
@@ -129,9 +131,11 @@ int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* a
   SPA_PTR(qkv); SPA_PTR(attn_out); SPA_PTR(lse); SPA_PTR(d_attn_out); SPA_PTR(seg_offsets); SPA_PTR(dqkv);
   SPA_OPT_PTR(workspace);
   SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
-  if (use_tc(p) && tc_attention_bwd_supported(*p) && workspace != nullptr)
-    return launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace, d_status,
-                                   (cudaStream_t)stream);
+  if (use_tc(p) && tc_attention_bwd_supported(*p) && workspace != nullptr) {
+    rc = launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace, d_status,
+                                 (cudaStream_t)stream);
+    if (rc != SPA_ERR_UNSUPPORTED) return rc;
+  }
   return launch_attention_bwd_simt(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv,
                                    (cudaStream_t)stream);
 }

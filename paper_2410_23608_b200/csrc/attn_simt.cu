@@ -18,20 +18,6 @@ namespace {
 constexpr int kRows = 64;   // packed rows per CTA and rows per staged tile
 constexpr int kPart = 32;   // head dimensions held by one thread
 
-struct RowSeg { int lo, hi; };
-
-// Segment bounds of packed row i (hi clamped to the valid rows); rows >= Np get an empty range.
-__device__ __forceinline__ RowSeg row_segment(const int32_t* __restrict__ seg, int n_seg, int Np, int i) {
-  RowSeg r{0, 0};
-  if (i < Np) {
-    const int s = find_segment(seg, n_seg, i);
-    r.lo = __ldg(seg + s);
-    const int hi = __ldg(seg + s + 1);
-    r.hi = hi < Np ? hi : Np;
-  }
-  return r;
-}
-
 // Stage rows [row0, row0 + kRows) of one head's slice (column offset col0 of a [*, ld] matrix) as fp32.
 template <typename T, int D>
 __device__ __forceinline__ void stage_rows(float (*dst)[D], const T* __restrict__ src, long long ld, int col0, int row0,

@@ -1,0 +1,266 @@
+// Segment-masked attention forward on the packed tokens with tcgen05 tensor cores (Sec. 3.2: packed
+// tokens attend only to tokens of the same image; the 2L^2C term of Eq. 9).
+//
+// A CTA owns 128 consecutive packed query rows of one head, wherever image boundaries fall, and
+// walks the key range spanned by the segments of those rows in tiles of 128 keys; cu_seqlens alone
+// decides the range, so no padding token is ever loaded or multiplied.  Per key tile:
+//   S = Q K^T        tcgen05.mma, Q and K tiles staged by TMA (K/V double-buffered), S in TMEM (fp32)
+//   P = exp2(S - m)  one thread per query row reads its S row from TMEM, masks keys outside the
+//                    row's own segment, updates the running max / sum, writes P back to TMEM as bf16
+//   O_t = P V        tcgen05.mma with P read from TMEM and V from shared memory
+//   O = alpha O + O_t in registers (fp32), so TMEM never needs a rescaling pass.
+// K/V rows past the last valid packed row are unspecified memory: K columns are masked after the
+// product and V lines are zeroed in shared memory before the product.
+#include <math_constants.h>
+
+#include "sm100_ptx.cuh"
+#include "spa_tc.cuh"
+
+namespace spa {
+namespace {
+
+constexpr int kQ = 128;        // query rows per CTA = TMEM lanes
+constexpr int kKV = 128;       // keys per tile
+constexpr int kFwdThreads = 128;
+constexpr uint32_t kTmemCols = 256;  // S: 128 fp32 columns, P: 64 (bf16 pairs), O tile: up to 64
+constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
+
+template <int D> struct HeadTile {
+  static constexpr int kRowBytes = D * 2;          // 128 (d = 64) or 64 (d = 32): also the swizzle span
+  static constexpr int kTileBytes = 128 * kRowBytes;
+  static constexpr int kSbo = 8 * kRowBytes;
+  // K-major operand (Q or K rows, head dimension contiguous), k-th group of 16 head dimensions
+  __device__ static __forceinline__ uint64_t kmajor(uint32_t addr, int k) {
+    return D == 64 ? ptx::smem_desc_sw128(addr + k * 32, 16, kSbo) : ptx::smem_desc_sw64(addr + k * 32, 16, kSbo);
+  }
+  // MN-major operand (V: key rows are the K dimension, head dimension contiguous), k-th group of 16 keys
+  __device__ static __forceinline__ uint64_t mnmajor(uint32_t addr, int k) {
+    return D == 64 ? ptx::smem_desc_sw128(addr + k * 16 * kRowBytes, 16, kSbo)
+                   : ptx::smem_desc_sw64(addr + k * 16 * kRowBytes, 16, kSbo);
+  }
+};
+
+template <int D> __host__ __device__ constexpr int fwd_smem_bytes() {
+  return 5 * 128 * D * 2 + 1024 + 128;  // Q + 2 x (K, V), alignment slack, barriers
+}
+
+template <int D>
+__global__ void __launch_bounds__(kFwdThreads)
+attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __restrict__ seg, int n_seg, int capacity,
+                   int C, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
+                   int32_t* d_status) {
+  using HT = HeadTile<D>;
+  constexpr int kTile = HT::kTileBytes;
+  const int Np = packed_rows(seg, n_seg, capacity);
+  const int q0 = blockIdx.x * kQ;
+  if (q0 >= Np) return;
+  const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  const uint32_t q_s = smem_base;
+  auto k_s = [&](int st) { return smem_base + kTile * (1 + 2 * st); };
+  auto v_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
+  const uint32_t bar_base = smem_base + 5 * kTile;
+  const uint32_t bar_q = bar_base, bar_s = bar_base + 24, bar_o = bar_base + 32;
+  auto bar_kv = [&](int st) { return bar_base + 8 + 8 * st; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 5 * kTile + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 68);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 72);
+
+  const int row = q0 + tid;
+  const RowSeg mine = row_segment(seg, n_seg, Np, row);
+  {
+    const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
+    if (row == q0) range[0] = mine.lo;
+    if (row == last) range[1] = mine.hi;
+  }
+  if (tid == 0) {
+    ptx::prefetch_tensormap(&tm);
+    ptx::mbar_init(bar_q, 1);
+    ptx::mbar_init(bar_kv(0), 1);
+    ptx::mbar_init(bar_kv(1), 1);
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_o, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;  // TMEM lanes this warp may touch
+  const int kv_lo = range[0], kv_hi = range[1];
+  const int n_tiles = (kv_hi - kv_lo + kKV - 1) / kKV;
+
+  constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(kQ, kKV, false, false);
+  constexpr uint32_t kIdescO = ptx::idesc_bf16_f32(kQ, D, false, true);
+
+  if (tid == 0) {
+    ptx::mbar_expect_tx(bar_q, kTile);
+    ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
+    ptx::mbar_expect_tx(bar_kv(0), 2 * kTile);
+    ptx::tma_load_2d(k_s(0), &tm, bar_kv(0), C + h * D, kv_lo);
+    ptx::tma_load_2d(v_s(0), &tm, bar_kv(0), 2 * C + h * D, kv_lo);
+  }
+
+  float o[D];
+#pragma unroll
+  for (int e = 0; e < D; ++e) o[e] = 0.f;
+  float m = -CUDART_INF_F, l = 0.f;
+  int issued_kv = 1;  // tiles whose loads thread 0 has issued
+
+  for (int t = 0; t < n_tiles; ++t) {
+    const int st = t & 1;
+    const int kv0 = kv_lo + t * kKV;
+    if (tid == 0) {
+      if (t + 1 < n_tiles) {  // the other stage is free: its P V product finished last iteration
+        ptx::mbar_expect_tx(bar_kv(st ^ 1), 2 * kTile);
+        ptx::tma_load_2d(k_s(st ^ 1), &tm, bar_kv(st ^ 1), C + h * D, kv0 + kKV);
+        ptx::tma_load_2d(v_s(st ^ 1), &tm, bar_kv(st ^ 1), 2 * C + h * D, kv0 + kKV);
+        issued_kv = t + 2;
+      }
+      bool ok = (t > 0) || ptx::mbar_wait(bar_q, 0);
+      ok = ok && ptx::mbar_wait(bar_kv(st), (t >> 1) & 1);
+      if (ok) {
+        ptx::tc_fence_after_sync();
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(k_s(st), k), kIdescS, k != 0 ? 1u : 0u);
+        ptx::mma_commit(bar_s);
+      } else {
+        record_status(d_status, SPA_ERR_TIMEOUT);
+        *abort_flag = 1;
+      }
+    }
+    // ---- softmax on this row of S
+    if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    ptx::tc_fence_after_sync();
+    const unsigned span = (unsigned)(mine.hi - mine.lo);
+    float mt = -CUDART_INF_F;
+#pragma unroll 1
+    for (int c = 0; c < kKV / 32; ++c) {
+      uint32_t r[32];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS + c * 32, r);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const bool valid = (unsigned)(kv0 + c * 32 + j - mine.lo) < span;
+        mt = fmaxf(mt, valid ? __uint_as_float(r[j]) * scale_log2e : -CUDART_INF_F);
+      }
+    }
+    const float m_new = fmaxf(m, mt);
+    const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
+    const float alpha = ptx::ex2_approx(m - m_use);
+    float rs = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < kKV / 32; ++c) {
+      uint32_t r[32], pk[16];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS + c * 32, r);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; j += 2) {
+        const bool v0 = (unsigned)(kv0 + c * 32 + j - mine.lo) < span;
+        const bool v1 = (unsigned)(kv0 + c * 32 + j + 1 - mine.lo) < span;
+        const float p0 = v0 ? ptx::ex2_approx(__uint_as_float(r[j]) * scale_log2e - m_use) : 0.f;
+        const float p1 = v1 ? ptx::ex2_approx(__uint_as_float(r[j + 1]) * scale_log2e - m_use) : 0.f;
+        rs += p0 + p1;
+        __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
+        pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
+      }
+      ptx::tmem_st_32x16(tmem + lane_base + kColP + c * 16, pk);
+    }
+    ptx::tmem_st_wait();
+    l = l * alpha + rs;
+    m = m_new;
+    // ---- V lines past the last valid packed row must not reach the product
+    if (kv0 + kKV > Np) {
+      ptx::mbar_wait(bar_kv(st), (t >> 1) & 1);  // already complete: K of this stage was consumed
+      const int first = Np - kv0;                // >= 1
+      constexpr int kChunks = HT::kRowBytes / 16;
+      for (int c = tid; c < (kKV - first) * kChunks; c += kFwdThreads)
+        *reinterpret_cast<uint4*>(smem_al + kTile * (2 + 2 * st) + (first + c / kChunks) * HT::kRowBytes +
+                                  (c % kChunks) * 16) = make_uint4(0, 0, 0, 0);
+      ptx::fence_proxy_async_smem();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) break;
+    if (tid == 0) {
+      ptx::tc_fence_after_sync();
+#pragma unroll
+      for (int k = 0; k < kKV / 16; ++k)
+        ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(v_s(st), k), kIdescO, k != 0 ? 1u : 0u);
+      ptx::mma_commit(bar_o);
+    }
+    if (!ptx::mbar_wait(bar_o, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    ptx::tc_fence_after_sync();
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t r[32];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColO + c * 32, r);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[c * 32 + j] = fmaf(o[c * 32 + j], alpha, __uint_as_float(r[j]));
+    }
+  }
+
+  if (!*abort_flag && row < Np) {
+    const float inv_l = 1.f / l;
+    __nv_bfloat16* dst = ao + (long long)row * C + h * D;
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) {
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = o[c * 8 + e] * inv_l;
+      *reinterpret_cast<uint4*>(dst + c * 8) = Vec16<__nv_bfloat16>::from_float(v);
+    }
+    lse[(long long)h * capacity + row] = (m + log2f(l)) * 0.6931471805599453f;
+  }
+  if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
+    for (int t = issued_kv > 2 ? issued_kv - 2 : 0; t < issued_kv; ++t) ptx::mbar_wait(bar_kv(t & 1), (t >> 1) & 1);
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+template <int D>
+int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
+               int32_t* d_status, cudaStream_t st) {
+  CUtensorMap tm;
+  if (!make_tmap_bf16_2d(&tm, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2)) return SPA_ERR_UNSUPPORTED;
+  auto kern = attn_fwd_tc_kernel<D>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem_bytes<D>());
+    if (e != cudaSuccess) { set_cuda_error(e, "attn_fwd_tc_kernel"); return SPA_ERR_CUDA; }
+    attr_set = true;
+  }
+  dim3 grid((p.capacity + kQ - 1) / kQ, p.H);
+  kern<<<grid, kFwdThreads, fwd_smem_bytes<D>(), st>>>(tm, seg, n_seg, p.capacity, p.C,
+                                                      softmax_scale_of(p) * 1.4426950408889634f,
+                                                      (__nv_bfloat16*)ao, lse, d_status);
+  SPA_CUDA_CHECK_LAUNCH("attn_fwd_tc_kernel");
+  return SPA_OK;
+}
+
+}  // namespace
+
+bool tc_attention_fwd_supported(const spa_params& p) {
+  const int d = p.C / p.H;
+  return p.dtype == SPA_BF16 && (d == 32 || d == 64) && tensor_maps_available();
+}
+
+int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
+                            int32_t* d_status, cudaStream_t st) {
+  return p.C / p.H == 64 ? fwd_launch<64>(p, qkv, seg, n_seg, ao, lse, d_status, st)
+                         : fwd_launch<32>(p, qkv, seg, n_seg, ao, lse, d_status, st);
+}
+
+}  // namespace spa

@@ -43,9 +43,12 @@ std::mutex g_tm_mutex;
 std::unordered_map<std::string, CUtensorMap> g_tm_cache;
 }  // namespace
 
+bool tensor_maps_available() { return encode_fn() != nullptr; }
+
 bool make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t rows, uint64_t row_stride_bytes,
-                       uint32_t box_inner, uint32_t box_rows) {
-  struct Key { const void* b; uint64_t i, r, s; uint32_t bi, br; } key{base, inner, rows, row_stride_bytes, box_inner, box_rows};
+                       uint32_t box_inner, uint32_t box_rows, int swizzle_bytes) {
+  struct Key { const void* b; uint64_t i, r, s; uint32_t bi, br; int sw; int pad; } key{base, inner, rows, row_stride_bytes,
+                                                                                     box_inner, box_rows, swizzle_bytes, 0};
   std::string k(reinterpret_cast<const char*>(&key), sizeof(key));
   std::lock_guard<std::mutex> lock(g_tm_mutex);
   auto it = g_tm_cache.find(k);
@@ -57,7 +60,9 @@ bool make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint6
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (g_tm_cache.size() > 4096) g_tm_cache.clear();

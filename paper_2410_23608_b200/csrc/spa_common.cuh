@@ -85,6 +85,20 @@ __device__ __forceinline__ int find_segment(const int32_t* __restrict__ offsets,
   return lo;
 }
 
+struct RowSeg { int lo, hi; };
+
+// Segment bounds of packed row i (hi clamped to the valid rows); rows >= Np get an empty range.
+__device__ __forceinline__ RowSeg row_segment(const int32_t* __restrict__ seg, int n_seg, int Np, int i) {
+  RowSeg r{0, 0};
+  if (i < Np) {
+    const int s = find_segment(seg, n_seg, i);
+    r.lo = __ldg(seg + s);
+    const int hi = __ldg(seg + s + 1);
+    r.hi = hi < Np ? hi : Np;
+  }
+  return r;
+}
+
 // ---- host side -------------------------------------------------------------------------------
 void set_cuda_error(cudaError_t e, const char* where);
 void count_launch();  // one more kernel of this library was enqueued (host-side tally)

@@ -5,9 +5,6 @@
 namespace spa {
 
 size_t tc_attention_workspace_bytes(const spa_params&) { return 0; }
-bool tc_attention_fwd_supported(const spa_params&) { return false; }
-int launch_attention_fwd_tc(const spa_params&, const void*, const int32_t*, int, void*, float*, int32_t*,
-                            cudaStream_t) { return SPA_ERR_UNSUPPORTED; }
 bool tc_attention_bwd_supported(const spa_params&) { return false; }
 int launch_attention_bwd_tc(const spa_params&, const void*, const void*, const float*, const void*, const int32_t*,
                             int, void*, void*, int32_t*, cudaStream_t) { return SPA_ERR_UNSUPPORTED; }
