@@ -1,4 +1,4 @@
-// Segment-masked attention forward on the packed tokens with tcgen05 tensor cores (Sec. 3.2: packed
+// Segment-masked attention, forward and backward, on the packed tokens with tcgen05 tensor cores (Sec. 3.2: packed
 // tokens attend only to tokens of the same image; the 2L^2C term of Eq. 9).
 //
 // A CTA owns 128 consecutive packed query rows of one head, wherever image boundaries fall, and
@@ -230,6 +230,292 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Backward.  Two passes over the same tile machinery, each accumulating its outputs in TMEM over the
+// whole loop, so that no sum is split across CTAs (no float atomics, bitwise reproducible):
+//   kDQ = true : a CTA owns 128 query rows i; per key tile   S = Q K^T, dP = dO V^T,
+//                dS = P (dP - D_i) written to TMEM as bf16,  dQ += dS K.  Also stores D_i = dO_i . O_i.
+//   kDQ = false: a CTA owns 128 key rows j; per query tile   S^T = K Q^T, dP^T = V dO^T,
+//                P^T and dS^T written to TMEM as bf16,       dV += P^T dO,  dK += dS^T Q.
+// "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through two stages.  The
+// bf16 operand written back to TMEM aliases the first half of the fp32 tile it was computed from
+// (column group c of the result only covers columns already consumed).
+constexpr int kBwdThreads = 128;
+constexpr uint32_t kBwdTmemCols = 512;
+constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320;
+
+template <int D> __host__ __device__ constexpr int bwd_smem_bytes() {
+  return 6 * 128 * D * 2 + 1024 + 1024 + 128;  // 6 tiles, alignment slack, row statistics, barriers
+}
+
+template <int D, bool kDQ>
+__global__ void __launch_bounds__(kBwdThreads)
+attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
+                   const __nv_bfloat16* __restrict__ ao, const __nv_bfloat16* __restrict__ dao,
+                   const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
+                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
+  using HT = HeadTile<D>;
+  constexpr int kTile = HT::kTileBytes;
+  constexpr float kLog2e = 1.4426950408889634f;
+  const int Np = packed_rows(seg, n_seg, capacity);
+  const int r0 = blockIdx.x * 128;
+  if (r0 >= Np) return;
+  const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
+  const float scale_log2e = scale * kLog2e;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
+  auto y1_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
+  auto y2_s = [&](int st) { return smem_base + kTile * (3 + 2 * st); };
+  float* stat_lse = reinterpret_cast<float*>(smem_al + 6 * kTile);        // [128] lse_i * log2e of the staged query tile
+  float* stat_D = stat_lse + 128;                                         // [128] D_i
+  const uint32_t bar_base = smem_base + 6 * kTile + 1024;
+  const uint32_t bar_x = bar_base, bar_s = bar_base + 24, bar_o = bar_base + 32;
+  auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 6 * kTile + 1024 + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 6 * kTile + 1024 + 68);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 6 * kTile + 1024 + 72);
+
+  const int row = r0 + tid;
+  const RowSeg mine = row_segment(seg, n_seg, Np, row);
+  {
+    const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
+    if (row == r0) range[0] = mine.lo;
+    if (row == last) range[1] = mine.hi;
+  }
+  if (tid == 0) {
+    ptx::prefetch_tensormap(&tm_qkv);
+    ptx::prefetch_tensormap(&tm_do);
+    ptx::mbar_init(bar_x, 1);
+    ptx::mbar_init(bar_y(0), 1);
+    ptx::mbar_init(bar_y(1), 1);
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_o, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
+  const int n_tiles = (o_hi - o_lo + 127) / 128;
+
+  // column offsets inside qkv of the own / other operands
+  const int x1_col = (kDQ ? 0 : C) + h * D;           // Q | K
+  const int y1_col = (kDQ ? C : 0) + h * D;           // K | Q
+  auto load_other = [&](int st, int y0) {
+    ptx::mbar_expect_tx(bar_y(st), 2 * kTile);
+    ptx::tma_load_2d(y1_s(st), &tm_qkv, bar_y(st), y1_col, y0);
+    if (kDQ) ptx::tma_load_2d(y2_s(st), &tm_qkv, bar_y(st), 2 * C + h * D, y0);   // V
+    else ptx::tma_load_2d(y2_s(st), &tm_do, bar_y(st), h * D, y0);                // dO
+  };
+  if (tid == 0) {
+    ptx::mbar_expect_tx(bar_x, 2 * kTile);
+    ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
+    if (kDQ) ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                    // dO
+    else ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);               // V
+    load_other(0, o_lo);
+  }
+
+  // per-row statistics of the query side
+  float my_lse = 0.f, my_D = 0.f;   // kDQ: this thread's query row
+  float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next staged query tile, row tid
+  if (kDQ) {
+    if (row < Np) {
+      const __nv_bfloat16* orow = ao + (long long)row * C + h * D;
+      const __nv_bfloat16* grow = dao + (long long)row * C + h * D;
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        float a[8], b[8];
+        Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(orow + c * 8), a);
+        Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(grow + c * 8), b);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
+      }
+      my_lse = lse[(long long)h * capacity + row] * kLog2e;
+      delta[(long long)h * capacity + row] = my_D;
+    }
+  } else {
+    const int i = o_lo + tid;
+    if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
+  }
+
+  constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, 128, false, false);
+  constexpr uint32_t kIdescAcc = ptx::idesc_bf16_f32(128, D, false, true);
+  const unsigned span = (unsigned)(mine.hi - mine.lo);
+  int issued = 1;
+
+  for (int t = 0; t < n_tiles; ++t) {
+    const int st = t & 1;
+    const int y0 = o_lo + t * 128;
+    if (tid == 0 && t + 1 < n_tiles) { load_other(st ^ 1, y0 + 128); issued = t + 2; }
+    if (!kDQ) {
+      stat_lse[tid] = nxt_lse;
+      stat_D[tid] = nxt_D;
+      const int i = y0 + 128 + tid;
+      nxt_lse = 0.f; nxt_D = 0.f;
+      if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
+    }
+    // other-side lines past the last valid packed row must not reach a product
+    bool ok = ptx::mbar_wait(bar_y(st), (t >> 1) & 1);
+    if (t == 0) ok = ptx::mbar_wait(bar_x, 0) && ok;
+    if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    if (y0 + 128 > Np) {
+      const int first = Np - y0;
+      constexpr int kChunks = HT::kRowBytes / 16;
+      for (int c = tid; c < (128 - first) * kChunks; c += kBwdThreads) {
+        const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
+        *reinterpret_cast<uint4*>(smem_al + kTile * (2 + 2 * st) + off) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(smem_al + kTile * (3 + 2 * st) + off) = make_uint4(0, 0, 0, 0);
+      }
+      ptx::fence_proxy_async_smem();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) break;
+    if (tid == 0) {
+      ptx::tc_fence_after_sync();
+#pragma unroll
+      for (int k = 0; k < D / 16; ++k)
+        ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1_s(st), k), kIdescS, k != 0 ? 1u : 0u);
+#pragma unroll
+      for (int k = 0; k < D / 16; ++k)
+        ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2_s(st), k), kIdescS, k != 0 ? 1u : 0u);
+      ptx::mma_commit(bar_s);
+    }
+    if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    ptx::tc_fence_after_sync();
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t rs[32], rp[32], pk_p[16], pk_ds[16];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + c * 32, rs);
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + c * 32, rp);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; j += 2) {
+        float pv[2], dsv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int col = c * 32 + j + u;
+          const bool valid = (unsigned)(y0 + col - mine.lo) < span;
+          const float l2 = kDQ ? my_lse : stat_lse[col];
+          const float Dv = kDQ ? my_D : stat_D[col];
+          const float pe = ptx::ex2_approx(__uint_as_float(rs[j + u]) * scale_log2e - l2);
+          pv[u] = valid ? pe : 0.f;
+          dsv[u] = valid ? pe * (__uint_as_float(rp[j + u]) - Dv) : 0.f;
+        }
+        __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
+        pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
+        if (!kDQ) {
+          __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
+          pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+        }
+      }
+      if (kDQ) {
+        ptx::tmem_st_32x16(tmem + lane_base + kColS1 + c * 16, pk_ds);   // dS over the consumed part of S
+      } else {
+        ptx::tmem_st_32x16(tmem + lane_base + kColS1 + c * 16, pk_p);    // P^T over S^T
+        ptx::tmem_st_32x16(tmem + lane_base + kColS2 + c * 16, pk_ds);   // dS^T over dP^T
+      }
+    }
+    ptx::tmem_st_wait();
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      ptx::tc_fence_after_sync();
+      const uint32_t acc = (t != 0) ? 1u : 0u;
+      if (kDQ) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)   // dQ += dS K
+          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS1 + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)   // dV += P^T dO
+          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS1 + k * 8, HT::mnmajor(y2_s(st), k), kIdescAcc, acc | (k != 0));
+#pragma unroll
+        for (int k = 0; k < 8; ++k)   // dK += dS^T Q
+          ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColS2 + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
+      }
+      ptx::mma_commit(bar_o);
+    }
+    if (!ptx::mbar_wait(bar_o, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    ptx::tc_fence_after_sync();
+  }
+
+  if (!*abort_flag && n_tiles > 0) {
+    const long long ld = 3LL * C;
+    auto store_acc = [&](uint32_t col0, __nv_bfloat16* dst, float mul) {
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem + lane_base + col0 + c * 32, r);
+        ptx::tmem_ld_wait();
+        if (row < Np) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul;
+            *reinterpret_cast<uint4*>(dst + c * 32 + g * 8) = Vec16<__nv_bfloat16>::from_float(v);
+          }
+        }
+      }
+    };
+    __nv_bfloat16* base = dqkv + (long long)row * ld + h * D;
+    if (kDQ) {
+      store_acc(kColAcc1, base, scale);
+    } else {
+      store_acc(kColAcc1, base + 2 * C, 1.f);     // dV
+      store_acc(kColAcc2, base + C, scale);       // dK
+    }
+  }
+  if (*abort_flag && tid == 0) {
+    for (int t = issued > 2 ? issued - 2 : 0; t < issued; ++t) ptx::mbar_wait(bar_y(t & 1), (t >> 1) & 1);
+    ptx::mbar_wait(bar_x, 0);
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem, kBwdTmemCols);
+  }
+}
+
+template <int D>
+int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
+               const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st) {
+  CUtensorMap tm_qkv, tm_do;
+  if (!make_tmap_bf16_2d(&tm_qkv, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2) ||
+      !make_tmap_bf16_2d(&tm_do, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2))
+    return SPA_ERR_UNSUPPORTED;
+  auto kq = attn_bwd_tc_kernel<D, true>;
+  auto kkv = attn_bwd_tc_kernel<D, false>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D>());
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D>());
+    if (e != cudaSuccess) { set_cuda_error(e, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
+    attr_set = true;
+  }
+  float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
+  dim3 grid((p.capacity + 127) / 128, p.H);
+  const float scale = softmax_scale_of(p);
+  kq<<<grid, kBwdThreads, bwd_smem_bytes<D>(), st>>>(tm_qkv, tm_do, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
+                                                    lse, delta, seg, n_seg, p.capacity, p.C, scale,
+                                                    (__nv_bfloat16*)dqkv, d_status);
+  SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
+  kkv<<<grid, kBwdThreads, bwd_smem_bytes<D>(), st>>>(tm_qkv, tm_do, (const __nv_bfloat16*)ao,
+                                                     (const __nv_bfloat16*)dao, lse, delta, seg, n_seg, p.capacity,
+                                                     p.C, scale, (__nv_bfloat16*)dqkv, d_status);
+  SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
+  return SPA_OK;
+}
+
 template <int D>
 int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
                int32_t* d_status, cudaStream_t st) {
@@ -255,6 +541,20 @@ int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_s
 bool tc_attention_fwd_supported(const spa_params& p) {
   const int d = p.C / p.H;
   return p.dtype == SPA_BF16 && (d == 32 || d == 64) && tensor_maps_available();
+}
+
+bool tc_attention_bwd_supported(const spa_params& p) { return tc_attention_fwd_supported(p); }
+
+size_t tc_attention_workspace_bytes(const spa_params& p) {
+  if (!tc_attention_fwd_supported(p)) return 0;
+  return ((size_t)p.H * p.capacity * sizeof(float) + 255) & ~(size_t)255;
+}
+
+int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
+                            const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
+                            cudaStream_t st) {
+  return p.C / p.H == 64 ? bwd_launch<64>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st)
+                         : bwd_launch<32>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st);
 }
 
 int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
