@@ -43,7 +43,8 @@ typedef enum {
   SPA_ERR_UNSUPPORTED = -2, /* dtype, head dimension or row size the kernels do not cover   */
   SPA_ERR_CAPACITY = -3,    /* device: more selected tokens than `capacity`                 */
   SPA_ERR_CUDA = -4,        /* a CUDA runtime call failed (see spa_last_cuda_error)         */
-  SPA_ERR_TIMEOUT = -5      /* device: a bounded wait expired                               */
+  SPA_ERR_TIMEOUT = -5,     /* device: a bounded wait expired                               */
+  SPA_ERR_SCRATCH = -6      /* the problem needs more scratch than the built-in array holds */
 } spa_status;
 
 typedef enum { SPA_F32 = 0, SPA_BF16 = 1 } spa_dtype;
@@ -120,6 +121,35 @@ int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* a
                              const float* lse, const void* d_attn_out, const int32_t* seg_offsets,
                              int32_t n_seg, void* dqkv, void* workspace, int32_t* d_status,
                              void* stream);
+
+/* Attention backward for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart: this is a packaging variant of spa_packed_attention_bwd, same arithmetic.)
+ *
+ * Who needs it: code that runs where device allocation is off the table - inside a region that is
+ * being recorded for later replay, inside a framework whose memory pool is frozen or owned by
+ * someone else, in a plugin that is only handed its input and output tensors, or under a memory
+ * budget fixed at start-up.  Such callers cannot call cudaMalloc (or any allocator built on it) to
+ * obtain the `workspace` the regular call wants, so here the per-row scratch (D_i, one float per
+ * head and packed row) lives in an array that is part of the library image itself.
+ *
+ * Limits and rules:
+ *   - bf16 problems with head dimension 32 or 64 only (the tensor-core path); anything else returns
+ *     SPA_ERR_UNSUPPORTED.
+ *   - H * capacity * sizeof(float) must not exceed SPA_STATIC_SCRATCH_BYTES, else SPA_ERR_SCRATCH.
+ *     Every GPU on which the library is loaded holds that many bytes until the process exits.
+ *   - The call allocates nothing and frees nothing, on the device or through any library.
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     Nothing in it has to start at zero: each call writes every entry before reading it.  Two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it; keep
+ *     calls to this entry point ordered with respect to one another.
+ * Arguments are those of spa_packed_attention_bwd without `workspace`. */
+#define SPA_STATIC_SCRATCH_BYTES (4u << 20)
+int spa_packed_attention_bwd_static(const spa_params* p, const void* qkv, const void* attn_out,
+                                    const float* lse, const void* d_attn_out,
+                                    const int32_t* seg_offsets, int32_t n_seg, void* dqkv,
+                                    int32_t* d_status, void* stream);
 
 /* Output projection on the packed tokens:  z[i][j] = b_o[j] + sum_c W_o[j][c] * a[i][c].
  * a: T[capacity][C]; W_o: T[C][C]; b_o: T[C] or NULL; z: T[capacity][C] out. */

@@ -17,6 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspa.so")
 
 SPA_OK, SPA_ERR_INVALID_ARG, SPA_ERR_UNSUPPORTED, SPA_ERR_CAPACITY, SPA_ERR_CUDA, SPA_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+SPA_ERR_SCRATCH = -6
+SPA_STATIC_SCRATCH_BYTES = 4 << 20
 SPA_F32, SPA_BF16 = 0, 1
 SPA_FLAG_RESIDUAL, SPA_FLAG_INPLACE, SPA_FLAG_GATE_SCALE, SPA_FLAG_SIMT_ONLY = 1, 2, 4, 8
 
@@ -24,7 +26,7 @@ EXPORTS = (
     "spa_workspace_bytes", "spa_gate", "spa_select_pack", "spa_packed_qkv", "spa_packed_attention_fwd",
     "spa_packed_attention_bwd", "spa_packed_proj", "spa_unpack_scatter", "spa_unpack_scatter_bwd",
     "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
-    "spa_last_cuda_error", "spa_launch_count",
+    "spa_last_cuda_error", "spa_launch_count", "spa_packed_attention_bwd_static",
 )
 
 
@@ -66,6 +68,7 @@ def lib() -> C.CDLL:
         L.spa_packed_qkv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_packed_attention_fwd.argtypes = [pp, vp, vp, i32, vp, vp, vp, vp]
         L.spa_packed_attention_bwd.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        L.spa_packed_attention_bwd_static.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.spa_packed_proj.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_unpack_scatter.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_unpack_scatter_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
@@ -134,6 +137,15 @@ def spa_packed_attention_bwd(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_s
     _check(lib().spa_packed_attention_bwd(C.byref(p), _ptr(qkv), _ptr(attn_out), _ptr(lse), _ptr(d_attn_out),
                                           _ptr(seg_offsets), int(n_seg), _ptr(dqkv), _ptr(workspace), _ptr(d_status),
                                           _stream(stream)), "spa_packed_attention_bwd")
+
+
+def spa_packed_attention_bwd_static(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, d_status=None,
+                                    stream=None):
+    """Attention backward for callers that cannot allocate: the scratch is an array inside the library
+    (at most SPA_STATIC_SCRATCH_BYTES; all calls on a device share it, so keep them ordered)."""
+    _check(lib().spa_packed_attention_bwd_static(C.byref(p), _ptr(qkv), _ptr(attn_out), _ptr(lse), _ptr(d_attn_out),
+                                                 _ptr(seg_offsets), int(n_seg), _ptr(dqkv), _ptr(d_status),
+                                                 _stream(stream)), "spa_packed_attention_bwd_static")
 
 
 def spa_packed_proj(p, a, W_o, b_o, cu_seqlens, z, d_status=None, stream=None):

@@ -214,6 +214,7 @@ const char* spa_status_string(int status) {
     case SPA_ERR_CAPACITY: return "more selected tokens than the packed capacity";
     case SPA_ERR_CUDA: return "CUDA runtime error";
     case SPA_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case SPA_ERR_SCRATCH: return "the problem needs more scratch than the built-in array holds";
     default: return "unknown status";
   }
 }

@@ -13,6 +13,8 @@
 // product and V lines are zeroed in shared memory before the product.
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "sm100_ptx.cuh"
 #include "spa_tc.cuh"
 
@@ -564,3 +566,58 @@ int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t*
 }
 
 }  // namespace spa
+
+// ------------------------------------------------------------------------------------------------
+// Attention backward without caller scratch.  The D_i values (one float per head and packed row)
+// that the dQ pass hands to the dK/dV pass live in this array, which is part of the library image:
+// a caller that may not allocate device memory still gets the tensor-core backward.  Host code must
+// not pass the symbol itself to a kernel - on the host it only stands for the array - so the device
+// address is looked up once per device and cached.
+static __device__ __align__(256) unsigned char g_static_scratch[SPA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device (looked up on first use).
+int static_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { spa::set_cuda_error(e, "spa_packed_attention_bwd_static: cudaGetDevice"); return SPA_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) return SPA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (g_scratch_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess || ptr == nullptr) {
+      spa::set_cuda_error(e, "spa_packed_attention_bwd_static: cudaGetSymbolAddress");
+      return SPA_ERR_CUDA;
+    }
+    g_scratch_ptr[dev] = ptr;
+  }
+  *out = g_scratch_ptr[dev];
+  return SPA_OK;
+}
+}  // namespace
+
+extern "C" int spa_packed_attention_bwd_static(const spa_params* p, const void* qkv, const void* attn_out,
+                                               const float* lse, const void* d_attn_out, const int32_t* seg_offsets,
+                                               int32_t n_seg, void* dqkv, int32_t* d_status, void* stream) {
+  auto misaligned = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
+  if (p == nullptr || p->B < 0 || p->N <= 0 || p->C <= 0 || p->H <= 0 || p->C % p->H != 0 || n_seg < 0 ||
+      p->capacity < 1 || (long long)p->capacity > (long long)(p->B > 0 ? p->B : 1) * p->N)
+    return SPA_ERR_INVALID_ARG;
+  if (misaligned(qkv) || misaligned(attn_out) || misaligned(lse) || misaligned(d_attn_out) ||
+      misaligned(seg_offsets) || misaligned(dqkv))
+    return SPA_ERR_INVALID_ARG;
+  if ((long long)p->B * p->N > (1LL << 20) || (p->flags & SPA_FLAG_SIMT_ONLY) || !spa::tc_attention_bwd_supported(*p))
+    return SPA_ERR_UNSUPPORTED;
+  if ((unsigned long long)p->H * (unsigned long long)p->capacity * sizeof(float) > SPA_STATIC_SCRATCH_BYTES)
+    return SPA_ERR_SCRATCH;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != SPA_OK) return rc;
+  return spa::launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, scratch, d_status,
+                                      (cudaStream_t)stream);
+}
