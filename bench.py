@@ -319,8 +319,8 @@ def main():
 
     def e2e_step(i):
         inp, d, blk, seq = sets[i % n_sets]
-        d["x"].copy_(hx[i % 2], non_blocking=True)
-        d["dY"].copy_(hdy[i % 2], non_blocking=True)
+        d["x"].copy_(hx[(i % n_sets) % 2], non_blocking=True)
+        d["dY"].copy_(hdy[(i % n_sets) % 2], non_blocking=True)
         step(i)
         hy.copy_(blk.y, non_blocking=True)
         hdx.copy_(blk.dX, non_blocking=True)

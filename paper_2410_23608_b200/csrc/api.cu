@@ -1,5 +1,6 @@
 // C boundary: argument validation and dispatch to the kernels.  Nothing here computes.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <atomic>
@@ -13,6 +14,11 @@ static thread_local char g_cuda_error[256] = "";
 
 void set_cuda_error(cudaError_t e, const char* where) {
   snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+}
+
+bool pdl_enabled() {
+  static const bool on = []() { const char* e = getenv("SPA_PDL"); return !(e != nullptr && e[0] == '0'); }();
+  return on;
 }
 
 static std::atomic<unsigned long long> g_launches{0};

@@ -93,6 +93,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kRows * (D / kPart))
 attn_fwd_simt_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ seg, int n_seg, int capacity, int C,
                      float scale, T* __restrict__ ao, float* __restrict__ lse) {
+  pdl_entry();
   constexpr int kSplit = D / kPart;
   constexpr int kThreads = kRows * kSplit;
   __shared__ __align__(16) float Ks[kRows][D];
@@ -166,6 +167,7 @@ __global__ void __launch_bounds__(kRows * (D / kPart))
 attn_bwd_dq_simt_kernel(const T* __restrict__ qkv, const T* __restrict__ ao, const float* __restrict__ lse,
                         const T* __restrict__ dao, const int32_t* __restrict__ seg, int n_seg, int capacity, int C,
                         float scale, T* __restrict__ dqkv) {
+  pdl_entry();
   constexpr int kSplit = D / kPart;
   constexpr int kThreads = kRows * kSplit;
   __shared__ __align__(16) float Ks[kRows][D];
@@ -224,6 +226,7 @@ __global__ void __launch_bounds__(kRows * (D / kPart))
 attn_bwd_dkv_simt_kernel(const T* __restrict__ qkv, const T* __restrict__ ao, const float* __restrict__ lse,
                          const T* __restrict__ dao, const int32_t* __restrict__ seg, int n_seg, int capacity, int C,
                          float scale, T* __restrict__ dqkv) {
+  pdl_entry();
   constexpr int kSplit = D / kPart;
   constexpr int kThreads = kRows * kSplit;
   constexpr int E = Vec16<T>::kElems;
@@ -296,7 +299,7 @@ template <typename T, int D>
 int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
                cudaStream_t st) {
   dim3 grid((p.capacity + kRows - 1) / kRows, p.H);
-  attn_fwd_simt_kernel<T, D><<<grid, kRows * (D / kPart), 0, st>>>((const T*)qkv, seg, n_seg, p.capacity, p.C,
+  launch_pdl(attn_fwd_simt_kernel<T, D>, grid, kRows * (D / kPart), 0, st, (const T*)qkv, seg, n_seg, p.capacity, p.C,
                                                                   softmax_scale_of(p), (T*)ao, lse);
   SPA_CUDA_CHECK_LAUNCH("attn_fwd_simt_kernel");
   return SPA_OK;
@@ -307,10 +310,10 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
                const int32_t* seg, int n_seg, void* dqkv, cudaStream_t st) {
   dim3 grid((p.capacity + kRows - 1) / kRows, p.H);
   const float scale = softmax_scale_of(p);
-  attn_bwd_dq_simt_kernel<T, D><<<grid, kRows * (D / kPart), 0, st>>>((const T*)qkv, (const T*)ao, lse, (const T*)dao,
+  launch_pdl(attn_bwd_dq_simt_kernel<T, D>, grid, kRows * (D / kPart), 0, st, (const T*)qkv, (const T*)ao, lse, (const T*)dao,
                                                                      seg, n_seg, p.capacity, p.C, scale, (T*)dqkv);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_dq_simt_kernel");
-  attn_bwd_dkv_simt_kernel<T, D><<<grid, kRows * (D / kPart), 0, st>>>((const T*)qkv, (const T*)ao, lse,
+  launch_pdl(attn_bwd_dkv_simt_kernel<T, D>, grid, kRows * (D / kPart), 0, st, (const T*)qkv, (const T*)ao, lse,
                                                                       (const T*)dao, seg, n_seg, p.capacity, p.C,
                                                                       scale, (T*)dqkv);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_dkv_simt_kernel");

@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(kFwdThreads)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __restrict__ seg, int n_seg, int capacity,
                    int C, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
                    int32_t* d_status) {
+  pdl_entry();
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
   const int Np = packed_rows(seg, n_seg, capacity);
@@ -256,6 +257,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
                    const __nv_bfloat16* __restrict__ ao, const __nv_bfloat16* __restrict__ dao,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
                    int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
+  pdl_entry();
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
   constexpr float kLog2e = 1.4426950408889634f;
@@ -507,11 +509,11 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
   dim3 grid((p.capacity + 127) / 128, p.H);
   const float scale = softmax_scale_of(p);
-  kq<<<grid, kBwdThreads, bwd_smem_bytes<D>(), st>>>(tm_qkv, tm_do, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
+  launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
                                                     lse, delta, seg, n_seg, p.capacity, p.C, scale,
                                                     (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
-  kkv<<<grid, kBwdThreads, bwd_smem_bytes<D>(), st>>>(tm_qkv, tm_do, (const __nv_bfloat16*)ao,
+  launch_pdl(kkv, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, (const __nv_bfloat16*)ao,
                                                      (const __nv_bfloat16*)dao, lse, delta, seg, n_seg, p.capacity,
                                                      p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
@@ -531,7 +533,7 @@ int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_s
     attr_set = true;
   }
   dim3 grid((p.capacity + kQ - 1) / kQ, p.H);
-  kern<<<grid, kFwdThreads, fwd_smem_bytes<D>(), st>>>(tm, seg, n_seg, p.capacity, p.C,
+  launch_pdl(kern, grid, kFwdThreads, fwd_smem_bytes<D>(), st, tm, seg, n_seg, p.capacity, p.C,
                                                       softmax_scale_of(p) * 1.4426950408889634f,
                                                       (__nv_bfloat16*)ao, lse, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_fwd_tc_kernel");

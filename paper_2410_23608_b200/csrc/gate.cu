@@ -15,6 +15,7 @@ template <typename T>
 __global__ void __launch_bounds__(kGateThreads)
 gate_kernel(const T* __restrict__ x, const T* __restrict__ w_g, float b_g, const float* __restrict__ s_up,
             float tau, int rows, int C, float* __restrict__ scores, uint8_t* __restrict__ mask) {
+  pdl_entry();
   constexpr int E = Vec16<T>::kElems;
   extern __shared__ float w_s[];
   for (int c = threadIdx.x; c < C; c += blockDim.x) w_s[c] = to_f32<T>(w_g[c]);
@@ -77,10 +78,10 @@ int launch_gate(const spa_params& p, const void* x, const void* w_g, float b_g, 
   if (grid > kNumSMs * 8) grid = kNumSMs * 8;
   const size_t smem = (size_t)p.C * sizeof(float);
   if (p.dtype == SPA_F32)
-    gate_kernel<float><<<grid, kGateThreads, smem, st>>>((const float*)x, (const float*)w_g, b_g, s_up, p.tau,
+    launch_pdl(gate_kernel<float>, grid, kGateThreads, smem, st, (const float*)x, (const float*)w_g, b_g, s_up, p.tau,
                                                          rows, p.C, scores, mask);
   else
-    gate_kernel<__nv_bfloat16><<<grid, kGateThreads, smem, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_g,
+    launch_pdl(gate_kernel<__nv_bfloat16>, grid, kGateThreads, smem, st, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_g,
                                                                  b_g, s_up, p.tau, rows, p.C, scores, mask);
   SPA_CUDA_CHECK_LAUNCH("gate_kernel");
   return SPA_OK;

@@ -18,6 +18,7 @@ __global__ void __launch_bounds__(kThreads)
 gemm_simt_kernel(const T* __restrict__ A, long long sAm, long long sAk, const T* __restrict__ Bm, long long sBn,
                  long long sBk, const T* __restrict__ bias, TO* __restrict__ out, long long ldo, int M, int N, int K,
                  const int32_t* __restrict__ cu, int n_seg, int capacity, int dyn_which) {
+  pdl_entry();
   if (dyn_which != 0) {
     const int rows = packed_rows(cu, n_seg, capacity);
     if (dyn_which == 1) M = rows; else K = rows;
@@ -80,6 +81,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 colsum_kernel(const T* __restrict__ dout, int n_out, const int32_t* __restrict__ cu, int n_seg, int capacity,
               float* __restrict__ db) {
+  pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
   __shared__ float part[4][64];
   const int c = threadIdx.x % 64, g = threadIdx.x / 64;
@@ -97,7 +99,7 @@ void launch_gemm(const T* A, long long sAm, long long sAk, const T* Bm, long lon
                  TO* out, long long ldo, int M, int N, int K, const int32_t* cu, int n_seg, int capacity,
                  int dyn_which, cudaStream_t st) {
   dim3 grid((N + kTile - 1) / kTile, (M + kTile - 1) / kTile);
-  gemm_simt_kernel<T, TO><<<grid, kThreads, 0, st>>>(A, sAm, sAk, Bm, sBn, sBk, bias, out, ldo, M, N, K, cu, n_seg,
+  launch_pdl(gemm_simt_kernel<T, TO>, grid, kThreads, 0, st, A, sAm, sAk, Bm, sBn, sBk, bias, out, ldo, M, N, K, cu, n_seg,
                                                     capacity, dyn_which);
 }
 
@@ -124,7 +126,7 @@ int linear_bwd(const spa_params& p, const void* a, const void* W, const void* do
     SPA_CUDA_CHECK_LAUNCH("gemm_simt_kernel(wgrad)");
   }
   if (db != nullptr) {
-    colsum_kernel<T><<<(n_out + 63) / 64, kThreads, 0, st>>>((const T*)dout, n_out, cu, p.B, p.capacity, db);
+    launch_pdl(colsum_kernel<T>, (n_out + 63) / 64, kThreads, 0, st, (const T*)dout, n_out, cu, p.B, p.capacity, db);
     SPA_CUDA_CHECK_LAUNCH("colsum_kernel");
   }
   return SPA_OK;

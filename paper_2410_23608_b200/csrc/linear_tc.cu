@@ -102,6 +102,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
                long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
                int dyn_which, int k_per_split, int32_t* d_status) {
+  pdl_entry();
   constexpr int kStage = stage_bytes<BN>();
   constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
   {
@@ -267,6 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 __global__ void __launch_bounds__(256)
 colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const int32_t* __restrict__ cu, int n_seg,
                       int capacity, int k_per_split, float* __restrict__ part) {
+  pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
   const int r_begin = blockIdx.y * k_per_split;
   int r_end = r_begin + k_per_split;
@@ -300,6 +302,7 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const i
 __global__ void __launch_bounds__(256)
 split_reduce_kernel(const float* __restrict__ part, long long n, long long split_stride, int k_per_split,
                     const int32_t* __restrict__ cu, int n_seg, int capacity, float* __restrict__ out) {
+  pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
   const int valid = (rows + k_per_split - 1) / k_per_split;
   const long long n4 = n >> 2;
@@ -348,7 +351,7 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
     attr_set = true;
   }
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, splits);
-  kern<<<grid, kGemmThreads, gemm_smem_bytes<BN>(), st>>>(tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu, n_seg,
+  launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu, n_seg,
                                                          capacity, dyn_which, k_per_split, d_status);
   SPA_CUDA_CHECK_LAUNCH(what);
   return SPA_OK;
@@ -407,15 +410,15 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
     const long long n = (long long)n_out * n_in;
     int grid = (int)((n / 4 + 255) / 256);
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
-    split_reduce_kernel<<<grid, 256, 0, st>>>(part_w, n, n, sp.k_per_split, cu, p.B, p.capacity, dW);
+    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n, n, sp.k_per_split, cu, p.B, p.capacity, dW);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(dW)");
   }
   if (db != nullptr) {
     dim3 grid((n_out + 63) / 64, sp.splits);
-    colsum_partial_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity, sp.k_per_split,
+    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity, sp.k_per_split,
                                                 part_b);
     SPA_CUDA_CHECK_LAUNCH("colsum_partial_kernel");
-    split_reduce_kernel<<<(n_out / 4 + 255) / 256, 256, 0, st>>>(part_b, n_out, n_out, sp.k_per_split, cu, p.B,
+    launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, part_b, n_out, n_out, sp.k_per_split, cu, p.B,
                                                                  p.capacity, db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
   }

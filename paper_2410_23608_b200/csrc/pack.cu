@@ -46,6 +46,7 @@ select_pack_kernel(const uint4* __restrict__ x16, const uint8_t* __restrict__ ma
                    int rows, int N, int B, int Q, int tile, int capacity, uint4* __restrict__ xp16,
                    int32_t* __restrict__ idx, int32_t* __restrict__ inv, int32_t* __restrict__ cu,
                    int32_t* d_status) {
+  pdl_entry();
   __shared__ int warp_cnt[kPackThreads / 32];
   __shared__ int warp_sel[kPackThreads / 32];
   __shared__ int sel_tok[kPackThreads];   // tile-local offsets of the selected tokens, in order
@@ -126,6 +127,7 @@ __global__ void __launch_bounds__(kPackThreads)
 unpack_scatter_kernel(const uint4* __restrict__ z16, const uint4* __restrict__ x16, const int32_t* __restrict__ inv,
                       const int32_t* __restrict__ cu, int B, int capacity, long long total, int Q,
                       uint4* __restrict__ y16) {
+  pdl_entry();
   const int Np = packed_rows(cu, B, capacity);
   const long long stride = (long long)gridDim.x * kPackThreads;
   for (long long k0 = (long long)blockIdx.x * kPackThreads + threadIdx.x; k0 < total; k0 += stride * kBatch) {
@@ -160,6 +162,7 @@ template <typename T, bool kAdd>
 __global__ void __launch_bounds__(kPackThreads)
 row_scatter_kernel(const uint4* __restrict__ src16, const uint4* addp, const int32_t* __restrict__ idx,
                    const int32_t* __restrict__ cu, int B, int capacity, int Q, uint4* dst16) {
+  pdl_entry();
   const long long total = (long long)packed_rows(cu, B, capacity) * Q;
   const long long stride = (long long)gridDim.x * kPackThreads;
   for (long long k0 = (long long)blockIdx.x * kPackThreads + threadIdx.x; k0 < total; k0 += stride * kBatch) {
@@ -189,6 +192,7 @@ __global__ void __launch_bounds__(kPackThreads)
 unpack_scatter_bwd_kernel(const uint4* __restrict__ dY16, const int32_t* __restrict__ inv,
                           const int32_t* __restrict__ cu, int B, int capacity, long long total, int Q,
                           uint4* __restrict__ dz16, uint4* dX16, bool copy_pass_through) {
+  pdl_entry();
   const int Np = packed_rows(cu, B, capacity);
   const long long stride = (long long)gridDim.x * kPackThreads;
   for (long long k0 = (long long)blockIdx.x * kPackThreads + threadIdx.x; k0 < total; k0 += stride * kBatch) {
@@ -235,7 +239,7 @@ int launch_select_pack(const spa_params& p, const void* x, const uint8_t* mask, 
   const int grid = (rows + tile - 1) / tile;
   const bool gs = (p.flags & SPA_FLAG_GATE_SCALE) != 0;
 #define SPA_PACK_LAUNCH(T, GS)                                                                              \
-  select_pack_kernel<T, GS><<<grid, kPackThreads, 0, st>>>((const uint4*)x, mask, scores, rows, p.N, p.B,    \
+  launch_pdl(select_pack_kernel<T, GS>, grid, kPackThreads, 0, st, (const uint4*)x, mask, scores, rows, p.N, p.B,    \
                                                           chunks_per_row<T>(p.C), tile, p.capacity,         \
                                                           (uint4*)xp, idx, inv, cu, d_status)
   if (p.dtype == SPA_F32) { if (gs) SPA_PACK_LAUNCH(float, true); else SPA_PACK_LAUNCH(float, false); }
@@ -246,7 +250,7 @@ int launch_select_pack(const spa_params& p, const void* x, const uint8_t* mask, 
 }
 
 #define SPA_SCATTER(T, ADD, SRC, ADDP, DST) \
-  row_scatter_kernel<T, ADD><<<grid, kPackThreads, 0, st>>>((const uint4*)(SRC), (const uint4*)(ADDP), idx, cu, p.B, p.capacity, Q, (uint4*)(DST))
+  launch_pdl(row_scatter_kernel<T, ADD>, grid, kPackThreads, 0, st, (const uint4*)(SRC), (const uint4*)(ADDP), idx, cu, p.B, p.capacity, Q, (uint4*)(DST))
 
 int launch_unpack_scatter(const spa_params& p, const void* z, const void* x, const int32_t* idx,
                           const int32_t* inv, const int32_t* cu, void* y, cudaStream_t st) {
@@ -263,7 +267,7 @@ int launch_unpack_scatter(const spa_params& p, const void* z, const void* x, con
   const long long total = (long long)p.B * p.N * Q;
   const int grid = stream_grid(total);
 #define SPA_UNPACK(T, RES) \
-  unpack_scatter_kernel<T, RES><<<grid, kPackThreads, 0, st>>>((const uint4*)z, (const uint4*)x, inv, cu, p.B, p.capacity, total, Q, (uint4*)y)
+  launch_pdl(unpack_scatter_kernel<T, RES>, grid, kPackThreads, 0, st, (const uint4*)z, (const uint4*)x, inv, cu, p.B, p.capacity, total, Q, (uint4*)y)
   if (f32) { if (res) SPA_UNPACK(float, true); else SPA_UNPACK(float, false); }
   else { if (res) SPA_UNPACK(__nv_bfloat16, true); else SPA_UNPACK(__nv_bfloat16, false); }
 #undef SPA_UNPACK
@@ -277,7 +281,7 @@ int launch_unpack_scatter_bwd(const spa_params& p, const void* dY, const int32_t
   const int Q = p.dtype == SPA_F32 ? chunks_per_row<float>(p.C) : chunks_per_row<__nv_bfloat16>(p.C);
   const long long total = (long long)p.B * p.N * Q;
   const bool copy = dX != nullptr && dX != dY;
-  unpack_scatter_bwd_kernel<<<stream_grid(total), kPackThreads, 0, st>>>((const uint4*)dY, inv, cu, p.B, p.capacity,
+  launch_pdl(unpack_scatter_bwd_kernel, stream_grid(total), kPackThreads, 0, st, (const uint4*)dY, inv, cu, p.B, p.capacity,
                                                                         total, Q, (uint4*)dz, (uint4*)dX, copy);
   SPA_CUDA_CHECK_LAUNCH("unpack_scatter_bwd_kernel");
   return SPA_OK;

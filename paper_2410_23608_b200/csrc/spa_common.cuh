@@ -21,6 +21,13 @@ __device__ __forceinline__ void record_status(int32_t* d_status, int code) {
   if (d_status != nullptr) atomicCAS(d_status, 0, code);
 }
 
+// Programmatic dependent launch: every kernel lets its successor in the stream start being scheduled at
+// once, and itself waits for its predecessor's results before touching global memory.  Launch
+// latency and CTA ramp-up of the next kernel overlap the tail of this one.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_entry() { pdl_launch_dependents(); pdl_wait(); }
+
 // ---- 16-byte vector access, converted to fp32 ------------------------------------------------
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {
@@ -108,6 +115,24 @@ void count_launch();  // one more kernel of this library was enqueued (host-side
     if (e__ != cudaSuccess) { ::spa::set_cuda_error(e__, where); return SPA_ERR_CUDA; } \
     ::spa::count_launch();                                             \
   } while (0)
+
+bool pdl_enabled();  // programmatic dependent launch is on unless the environment sets SPA_PDL=0
+
+// Launch `kern` on `st`, allowing it to overlap the tail of the previous kernel of the stream.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 // launchers implemented per .cu file; every one enqueues on `st` and returns a spa_status
 int launch_gate(const spa_params& p, const void* x, const void* w_g, float b_g, const float* s_up,
