@@ -95,147 +95,227 @@ template <> struct OutStore<float> {
   }
 };
 
+// Tile bookkeeping shared by the three roles of the persistent kernel.
+struct TileCoord { int m0, n0, z, n_t; };
+
 // dyn_which: 1 = M is the device-side packed row count, 2 = K is.
-template <int BN, bool kAMn, bool kBMn, typename OutT>
+// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... of the (m, n, split) space
+// that the device-side row count leaves; two accumulator stages in TMEM let the epilogue of one tile
+// overlap the main loop of the next, and the TMA ring runs ahead across tile boundaries.
+// kColSum (wgrad only): while the MMAs run, the epilogue warps add up the columns of the dout tiles
+// that stream through shared memory, which gives the bias gradient at no extra HBM traffic.
+template <int BN, bool kAMn, bool kBMn, typename OutT, bool kColSum>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
                long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
-               int dyn_which, int k_per_split, int32_t* d_status) {
-  pdl_entry();
+               int dyn_which, int k_per_split, float* __restrict__ colsum_part, int32_t* d_status) {
   constexpr int kStage = stage_bytes<BN>();
   constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
-  {
-    const int rows = packed_rows(cu, n_seg, capacity);
-    if (dyn_which == 1) M = rows; else if (dyn_which == 2) K = rows;
-  }
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int k_begin = blockIdx.z * k_per_split;
-  int k_end = k_begin + k_per_split;
-  if (k_end > K) k_end = K;
-  if (m0 >= M || k_begin >= k_end) return;
-  const int nkb = (k_end - k_begin + BK - 1) / BK;
+  pdl_launch_dependents();
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kStages * kStage;  // full[kStages], empty[kStages], tmem_full
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kStages * kStage + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStages * kStage + 68);
+  const uint32_t bar_base = smem_base + kStages * kStage;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
-  const uint32_t tmem_full_bar = bar_base + 8u * (2 * kStages);
+  auto tmem_full_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto tmem_empty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kStages * kStage + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStages * kStage + 100);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
-    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    ptx::mbar_init(tmem_full_bar, 1);
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), kColSum ? 2 : 1);
+    }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(tmem_full_bar(a), 1); ptx::mbar_init(tmem_empty_bar(a), 4); }
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
-  if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), BN);
+  if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), 2 * BN);
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
+  pdl_wait();  // everything above touched no global memory; the predecessor's results are needed from here on
+  {
+    const int rows = packed_rows(cu, n_seg, capacity);
+    if (dyn_which == 1) M = rows; else if (dyn_which == 2) K = rows;
+  }
+  const int tiles_n = (N + BN - 1) / BN;
+  const int tiles_m = (M + BM - 1) / BM;
+  const int n_splits = K > 0 ? (K + k_per_split - 1) / k_per_split : 0;
+  const int total = tiles_m * tiles_n * n_splits;
+  auto coord = [&](int tile) {
+    TileCoord c;
+    c.n_t = tile % tiles_n;
+    const int rest = tile / tiles_n;
+    c.m0 = (rest % tiles_m) * BM;
+    c.z = rest / tiles_m;
+    c.n0 = c.n_t * BN;
+    return c;
+  };
+  auto k_range = [&](int z, int& k_begin, int& k_end) {
+    k_begin = z * k_per_split;
+    k_end = k_begin + k_per_split;
+    if (k_end > K) k_end = K;
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % kStages;
-        if (kb >= kStages && !ptx::mbar_wait(empty_bar(s), ((kb / kStages) - 1) & 1)) {
-          record_status(d_status, SPA_ERR_TIMEOUT);
-          *abort_flag = 1;
-          break;
-        }
-        if (*abort_flag) break;
-        const uint32_t a_dst = smem_base + s * kStage, b_dst = a_dst + kABytes;
-        const int k0 = k_begin + kb * BK;
-        ptx::mbar_expect_tx(full_bar(s), kStage);
-        if (!kAMn) {
-          ptx::tma_load_2d(a_dst, &tmA, full_bar(s), k0, m0);
-        } else {
+      int it = 0;  // k-block counter over all tiles of this CTA: ring position and phase
+      for (int tile = blockIdx.x; tile < total && !*abort_flag; tile += gridDim.x) {
+        const TileCoord c = coord(tile);
+        int k_begin, k_end;
+        k_range(c.z, k_begin, k_end);
+        for (int k0 = k_begin; k0 < k_end; k0 += BK, ++it) {
+          const int s = it % kStages;
+          if (it >= kStages && !ptx::mbar_wait(empty_bar(s), ((it / kStages) - 1) & 1)) {
+            record_status(d_status, SPA_ERR_TIMEOUT);
+            *abort_flag = 1;
+          }
+          if (*abort_flag) break;
+          const uint32_t a_dst = smem_base + s * kStage, b_dst = a_dst + kABytes;
+          ptx::mbar_expect_tx(full_bar(s), kStage);
+          if (!kAMn) {
+            ptx::tma_load_2d(a_dst, &tmA, full_bar(s), k0, c.m0);
+          } else {
 #pragma unroll
-          for (int j = 0; j < BM / 64; ++j) ptx::tma_load_2d(a_dst + j * (BK * 128), &tmA, full_bar(s), m0 + 64 * j, k0);
-        }
-        if (!kBMn) {
-          ptx::tma_load_2d(b_dst, &tmB, full_bar(s), k0, n0);
-        } else {
+            for (int j = 0; j < BM / 64; ++j)
+              ptx::tma_load_2d(a_dst + j * (BK * 128), &tmA, full_bar(s), c.m0 + 64 * j, k0);
+          }
+          if (!kBMn) {
+            ptx::tma_load_2d(b_dst, &tmB, full_bar(s), k0, c.n0);
+          } else {
 #pragma unroll
-          for (int j = 0; j < BN / 64; ++j) ptx::tma_load_2d(b_dst + j * (BK * 128), &tmB, full_bar(s), n0 + 64 * j, k0);
+            for (int j = 0; j < BN / 64; ++j)
+              ptx::tma_load_2d(b_dst + j * (BK * 128), &tmB, full_bar(s), c.n0 + 64 * j, k0);
+          }
         }
-        issued = kb + 1;
       }
       if (*abort_flag) {  // let our own copies land before the CTA's shared memory goes away
-        for (int kb = issued > kStages ? issued - kStages : 0; kb < issued; ++kb)
-          ptx::mbar_wait(full_bar(kb % kStages), (kb / kStages) & 1);
+        for (int j = it > kStages ? it - kStages : 0; j < it; ++j)
+          ptx::mbar_wait(full_bar(j % kStages), (j / kStages) & 1);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    bool issued_any = false;
-    for (int kb = 0; kb < nkb; ++kb) {
-      const int s = kb % kStages;
-      if (*abort_flag) break;
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(full_bar(s), (kb / kStages) & 1))) {
+    int it = 0, tl = 0;  // k-block counter, tile counter of this CTA
+    bool dead = false;   // warp-uniform: a wait of this warp ran out, or another role gave up
+    for (int tile = blockIdx.x; tile < total && !dead; tile += gridDim.x, ++tl) {
+      if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
+      const TileCoord c = coord(tile);
+      int k_begin, k_end;
+      k_range(c.z, k_begin, k_end);
+      const int acc = tl & 1;
+      if (tl >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(tmem_empty_bar(acc), ((tl >> 1) - 1) & 1))) {
         if (lane == 0) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
         break;
       }
-      const uint32_t a_src = smem_base + s * kStage, b_src = a_src + kABytes;
-      const int k_valid = k_end - (k_begin + kb * BK);
-      if ((kAMn || kBMn) && k_valid < BK) {
-        // K rows beyond the end of the reduction: zero them (a K row is one 128-byte line per 64-wide box)
-        const int n_lines = BK - k_valid;
-        if (kAMn)
-          for (int j = 0; j < BM / 64; ++j)
-            for (int c = lane; c < n_lines * 8; c += 32)
-              *reinterpret_cast<uint4*>(smem_al + s * kStage + j * (BK * 128) + (k_valid + c / 8) * 128 + (c % 8) * 16) =
-                  make_uint4(0, 0, 0, 0);
-        if (kBMn)
-          for (int j = 0; j < BN / 64; ++j)
-            for (int c = lane; c < n_lines * 8; c += 32)
-              *reinterpret_cast<uint4*>(smem_al + s * kStage + kABytes + j * (BK * 128) + (k_valid + c / 8) * 128 +
-                                        (c % 8) * 16) = make_uint4(0, 0, 0, 0);
-        ptx::fence_proxy_async_smem();
+      ptx::tc_fence_after_sync();
+      const uint32_t tmem_d = tmem_base + acc * BN;
+      bool first = true;
+      for (int k0 = k_begin; k0 < k_end; k0 += BK, ++it) {
+        const int s = it % kStages;
+        if (__any_sync(0xffffffffu, *abort_flag != 0)) { dead = true; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(full_bar(s), (it / kStages) & 1))) {
+          if (lane == 0) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+          dead = true;
+          break;
+        }
+        const uint32_t a_src = smem_base + s * kStage, b_src = a_src + kABytes;
+        const int k_valid = k_end - k0;
+        if ((kAMn || kBMn) && k_valid < BK) {
+          // K rows beyond the end of the reduction: zero them (a K row is one 128-byte line per 64-wide box)
+          const int n_lines = BK - k_valid;
+          if (kAMn)
+            for (int j = 0; j < BM / 64; ++j)
+              for (int q = lane; q < n_lines * 8; q += 32)
+                *reinterpret_cast<uint4*>(smem_al + s * kStage + j * (BK * 128) + (k_valid + q / 8) * 128 + (q % 8) * 16) =
+                    make_uint4(0, 0, 0, 0);
+          if (kBMn)
+            for (int j = 0; j < BN / 64; ++j)
+              for (int q = lane; q < n_lines * 8; q += 32)
+                *reinterpret_cast<uint4*>(smem_al + s * kStage + kABytes + j * (BK * 128) + (k_valid + q / 8) * 128 +
+                                          (q % 8) * 16) = make_uint4(0, 0, 0, 0);
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+        }
+        ptx::tc_fence_after_sync();
+        if (lane == 0) {
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t adesc = kAMn ? ptx::smem_desc_sw128(a_src + k * 2048, BK * 128, 1024)
+                                        : ptx::smem_desc_sw128(a_src + k * 32, 16, 1024);
+            const uint64_t bdesc = kBMn ? ptx::smem_desc_sw128(b_src + k * 2048, BK * 128, 1024)
+                                        : ptx::smem_desc_sw128(b_src + k * 32, 16, 1024);
+            ptx::mma_bf16(tmem_d, adesc, bdesc, kIdesc, (first && k == 0) ? 0u : 1u);
+          }
+          ptx::mma_commit(empty_bar(s));
+        }
+        first = false;
         __syncwarp();
       }
-      ptx::tc_fence_after_sync();
-      if (lane == 0) {
-#pragma unroll
-        for (int k = 0; k < BK / 16; ++k) {
-          const uint64_t adesc = kAMn ? ptx::smem_desc_sw128(a_src + k * 2048, BK * 128, 1024)
-                                      : ptx::smem_desc_sw128(a_src + k * 32, 16, 1024);
-          const uint64_t bdesc = kBMn ? ptx::smem_desc_sw128(b_src + k * 2048, BK * 128, 1024)
-                                      : ptx::smem_desc_sw128(b_src + k * 32, 16, 1024);
-          ptx::mma_bf16(tmem_base, adesc, bdesc, kIdesc, (kb | k) != 0 ? 1u : 0u);
-        }
-        ptx::mma_commit(empty_bar(s));
-      }
-      issued_any = true;
-      __syncwarp();
+      if (lane == 0 && !first) ptx::mma_commit(tmem_full_bar(acc));
     }
-    if (lane == 0 && issued_any) ptx::mma_commit(tmem_full_bar);
-    if (*abort_flag && issued_any) ptx::mbar_wait(tmem_full_bar, 0);  // drain before TMEM is freed
   } else {
-    // ------------------------------------------------------------------ epilogue: TMEM -> registers -> global
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
-    if (__all_sync(0xffffffffu, ptx::mbar_wait(tmem_full_bar, 0) && !*abort_flag)) {
+    // ------------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;          // TMEM lane quarter this warp may read
+    const int et = threadIdx.x - 64; // 0..127 over the four epilogue warps, any order of quarters
+    int it = 0, tl = 0;
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++tl) {
+      if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
+      const TileCoord c = coord(tile);
+      int k_begin, k_end;
+      k_range(c.z, k_begin, k_end);
+      if (kColSum) {
+        // column sums of the dout tiles (A operand, MN-major: K row k of 64-wide box j is the 128-byte line
+        // at j*8192 + k*128, 16-byte chunks XOR-swizzled by k mod 8); thread et owns column m0 + et
+        float sum = 0.f;
+        for (int k0 = k_begin; k0 < k_end; k0 += BK, ++it) {
+          const int s = it % kStages;
+          bool ok = true;
+          if (c.n_t == 0 || et == 0) ok = ptx::mbar_wait(full_bar(s), (it / kStages) & 1);
+          if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+          if (c.n_t == 0) {
+            const int k_valid = (k_end - k0) < BK ? (k_end - k0) : BK;
+            const uint8_t* box = smem_al + s * kStage + (et >> 6) * (BK * 128);
+            const int ml = et & 63;
+            for (int k = 0; k < k_valid; ++k) {
+              const uint16_t raw = *reinterpret_cast<const uint16_t*>(box + k * 128 + (((ml >> 3) ^ (k & 7)) << 4) + (ml & 7) * 2);
+              sum += __uint_as_float((uint32_t)raw << 16);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");  // all four warps are done with this stage
+          }
+          if (et == 0) ptx::mbar_arrive(empty_bar(s));
+        }
+        if (c.n_t == 0 && c.m0 + et < M) colsum_part[(long long)c.z * M + c.m0 + et] = sum;
+      }
+      const int acc = tl & 1;
+      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(tmem_full_bar(acc), (tl >> 1) & 1) && !*abort_flag);
+      if (!ok) {
+        if (lane == 0) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+        break;
+      }
       ptx::tc_fence_after_sync();
-      const int row = m0 + q * 32 + lane;
-      OutT* orow = out + (long long)blockIdx.z * split_stride + (long long)row * ldo;
+      const int row = c.m0 + q * 32 + lane;
+      OutT* orow = out + (long long)c.z * split_stride + (long long)row * ldo;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int cc = 0; cc < BN / 32; ++cc) {
         uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, r);
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + cc * 32, r);
         ptx::tmem_ld_wait();
         if (row < M) {
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            const int col = n0 + c * 32 + g * 8;
+            const int col = c.n0 + cc * 32 + g * 8;
             if (col < N) {
               float v[8];
 #pragma unroll
@@ -251,15 +331,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       }
-    } else if (lane == 0) {
-      record_status(d_status, SPA_ERR_TIMEOUT);
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tmem_empty_bar(acc));  // this warp has drained its quarter of the accumulator
     }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, BN);
+    ptx::tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 
@@ -299,20 +380,26 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const i
 }
 
 // out[e] = sum over the splits that hold rows (in split order) of part[s][e]; zero if there are none.
+// Two arrays (the weight-gradient partials and, optionally, the bias-gradient partials) in one launch.
 __global__ void __launch_bounds__(256)
-split_reduce_kernel(const float* __restrict__ part, long long n, long long split_stride, int k_per_split,
-                    const int32_t* __restrict__ cu, int n_seg, int capacity, float* __restrict__ out) {
+split_reduce_kernel(const float* __restrict__ part, long long n, const float* __restrict__ part2, long long n2,
+                    int k_per_split, const int32_t* __restrict__ cu, int n_seg, int capacity, float* __restrict__ out,
+                    float* __restrict__ out2) {
   pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
   const int valid = (rows + k_per_split - 1) / k_per_split;
-  const long long n4 = n >> 2;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  const long long n4 = n >> 2, m4 = n2 >> 2;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4 + m4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const bool second = i >= n4;
+    const float* src = second ? part2 : part;
+    const long long stride = second ? n2 : n, j = second ? i - n4 : i;
+    float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int z = 0; z < valid; ++z) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(part + (long long)z * split_stride) + i);
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      const float4 v = __ldg(reinterpret_cast<const float4*>(src + (long long)z * stride) + j);
+      s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w;
     }
-    reinterpret_cast<float4*>(out)[i] = s;
+    reinterpret_cast<float4*>(second ? out2 : out)[j] = s4;
   }
 }
 
@@ -339,20 +426,23 @@ size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
   return w + (size_t)sp.splits * n_out * sizeof(float) + 256;
 }
 
-template <int BN, bool kAMn, bool kBMn, typename OutT>
+template <int BN, bool kAMn, bool kBMn, typename OutT, bool kColSum>
 int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloat16* bias, OutT* out, long long ldo,
                 long long split_stride, int M, int N, int K, const int32_t* cu, int n_seg, int capacity, int dyn_which,
-                int k_per_split, int splits, int32_t* d_status, cudaStream_t st, const char* what) {
-  auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT>;
+                int k_per_split, int splits, float* colsum_part, int32_t* d_status, cudaStream_t st, const char* what) {
+  auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT, kColSum>;
   static bool attr_set = false;  // per instantiation
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes<BN>());
     if (e != cudaSuccess) { set_cuda_error(e, what); return SPA_ERR_CUDA; }
     attr_set = true;
   }
-  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, splits);
-  launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu, n_seg,
-                                                         capacity, dyn_which, k_per_split, d_status);
+  // persistent grid: two CTAs per SM (99 KB of shared memory and 256 TMEM columns each), never more
+  // CTAs than there are tiles when every allocated row is in use
+  long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * splits;
+  const int grid = (int)(tiles < 2 * kNumSMs ? (tiles < 1 ? 1 : tiles) : 2 * kNumSMs);
+  launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu,
+             n_seg, capacity, dyn_which, k_per_split, colsum_part, d_status);
   SPA_CUDA_CHECK_LAUNCH(what);
   return SPA_OK;
 }
@@ -376,9 +466,10 @@ int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, cons
   if (!make_tmap_bf16_2d(&tmA, a, n_in, p.capacity, (uint64_t)n_in * 2, BK, BM) ||
       !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, BK, 128))
     return SPA_ERR_UNSUPPORTED;
-  return launch_gemm<128, false, false, __nv_bfloat16>(tmA, tmB, (const __nv_bfloat16*)bias, (__nv_bfloat16*)out, n_out,
-                                                       0, p.capacity, n_out, n_in, cu, p.B, p.capacity, 1, n_in, 1,
-                                                       d_status, st, "gemm_tc_kernel(fwd)");
+  return launch_gemm<128, false, false, __nv_bfloat16, false>(tmA, tmB, (const __nv_bfloat16*)bias,
+                                                              (__nv_bfloat16*)out, n_out, 0, p.capacity, n_out, n_in,
+                                                              cu, p.B, p.capacity, 1, n_in, 1, nullptr, d_status, st,
+                                                              "gemm_tc_kernel(fwd)");
 }
 
 int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
@@ -392,9 +483,9 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
                         !make_tmap_bf16_2d(&tmB2, a, n_in, p.capacity, (uint64_t)n_in * 2, 64, BK)))
     return SPA_ERR_UNSUPPORTED;
   if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
-    int rc = launch_gemm<128, false, true, __nv_bfloat16>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0, p.capacity,
-                                                          n_in, n_out, cu, p.B, p.capacity, 1, n_out, 1, d_status, st,
-                                                          "gemm_tc_kernel(dgrad)");
+    int rc = launch_gemm<128, false, true, __nv_bfloat16, false>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
+                                                                 p.capacity, n_in, n_out, cu, p.B, p.capacity, 1, n_out,
+                                                                 1, nullptr, d_status, st, "gemm_tc_kernel(dgrad)");
     if (rc != SPA_OK) return rc;
   }
   if (dW == nullptr && db == nullptr) return SPA_OK;
@@ -402,24 +493,31 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   float* part_w = reinterpret_cast<float*>(workspace);
   size_t off = ((size_t)sp.splits * n_out * n_in * sizeof(float) + 255) & ~(size_t)255;
   float* part_b = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + off);
-  if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]
-    int rc = launch_gemm<128, true, true, float>(tmA2, tmB2, nullptr, part_w, n_in, (long long)n_out * n_in, n_out, n_in,
-                                                 p.capacity, cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits,
-                                                 d_status, st, "gemm_tc_kernel(wgrad)");
+  const long long n_w = (long long)n_out * n_in;
+  if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]; db rides along as column sums of dout
+    int rc;
+    if (db != nullptr)
+      rc = launch_gemm<128, true, true, float, true>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity, cu,
+                                                     p.B, p.capacity, 2, sp.k_per_split, sp.splits, part_b, d_status, st,
+                                                     "gemm_tc_kernel(wgrad+colsum)");
+    else
+      rc = launch_gemm<128, true, true, float, false>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity,
+                                                      cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr,
+                                                      d_status, st, "gemm_tc_kernel(wgrad)");
     if (rc != SPA_OK) return rc;
-    const long long n = (long long)n_out * n_in;
-    int grid = (int)((n / 4 + 255) / 256);
+    const long long n_b = db != nullptr ? n_out : 0;
+    int grid = (int)(((n_w + n_b) / 4 + 255) / 256);
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
-    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n, n, sp.k_per_split, cu, p.B, p.capacity, dW);
-    SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(dW)");
-  }
-  if (db != nullptr) {
+    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.k_per_split, cu, p.B, p.capacity, dW,
+               db);
+    SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel");
+  } else {  // db alone
     dim3 grid((n_out + 63) / 64, sp.splits);
-    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity, sp.k_per_split,
-                                                part_b);
+    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity,
+               sp.k_per_split, part_b);
     SPA_CUDA_CHECK_LAUNCH("colsum_partial_kernel");
-    launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, part_b, n_out, n_out, sp.k_per_split, cu, p.B,
-                                                                 p.capacity, db);
+    launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, part_b, (long long)n_out, (const float*)nullptr,
+               0LL, sp.k_per_split, cu, p.B, p.capacity, db, (float*)nullptr);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
   }
   return SPA_OK;
