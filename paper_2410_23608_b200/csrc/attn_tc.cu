@@ -4,11 +4,13 @@
 // A CTA owns 128 consecutive packed query rows of one head, wherever image boundaries fall, and
 // walks the key range spanned by the segments of those rows in tiles of 128 keys; cu_seqlens alone
 // decides the range, so no padding token is ever loaded or multiplied.  Per key tile:
-//   S = Q K^T        tcgen05.mma, Q and K tiles staged by TMA (K/V double-buffered), S in TMEM (fp32)
-//   P = exp2(S - m)  one thread per query row reads its S row from TMEM, masks keys outside the
-//                    row's own segment, updates the running max / sum, writes P back to TMEM as bf16
+//   S = Q K^T        tcgen05.mma, Q and K tiles staged by TMA (K two tiles ahead, V one), S in TMEM (fp32)
+//   P = exp2(S - m)  one thread per query row pulls its S row into registers in one TMEM pass, masks keys
+//                    outside the row's own segment, updates the running max / sum, writes P back as bf16
 //   O_t = P V        tcgen05.mma with P read from TMEM and V from shared memory
 //   O = alpha O + O_t in registers (fp32), so TMEM never needs a rescaling pass.
+// The next tile's S product is issued as soon as every thread holds the current S row, so the tensor
+// core works under the softmax; the O tile is folded in one iteration late for the same reason.
 // K/V rows past the last valid packed row are unspecified memory: K columns are masked after the
 // product and V lines are zeroed in shared memory before the product.
 #include <math_constants.h>
@@ -66,8 +68,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   auto k_s = [&](int st) { return smem_base + kTile * (1 + 2 * st); };
   auto v_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
   const uint32_t bar_base = smem_base + 5 * kTile;
-  const uint32_t bar_q = bar_base, bar_s = bar_base + 24, bar_o = bar_base + 32;
-  auto bar_kv = [&](int st) { return bar_base + 8 + 8 * st; };
+  const uint32_t bar_q = bar_base, bar_s = bar_base + 40, bar_o = bar_base + 48;
+  auto bar_k = [&](int st) { return bar_base + 8 + 8 * st; };
+  auto bar_v = [&](int st) { return bar_base + 24 + 8 * st; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 5 * kTile + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 68);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 72);
@@ -82,8 +85,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   if (tid == 0) {
     ptx::prefetch_tensormap(&tm);
     ptx::mbar_init(bar_q, 1);
-    ptx::mbar_init(bar_kv(0), 1);
-    ptx::mbar_init(bar_kv(1), 1);
+    for (int s = 0; s < 2; ++s) { ptx::mbar_init(bar_k(s), 1); ptx::mbar_init(bar_v(s), 1); }
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_o, 1);
     *abort_flag = 0;
@@ -101,74 +103,92 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(kQ, kKV, false, false);
   constexpr uint32_t kIdescO = ptx::idesc_bf16_f32(kQ, D, false, true);
 
+  auto load_k = [&](int t) {
+    ptx::mbar_expect_tx(bar_k(t & 1), kTile);
+    ptx::tma_load_2d(k_s(t & 1), &tm, bar_k(t & 1), C + h * D, kv_lo + t * kKV);
+  };
+  auto load_v = [&](int t) {
+    ptx::mbar_expect_tx(bar_v(t & 1), kTile);
+    ptx::tma_load_2d(v_s(t & 1), &tm, bar_v(t & 1), 2 * C + h * D, kv_lo + t * kKV);
+  };
+  auto issue_qk = [&](int t) {  // S = Q K_t^T into TMEM; bar_s completes when it is done
+    bool ok = (t > 0) || ptx::mbar_wait(bar_q, 0);
+    ok = ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1) && ok;
+    if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; return; }
+    ptx::tc_fence_after_sync();
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(k_s(t & 1), k), kIdescS, k != 0 ? 1u : 0u);
+    ptx::mma_commit(bar_s);
+  };
+  int loads_k = 0, loads_v = 0;  // tiles whose loads thread 0 has issued
   if (tid == 0) {
     ptx::mbar_expect_tx(bar_q, kTile);
     ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
-    ptx::mbar_expect_tx(bar_kv(0), 2 * kTile);
-    ptx::tma_load_2d(k_s(0), &tm, bar_kv(0), C + h * D, kv_lo);
-    ptx::tma_load_2d(v_s(0), &tm, bar_kv(0), 2 * C + h * D, kv_lo);
+    load_k(0);
+    load_v(0);
+    loads_k = loads_v = 1;
+    if (n_tiles > 1) { load_k(1); loads_k = 2; }
+    issue_qk(0);
   }
 
   float o[D];
 #pragma unroll
   for (int e = 0; e < D; ++e) o[e] = 0.f;
-  float m = -CUDART_INF_F, l = 0.f;
-  int issued_kv = 1;  // tiles whose loads thread 0 has issued
+  float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
+  const unsigned span = (unsigned)(mine.hi - mine.lo);
+
+  // O = alpha O + (P V of tile t_prev), read from TMEM once that product has completed
+  auto fold_o = [&](int t_prev) {
+    if (!ptx::mbar_wait(bar_o, t_prev & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    ptx::tc_fence_after_sync();
+    uint32_t r[D];
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColO + c * 32, r + c * 32);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int e = 0; e < D; ++e) o[e] = fmaf(o[e], alpha_prev, __uint_as_float(r[e]));
+  };
 
   for (int t = 0; t < n_tiles; ++t) {
     const int st = t & 1;
     const int kv0 = kv_lo + t * kKV;
-    if (tid == 0) {
-      if (t + 1 < n_tiles) {  // the other stage is free: its P V product finished last iteration
-        ptx::mbar_expect_tx(bar_kv(st ^ 1), 2 * kTile);
-        ptx::tma_load_2d(k_s(st ^ 1), &tm, bar_kv(st ^ 1), C + h * D, kv0 + kKV);
-        ptx::tma_load_2d(v_s(st ^ 1), &tm, bar_kv(st ^ 1), 2 * C + h * D, kv0 + kKV);
-        issued_kv = t + 2;
-      }
-      bool ok = (t > 0) || ptx::mbar_wait(bar_q, 0);
-      ok = ok && ptx::mbar_wait(bar_kv(st), (t >> 1) & 1);
-      if (ok) {
-        ptx::tc_fence_after_sync();
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(k_s(st), k), kIdescS, k != 0 ? 1u : 0u);
-        ptx::mma_commit(bar_s);
-      } else {
-        record_status(d_status, SPA_ERR_TIMEOUT);
-        *abort_flag = 1;
-      }
-    }
-    // ---- softmax on this row of S
+    // ---- fold in the previous tile's P V (it was issued after this tile's S, so both are complete by then)
+    if (t > 0) fold_o(t - 1);
+    if (tid == 0 && t + 1 < n_tiles) { load_v(t + 1); loads_v = t + 2; }  // V stage of tile t-1 is free
+    // ---- S_t into registers: four TMEM loads in flight, one wait
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-    const unsigned span = (unsigned)(mine.hi - mine.lo);
-    float mt = -CUDART_INF_F;
-#pragma unroll 1
-    for (int c = 0; c < kKV / 32; ++c) {
-      uint32_t r[32];
-      ptx::tmem_ld_32x32(tmem + lane_base + kColS + c * 32, r);
-      ptx::tmem_ld_wait();
+    uint32_t s[kKV];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const bool valid = (unsigned)(kv0 + c * 32 + j - mine.lo) < span;
-        mt = fmaxf(mt, valid ? __uint_as_float(r[j]) * scale_log2e : -CUDART_INF_F);
-      }
+    for (int c = 0; c < kKV / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColS + c * 32, s + c * 32);
+    ptx::tmem_ld_wait();
+    if (tid == 0 && t + 2 < n_tiles) { load_k(t + 2); loads_k = t + 3; }  // K stage st is free: S_t is complete
+    ptx::tc_fence_before_sync();
+    __syncthreads();  // A: every thread holds its S row and has consumed the previous O tile
+    if (*abort_flag) break;
+    if (tid == 0 && t + 1 < n_tiles) issue_qk(t + 1);  // runs on the tensor core under the softmax below
+
+    // ---- masked online softmax of this row (exp2 domain)
+    float mt = -CUDART_INF_F;
+#pragma unroll
+    for (int j = 0; j < kKV; ++j) {
+      const bool valid = (unsigned)(kv0 + j - mine.lo) < span;
+      const float v = valid ? __uint_as_float(s[j]) * scale_log2e : -CUDART_INF_F;
+      s[j] = __float_as_uint(v);
+      mt = fmaxf(mt, v);
     }
     const float m_new = fmaxf(m, mt);
     const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
     const float alpha = ptx::ex2_approx(m - m_use);
     float rs = 0.f;
-#pragma unroll 1
+#pragma unroll
     for (int c = 0; c < kKV / 32; ++c) {
-      uint32_t r[32], pk[16];
-      ptx::tmem_ld_32x32(tmem + lane_base + kColS + c * 32, r);
-      ptx::tmem_ld_wait();
+      uint32_t pk[16];
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
-        const bool v0 = (unsigned)(kv0 + c * 32 + j - mine.lo) < span;
-        const bool v1 = (unsigned)(kv0 + c * 32 + j + 1 - mine.lo) < span;
-        const float p0 = v0 ? ptx::ex2_approx(__uint_as_float(r[j]) * scale_log2e - m_use) : 0.f;
-        const float p1 = v1 ? ptx::ex2_approx(__uint_as_float(r[j + 1]) * scale_log2e - m_use) : 0.f;
+        const float p0 = ptx::ex2_approx(__uint_as_float(s[c * 32 + j]) - m_use);  // masked entries: 2^-inf = 0
+        const float p1 = ptx::ex2_approx(__uint_as_float(s[c * 32 + j + 1]) - m_use);
         rs += p0 + p1;
         __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
         pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
@@ -178,10 +198,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     ptx::tmem_st_wait();
     l = l * alpha + rs;
     m = m_new;
+    alpha_prev = alpha;
     // ---- V lines past the last valid packed row must not reach the product
     if (kv0 + kKV > Np) {
-      ptx::mbar_wait(bar_kv(st), (t >> 1) & 1);  // already complete: K of this stage was consumed
-      const int first = Np - kv0;                // >= 1
+      if (!ptx::mbar_wait(bar_v(st), (t >> 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+      const int first = Np - kv0;  // >= 1
       constexpr int kChunks = HT::kRowBytes / 16;
       for (int c = tid; c < (kKV - first) * kChunks; c += kFwdThreads)
         *reinterpret_cast<uint4*>(smem_al + kTile * (2 + 2 * st) + (first + c / kChunks) * HT::kRowBytes +
@@ -189,26 +210,22 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       ptx::fence_proxy_async_smem();
     }
     ptx::tc_fence_before_sync();
-    __syncthreads();
+    __syncthreads();  // B: P_t is complete in TMEM
     if (*abort_flag) break;
     if (tid == 0) {
-      ptx::tc_fence_after_sync();
+      if (ptx::mbar_wait(bar_v(st), (t >> 1) & 1)) {
+        ptx::tc_fence_after_sync();
 #pragma unroll
-      for (int k = 0; k < kKV / 16; ++k)
-        ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(v_s(st), k), kIdescO, k != 0 ? 1u : 0u);
-      ptx::mma_commit(bar_o);
-    }
-    if (!ptx::mbar_wait(bar_o, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-    ptx::tc_fence_after_sync();
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t r[32];
-      ptx::tmem_ld_32x32(tmem + lane_base + kColO + c * 32, r);
-      ptx::tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) o[c * 32 + j] = fmaf(o[c * 32 + j], alpha, __uint_as_float(r[j]));
+        for (int k = 0; k < kKV / 16; ++k)
+          ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(v_s(st), k), kIdescO, k != 0 ? 1u : 0u);
+        ptx::mma_commit(bar_o);
+      } else {
+        record_status(d_status, SPA_ERR_TIMEOUT);
+        *abort_flag = 1;
+      }
     }
   }
+  if (!*abort_flag && n_tiles > 0) fold_o(n_tiles - 1);
 
   if (!*abort_flag && row < Np) {
     const float inv_l = 1.f / l;
@@ -223,7 +240,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     lse[(long long)h * capacity + row] = (m + log2f(l)) * 0.6931471805599453f;
   }
   if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
-    for (int t = issued_kv > 2 ? issued_kv - 2 : 0; t < issued_kv; ++t) ptx::mbar_wait(bar_kv(t & 1), (t >> 1) & 1);
+    for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
+    for (int t = loads_v > 2 ? loads_v - 2 : 0; t < loads_v; ++t) ptx::mbar_wait(bar_v(t & 1), (t >> 1) & 1);
+    ptx::mbar_wait(bar_q, 0);
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
