@@ -169,16 +169,18 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     if (*abort_flag) break;
     if (tid == 0 && t + 1 < n_tiles) issue_qk(t + 1);  // runs on the tensor core under the softmax below
 
-    // ---- masked online softmax of this row (exp2 domain)
+    // ---- masked online softmax of this row (exp2 domain).  Only tiles that straddle a boundary of the
+    // row's own segment pay for the mask; interior tiles cost one max, one fma, one ex2 and one add per key.
+    const bool interior = kv0 >= mine.lo && kv0 + kKV <= mine.hi;
+    if (!interior) {
+#pragma unroll
+      for (int j = 0; j < kKV; ++j)
+        if ((unsigned)(kv0 + j - mine.lo) >= span) s[j] = 0xff800000u;  // -inf
+    }
     float mt = -CUDART_INF_F;
 #pragma unroll
-    for (int j = 0; j < kKV; ++j) {
-      const bool valid = (unsigned)(kv0 + j - mine.lo) < span;
-      const float v = valid ? __uint_as_float(s[j]) * scale_log2e : -CUDART_INF_F;
-      s[j] = __float_as_uint(v);
-      mt = fmaxf(mt, v);
-    }
-    const float m_new = fmaxf(m, mt);
+    for (int j = 0; j < kKV; ++j) mt = fmaxf(mt, __uint_as_float(s[j]));
+    const float m_new = fmaxf(m, mt * scale_log2e);  // the scale is positive: max commutes with it
     const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
     const float alpha = ptx::ex2_approx(m - m_use);
     float rs = 0.f;
@@ -187,8 +189,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       uint32_t pk[16];
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
-        const float p0 = ptx::ex2_approx(__uint_as_float(s[c * 32 + j]) - m_use);  // masked entries: 2^-inf = 0
-        const float p1 = ptx::ex2_approx(__uint_as_float(s[c * 32 + j + 1]) - m_use);
+        const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j]), scale_log2e, -m_use));  // -inf -> 0
+        const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j + 1]), scale_log2e, -m_use));
         rs += p0 + p1;
         __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
         pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
