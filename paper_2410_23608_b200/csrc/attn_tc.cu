@@ -25,7 +25,7 @@ namespace {
 
 constexpr int kQ = 128;        // query rows per CTA = TMEM lanes
 constexpr int kKV = 128;       // keys per tile
-constexpr int kFwdThreads = 128;
+constexpr int kFwdThreads = 256;  // two threads per query row: each owns half of the key columns and half of d
 constexpr uint32_t kTmemCols = 256;  // S: 128 fp32 columns, P: 64 (bf16 pairs), O tile: up to 64
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
 
@@ -45,7 +45,7 @@ template <int D> struct HeadTile {
 };
 
 template <int D> __host__ __device__ constexpr int fwd_smem_bytes() {
-  return 5 * 128 * D * 2 + 1024 + 128;  // Q + 2 x (K, V), alignment slack, barriers
+  return 5 * 128 * D * 2 + 1024 + 128 + 2048;  // Q + 2 x (K, V), alignment slack, barriers, row-max exchange
 }
 
 template <int D>
@@ -60,6 +60,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   const int q0 = blockIdx.x * kQ;
   if (q0 >= Np) return;
   const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
+  // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 query rows and split
+  // the work of each row (key columns of S and P, head dimensions of O) in two halves
+  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -74,10 +77,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 5 * kTile + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 68);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 72);
+  float* xch = reinterpret_cast<float*>(smem_al + 5 * kTile + 128);  // [2 tile parities][2 halves][128 rows]
 
-  const int row = q0 + tid;
+  const int row = q0 + rl;
   const RowSeg mine = row_segment(seg, n_seg, Np, row);
-  {
+  if (half == 0) {
     const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
     if (row == q0) range[0] = mine.lo;
     if (row == last) range[1] = mine.hi;
@@ -96,7 +100,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;  // TMEM lanes this warp may touch
+  const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;  // TMEM lanes this warp may touch
+  constexpr int kCols = kKV / 2;  // key columns of each tile owned by this thread
+  constexpr int kDh = D / 2;      // head dimensions of O owned by this thread
+  const int col0 = half * kCols;
   const int kv_lo = range[0], kv_hi = range[1];
   const int n_tiles = (kv_hi - kv_lo + kKV - 1) / kKV;
 
@@ -132,9 +139,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     issue_qk(0);
   }
 
-  float o[D];
+  float o[kDh];
 #pragma unroll
-  for (int e = 0; e < D; ++e) o[e] = 0.f;
+  for (int e = 0; e < kDh; ++e) o[e] = 0.f;
   float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
   const unsigned span = (unsigned)(mine.hi - mine.lo);
 
@@ -142,12 +149,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   auto fold_o = [&](int t_prev) {
     if (!ptx::mbar_wait(bar_o, t_prev & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-    uint32_t r[D];
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColO + c * 32, r + c * 32);
+    uint32_t r[kDh];
+    if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + kColO + half * kDh, r);
+    else ptx::tmem_ld_32x16(tmem + lane_base + kColO + half * kDh, r);
     ptx::tmem_ld_wait();
 #pragma unroll
-    for (int e = 0; e < D; ++e) o[e] = fmaf(o[e], alpha_prev, __uint_as_float(r[e]));
+    for (int e = 0; e < kDh; ++e) o[e] = fmaf(o[e], alpha_prev, __uint_as_float(r[e]));
   };
 
   for (int t = 0; t < n_tiles; ++t) {
@@ -159,44 +166,53 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     // ---- S_t into registers: four TMEM loads in flight, one wait
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-    uint32_t s[kKV];
+    uint32_t s[kCols];
 #pragma unroll
-    for (int c = 0; c < kKV / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColS + c * 32, s + c * 32);
+    for (int c = 0; c < kCols / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColS + col0 + c * 32, s + c * 32);
     ptx::tmem_ld_wait();
+    // mask (boundary tiles only) and this half's row maximum, handed to the partner thread through shared memory
+    const int kc0 = kv0 + col0;
+    const bool interior = kc0 >= mine.lo && kc0 + kCols <= mine.hi;
+    if (!interior) {
+#pragma unroll
+      for (int j = 0; j < kCols; ++j)
+        if ((unsigned)(kc0 + j - mine.lo) >= span) s[j] = 0xff800000u;  // -inf
+    }
+    float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+    for (int j = 0; j < kCols; j += 4) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[j + u]));
+    }
+    float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+    xch[((t & 1) * 2 + half) * 128 + rl] = mt;
     if (tid == 0 && t + 2 < n_tiles) { load_k(t + 2); loads_k = t + 3; }  // K stage st is free: S_t is complete
     ptx::tc_fence_before_sync();
     __syncthreads();  // A: every thread holds its S row and has consumed the previous O tile
     if (*abort_flag) break;
     if (tid == 0 && t + 1 < n_tiles) issue_qk(t + 1);  // runs on the tensor core under the softmax below
 
-    // ---- masked online softmax of this row (exp2 domain).  Only tiles that straddle a boundary of the
-    // row's own segment pay for the mask; interior tiles cost one max, one fma, one ex2 and one add per key.
-    const bool interior = kv0 >= mine.lo && kv0 + kKV <= mine.hi;
-    if (!interior) {
-#pragma unroll
-      for (int j = 0; j < kKV; ++j)
-        if ((unsigned)(kv0 + j - mine.lo) >= span) s[j] = 0xff800000u;  // -inf
-    }
-    float mt = -CUDART_INF_F;
-#pragma unroll
-    for (int j = 0; j < kKV; ++j) mt = fmaxf(mt, __uint_as_float(s[j]));
+    // ---- online softmax of this half row (exp2 domain): one fma, one ex2 and one add per key
+    mt = fmaxf(mt, xch[((t & 1) * 2 + (half ^ 1)) * 128 + rl]);
     const float m_new = fmaxf(m, mt * scale_log2e);  // the scale is positive: max commutes with it
     const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
     const float alpha = ptx::ex2_approx(m - m_use);
-    float rs = 0.f;
+    float rs0 = 0.f, rs1 = 0.f;
 #pragma unroll
-    for (int c = 0; c < kKV / 32; ++c) {
+    for (int c = 0; c < kCols / 32; ++c) {
       uint32_t pk[16];
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
         const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j]), scale_log2e, -m_use));  // -inf -> 0
         const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j + 1]), scale_log2e, -m_use));
-        rs += p0 + p1;
+        rs0 += p0;
+        rs1 += p1;
         __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
         pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
       }
-      ptx::tmem_st_32x16(tmem + lane_base + kColP + c * 16, pk);
+      ptx::tmem_st_32x16(tmem + lane_base + kColP + (col0 >> 1) + c * 16, pk);
     }
+    const float rs = rs0 + rs1;
     ptx::tmem_st_wait();
     l = l * alpha + rs;
     m = m_new;
@@ -229,17 +245,21 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   }
   if (!*abort_flag && n_tiles > 0) fold_o(n_tiles - 1);
 
+  // the two halves of a row share the running max but kept separate sums: combine them
+  xch[half * 128 + rl] = l;
+  __syncthreads();
   if (!*abort_flag && row < Np) {
-    const float inv_l = 1.f / l;
-    __nv_bfloat16* dst = ao + (long long)row * C + h * D;
+    const float l_row = l + xch[(half ^ 1) * 128 + rl];
+    const float inv_l = 1.f / l_row;
+    __nv_bfloat16* dst = ao + (long long)row * C + h * D + half * kDh;
 #pragma unroll
-    for (int c = 0; c < D / 8; ++c) {
+    for (int c = 0; c < kDh / 8; ++c) {
       float v[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] = o[c * 8 + e] * inv_l;
       *reinterpret_cast<uint4*>(dst + c * 8) = Vec16<__nv_bfloat16>::from_float(v);
     }
-    lse[(long long)h * capacity + row] = (m + log2f(l)) * 0.6931471805599453f;
+    if (half == 0) lse[(long long)h * capacity + row] = (m + log2f(l_row)) * 0.6931471805599453f;
   }
   if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
     for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
