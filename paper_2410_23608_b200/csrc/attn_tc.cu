@@ -284,9 +284,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 // "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through two stages.  The
 // bf16 operand written back to TMEM aliases the first half of the fp32 tile it was computed from
 // (column group c of the result only covers columns already consumed).
-constexpr int kBwdThreads = 128;
+constexpr int kBwdThreads = 256;  // two threads per TMEM lane (row): each owns half of the columns
 constexpr uint32_t kBwdTmemCols = 512;
-constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320;
+constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320, kColOpA = 384, kColOpB = 448;
 
 template <int D> __host__ __device__ constexpr int bwd_smem_bytes() {
   return 6 * 128 * D * 2 + 1024 + 1024 + 128;  // 6 tiles, alignment slack, row statistics, barriers
@@ -306,6 +306,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const int r0 = blockIdx.x * 128;
   if (r0 >= Np) return;
   const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
+  // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
+  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
   const float scale_log2e = scale * kLog2e;
 
   extern __shared__ uint8_t smem_raw[];
@@ -323,9 +325,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 6 * kTile + 1024 + 68);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + 6 * kTile + 1024 + 72);
 
-  const int row = r0 + tid;
+  const int row = r0 + rl;
   const RowSeg mine = row_segment(seg, n_seg, Np, row);
-  {
+  if (half == 0) {
     const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
     if (row == r0) range[0] = mine.lo;
     if (row == last) range[1] = mine.hi;
@@ -346,7 +348,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
   const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
   const int n_tiles = (o_hi - o_lo + 127) / 128;
 
@@ -383,11 +385,11 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
         for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
       }
       my_lse = lse[(long long)h * capacity + row] * kLog2e;
-      delta[(long long)h * capacity + row] = my_D;
+      if (half == 0) delta[(long long)h * capacity + row] = my_D;
     }
   } else {
-    const int i = o_lo + tid;
-    if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
+    const int i = o_lo + rl;
+    if (half == 0 && i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
   }
 
   constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, 128, false, false);
@@ -399,10 +401,10 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     const int st = t & 1;
     const int y0 = o_lo + t * 128;
     if (tid == 0 && t + 1 < n_tiles) { load_other(st ^ 1, y0 + 128); issued = t + 2; }
-    if (!kDQ) {
-      stat_lse[tid] = nxt_lse;
-      stat_D[tid] = nxt_D;
-      const int i = y0 + 128 + tid;
+    if (!kDQ && half == 0) {
+      stat_lse[rl] = nxt_lse;
+      stat_D[rl] = nxt_D;
+      const int i = y0 + 128 + rl;
       nxt_lse = 0.f; nxt_D = 0.f;
       if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
     }
@@ -435,24 +437,34 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     }
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      uint32_t rs[32], rp[32], pk_p[16], pk_ds[16];
-      ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + c * 32, rs);
-      ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + c * 32, rp);
-      ptx::tmem_ld_wait();
+    // this thread's 64 columns of both fp32 tiles: four TMEM loads in flight, one wait
+    const int col0 = half * 64;
+    uint32_t rs[64], rp[64];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0 + c * 32, rs + c * 32);
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0 + c * 32, rp + c * 32);
+    }
+    ptx::tmem_ld_wait();
+    const int yc0 = y0 + col0;
+    if (!(yc0 >= mine.lo && yc0 + 64 <= mine.hi)) {  // a boundary of this row's segment crosses these columns
+#pragma unroll
+      for (int j = 0; j < 64; ++j)
+        if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t pk_p[16], pk_ds[16];
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
         float pv[2], dsv[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-          const int col = c * 32 + j + u;
-          const bool valid = (unsigned)(y0 + col - mine.lo) < span;
-          const float l2 = kDQ ? my_lse : stat_lse[col];
-          const float Dv = kDQ ? my_D : stat_D[col];
-          const float pe = ptx::ex2_approx(__uint_as_float(rs[j + u]) * scale_log2e - l2);
-          pv[u] = valid ? pe : 0.f;
-          dsv[u] = valid ? pe * (__uint_as_float(rp[j + u]) - Dv) : 0.f;
+          const int jj = c * 32 + j + u;
+          const float l2 = kDQ ? my_lse : stat_lse[col0 + jj];
+          const float Dv = kDQ ? my_D : stat_D[col0 + jj];
+          pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[jj]), scale_log2e, -l2));
+          dsv[u] = pv[u] * (__uint_as_float(rp[jj]) - Dv);
         }
         __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
         pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
@@ -461,12 +473,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
           pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
         }
       }
-      if (kDQ) {
-        ptx::tmem_st_32x16(tmem + lane_base + kColS1 + c * 16, pk_ds);   // dS over the consumed part of S
-      } else {
-        ptx::tmem_st_32x16(tmem + lane_base + kColS1 + c * 16, pk_p);    // P^T over S^T
-        ptx::tmem_st_32x16(tmem + lane_base + kColS2 + c * 16, pk_ds);   // dS^T over dP^T
-      }
+      const uint32_t pc = (uint32_t)(col0 >> 1) + c * 16;  // packed bf16 pairs: column pair index
+      if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColOpA + pc, pk_p);   // P^T (dK/dV pass only)
+      ptx::tmem_st_32x16(tmem + lane_base + kColOpB + pc, pk_ds);            // dS or dS^T
     }
     ptx::tmem_st_wait();
     ptx::tc_fence_before_sync();
@@ -477,14 +486,14 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       if (kDQ) {
 #pragma unroll
         for (int k = 0; k < 8; ++k)   // dQ += dS K
-          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS1 + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
+          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpB + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
       } else {
 #pragma unroll
         for (int k = 0; k < 8; ++k)   // dV += P^T dO
-          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS1 + k * 8, HT::mnmajor(y2_s(st), k), kIdescAcc, acc | (k != 0));
+          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpA + k * 8, HT::mnmajor(y2_s(st), k), kIdescAcc, acc | (k != 0));
 #pragma unroll
         for (int k = 0; k < 8; ++k)   // dK += dS^T Q
-          ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColS2 + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
+          ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColOpB + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
       }
       ptx::mma_commit(bar_o);
     }
@@ -494,20 +503,19 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
 
   if (!*abort_flag && n_tiles > 0) {
     const long long ld = 3LL * C;
-    auto store_acc = [&](uint32_t col0, __nv_bfloat16* dst, float mul) {
+    constexpr int kDh = D / 2;  // head dimensions stored by this thread
+    auto store_acc = [&](uint32_t acc_col, __nv_bfloat16* dst, float mul) {
+      uint32_t r[kDh];
+      if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + acc_col + half * kDh, r);
+      else ptx::tmem_ld_32x16(tmem + lane_base + acc_col + half * kDh, r);
+      ptx::tmem_ld_wait();
+      if (row < Np) {
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem + lane_base + col0 + c * 32, r);
-        ptx::tmem_ld_wait();
-        if (row < Np) {
+        for (int g = 0; g < kDh / 8; ++g) {
+          float v[8];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul;
-            *reinterpret_cast<uint4*>(dst + c * 32 + g * 8) = Vec16<__nv_bfloat16>::from_float(v);
-          }
+          for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul;
+          *reinterpret_cast<uint4*>(dst + half * kDh + g * 8) = Vec16<__nv_bfloat16>::from_float(v);
         }
       }
     };
