@@ -284,7 +284,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 // "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through two stages.  The
 // bf16 operand written back to TMEM aliases the first half of the fp32 tile it was computed from
 // (column group c of the result only covers columns already consumed).
-constexpr int kBwdThreads = 256;  // two threads per TMEM lane (row): each owns half of the columns
+constexpr int kBwdThreads = 512;  // four threads per TMEM lane (row): each owns a quarter of the columns
+constexpr int kBwdPc = 128 / (kBwdThreads / 128);  // fp32 columns of S / dP per thread
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320, kColOpA = 384, kColOpB = 448;
 
@@ -307,7 +308,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   if (r0 >= Np) return;
   const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
-  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
+  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);  // half: column part 0..3
   const float scale_log2e = scale * kLog2e;
 
   extern __shared__ uint8_t smem_raw[];
@@ -437,23 +438,24 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     }
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-    // this thread's 64 columns of both fp32 tiles: four TMEM loads in flight, one wait
-    const int col0 = half * 64;
-    uint32_t rs[64], rp[64];
+    // this thread's columns of both fp32 tiles: all TMEM loads in flight, one wait
+    constexpr int kPc = kBwdPc;
+    const int col0 = half * kPc;
+    uint32_t rs[kPc], rp[kPc];
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    for (int c = 0; c < kPc / 32; ++c) {
       ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0 + c * 32, rs + c * 32);
       ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0 + c * 32, rp + c * 32);
     }
     ptx::tmem_ld_wait();
     const int yc0 = y0 + col0;
-    if (!(yc0 >= mine.lo && yc0 + 64 <= mine.hi)) {  // a boundary of this row's segment crosses these columns
+    if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {  // a boundary of this row's segment crosses these columns
 #pragma unroll
-      for (int j = 0; j < 64; ++j)
+      for (int j = 0; j < kPc; ++j)
         if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
     }
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    for (int c = 0; c < kPc / 32; ++c) {
       uint32_t pk_p[16], pk_ds[16];
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
@@ -501,7 +503,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     ptx::tc_fence_after_sync();
   }
 
-  if (!*abort_flag && n_tiles > 0) {
+  if (!*abort_flag && n_tiles > 0 && half < 2) {  // two of the column parts drain the accumulators, d/2 columns each
     const long long ld = 3LL * C;
     constexpr int kDh = D / 2;  // head dimensions stored by this thread
     auto store_acc = [&](uint32_t acc_col, __nv_bfloat16* dst, float mul) {
