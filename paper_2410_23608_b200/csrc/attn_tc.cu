@@ -281,7 +281,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 //                dS = P (dP - D_i) written to TMEM as bf16,  dQ += dS K.  Also stores D_i = dO_i . O_i.
 //   kDQ = false: a CTA owns 128 key rows j; per query tile   S^T = K Q^T, dP^T = V dO^T,
 //                P^T and dS^T written to TMEM as bf16,       dV += P^T dO,  dK += dS^T Q.
-// "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through two stages.  The
+// "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through three stages.  The fp32
+// tiles of the next streamed tile are issued as soon as every thread holds the current ones in
+// registers, and the accumulating products of a tile run under the arithmetic of the next one.  The
 // bf16 operand written back to TMEM aliases the first half of the fp32 tile it was computed from
 // (column group c of the result only covers columns already consumed).
 constexpr int kBwdThreads = 512;  // four threads per TMEM lane (row): each owns a quarter of the columns
@@ -290,7 +292,7 @@ constexpr uint32_t kBwdTmemCols = 512;
 constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320, kColOpA = 384, kColOpB = 448;
 
 template <int D> __host__ __device__ constexpr int bwd_smem_bytes() {
-  return 6 * 128 * D * 2 + 1024 + 1024 + 128;  // 6 tiles, alignment slack, row statistics, barriers
+  return 8 * 128 * D * 2 + 1024 + 1024 + 128;  // 2 own + 3 x 2 streamed tiles, alignment slack, row statistics, barriers
 }
 
 template <int D, bool kDQ>
@@ -315,16 +317,17 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
+  constexpr int kYStages = 3;  // streamed tiles: one being multiplied, one staged for the next product, one in flight
   auto y1_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
   auto y2_s = [&](int st) { return smem_base + kTile * (3 + 2 * st); };
-  float* stat_lse = reinterpret_cast<float*>(smem_al + 6 * kTile);        // [128] lse_i * log2e of the staged query tile
+  float* stat_lse = reinterpret_cast<float*>(smem_al + 8 * kTile);        // [128] lse_i * log2e of the staged query tile
   float* stat_D = stat_lse + 128;                                         // [128] D_i
-  const uint32_t bar_base = smem_base + 6 * kTile + 1024;
-  const uint32_t bar_x = bar_base, bar_s = bar_base + 24, bar_o = bar_base + 32;
+  const uint32_t bar_base = smem_base + 8 * kTile + 1024;
+  const uint32_t bar_x = bar_base, bar_s = bar_base + 32, bar_o = bar_base + 40;
   auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 6 * kTile + 1024 + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 6 * kTile + 1024 + 68);
-  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 6 * kTile + 1024 + 72);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 8 * kTile + 1024 + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 8 * kTile + 1024 + 68);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 8 * kTile + 1024 + 72);
 
   const int row = r0 + rl;
   const RowSeg mine = row_segment(seg, n_seg, Np, row);
@@ -337,8 +340,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     ptx::prefetch_tensormap(&tm_qkv);
     ptx::prefetch_tensormap(&tm_do);
     ptx::mbar_init(bar_x, 1);
-    ptx::mbar_init(bar_y(0), 1);
-    ptx::mbar_init(bar_y(1), 1);
+    for (int s3 = 0; s3 < kYStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_o, 1);
     *abort_flag = 0;
@@ -356,7 +358,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   // column offsets inside qkv of the own / other operands
   const int x1_col = (kDQ ? 0 : C) + h * D;           // Q | K
   const int y1_col = (kDQ ? C : 0) + h * D;           // K | Q
-  auto load_other = [&](int st, int y0) {
+  auto load_other = [&](int t_) {  // tile t_ of the other side into stage t_ mod 3
+    const int st = t_ % kYStages, y0 = o_lo + t_ * 128;
     ptx::mbar_expect_tx(bar_y(st), 2 * kTile);
     ptx::tma_load_2d(y1_s(st), &tm_qkv, bar_y(st), y1_col, y0);
     if (kDQ) ptx::tma_load_2d(y2_s(st), &tm_qkv, bar_y(st), 2 * C + h * D, y0);   // V
@@ -367,7 +370,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
     if (kDQ) ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                    // dO
     else ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);               // V
-    load_other(0, o_lo);
+    load_other(0);
+    if (n_tiles > 1) load_other(1);
   }
 
   // per-row statistics of the query side
@@ -396,25 +400,17 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, 128, false, false);
   constexpr uint32_t kIdescAcc = ptx::idesc_bf16_f32(128, D, false, true);
   const unsigned span = (unsigned)(mine.hi - mine.lo);
-  int issued = 1;
+  int issued = n_tiles > 1 ? 2 : 1;  // streamed tiles whose loads thread 0 has issued
 
-  for (int t = 0; t < n_tiles; ++t) {
-    const int st = t & 1;
-    const int y0 = o_lo + t * 128;
-    if (tid == 0 && t + 1 < n_tiles) { load_other(st ^ 1, y0 + 128); issued = t + 2; }
-    if (!kDQ && half == 0) {
-      stat_lse[rl] = nxt_lse;
-      stat_D[rl] = nxt_D;
-      const int i = y0 + 128 + rl;
-      nxt_lse = 0.f; nxt_D = 0.f;
-      if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
-    }
-    // other-side lines past the last valid packed row must not reach a product
-    bool ok = ptx::mbar_wait(bar_y(st), (t >> 1) & 1);
-    if (t == 0) ok = ptx::mbar_wait(bar_x, 0) && ok;
+  // Lines of a streamed tile that lie past the last valid packed row are unspecified memory: zero them
+  // before any product sums over them.
+  auto wait_and_clean = [&](int t_) {
+    bool ok = ptx::mbar_wait(bar_y(t_ % kYStages), (t_ / kYStages) & 1);
+    if (t_ == 0) ok = ptx::mbar_wait(bar_x, 0) && ok;
     if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    const int y0 = o_lo + t_ * 128;
     if (y0 + 128 > Np) {
-      const int first = Np - y0;
+      const int first = Np - y0, st = t_ % kYStages;
       constexpr int kChunks = HT::kRowBytes / 16;
       for (int c = tid; c < (128 - first) * kChunks; c += kBwdThreads) {
         const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
@@ -423,24 +419,38 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       }
       ptx::fence_proxy_async_smem();
     }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    if (*abort_flag) break;
-    if (tid == 0) {
-      ptx::tc_fence_after_sync();
+  };
+  auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
+    const int st = t_ % kYStages;
+    ptx::tc_fence_after_sync();
 #pragma unroll
-      for (int k = 0; k < D / 16; ++k)
-        ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1_s(st), k), kIdescS, k != 0 ? 1u : 0u);
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1_s(st), k), kIdescS, k != 0 ? 1u : 0u);
 #pragma unroll
-      for (int k = 0; k < D / 16; ++k)
-        ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2_s(st), k), kIdescS, k != 0 ? 1u : 0u);
-      ptx::mma_commit(bar_s);
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2_s(st), k), kIdescS, k != 0 ? 1u : 0u);
+    ptx::mma_commit(bar_s);
+  };
+  wait_and_clean(0);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && !*abort_flag) issue_s(0);
+
+  constexpr int kPc = kBwdPc;
+  const int col0 = half * kPc;
+  for (int t = 0; t < n_tiles; ++t) {
+    const int st = t % kYStages;
+    const int y0 = o_lo + t * 128;
+    if (!kDQ && half == 0) {  // statistics of the query rows of tile t (rows of the staged tile = columns here)
+      stat_lse[rl] = nxt_lse;
+      stat_D[rl] = nxt_D;
+      const int i = y0 + 128 + rl;
+      nxt_lse = 0.f; nxt_D = 0.f;
+      if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
     }
+    // ---- this thread's columns of both fp32 tiles into registers
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-    // this thread's columns of both fp32 tiles: all TMEM loads in flight, one wait
-    constexpr int kPc = kBwdPc;
-    const int col0 = half * kPc;
     uint32_t rs[kPc], rp[kPc];
 #pragma unroll
     for (int c = 0; c < kPc / 32; ++c) {
@@ -448,40 +458,51 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0 + c * 32, rp + c * 32);
     }
     ptx::tmem_ld_wait();
+    if (t + 1 < n_tiles) wait_and_clean(t + 1);  // its load was issued a whole iteration ago
+    ptx::tc_fence_before_sync();
+    __syncthreads();  // A: both fp32 tiles are in registers, the next streamed tile is clean
+    if (*abort_flag) break;
+    if (tid == 0 && t + 1 < n_tiles) issue_s(t + 1);  // runs on the tensor core under the arithmetic below
+
+    // ---- P = 2^(S - lse), dS = P (dP - D): masked only where a boundary of this row's segment crosses
     const int yc0 = y0 + col0;
-    if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {  // a boundary of this row's segment crosses these columns
+    if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {
 #pragma unroll
       for (int j = 0; j < kPc; ++j)
         if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
     }
+    uint32_t pk_p[kPc / 2], pk_ds[kPc / 2];
+#pragma unroll
+    for (int j = 0; j < kPc; j += 2) {
+      float pv[2], dsv[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const float l2 = kDQ ? my_lse : stat_lse[col0 + j + u];
+        const float Dv = kDQ ? my_D : stat_D[col0 + j + u];
+        pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + u]), scale_log2e, -l2));
+        dsv[u] = pv[u] * (__uint_as_float(rp[j + u]) - Dv);
+      }
+      __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
+      pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
+      __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
+      pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+    }
+    // ---- the bf16 operand columns and the streamed stage of tile t-1 are free once its products are done
+    if (t > 0) {
+      if (!ptx::mbar_wait(bar_o, (t - 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+      ptx::tc_fence_after_sync();
+    }
+    if (tid == 0 && t + 2 < n_tiles) { load_other(t + 2); issued = t + 3; }
 #pragma unroll
     for (int c = 0; c < kPc / 32; ++c) {
-      uint32_t pk_p[16], pk_ds[16];
-#pragma unroll
-      for (int j = 0; j < 32; j += 2) {
-        float pv[2], dsv[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int jj = c * 32 + j + u;
-          const float l2 = kDQ ? my_lse : stat_lse[col0 + jj];
-          const float Dv = kDQ ? my_D : stat_D[col0 + jj];
-          pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[jj]), scale_log2e, -l2));
-          dsv[u] = pv[u] * (__uint_as_float(rp[jj]) - Dv);
-        }
-        __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
-        pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
-        if (!kDQ) {
-          __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
-          pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
-        }
-      }
       const uint32_t pc = (uint32_t)(col0 >> 1) + c * 16;  // packed bf16 pairs: column pair index
-      if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColOpA + pc, pk_p);   // P^T (dK/dV pass only)
-      ptx::tmem_st_32x16(tmem + lane_base + kColOpB + pc, pk_ds);            // dS or dS^T
+      if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColOpA + pc, pk_p + c * 16);   // P^T (dK/dV pass only)
+      ptx::tmem_st_32x16(tmem + lane_base + kColOpB + pc, pk_ds + c * 16);            // dS or dS^T
     }
     ptx::tmem_st_wait();
     ptx::tc_fence_before_sync();
-    __syncthreads();
+    __syncthreads();  // B: the bf16 operands of tile t are complete in TMEM
+    if (*abort_flag) break;
     if (tid == 0) {
       ptx::tc_fence_after_sync();
       const uint32_t acc = (t != 0) ? 1u : 0u;
@@ -499,7 +520,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       }
       ptx::mma_commit(bar_o);
     }
-    if (!ptx::mbar_wait(bar_o, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+  }
+  if (!*abort_flag && n_tiles > 0) {
+    if (!ptx::mbar_wait(bar_o, (n_tiles - 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
   }
 
@@ -530,7 +553,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     }
   }
   if (*abort_flag && tid == 0) {
-    for (int t = issued > 2 ? issued - 2 : 0; t < issued; ++t) ptx::mbar_wait(bar_y(t & 1), (t >> 1) & 1);
+    for (int t = issued > kYStages ? issued - kYStages : 0; t < issued; ++t)
+      ptx::mbar_wait(bar_y(t % kYStages), (t / kYStages) & 1);
     ptx::mbar_wait(bar_x, 0);
   }
   ptx::tc_fence_before_sync();
