@@ -281,7 +281,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 //                dS = P (dP - D_i) written to TMEM as bf16,  dQ += dS K.  Also stores D_i = dO_i . O_i.
 //   kDQ = false: a CTA owns 128 key rows j; per query tile   S^T = K Q^T, dP^T = V dO^T,
 //                P^T and dS^T written to TMEM as bf16,       dV += P^T dO,  dK += dS^T Q.
-// "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through three stages.  The fp32
+// "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through four stages.  The fp32
 // tiles of the next streamed tile are issued as soon as every thread holds the current ones in
 // registers, and the accumulating products of a tile run under the arithmetic of the next one.  The
 // bf16 operand written back to TMEM aliases the first half of the fp32 tile it was computed from
@@ -292,7 +292,7 @@ constexpr uint32_t kBwdTmemCols = 512;
 constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320, kColOpA = 384, kColOpB = 448;
 
 template <int D> __host__ __device__ constexpr int bwd_smem_bytes() {
-  return 8 * 128 * D * 2 + 1024 + 1024 + 128;  // 2 own + 3 x 2 streamed tiles, alignment slack, row statistics, barriers
+  return 10 * 128 * D * 2 + 1024 + 1024 + 128;  // 2 own + 4 x 2 streamed tiles, alignment slack, row statistics, barriers
 }
 
 template <int D, bool kDQ>
@@ -317,17 +317,17 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
-  constexpr int kYStages = 3;  // streamed tiles: one being multiplied, one staged for the next product, one in flight
+  constexpr int kYStages = 4;  // streamed tiles: one being multiplied, one staged for the next product, two in flight
   auto y1_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
   auto y2_s = [&](int st) { return smem_base + kTile * (3 + 2 * st); };
-  float* stat_lse = reinterpret_cast<float*>(smem_al + 8 * kTile);        // [128] lse_i * log2e of the staged query tile
+  float* stat_lse = reinterpret_cast<float*>(smem_al + 10 * kTile);       // [128] lse_i * log2e of the staged query tile
   float* stat_D = stat_lse + 128;                                         // [128] D_i
-  const uint32_t bar_base = smem_base + 8 * kTile + 1024;
-  const uint32_t bar_x = bar_base, bar_s = bar_base + 32, bar_o = bar_base + 40;
+  const uint32_t bar_base = smem_base + 10 * kTile + 1024;
+  const uint32_t bar_x = bar_base, bar_s = bar_base + 40, bar_o = bar_base + 48;
   auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 8 * kTile + 1024 + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 8 * kTile + 1024 + 68);
-  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 8 * kTile + 1024 + 72);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 10 * kTile + 1024 + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 10 * kTile + 1024 + 68);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 10 * kTile + 1024 + 72);
 
   const int row = r0 + rl;
   const RowSeg mine = row_segment(seg, n_seg, Np, row);
@@ -372,6 +372,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     else ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);               // V
     load_other(0);
     if (n_tiles > 1) load_other(1);
+    if (n_tiles > 2) load_other(2);
   }
 
   // per-row statistics of the query side
@@ -400,7 +401,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, 128, false, false);
   constexpr uint32_t kIdescAcc = ptx::idesc_bf16_f32(128, D, false, true);
   const unsigned span = (unsigned)(mine.hi - mine.lo);
-  int issued = n_tiles > 1 ? 2 : 1;  // streamed tiles whose loads thread 0 has issued
+  int issued = n_tiles > 2 ? 3 : n_tiles;  // streamed tiles whose loads thread 0 has issued
 
   // Lines of a streamed tile that lie past the last valid packed row are unspecified memory: zero them
   // before any product sums over them.
@@ -492,7 +493,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       if (!ptx::mbar_wait(bar_o, (t - 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
       ptx::tc_fence_after_sync();
     }
-    if (tid == 0 && t + 2 < n_tiles) { load_other(t + 2); issued = t + 3; }
+    if (tid == 0 && t + 3 < n_tiles) { load_other(t + 3); issued = t + 4; }  // into the stage of tile t-1
 #pragma unroll
     for (int c = 0; c < kPc / 32; ++c) {
       const uint32_t pc = (uint32_t)(col0 >> 1) + c * 16;  // packed bf16 pairs: column pair index
