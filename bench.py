@@ -41,6 +41,22 @@ def peaks():
     return dict(hbm=6650.0, tensor=1590.0, source="fallback")
 
 
+def measured_traffic(workload, unit):
+    """DRAM bytes per launch of `unit` from the committed ncu summary, or None when there is no figure
+    or the kernel's source has changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", f"traffic_{workload}.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        parts = line.split()
+        if len(parts) == 4 and parts[0] == unit:
+            src = os.path.join(ROOT, "paper_2410_23608_b200", "csrc", parts[2])
+            if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] == parts[3]:
+                return int(parts[1])
+    return None
+
+
 # ----------------------------------------------------------------------------- work model
 def work_model(cfg, cu):
     """Algorithmic bytes and FLOPs of every call for the realised selection (FLOPs = 2 x MACs)."""
@@ -375,7 +391,9 @@ def main():
     top = max(call_ms, key=call_ms.get)
     tr = per_call[top]
     roofline = {"kernel": top, "bound": tr["bound"], "achieved": tr["achieved"], "peak": pk[tr["bound"]],
-                "unit": "TFLOP/s" if tr["bound"] == "tensor" else "GB/s", "frac": tr["frac"], "traffic": None,
+                "unit": "TFLOP/s" if tr["bound"] == "tensor" else "GB/s", "frac": tr["frac"],
+                "traffic": measured_traffic(cfg.name, top), "algorithmic_bytes": work[top]["bytes"],
+                "algorithmic_flops": work[top]["flops"],
                 "peak_source": pk["source"], "us_per_launch": tr["us"]}
 
     # ---- forward-only time (same rotation), reported beside the headline
