@@ -57,9 +57,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
   const int Np = packed_rows(seg, n_seg, capacity);
-  const int q0 = blockIdx.x * kQ;
+  const int q0 = blockIdx.y * kQ;  // grid = (heads, tiles): CTAs past the last valid tile are dispatched last
   if (q0 >= Np) return;
-  const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
+  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 query rows and split
   // the work of each row (key columns of S and P, head dimensions of O) in two halves
   const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
@@ -306,9 +306,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   constexpr int kTile = HT::kTileBytes;
   constexpr float kLog2e = 1.4426950408889634f;
   const int Np = packed_rows(seg, n_seg, capacity);
-  const int r0 = blockIdx.x * 128;
+  const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
   if (r0 >= Np) return;
-  const int h = blockIdx.y, tid = threadIdx.x, warp = tid >> 5;
+  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
   const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);  // half: column part 0..3
   const float scale_log2e = scale * kLog2e;
@@ -583,7 +583,7 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
     attr_set = true;
   }
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
-  dim3 grid((p.capacity + 127) / 128, p.H);
+  dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
   launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
                                                     lse, delta, seg, n_seg, p.capacity, p.C, scale,
@@ -608,7 +608,7 @@ int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_s
     if (e != cudaSuccess) { set_cuda_error(e, "attn_fwd_tc_kernel"); return SPA_ERR_CUDA; }
     attr_set = true;
   }
-  dim3 grid((p.capacity + kQ - 1) / kQ, p.H);
+  dim3 grid(p.H, (p.capacity + kQ - 1) / kQ);
   launch_pdl(kern, grid, kFwdThreads, fwd_smem_bytes<D>(), st, tm, seg, n_seg, p.capacity, p.C,
                                                       softmax_scale_of(p) * 1.4426950408889634f,
                                                       (__nv_bfloat16*)ao, lse, d_status);
