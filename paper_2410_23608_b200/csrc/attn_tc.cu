@@ -275,59 +275,65 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 }
 
 // ------------------------------------------------------------------------------------------------
-// Backward.  Two passes over the same tile machinery, each accumulating its outputs in TMEM over the
-// whole loop, so that no sum is split across CTAs (no float atomics, bitwise reproducible):
-//   kDQ = true : a CTA owns 128 query rows i; per key tile   S = Q K^T, dP = dO V^T,
-//                dS = P (dP - D_i) written to TMEM as bf16,  dQ += dS K.  Also stores D_i = dO_i . O_i.
-//   kDQ = false: a CTA owns 128 key rows j; per query tile   S^T = K Q^T, dP^T = V dO^T,
-//                P^T and dS^T written to TMEM as bf16,       dV += P^T dO,  dK += dS^T Q.
-// "own" tiles (X1, X2) are loaded once, "other" tiles (Y1, Y2) stream through four stages.  The fp32
-// tiles of the next streamed tile are issued as soon as every thread holds the current ones in
-// registers, and the accumulating products of a tile run under the arithmetic of the next one.  The
-// bf16 operand written back to TMEM aliases the first half of the fp32 tile it was computed from
-// (column group c of the result only covers columns already consumed).
-constexpr int kBwdThreads = 512;  // four threads per TMEM lane (row): each owns a quarter of the columns
-constexpr int kBwdPc = 128 / (kBwdThreads / 128);  // fp32 columns of S / dP per thread
-constexpr uint32_t kBwdTmemCols = 512;
-constexpr uint32_t kColS1 = 0, kColS2 = 128, kColAcc1 = 256, kColAcc2 = 320, kColOpA = 384, kColOpB = 448;
+// Backward.
+// Two passes over the same tile machinery, each accumulating its outputs in TMEM over its whole loop, so
+// that no sum is split across CTAs (no float atomics, bitwise reproducible):
+//   kDQ = true : a CTA owns 128 query rows i; per streamed tile of 64 keys   S = Q K^T, dP = dO V^T,
+//                dS = P (dP - D_i) written to TMEM as bf16,   dQ += dS K.   Also stores D_i = dO_i . O_i.
+//   kDQ = false: a CTA owns 128 key rows j; per streamed tile of 64 queries  S^T = K Q^T, dP^T = V dO^T,
+//                P^T and dS^T written to TMEM as bf16,        dV += P^T dO,  dK += dS^T Q.
+// The footprint is kept to 256 TMEM columns and about 80 KB of shared memory so that two CTAs share an
+// SM: one CTA's arithmetic runs under the other's MMA round trips and prologue.  To fit, the streamed
+// tiles are 64 rows, and the bf16 operands (P^T, dS) are written over the first half of the fp32 tiles
+// they were computed from - after a barrier, once every thread holds its fp32 columns in registers.
+// MMAs execute in issue order, so the next tile's fp32 products (which overwrite those columns) are
+// simply issued behind the accumulating products that read them.
+constexpr int kBwdThreads = 256;   // two threads per TMEM lane (row): each owns 32 of the 64 streamed columns
+constexpr int kBwdY = 64;          // rows of a streamed tile
+constexpr int kBwdStages = 3;      // streamed tiles in shared memory
+constexpr uint32_t kBwdTmemCols = 256;
+constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;  // operands alias S1 / S2 columns [0, 32)
 
 template <int D> __host__ __device__ constexpr int bwd_smem_bytes() {
-  return 10 * 128 * D * 2 + 1024 + 1024 + 128;  // 2 own + 4 x 2 streamed tiles, alignment slack, row statistics, barriers
+  return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128;  // own, streamed, slack, statistics, barriers
 }
 
 template <int D, bool kDQ>
 __global__ void __launch_bounds__(kBwdThreads)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
+                   const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __nv_bfloat16* __restrict__ ao, const __nv_bfloat16* __restrict__ dao,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
                    int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
   pdl_entry();
   using HT = HeadTile<D>;
-  constexpr int kTile = HT::kTileBytes;
+  constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
+  constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
   constexpr float kLog2e = 1.4426950408889634f;
   const int Np = packed_rows(seg, n_seg, capacity);
   const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
   if (r0 >= Np) return;
   const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
-  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);  // half: column part 0..3
+  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
   const float scale_log2e = scale * kLog2e;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
-  constexpr int kYStages = 4;  // streamed tiles: one being multiplied, one staged for the next product, two in flight
-  auto y1_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
-  auto y2_s = [&](int st) { return smem_base + kTile * (3 + 2 * st); };
-  float* stat_lse = reinterpret_cast<float*>(smem_al + 10 * kTile);       // [128] lse_i * log2e of the staged query tile
-  float* stat_D = stat_lse + 128;                                         // [128] D_i
-  const uint32_t bar_base = smem_base + 10 * kTile + 1024;
+  constexpr int kYBase = 2 * kTile;
+  auto y1_off = [&](int st) { return kYBase + kYTile * (2 * st); };
+  auto y2_off = [&](int st) { return kYBase + kYTile * (2 * st + 1); };
+  constexpr int kStatBase = kYBase + kBwdStages * 2 * kYTile;
+  float* stat_lse = reinterpret_cast<float*>(smem_al + kStatBase);  // [2][64] lse_i * log2e of the staged query tile
+  float* stat_D = stat_lse + 2 * kBwdY;                              // [2][64] D_i
+  const uint32_t bar_base = smem_base + kStatBase + 1024;
   const uint32_t bar_x = bar_base, bar_s = bar_base + 40, bar_o = bar_base + 48;
   auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 10 * kTile + 1024 + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 10 * kTile + 1024 + 68);
-  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 10 * kTile + 1024 + 72);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kStatBase + 1024 + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 68);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 72);
 
   const int row = r0 + rl;
   const RowSeg mine = row_segment(seg, n_seg, Np, row);
@@ -339,8 +345,10 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   if (tid == 0) {
     ptx::prefetch_tensormap(&tm_qkv);
     ptx::prefetch_tensormap(&tm_do);
+    ptx::prefetch_tensormap(&tm_qkv_y);
+    ptx::prefetch_tensormap(&tm_do_y);
     ptx::mbar_init(bar_x, 1);
-    for (int s3 = 0; s3 < kYStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
+    for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_o, 1);
     *abort_flag = 0;
@@ -353,31 +361,30 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const uint32_t tmem = *tmem_slot;
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
   const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
-  const int n_tiles = (o_hi - o_lo + 127) / 128;
+  const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
 
-  // column offsets inside qkv of the own / other operands
+  // column offsets inside qkv of the own / streamed operands
   const int x1_col = (kDQ ? 0 : C) + h * D;           // Q | K
   const int y1_col = (kDQ ? C : 0) + h * D;           // K | Q
-  auto load_other = [&](int t_) {  // tile t_ of the other side into stage t_ mod 3
-    const int st = t_ % kYStages, y0 = o_lo + t_ * 128;
-    ptx::mbar_expect_tx(bar_y(st), 2 * kTile);
-    ptx::tma_load_2d(y1_s(st), &tm_qkv, bar_y(st), y1_col, y0);
-    if (kDQ) ptx::tma_load_2d(y2_s(st), &tm_qkv, bar_y(st), 2 * C + h * D, y0);   // V
-    else ptx::tma_load_2d(y2_s(st), &tm_do, bar_y(st), h * D, y0);                // dO
+  auto load_other = [&](int t_) {  // streamed tile t_ into stage t_ mod kBwdStages
+    const int st = t_ % kBwdStages, y0 = o_lo + t_ * kBwdY;
+    ptx::mbar_expect_tx(bar_y(st), 2 * kYTile);
+    ptx::tma_load_2d(smem_base + y1_off(st), &tm_qkv_y, bar_y(st), y1_col, y0);
+    if (kDQ) ptx::tma_load_2d(smem_base + y2_off(st), &tm_qkv_y, bar_y(st), 2 * C + h * D, y0);   // V
+    else ptx::tma_load_2d(smem_base + y2_off(st), &tm_do_y, bar_y(st), h * D, y0);                // dO
   };
+  int issued = 0;  // streamed tiles whose loads thread 0 has issued
   if (tid == 0) {
     ptx::mbar_expect_tx(bar_x, 2 * kTile);
     ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
     if (kDQ) ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                    // dO
     else ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);               // V
-    load_other(0);
-    if (n_tiles > 1) load_other(1);
-    if (n_tiles > 2) load_other(2);
+    for (int t_ = 0; t_ < n_tiles && t_ < 2; ++t_) load_other(t_);
+    issued = n_tiles < 2 ? n_tiles : 2;
   }
-
   // per-row statistics of the query side
   float my_lse = 0.f, my_D = 0.f;   // kDQ: this thread's query row
-  float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next staged query tile, row tid
+  float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next streamed query tile, row rl < 64
   if (kDQ) {
     if (row < Np) {
       const __nv_bfloat16* orow = ao + (long long)row * C + h * D;
@@ -393,77 +400,75 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       my_lse = lse[(long long)h * capacity + row] * kLog2e;
       if (half == 0) delta[(long long)h * capacity + row] = my_D;
     }
-  } else {
+  } else if (half == 0 && rl < kBwdY) {
     const int i = o_lo + rl;
-    if (half == 0 && i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
+    if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
   }
 
-  constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, 128, false, false);
+  constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, kBwdY, false, false);
   constexpr uint32_t kIdescAcc = ptx::idesc_bf16_f32(128, D, false, true);
   const unsigned span = (unsigned)(mine.hi - mine.lo);
-  int issued = n_tiles > 2 ? 3 : n_tiles;  // streamed tiles whose loads thread 0 has issued
 
-  // Lines of a streamed tile that lie past the last valid packed row are unspecified memory: zero them
-  // before any product sums over them.
-  auto wait_and_clean = [&](int t_) {
-    bool ok = ptx::mbar_wait(bar_y(t_ % kYStages), (t_ / kYStages) & 1);
+  // Make streamed tile t_ ready for the products: its load has landed, lines past the last valid packed row
+  // are zeroed (they are unspecified memory and would be summed over), its query statistics are staged.
+  auto prep = [&](int t_) {
+    const int st = t_ % kBwdStages;
+    bool ok = ptx::mbar_wait(bar_y(st), (t_ / kBwdStages) & 1);
     if (t_ == 0) ok = ptx::mbar_wait(bar_x, 0) && ok;
     if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-    const int y0 = o_lo + t_ * 128;
-    if (y0 + 128 > Np) {
-      const int first = Np - y0, st = t_ % kYStages;
+    const int y0 = o_lo + t_ * kBwdY;
+    if (y0 + kBwdY > Np) {
+      const int first = Np - y0;
       constexpr int kChunks = HT::kRowBytes / 16;
-      for (int c = tid; c < (128 - first) * kChunks; c += kBwdThreads) {
+      for (int c = tid; c < (kBwdY - first) * kChunks; c += kBwdThreads) {
         const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
-        *reinterpret_cast<uint4*>(smem_al + kTile * (2 + 2 * st) + off) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(smem_al + kTile * (3 + 2 * st) + off) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(smem_al + y1_off(st) + off) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(smem_al + y2_off(st) + off) = make_uint4(0, 0, 0, 0);
       }
       ptx::fence_proxy_async_smem();
     }
-  };
-  auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
-    const int st = t_ % kYStages;
-    ptx::tc_fence_after_sync();
-#pragma unroll
-    for (int k = 0; k < D / 16; ++k)
-      ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1_s(st), k), kIdescS, k != 0 ? 1u : 0u);
-#pragma unroll
-    for (int k = 0; k < D / 16; ++k)
-      ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2_s(st), k), kIdescS, k != 0 ? 1u : 0u);
-    ptx::mma_commit(bar_s);
-  };
-  wait_and_clean(0);
-  ptx::tc_fence_before_sync();
-  __syncthreads();
-  if (tid == 0 && !*abort_flag) issue_s(0);
-
-  constexpr int kPc = kBwdPc;
-  const int col0 = half * kPc;
-  for (int t = 0; t < n_tiles; ++t) {
-    const int st = t % kYStages;
-    const int y0 = o_lo + t * 128;
-    if (!kDQ && half == 0) {  // statistics of the query rows of tile t (rows of the staged tile = columns here)
-      stat_lse[rl] = nxt_lse;
-      stat_D[rl] = nxt_D;
-      const int i = y0 + 128 + rl;
+    if (!kDQ && half == 0 && rl < kBwdY) {
+      stat_lse[(t_ & 1) * kBwdY + rl] = nxt_lse;
+      stat_D[(t_ & 1) * kBwdY + rl] = nxt_D;
+      const int i = y0 + kBwdY + rl;
       nxt_lse = 0.f; nxt_D = 0.f;
       if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
     }
-    // ---- this thread's columns of both fp32 tiles into registers
+  };
+  auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
+    const int st = t_ % kBwdStages;
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(smem_base + y1_off(st), k), kIdescS, k != 0 ? 1u : 0u);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(smem_base + y2_off(st), k), kIdescS, k != 0 ? 1u : 0u);
+    ptx::mma_commit(bar_s);
+  };
+
+  prep(0);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && !*abort_flag) { ptx::tc_fence_after_sync(); issue_s(0); }
+
+  constexpr int kPc = kBwdY / 2;  // fp32 columns of each tile owned by this thread
+  const int col0 = half * kPc;
+  bool dead = false;
+  for (int t = 0; t < n_tiles; ++t) {
+    const int st = t % kBwdStages;
+    const int y0 = o_lo + t * kBwdY;
+    // ---- this thread's columns of both fp32 tiles into registers.  bar_s also covers the accumulating
+    // products of tile t-1 (commits are in issue order), so its streamed stage is free again.
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
+    if (tid == 0 && t + 2 < n_tiles) { load_other(t + 2); issued = t + 3; }
     uint32_t rs[kPc], rp[kPc];
-#pragma unroll
-    for (int c = 0; c < kPc / 32; ++c) {
-      ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0 + c * 32, rs + c * 32);
-      ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0 + c * 32, rp + c * 32);
-    }
+    ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0, rs);
+    ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0, rp);
     ptx::tmem_ld_wait();
-    if (t + 1 < n_tiles) wait_and_clean(t + 1);  // its load was issued a whole iteration ago
     ptx::tc_fence_before_sync();
-    __syncthreads();  // A: both fp32 tiles are in registers, the next streamed tile is clean
-    if (*abort_flag) break;
-    if (tid == 0 && t + 1 < n_tiles) issue_s(t + 1);  // runs on the tensor core under the arithmetic below
+    __syncthreads();  // A: every thread holds its fp32 columns; their TMEM columns may now take the bf16 operands
+    if (*abort_flag) { dead = true; break; }
 
     // ---- P = 2^(S - lse), dS = P (dP - D): masked only where a boundary of this row's segment crosses
     const int yc0 = y0 + col0;
@@ -473,13 +478,15 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
         if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
     }
     uint32_t pk_p[kPc / 2], pk_ds[kPc / 2];
+    const float* sl = stat_lse + (t & 1) * kBwdY + col0;
+    const float* sd = stat_D + (t & 1) * kBwdY + col0;
 #pragma unroll
     for (int j = 0; j < kPc; j += 2) {
       float pv[2], dsv[2];
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
-        const float l2 = kDQ ? my_lse : stat_lse[col0 + j + u];
-        const float Dv = kDQ ? my_D : stat_D[col0 + j + u];
+        const float l2 = kDQ ? my_lse : sl[j + u];
+        const float Dv = kDQ ? my_D : sd[j + u];
         pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + u]), scale_log2e, -l2));
         dsv[u] = pv[u] * (__uint_as_float(rp[j + u]) - Dv);
       }
@@ -488,48 +495,41 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
       pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
     }
-    // ---- the bf16 operand columns and the streamed stage of tile t-1 are free once its products are done
-    if (t > 0) {
-      if (!ptx::mbar_wait(bar_o, (t - 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-      ptx::tc_fence_after_sync();
-    }
-    if (tid == 0 && t + 3 < n_tiles) { load_other(t + 3); issued = t + 4; }  // into the stage of tile t-1
-#pragma unroll
-    for (int c = 0; c < kPc / 32; ++c) {
-      const uint32_t pc = (uint32_t)(col0 >> 1) + c * 16;  // packed bf16 pairs: column pair index
-      if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColOpA + pc, pk_p + c * 16);   // P^T (dK/dV pass only)
-      ptx::tmem_st_32x16(tmem + lane_base + kColOpB + pc, pk_ds + c * 16);            // dS or dS^T
-    }
+    if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColS1 + (col0 >> 1), pk_p);   // P^T over the consumed S^T
+    ptx::tmem_st_32x16(tmem + lane_base + kColS2 + (col0 >> 1), pk_ds);            // dS (or dS^T) over the consumed dP
     ptx::tmem_st_wait();
+    if (t + 1 < n_tiles) prep(t + 1);
     ptx::tc_fence_before_sync();
-    __syncthreads();  // B: the bf16 operands of tile t are complete in TMEM
-    if (*abort_flag) break;
+    __syncthreads();  // B: the bf16 operands of tile t are complete, tile t+1 is ready
+    if (*abort_flag) { dead = true; break; }
     if (tid == 0) {
       ptx::tc_fence_after_sync();
       const uint32_t acc = (t != 0) ? 1u : 0u;
+      const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
       if (kDQ) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k)   // dQ += dS K
-          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpB + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
+        for (int k = 0; k < kBwdY / 16; ++k)   // dQ += dS K
+          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS2 + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
       } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k)   // dV += P^T dO
-          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpA + k * 8, HT::mnmajor(y2_s(st), k), kIdescAcc, acc | (k != 0));
+        for (int k = 0; k < kBwdY / 16; ++k)   // dV += P^T dO
+          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS1 + k * 8, HT::mnmajor(y2a, k), kIdescAcc, acc | (k != 0));
 #pragma unroll
-        for (int k = 0; k < 8; ++k)   // dK += dS^T Q
-          ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColOpB + k * 8, HT::mnmajor(y1_s(st), k), kIdescAcc, acc | (k != 0));
+        for (int k = 0; k < kBwdY / 16; ++k)   // dK += dS^T Q
+          ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColS2 + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
       }
-      ptx::mma_commit(bar_o);
+      if (t + 1 < n_tiles) issue_s(t + 1);  // queued behind the products above, which read the columns it overwrites
+      else ptx::mma_commit(bar_o);
     }
   }
-  if (!*abort_flag && n_tiles > 0) {
-    if (!ptx::mbar_wait(bar_o, (n_tiles - 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+  if (!dead && n_tiles > 0) {
+    if (!ptx::mbar_wait(bar_o, 0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
   }
 
-  if (!*abort_flag && n_tiles > 0 && half < 2) {  // two of the column parts drain the accumulators, d/2 columns each
+  if (!*abort_flag && n_tiles > 0) {  // each thread drains d/2 columns of its row of the accumulators
     const long long ld = 3LL * C;
-    constexpr int kDh = D / 2;  // head dimensions stored by this thread
+    constexpr int kDh = D / 2;
     auto store_acc = [&](uint32_t acc_col, __nv_bfloat16* dst, float mul) {
       uint32_t r[kDh];
       if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + acc_col + half * kDh, r);
@@ -553,9 +553,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       store_acc(kColAcc2, base + C, scale);       // dK
     }
   }
-  if (*abort_flag && tid == 0) {
-    for (int t = issued > kYStages ? issued - kYStages : 0; t < issued; ++t)
-      ptx::mbar_wait(bar_y(t % kYStages), (t / kYStages) & 1);
+  if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
+    for (int t = issued > kBwdStages ? issued - kBwdStages : 0; t < issued; ++t)
+      ptx::mbar_wait(bar_y(t % kBwdStages), (t / kBwdStages) & 1);
     ptx::mbar_wait(bar_x, 0);
   }
   ptx::tc_fence_before_sync();
@@ -569,9 +569,11 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
 template <int D>
 int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st) {
-  CUtensorMap tm_qkv, tm_do;
+  CUtensorMap tm_qkv, tm_do, tm_qkv_y, tm_do_y;  // own tiles: 128-row boxes; streamed tiles: 64-row boxes
   if (!make_tmap_bf16_2d(&tm_qkv, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2) ||
-      !make_tmap_bf16_2d(&tm_do, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2))
+      !make_tmap_bf16_2d(&tm_do, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2) ||
+      !make_tmap_bf16_2d(&tm_qkv_y, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, kBwdY, D * 2) ||
+      !make_tmap_bf16_2d(&tm_do_y, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, kBwdY, D * 2))
     return SPA_ERR_UNSUPPORTED;
   auto kq = attn_bwd_tc_kernel<D, true>;
   auto kkv = attn_bwd_tc_kernel<D, false>;
@@ -585,11 +587,11 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
   dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
-  launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
+  launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
                                                     lse, delta, seg, n_seg, p.capacity, p.C, scale,
                                                     (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
-  launch_pdl(kkv, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, (const __nv_bfloat16*)ao,
+  launch_pdl(kkv, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, (const __nv_bfloat16*)ao,
                                                      (const __nv_bfloat16*)dao, lse, delta, seg, n_seg, p.capacity,
                                                      p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
