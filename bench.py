@@ -233,6 +233,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="issue the weight gradients on the main stream too")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 2000 and args.warmup == 50:
@@ -290,7 +291,14 @@ def main():
         for _, fn in sets[s_][3]:
             fn()
     torch.cuda.synchronize()
-    step_graphs = [capture([fn for _, fn in sets[s_][3]]) for s_ in range(n_sets)]
+    def whole_step(s_):
+        inp_, d_, blk_, _ = sets[s_]
+        def run():
+            blk_.forward(d_["x"], d_["w_g"], inp_.b_g, d_["W_qkv"], d_["b_qkv"], d_["W_o"], d_["b_o"])
+            blk_.backward(d_["dY"], overlap=not args.no_overlap)
+        return run
+
+    step_graphs = [capture([whole_step(s_)]) for s_ in range(n_sets)]
     launches_per_step = step_graphs[0][1]
 
     def step(i):

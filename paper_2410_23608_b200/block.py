@@ -44,6 +44,10 @@ class SpaBlock:
         self.status = torch.zeros(4, dtype=torch.int32, device=dev)
         ws = L.spa_workspace_bytes(self.p)
         self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if ws > 0 else None
+        # the weight gradients do not feed the rest of the backward chain: they run on a second stream,
+        # with a scratch area of their own, beside the attention backward and the input gradients
+        self.side_stream = torch.cuda.Stream(device=dev) if backward else None
+        self.workspace_side = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if (ws > 0 and backward) else None
         if backward:
             self.dz = e(cap, C)
             self.dao = e(cap, C)
@@ -74,21 +78,40 @@ class SpaBlock:
         return y
 
     # ------------------------------------------------------------------ backward
-    def backward(self, dY, dX=None):
+    def backward(self, dY, dX=None, overlap=True):
         """Gradients for the last forward(): returns dX; parameter gradients land in dW_qkv, db_qkv,
-        dW_o, db_o (fp32).  No gradient reaches the gate (hard threshold)."""
+        dW_o, db_o (fp32).  No gradient reaches the gate (hard threshold).  With overlap=True the two
+        weight-gradient calls are issued on a second stream and joined before returning."""
         p = self.p
         W_qkv, W_o = self._saved
         dX = self.dX if dX is None else dX
         C = self.C
+        main = torch.cuda.current_stream()
+        side = self.side_stream if (overlap and self.side_stream is not None) else None
         L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
-        L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
-                                self.workspace, self.status)
+        if side is None:
+            L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
+                                    self.workspace, self.status)
+        else:
+            side.wait_stream(main)
+            L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, None, self.dW_o, self.db_o,
+                                    self.workspace_side, self.status, stream=side)
+            L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, None, None,
+                                    self.workspace, self.status)
         L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self.cu, self.B, self.dqkv,
                                    self.workspace, self.status)
-        L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv, self.db_qkv,
-                                self.workspace, self.status)
+        if side is None:
+            L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv,
+                                    self.db_qkv, self.workspace, self.status)
+        else:
+            side.wait_stream(main)
+            L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, None, self.dW_qkv, self.db_qkv,
+                                    self.workspace_side, self.status, stream=side)
+            L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, None, None,
+                                    self.workspace, self.status)
         L.spa_select_pack_bwd(p, self.dxp, dY, self.idx, self.cu, dX)
+        if side is not None:
+            main.wait_stream(side)
         return dX
 
     def read_status(self) -> int:
