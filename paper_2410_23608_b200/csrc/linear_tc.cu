@@ -79,21 +79,8 @@ constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, war
 constexpr int kABytes = BM * BK * 2;
 
 template <int BN> __host__ __device__ constexpr int stage_bytes() { return kABytes + BN * BK * 2; }
-template <int BN> __host__ __device__ constexpr int gemm_smem_bytes() { return kStages * stage_bytes<BN>() + 1024 + 128; }
-
-template <typename OutT> struct OutStore;
-template <> struct OutStore<__nv_bfloat16> {
-  // 8 consecutive columns as one 16-byte store
-  __device__ static __forceinline__ void store8(__nv_bfloat16* dst, const float* v) {
-    *reinterpret_cast<uint4*>(dst) = Vec16<__nv_bfloat16>::from_float(v);
-  }
-};
-template <> struct OutStore<float> {
-  __device__ static __forceinline__ void store8(float* dst, const float* v) {
-    reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
-    reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
-  }
-};
+// operand ring, alignment slack, barriers, 2 KB per epilogue warp for the output transposition
+template <int BN> __host__ __device__ constexpr int gemm_smem_bytes() { return kStages * stage_bytes<BN>() + 1024 + 128 + 4 * 2048; }
 
 // Tile bookkeeping shared by the three roles of the persistent kernel.
 struct TileCoord { int m0, n0, z, n_t; };
@@ -269,6 +256,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ epilogue warps
     const int q = warp & 3;          // TMEM lane quarter this warp may read
     const int et = threadIdx.x - 64; // 0..127 over the four epilogue warps, any order of quarters
+    uint8_t* stage = smem_al + kStages * kStage + 128 + (warp - 2) * 2048;  // this warp's transposition buffer
     int it = 0, tl = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++tl) {
       if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
@@ -305,30 +293,51 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         break;
       }
       ptx::tc_fence_after_sync();
-      const int row = c.m0 + q * 32 + lane;
-      OutT* orow = out + (long long)c.z * split_stride + (long long)row * ldo;
+      // Thread `lane` receives row (q*32 + lane) of the accumulator.  Written straight from there, every
+      // store instruction would touch 32 rows with 16 bytes each; instead the warp turns 64-byte row
+      // segments around in its private 2 KB of shared memory, so that a store instruction covers 8 rows
+      // with 64 contiguous bytes each (whole 32-byte sectors only).
+      OutT* obase = out + (long long)c.z * split_stride;
+      constexpr int kPasses = sizeof(OutT) == 2 ? 1 : 2;        // 64-byte segments per 32 accumulator columns
+      constexpr int kSegCols = 64 / (int)sizeof(OutT);          // output columns per segment
+      const int my_chunk = lane & 3, my_row = lane >> 2;        // role of this lane on the store side
 #pragma unroll 1
       for (int cc = 0; cc < BN / 32; ++cc) {
         uint32_t r[32];
         ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + cc * 32, r);
         ptx::tmem_ld_wait();
-        if (row < M) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int col = c.n0 + cc * 32 + g * 8;
-            if (col < N) {
+        for (int ps = 0; ps < kPasses; ++ps) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {  // 16-byte chunk i of this row's segment
+            uint4 packed;
+            if (sizeof(OutT) == 2) {
               float v[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]);
-              if (bias != nullptr) {
+              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[i * 8 + e]);
+              const int col = c.n0 + cc * 32 + i * 8;
+              if (bias != nullptr && col < N) {
                 float b[8];
                 Vec16<__nv_bfloat16>::to_float(__ldg(reinterpret_cast<const uint4*>(bias + col)), b);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[e] += b[e];
               }
-              OutStore<OutT>::store8(orow + col, v);
+              packed = Vec16<__nv_bfloat16>::from_float(v);
+            } else {
+              packed = make_uint4(r[ps * 16 + i * 4], r[ps * 16 + i * 4 + 1], r[ps * 16 + i * 4 + 2], r[ps * 16 + i * 4 + 3]);
             }
+            *reinterpret_cast<uint4*>(stage + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = packed;
           }
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int rr = my_row + 8 * j;
+            const uint4 v4 = *reinterpret_cast<const uint4*>(stage + rr * 64 + ((my_chunk ^ ((rr >> 1) & 3)) << 4));
+            const int grow = c.m0 + q * 32 + rr;
+            const int gcol = c.n0 + cc * 32 + ps * kSegCols + my_chunk * (16 / (int)sizeof(OutT));
+            if (grow < M && gcol < N) *reinterpret_cast<uint4*>(obase + (long long)grow * ldo + gcol) = v4;
+          }
+          __syncwarp();
         }
       }
       ptx::tc_fence_before_sync();
