@@ -44,8 +44,46 @@ template <int D> struct HeadTile {
   }
 };
 
+constexpr int kSegStage = 512;  // segment offsets are searched in shared memory when there are at most this many
+
+// Segment bounds of packed row i (hi clamped to the valid rows) from offsets held in shared memory.
+__device__ __forceinline__ RowSeg row_segment_staged(const int32_t* s_off, int n_seg, int Np, int i) {
+  RowSeg r{0, 0};
+  if (i < Np) {
+    int lo = 0, hi = n_seg;  // invariant: s_off[lo] <= i < s_off[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_off[mid] <= i) lo = mid; else hi = mid;
+    }
+    r.lo = s_off[lo];
+    const int h2 = s_off[lo + 1];
+    r.hi = h2 < Np ? h2 : Np;
+  }
+  return r;
+}
+
+// Rotation of the 16-byte chunks of row r of a [128][D] bf16 tile in shared memory that makes the
+// accesses of 8 neighbouring rows to one chunk index fall into different banks.
+template <int D> __device__ __forceinline__ int chunk_rot(int r) { return D == 64 ? (r & 7) : ((r >> 1) & 3); }
+
+// Copy a [128][D] bf16 tile that the threads wrote to shared memory (chunk c of row r at position
+// c ^ chunk_rot(r)) to rows r0.. of a matrix with `ld` elements per row: a warp covers whole rows, so the
+// stores are full 64- or 128-byte lines.  Rows from Np on are not written.
+template <int D, int kThreads>
+__device__ __forceinline__ void copy_tile_out(const uint8_t* tile, __nv_bfloat16* dst, long long ld, int r0, int Np, int tid) {
+  constexpr int kChunks = D * 2 / 16;
+#pragma unroll
+  for (int i = tid; i < 128 * kChunks; i += kThreads) {
+    const int r = i / kChunks, c = i % kChunks;
+    if (r0 + r < Np)
+      *reinterpret_cast<uint4*>(dst + (long long)(r0 + r) * ld + c * 8) =
+          *reinterpret_cast<const uint4*>(tile + r * (D * 2) + ((c ^ chunk_rot<D>(r)) << 4));
+  }
+}
+
 template <int D> __host__ __device__ constexpr int fwd_smem_bytes() {
-  return 5 * 128 * D * 2 + 1024 + 128 + 2048;  // Q + 2 x (K, V), alignment slack, barriers, row-max exchange
+  // Q + 2 x (K, V), alignment slack, barriers, row-max exchange, segment offsets
+  return 5 * 128 * D * 2 + 1024 + 128 + 2048 + kSegStage * 4 + 64;
 }
 
 template <int D>
@@ -53,12 +91,9 @@ __global__ void __launch_bounds__(kFwdThreads)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __restrict__ seg, int n_seg, int capacity,
                    int C, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
                    int32_t* d_status) {
-  pdl_entry();
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
-  const int Np = packed_rows(seg, n_seg, capacity);
   const int q0 = blockIdx.y * kQ;  // grid = (heads, tiles): CTAs past the last valid tile are dispatched last
-  if (q0 >= Np) return;
   const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 query rows and split
   // the work of each row (key columns of S and P, head dimensions of O) in two halves
@@ -78,14 +113,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 68);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 72);
   float* xch = reinterpret_cast<float*>(smem_al + 5 * kTile + 128);  // [2 tile parities][2 halves][128 rows]
+  int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + 5 * kTile + 128 + 2048);  // [kSegStage + 1]
 
-  const int row = q0 + rl;
-  const RowSeg mine = row_segment(seg, n_seg, Np, row);
-  if (half == 0) {
-    const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
-    if (row == q0) range[0] = mine.lo;
-    if (row == last) range[1] = mine.hi;
-  }
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
   if (tid == 0) {
     ptx::prefetch_tensormap(&tm);
     ptx::mbar_init(bar_q, 1);
@@ -95,11 +125,30 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
+  pdl_entry();
+  const bool staged = n_seg < kSegStage;
+  if (staged)
+    for (int i = tid; i <= n_seg; i += kFwdThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  if (q0 >= Np) return;
+  if (tid == 0) {  // the Q tile depends only on q0: fetch it under the segment search
+    ptx::mbar_expect_tx(bar_q, kTile);
+    ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
+  }
   if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  __syncthreads();  // barriers, TMEM address and staged offsets are visible
   ptx::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+
+  const int row = q0 + rl;
+  const RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+  if (half == 0) {
+    const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
+    if (row == q0) range[0] = mine.lo;
+    if (row == last) range[1] = mine.hi;
+  }
+  __syncthreads();
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;  // TMEM lanes this warp may touch
   constexpr int kCols = kKV / 2;  // key columns of each tile owned by this thread
   constexpr int kDh = D / 2;      // head dimensions of O owned by this thread
@@ -130,8 +179,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   };
   int loads_k = 0, loads_v = 0;  // tiles whose loads thread 0 has issued
   if (tid == 0) {
-    ptx::mbar_expect_tx(bar_q, kTile);
-    ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
     load_k(0);
     load_v(0);
     loads_k = loads_v = 1;
@@ -170,19 +217,31 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 #pragma unroll
     for (int c = 0; c < kCols / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColS + col0 + c * 32, s + c * 32);
     ptx::tmem_ld_wait();
-    // mask (boundary tiles only) and this half's row maximum, handed to the partner thread through shared memory
+    // Which of this thread's groups of 32 key columns meet its row's segment at all (the others take no
+    // arithmetic: their P is zero); the mask is applied only where a boundary of the segment crosses a group.
+    // This half's row maximum is handed to the partner thread through shared memory.
     const int kc0 = kv0 + col0;
-    const bool interior = kc0 >= mine.lo && kc0 + kCols <= mine.hi;
-    if (!interior) {
+    bool need[kCols / 32];
 #pragma unroll
-      for (int j = 0; j < kCols; ++j)
-        if ((unsigned)(kc0 + j - mine.lo) >= span) s[j] = 0xff800000u;  // -inf
+    for (int c = 0; c < kCols / 32; ++c) {
+      const int g0 = kc0 + c * 32;
+      need[c] = g0 < mine.hi && g0 + 32 > mine.lo;
+      if (need[c] && !(g0 >= mine.lo && g0 + 32 <= mine.hi)) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if ((unsigned)(g0 + j - mine.lo) >= span) s[c * 32 + j] = 0xff800000u;  // -inf
+      }
     }
     float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-    for (int j = 0; j < kCols; j += 4) {
+    for (int c = 0; c < kCols / 32; ++c) {
+      if (need[c]) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[j + u]));
+        for (int j = 0; j < 32; j += 4) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c * 32 + j + u]));
+        }
+      }
     }
     float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
     xch[((t & 1) * 2 + half) * 128 + rl] = mt;
@@ -201,14 +260,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 #pragma unroll
     for (int c = 0; c < kCols / 32; ++c) {
       uint32_t pk[16];
+      if (need[c]) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 2) {
-        const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j]), scale_log2e, -m_use));  // -inf -> 0
-        const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j + 1]), scale_log2e, -m_use));
-        rs0 += p0;
-        rs1 += p1;
-        __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
-        pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j]), scale_log2e, -m_use));  // -inf -> 0
+          const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j + 1]), scale_log2e, -m_use));
+          rs0 += p0;
+          rs1 += p1;
+          __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
+          pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) pk[j] = 0u;
       }
       ptx::tmem_st_32x16(tmem + lane_base + kColP + (col0 >> 1) + c * 16, pk);
     }
@@ -247,19 +311,24 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 
   // the two halves of a row share the running max but kept separate sums: combine them
   xch[half * 128 + rl] = l;
-  __syncthreads();
-  if (!*abort_flag && row < Np) {
+  __syncthreads();  // nobody sets the flag from here on: the branch below is taken by all threads or by none
+  if (!*abort_flag) {
+    // normalised rows go to the Q tile's shared memory (idle now: every product has completed) as bf16 and
+    // leave from there as whole lines
     const float l_row = l + xch[(half ^ 1) * 128 + rl];
-    const float inv_l = 1.f / l_row;
-    __nv_bfloat16* dst = ao + (long long)row * C + h * D + half * kDh;
+    const float inv_l = row < Np ? 1.f / l_row : 0.f;
+    const int rot = chunk_rot<D>(rl);
 #pragma unroll
     for (int c = 0; c < kDh / 8; ++c) {
       float v[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] = o[c * 8 + e] * inv_l;
-      *reinterpret_cast<uint4*>(dst + c * 8) = Vec16<__nv_bfloat16>::from_float(v);
+      *reinterpret_cast<uint4*>(smem_al + rl * HT::kRowBytes + (((half * (kDh / 8) + c) ^ rot) << 4)) =
+          Vec16<__nv_bfloat16>::from_float(v);
     }
-    if (half == 0) lse[(long long)h * capacity + row] = (m + log2f(l_row)) * 0.6931471805599453f;
+    if (half == 0 && row < Np) lse[(long long)h * capacity + row] = (m + log2f(l_row)) * 0.6931471805599453f;
+    __syncthreads();
+    copy_tile_out<D, kFwdThreads>(smem_al, ao + h * D, C, q0, Np, tid);
   }
   if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
     for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
@@ -294,25 +363,24 @@ constexpr int kBwdStages = 3;      // streamed tiles in shared memory
 constexpr uint32_t kBwdTmemCols = 256;
 constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;  // operands alias S1 / S2 columns [0, 32)
 
-template <int D> __host__ __device__ constexpr int bwd_smem_bytes() {
-  return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128;  // own, streamed, slack, statistics, barriers
+template <int D, bool kDQ> __host__ __device__ constexpr int bwd_smem_bytes() {
+  // own tiles (the dQ pass also holds the O tile), streamed tiles, alignment slack, statistics, barriers, segment offsets
+  return (kDQ ? 3 : 2) * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64;
 }
 
 template <int D, bool kDQ>
 __global__ void __launch_bounds__(kBwdThreads)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
-                   const __nv_bfloat16* __restrict__ ao, const __nv_bfloat16* __restrict__ dao,
+                   const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
                    int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
-  pdl_entry();
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
+  constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
   constexpr float kLog2e = 1.4426950408889634f;
-  const int Np = packed_rows(seg, n_seg, capacity);
   const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
-  if (r0 >= Np) return;
   const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
   const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
@@ -321,8 +389,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
-  constexpr int kYBase = 2 * kTile;
+  const uint32_t x1_s = smem_base, x2_s = smem_base + kTile, x3_s = smem_base + 2 * kTile;
+  constexpr int kYBase = kOwn * kTile;
   auto y1_off = [&](int st) { return kYBase + kYTile * (2 * st); };
   auto y2_off = [&](int st) { return kYBase + kYTile * (2 * st + 1); };
   constexpr int kStatBase = kYBase + kBwdStages * 2 * kYTile;
@@ -334,19 +402,15 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kStatBase + 1024 + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 68);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 72);
+  int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kStatBase + 1024 + 128);  // [kSegStage + 1]
 
-  const int row = r0 + rl;
-  const RowSeg mine = row_segment(seg, n_seg, Np, row);
-  if (half == 0) {
-    const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
-    if (row == r0) range[0] = mine.lo;
-    if (row == last) range[1] = mine.hi;
-  }
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
   if (tid == 0) {
     ptx::prefetch_tensormap(&tm_qkv);
     ptx::prefetch_tensormap(&tm_do);
     ptx::prefetch_tensormap(&tm_qkv_y);
     ptx::prefetch_tensormap(&tm_do_y);
+    if (kDQ) ptx::prefetch_tensormap(&tm_o);
     ptx::mbar_init(bar_x, 1);
     for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
@@ -354,18 +418,42 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
+  pdl_entry();
+  const bool staged = n_seg < kSegStage;
+  if (staged)
+    for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  if (r0 >= Np) return;
+  const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
+  if (tid == 0) {  // the own tiles depend only on r0: fetch them under the segment search
+    ptx::mbar_expect_tx(bar_x, kOwn * kTile);
+    ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
+    if (kDQ) {
+      ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                  // dO
+      ptx::tma_load_2d(x3_s, &tm_o, bar_x, h * D, r0);                   // O, for D_i = dO_i . O_i
+    } else {
+      ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
+    }
+  }
   if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  __syncthreads();  // barriers, TMEM address and staged offsets are visible
   ptx::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+
+  const int row = r0 + rl;
+  const RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+  if (half == 0) {
+    const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
+    if (row == r0) range[0] = mine.lo;
+    if (row == last) range[1] = mine.hi;
+  }
+  __syncthreads();
   const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
   const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
 
-  // column offsets inside qkv of the own / streamed operands
-  const int x1_col = (kDQ ? 0 : C) + h * D;           // Q | K
-  const int y1_col = (kDQ ? C : 0) + h * D;           // K | Q
+  const int y1_col = (kDQ ? C : 0) + h * D;           // streamed operand inside qkv: K | Q
   auto load_other = [&](int t_) {  // streamed tile t_ into stage t_ mod kBwdStages
     const int st = t_ % kBwdStages, y0 = o_lo + t_ * kBwdY;
     ptx::mbar_expect_tx(bar_y(st), 2 * kYTile);
@@ -375,10 +463,6 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   };
   int issued = 0;  // streamed tiles whose loads thread 0 has issued
   if (tid == 0) {
-    ptx::mbar_expect_tx(bar_x, 2 * kTile);
-    ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
-    if (kDQ) ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                    // dO
-    else ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);               // V
     for (int t_ = 0; t_ < n_tiles && t_ < 2; ++t_) load_other(t_);
     issued = n_tiles < 2 ? n_tiles : 2;
   }
@@ -386,20 +470,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   float my_lse = 0.f, my_D = 0.f;   // kDQ: this thread's query row
   float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next streamed query tile, row rl < 64
   if (kDQ) {
-    if (row < Np) {
-      const __nv_bfloat16* orow = ao + (long long)row * C + h * D;
-      const __nv_bfloat16* grow = dao + (long long)row * C + h * D;
-#pragma unroll
-      for (int c = 0; c < D / 8; ++c) {
-        float a[8], b[8];
-        Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(orow + c * 8), a);
-        Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(grow + c * 8), b);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
-      }
-      my_lse = lse[(long long)h * capacity + row] * kLog2e;
-      if (half == 0) delta[(long long)h * capacity + row] = my_D;
-    }
+    if (row < Np) my_lse = lse[(long long)h * capacity + row] * kLog2e;
   } else if (half == 0 && rl < kBwdY) {
     const int i = o_lo + rl;
     if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
@@ -450,6 +521,24 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (tid == 0 && !*abort_flag) { ptx::tc_fence_after_sync(); issue_s(0); }
+  if (kDQ && row < Np) {
+    // D_i = dO_i . O_i from the two staged tiles (their load has completed: prep(0) waited for it).  Both
+    // carry the same swizzle, so equal positions hold equal columns and the order of the chunks is free:
+    // each row starts at a different chunk to keep 8 neighbouring rows off one bank.
+    constexpr int kChunks = HT::kRowBytes / 16;
+    const uint8_t* po = smem_al + 2 * kTile + rl * HT::kRowBytes;
+    const uint8_t* pg = smem_al + kTile + rl * HT::kRowBytes;
+    const int rot = chunk_rot<D>(rl);
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      float a[8], b[8];
+      Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(po + ((c ^ rot) << 4)), a);
+      Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(pg + ((c ^ rot) << 4)), b);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
+    }
+    if (half == 0) delta[(long long)h * capacity + row] = my_D;
+  }
 
   constexpr int kPc = kBwdY / 2;  // fp32 columns of each tile owned by this thread
   const int col0 = half * kPc;
@@ -470,30 +559,36 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     __syncthreads();  // A: every thread holds its fp32 columns; their TMEM columns may now take the bf16 operands
     if (*abort_flag) { dead = true; break; }
 
-    // ---- P = 2^(S - lse), dS = P (dP - D): masked only where a boundary of this row's segment crosses
+    // ---- P = 2^(S - lse), dS = P (dP - D).  A thread whose 32 columns lie wholly outside its row's segment
+    // writes zeros without doing the arithmetic; the mask costs something only where a boundary crosses.
     const int yc0 = y0 + col0;
-    if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {
-#pragma unroll
-      for (int j = 0; j < kPc; ++j)
-        if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
-    }
     uint32_t pk_p[kPc / 2], pk_ds[kPc / 2];
-    const float* sl = stat_lse + (t & 1) * kBwdY + col0;
-    const float* sd = stat_D + (t & 1) * kBwdY + col0;
+    if (yc0 < mine.hi && yc0 + kPc > mine.lo) {
+      if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {
 #pragma unroll
-    for (int j = 0; j < kPc; j += 2) {
-      float pv[2], dsv[2];
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const float l2 = kDQ ? my_lse : sl[j + u];
-        const float Dv = kDQ ? my_D : sd[j + u];
-        pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + u]), scale_log2e, -l2));
-        dsv[u] = pv[u] * (__uint_as_float(rp[j + u]) - Dv);
+        for (int j = 0; j < kPc; ++j)
+          if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
       }
-      __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
-      pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
-      __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
-      pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+      const float* sl = stat_lse + (t & 1) * kBwdY + col0;
+      const float* sd = stat_D + (t & 1) * kBwdY + col0;
+#pragma unroll
+      for (int j = 0; j < kPc; j += 2) {
+        float pv[2], dsv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const float l2 = kDQ ? my_lse : sl[j + u];
+          const float Dv = kDQ ? my_D : sd[j + u];
+          pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + u]), scale_log2e, -l2));
+          dsv[u] = pv[u] * (__uint_as_float(rp[j + u]) - Dv);
+        }
+        __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
+        pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
+        __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
+        pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < kPc / 2; ++j) { pk_p[j] = 0u; pk_ds[j] = 0u; }
     }
     if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColS1 + (col0 >> 1), pk_p);   // P^T over the consumed S^T
     ptx::tmem_st_32x16(tmem + lane_base + kColS2 + (col0 >> 1), pk_ds);            // dS (or dS^T) over the consumed dP
@@ -526,31 +621,38 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     if (!ptx::mbar_wait(bar_o, 0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
   }
+  __syncthreads();  // nobody sets the flag from here on: the branch below is taken by all threads or by none
 
-  if (!*abort_flag && n_tiles > 0) {  // each thread drains d/2 columns of its row of the accumulators
-    const long long ld = 3LL * C;
+  if (!*abort_flag && n_tiles > 0) {
+    // Each thread drains d/2 columns of its row of the accumulators into the own tiles' shared memory (idle
+    // now: every product has completed), from where whole rows go out as full lines.
     constexpr int kDh = D / 2;
-    auto store_acc = [&](uint32_t acc_col, __nv_bfloat16* dst, float mul) {
+    auto stage_acc = [&](uint32_t acc_col, uint8_t* tile, float mul) {
       uint32_t r[kDh];
       if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + acc_col + half * kDh, r);
       else ptx::tmem_ld_32x16(tmem + lane_base + acc_col + half * kDh, r);
       ptx::tmem_ld_wait();
-      if (row < Np) {
+      const int rot = chunk_rot<D>(rl);
 #pragma unroll
-        for (int g = 0; g < kDh / 8; ++g) {
-          float v[8];
+      for (int g = 0; g < kDh / 8; ++g) {
+        float v[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul;
-          *reinterpret_cast<uint4*>(dst + half * kDh + g * 8) = Vec16<__nv_bfloat16>::from_float(v);
-        }
+        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul;
+        *reinterpret_cast<uint4*>(tile + rl * HT::kRowBytes + (((half * (kDh / 8) + g) ^ rot) << 4)) =
+            Vec16<__nv_bfloat16>::from_float(v);
       }
     };
-    __nv_bfloat16* base = dqkv + (long long)row * ld + h * D;
+    const long long ld = 3LL * C;
     if (kDQ) {
-      store_acc(kColAcc1, base, scale);
+      stage_acc(kColAcc1, smem_al, scale);
+      __syncthreads();
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
     } else {
-      store_acc(kColAcc1, base + 2 * C, 1.f);     // dV
-      store_acc(kColAcc2, base + C, scale);       // dK
+      stage_acc(kColAcc1, smem_al, 1.f);             // dV
+      stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
+      __syncthreads();
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
     }
   }
   if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
@@ -569,31 +671,31 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
 template <int D>
 int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st) {
-  CUtensorMap tm_qkv, tm_do, tm_qkv_y, tm_do_y;  // own tiles: 128-row boxes; streamed tiles: 64-row boxes
+  CUtensorMap tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o;  // own tiles: 128-row boxes; streamed tiles: 64-row boxes
   if (!make_tmap_bf16_2d(&tm_qkv, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2) ||
       !make_tmap_bf16_2d(&tm_do, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2) ||
       !make_tmap_bf16_2d(&tm_qkv_y, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, kBwdY, D * 2) ||
-      !make_tmap_bf16_2d(&tm_do_y, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, kBwdY, D * 2))
+      !make_tmap_bf16_2d(&tm_do_y, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, kBwdY, D * 2) ||
+      !make_tmap_bf16_2d(&tm_o, ao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2))
     return SPA_ERR_UNSUPPORTED;
   auto kq = attn_bwd_tc_kernel<D, true>;
   auto kkv = attn_bwd_tc_kernel<D, false>;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D>());
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D>());
+    cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, true>());
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, false>());
     if (e != cudaSuccess) { set_cuda_error(e, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
     attr_set = true;
   }
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
   dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
-  launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, (const __nv_bfloat16*)ao, (const __nv_bfloat16*)dao,
-                                                    lse, delta, seg, n_seg, p.capacity, p.C, scale,
-                                                    (__nv_bfloat16*)dqkv, d_status);
+  launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D, true>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
-  launch_pdl(kkv, grid, kBwdThreads, bwd_smem_bytes<D>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, (const __nv_bfloat16*)ao,
-                                                     (const __nv_bfloat16*)dao, lse, delta, seg, n_seg, p.capacity,
-                                                     p.C, scale, (__nv_bfloat16*)dqkv, d_status);
+  launch_pdl(kkv, grid, kBwdThreads, bwd_smem_bytes<D, false>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
   return SPA_OK;
 }
