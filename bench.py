@@ -304,7 +304,8 @@ def main():
         step(i)
     torch.cuda.synchronize()
     Np_sets = [int(b.cu[-1].item()) for _, _, b, _ in sets]
-    assert all(b.read_status() == 0 for _, _, b, _ in sets)
+    statuses = [b.read_status() for _, _, b, _ in sets]
+    assert all(st == 0 for st in statuses), f"device status after warm-up: {statuses}"
     tokens_per_step = float(np.mean([Np_sets[i % n_sets] for i in range(args.steps)]))
 
     def barrier():
