@@ -186,6 +186,33 @@ int spa_packed_linear_bwd(const spa_params* p, const void* a, const void* W, con
                           int32_t n_in, int32_t n_out, const int32_t* cu_seqlens, void* da,
                           float* dW, float* db, void* workspace, int32_t* d_status, void* stream);
 
+/* Fused unpack (Sec. 3.2: selected tokens are replaced by the block's output, the others pass through).
+ * The three calls below give the same results as spa_packed_proj + spa_unpack_scatter and as
+ * spa_packed_linear_bwd + spa_select_pack_bwd, without the packed intermediate (z, dx_packed) and
+ * without the separate scatter kernel: the matrix product writes its rows straight to their tokens.
+ * Tensor-core problems only (bf16, C a multiple of 8, C >= 64): spa_fused_scatter_supported says
+ * whether they apply; otherwise they return SPA_ERR_UNSUPPORTED and the unfused calls must be used. */
+int spa_fused_scatter_supported(const spa_params* p);
+
+/* dst[B][N][C] = src[B][N][C]: writes the pass-through rows ahead of the scatter (y = x in the
+ * forward pass, dX = dY in the backward pass).  A no-op when dst == src. */
+int spa_unpack_prefill(const spa_params* p, const void* src, void* dst, void* stream);
+
+/* Output projection with the unpack scatter in its epilogue:  y[idx[i]][:] = b_o + W_o a[i][:]
+ * (added to y[idx[i]][:] under SPA_FLAG_RESIDUAL).  y: T[B][N][C] must already hold x
+ * (spa_unpack_prefill, or y aliasing x); rows of unselected tokens are not touched. */
+int spa_packed_proj_scatter(const spa_params* p, const void* a, const void* W_o, const void* b_o,
+                            const int32_t* idx, const int32_t* cu_seqlens, void* y, int32_t* d_status,
+                            void* stream);
+
+/* spa_packed_linear_bwd with the transpose of the pack gather in the epilogue of the input gradient:
+ * dX[idx[i]][:] = dout[i][:] W  (added to dX[idx[i]][:] under SPA_FLAG_RESIDUAL, where dX must
+ * already hold dY).  n_in must equal C; dW, db and workspace as in spa_packed_linear_bwd. */
+int spa_packed_linear_bwd_scatter(const spa_params* p, const void* a, const void* W, const void* dout,
+                                  int32_t n_in, int32_t n_out, const int32_t* idx,
+                                  const int32_t* cu_seqlens, void* dX, float* dW, float* db,
+                                  void* workspace, int32_t* d_status, void* stream);
+
 /* Blocking read of the device status word: synchronises `stream` and returns its value. */
 int spa_read_status(const int32_t* d_status, void* stream);
 

@@ -27,6 +27,7 @@ EXPORTS = (
     "spa_packed_attention_bwd", "spa_packed_proj", "spa_unpack_scatter", "spa_unpack_scatter_bwd",
     "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
     "spa_last_cuda_error", "spa_launch_count", "spa_packed_attention_bwd_static",
+    "spa_fused_scatter_supported", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
 )
 
 
@@ -74,6 +75,10 @@ def lib() -> C.CDLL:
         L.spa_unpack_scatter_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_select_pack_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp]
         L.spa_packed_linear_bwd.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_fused_scatter_supported.argtypes = [pp]
+        L.spa_unpack_prefill.argtypes = [pp, vp, vp, vp]
+        L.spa_packed_proj_scatter.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_packed_linear_bwd_scatter.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
             if name not in ("spa_workspace_bytes", "spa_status_string", "spa_last_cuda_error", "spa_launch_count"):
@@ -173,6 +178,27 @@ def spa_packed_linear_bwd(p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, wo
     _check(lib().spa_packed_linear_bwd(C.byref(p), _ptr(a), _ptr(W), _ptr(dout), int(n_in), int(n_out),
                                        _ptr(cu_seqlens), _ptr(da), _ptr(dW), _ptr(db), _ptr(workspace),
                                        _ptr(d_status), _stream(stream)), "spa_packed_linear_bwd")
+
+
+def spa_fused_scatter_supported(p) -> bool:
+    return bool(lib().spa_fused_scatter_supported(C.byref(p)))
+
+
+def spa_unpack_prefill(p, src, dst, stream=None):
+    _check(lib().spa_unpack_prefill(C.byref(p), _ptr(src), _ptr(dst), _stream(stream)), "spa_unpack_prefill")
+
+
+def spa_packed_proj_scatter(p, a, W_o, b_o, idx, cu_seqlens, y, d_status=None, stream=None):
+    _check(lib().spa_packed_proj_scatter(C.byref(p), _ptr(a), _ptr(W_o), _ptr(b_o), _ptr(idx), _ptr(cu_seqlens),
+                                         _ptr(y), _ptr(d_status), _stream(stream)), "spa_packed_proj_scatter")
+
+
+def spa_packed_linear_bwd_scatter(p, a, W, dout, n_in, n_out, idx, cu_seqlens, dX, dW, db, workspace=None,
+                                  d_status=None, stream=None):
+    _check(lib().spa_packed_linear_bwd_scatter(C.byref(p), _ptr(a), _ptr(W), _ptr(dout), int(n_in), int(n_out),
+                                               _ptr(idx), _ptr(cu_seqlens), _ptr(dX), _ptr(dW), _ptr(db),
+                                               _ptr(workspace), _ptr(d_status), _stream(stream)),
+           "spa_packed_linear_bwd_scatter")
 
 
 def spa_read_status(d_status, stream=None) -> int:

@@ -18,7 +18,8 @@ class SpaBlock:
     (paper Sec. 3.2) and the matching backward pass."""
 
     def __init__(self, B: int, N: int, C: int, H: int, dtype: str, tau: float = 0.0, flags: int = 0,
-                 capacity: Optional[int] = None, backward: bool = True, device: str = "cuda"):
+                 capacity: Optional[int] = None, backward: bool = True, device: str = "cuda",
+                 fused: Optional[bool] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("SpaBlock needs a CUDA device; there is no CPU path")
         L.lib()
@@ -27,6 +28,12 @@ class SpaBlock:
         cap = capacity if capacity is not None else max(B * N, 1)
         self.p = L.make_params(B, N, C, H, dtype, cap, flags, tau)
         self.cap = cap
+        # fused unpack: the projection and the QKV input gradient scatter their rows to the tokens themselves
+        # (tensor-core problems only); None = use it where the library offers it
+        can_fuse = L.spa_fused_scatter_supported(self.p)
+        if fused and not can_fuse:
+            raise ValueError("the fused scatter calls do not apply to this problem (needs bf16 tensor-core sizes)")
+        self.fused = can_fuse if fused is None else bool(fused)
         dev = torch.device(device)
         T = self.tdtype
         e = lambda *s, dt=T: torch.empty(*s, dtype=dt, device=dev)
@@ -46,7 +53,8 @@ class SpaBlock:
         self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if ws > 0 else None
         # the weight gradients do not feed the rest of the backward chain: they run on a second stream,
         # with a scratch area of their own, beside the attention backward and the input gradients
-        self.side_stream = torch.cuda.Stream(device=dev) if backward else None
+        self.side_stream = torch.cuda.Stream(device=dev) if (backward or self.fused) else None
+        self._prefilled = torch.cuda.Event() if self.fused else None
         self.workspace_side = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if (ws > 0 and backward) else None
         if backward:
             self.dz = e(cap, C)
@@ -64,16 +72,29 @@ class SpaBlock:
     def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None):
         p = self.p
         y = self.y if y is None else y
+        inplace = bool(p.flags & L.SPA_FLAG_INPLACE)
+        if self.fused and not inplace:
+            # the pass-through rows do not depend on anything the block computes: y = x runs beside the chain
+            main, side = torch.cuda.current_stream(), self.side_stream
+            side.wait_stream(main)
+            L.spa_unpack_prefill(p, x, y, stream=side)
         L.spa_gate(p, x, w_g, b_g, s_up, self.scores, self.mask)
         L.spa_select_pack(p, x, self.mask, self.scores, self.xp, self.idx, self.inv, self.cu, self.status)
         L.spa_packed_qkv(p, self.xp, W_qkv, b_qkv, self.cu, self.qkv, self.status)
         L.spa_packed_attention_fwd(p, self.qkv, self.cu, self.B, self.ao, self.lse, self.status)
-        L.spa_packed_proj(p, self.ao, W_o, b_o, self.cu, self.z, self.status)
-        if p.flags & L.SPA_FLAG_INPLACE:
-            L.spa_unpack_scatter(p, self.z, None, self.idx, self.inv, self.cu, x, self.status)
-            y = x
+        if self.fused:
+            if inplace:
+                y = x
+            else:
+                main.wait_stream(side)
+            L.spa_packed_proj_scatter(p, self.ao, W_o, b_o, self.idx, self.cu, y, self.status)
         else:
-            L.spa_unpack_scatter(p, self.z, x, self.idx, self.inv, self.cu, y, self.status)
+            L.spa_packed_proj(p, self.ao, W_o, b_o, self.cu, self.z, self.status)
+            if inplace:
+                L.spa_unpack_scatter(p, self.z, None, self.idx, self.inv, self.cu, x, self.status)
+                y = x
+            else:
+                L.spa_unpack_scatter(p, self.z, x, self.idx, self.inv, self.cu, y, self.status)
         self._saved = (W_qkv, W_o)
         return y
 
@@ -88,7 +109,21 @@ class SpaBlock:
         C = self.C
         main = torch.cuda.current_stream()
         side = self.side_stream if (overlap and self.side_stream is not None) else None
-        L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
+        if self.fused:
+            # dX = dY ahead of time (beside the chain when there is a second stream); the QKV input gradient
+            # then scatters its rows to the selected tokens itself, and dz is a plain gather
+            prefill_on_side = False
+            if dX is not dY and dX.data_ptr() != dY.data_ptr():
+                if side is not None:
+                    prefill_on_side = True
+                    side.wait_stream(main)
+                    L.spa_unpack_prefill(p, dY, dX, stream=side)
+                    self._prefilled.record(side)
+                else:
+                    L.spa_unpack_prefill(p, dY, dX)
+            L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, None)
+        else:
+            L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
         if side is None:
             L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
                                     self.workspace, self.status)
@@ -100,6 +135,20 @@ class SpaBlock:
                                     self.workspace, self.status)
         L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self.cu, self.B, self.dqkv,
                                    self.workspace, self.status)
+        if self.fused:
+            if side is None:
+                L.spa_packed_linear_bwd_scatter(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.idx, self.cu, dX,
+                                                self.dW_qkv, self.db_qkv, self.workspace, self.status)
+            else:
+                side.wait_stream(main)
+                L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, None, self.dW_qkv,
+                                        self.db_qkv, self.workspace_side, self.status, stream=side)
+                if prefill_on_side:
+                    main.wait_event(self._prefilled)
+                L.spa_packed_linear_bwd_scatter(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.idx, self.cu, dX,
+                                                None, None, None, self.status)
+                main.wait_stream(side)
+            return dX
         if side is None:
             L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv,
                                     self.db_qkv, self.workspace, self.status)

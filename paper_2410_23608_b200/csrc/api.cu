@@ -203,6 +203,45 @@ int spa_packed_linear_bwd(const spa_params* p, const void* a, const void* W, con
   return launch_linear_bwd_simt(*p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, (cudaStream_t)stream);
 }
 
+int spa_fused_scatter_supported(const spa_params* p) {
+  if (check_params(p) != SPA_OK) return 0;
+  return (use_tc(p) && tc_linear_supported(p->C, p->C) && tc_linear_supported(p->C, 3 * p->C)) ? 1 : 0;
+}
+
+int spa_unpack_prefill(const spa_params* p, const void* src, void* dst, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(src); SPA_PTR(dst);
+  if (src == dst || p->B == 0) return SPA_OK;
+  return launch_copy_tokens(*p, src, dst, (cudaStream_t)stream);
+}
+
+int spa_packed_proj_scatter(const spa_params* p, const void* a, const void* W_o, const void* b_o, const int32_t* idx,
+                            const int32_t* cu_seqlens, void* y, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(a); SPA_PTR(W_o); SPA_PTR(idx); SPA_PTR(cu_seqlens); SPA_PTR(y); SPA_OPT_PTR(b_o);
+  if (!spa_fused_scatter_supported(p)) return SPA_ERR_UNSUPPORTED;
+  return launch_linear_fwd_tc(*p, a, W_o, b_o, p->C, p->C, cu_seqlens, y, d_status, (cudaStream_t)stream, idx,
+                              (p->flags & SPA_FLAG_RESIDUAL) != 0);
+}
+
+int spa_packed_linear_bwd_scatter(const spa_params* p, const void* a, const void* W, const void* dout, int32_t n_in,
+                                  int32_t n_out, const int32_t* idx, const int32_t* cu_seqlens, void* dX, float* dW,
+                                  float* db, void* workspace, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dout); SPA_PTR(W); SPA_PTR(idx); SPA_PTR(cu_seqlens); SPA_PTR(dX);
+  SPA_OPT_PTR(dW); SPA_OPT_PTR(db); SPA_OPT_PTR(workspace);
+  if (dW != nullptr) SPA_PTR(a);
+  SPA_REQUIRE(n_in == p->C && n_out > 0, SPA_ERR_INVALID_ARG);  // rows of dX are C wide
+  SPA_REQUIRE(n_out % 8 == 0, SPA_ERR_UNSUPPORTED);
+  if (!spa_fused_scatter_supported(p) || !tc_linear_supported(n_in, n_out)) return SPA_ERR_UNSUPPORTED;
+  if ((dW != nullptr || db != nullptr) && workspace == nullptr) return SPA_ERR_INVALID_ARG;
+  return launch_linear_bwd_tc(*p, a, W, dout, n_in, n_out, cu_seqlens, dX, dW, db, workspace, d_status,
+                              (cudaStream_t)stream, idx, (p->flags & SPA_FLAG_RESIDUAL) != 0);
+}
+
 int spa_read_status(const int32_t* d_status, void* stream) {
   if (d_status == nullptr) return SPA_ERR_INVALID_ARG;
   int32_t v = 0;

@@ -89,6 +89,8 @@ struct TileCoord { int m0, n0, z, n_t; };
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... of the (m, n, split) space
 // that the device-side row count leaves; two accumulator stages in TMEM let the epilogue of one tile
 // overlap the main loop of the next, and the TMA ring runs ahead across tile boundaries.
+// row_map (optional): output row i goes to row row_map[i] of `out` (the unpack scatter fused into the
+// epilogue); with `accumulate` the bf16 result is added to what that row holds.
 // kColSum (wgrad only): while the MMAs run, the epilogue warps add up the columns of the dout tiles
 // that stream through shared memory, which gives the bias gradient at no extra HBM traffic.
 template <int BN, bool kAMn, bool kBMn, typename OutT, bool kColSum>
@@ -96,7 +98,8 @@ __global__ void __launch_bounds__(kGemmThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
                long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
-               int dyn_which, int k_per_split, float* __restrict__ colsum_part, int32_t* d_status) {
+               int dyn_which, int k_per_split, float* __restrict__ colsum_part, const int32_t* __restrict__ row_map,
+               int accumulate, int32_t* d_status) {
   constexpr int kStage = stage_bytes<BN>();
   constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
   pdl_launch_dependents();
@@ -301,6 +304,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       constexpr int kPasses = sizeof(OutT) == 2 ? 1 : 2;        // 64-byte segments per 32 accumulator columns
       constexpr int kSegCols = 64 / (int)sizeof(OutT);          // output columns per segment
       const int my_chunk = lane & 3, my_row = lane >> 2;        // role of this lane on the store side
+      long long orow[4];                                        // destination rows of the four rows this lane stores
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int grow = c.m0 + q * 32 + my_row + 8 * j;
+        orow[j] = (row_map != nullptr && grow < M) ? (long long)__ldg(row_map + grow) : (long long)grow;
+      }
 #pragma unroll 1
       for (int cc = 0; cc < BN / 32; ++cc) {
         uint32_t r[32];
@@ -335,7 +344,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint4 v4 = *reinterpret_cast<const uint4*>(stage + rr * 64 + ((my_chunk ^ ((rr >> 1) & 3)) << 4));
             const int grow = c.m0 + q * 32 + rr;
             const int gcol = c.n0 + cc * 32 + ps * kSegCols + my_chunk * (16 / (int)sizeof(OutT));
-            if (grow < M && gcol < N) *reinterpret_cast<uint4*>(obase + (long long)grow * ldo + gcol) = v4;
+            if (grow < M && gcol < N) {
+              uint4* dst = reinterpret_cast<uint4*>(obase + orow[j] * ldo + gcol);
+              if (sizeof(OutT) == 2 && accumulate) {
+                float fa[8], fb[8];
+                Vec16<__nv_bfloat16>::to_float(*dst, fa);
+                Vec16<__nv_bfloat16>::to_float(v4, fb);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) fa[e] += fb[e];
+                *dst = Vec16<__nv_bfloat16>::from_float(fa);
+              } else {
+                *dst = v4;
+              }
+            }
           }
           __syncwarp();
         }
@@ -438,7 +459,8 @@ size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
 template <int BN, bool kAMn, bool kBMn, typename OutT, bool kColSum>
 int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloat16* bias, OutT* out, long long ldo,
                 long long split_stride, int M, int N, int K, const int32_t* cu, int n_seg, int capacity, int dyn_which,
-                int k_per_split, int splits, float* colsum_part, int32_t* d_status, cudaStream_t st, const char* what) {
+                int k_per_split, int splits, float* colsum_part, const int32_t* row_map, int accumulate,
+                int32_t* d_status, cudaStream_t st, const char* what) {
   auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT, kColSum>;
   static bool attr_set = false;  // per instantiation
   if (!attr_set) {
@@ -451,7 +473,7 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
   long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * splits;
   const int grid = (int)(tiles < 2 * kNumSMs ? (tiles < 1 ? 1 : tiles) : 2 * kNumSMs);
   launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu,
-             n_seg, capacity, dyn_which, k_per_split, colsum_part, d_status);
+             n_seg, capacity, dyn_which, k_per_split, colsum_part, row_map, accumulate, d_status);
   SPA_CUDA_CHECK_LAUNCH(what);
   return SPA_OK;
 }
@@ -470,20 +492,21 @@ size_t tc_linear_workspace_bytes(const spa_params& p) {
 }
 
 int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
-                         const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st) {
+                         const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st, const int32_t* row_map,
+                         bool accumulate) {
   CUtensorMap tmA, tmB;
   if (!make_tmap_bf16_2d(&tmA, a, n_in, p.capacity, (uint64_t)n_in * 2, BK, BM) ||
       !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, BK, 128))
     return SPA_ERR_UNSUPPORTED;
   return launch_gemm<128, false, false, __nv_bfloat16, false>(tmA, tmB, (const __nv_bfloat16*)bias,
                                                               (__nv_bfloat16*)out, n_out, 0, p.capacity, n_out, n_in,
-                                                              cu, p.B, p.capacity, 1, n_in, 1, nullptr, d_status, st,
-                                                              "gemm_tc_kernel(fwd)");
+                                                              cu, p.B, p.capacity, 1, n_in, 1, nullptr, row_map,
+                                                              accumulate ? 1 : 0, d_status, st, "gemm_tc_kernel(fwd)");
 }
 
 int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
                          const int32_t* cu, void* da, float* dW, float* db, void* workspace, int32_t* d_status,
-                         cudaStream_t st) {
+                         cudaStream_t st, const int32_t* row_map, bool accumulate) {
   CUtensorMap tmA, tmB, tmA2, tmB2;
   if (da != nullptr && (!make_tmap_bf16_2d(&tmA, dout, n_out, p.capacity, (uint64_t)n_out * 2, BK, BM) ||
                         !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, 64, BK)))
@@ -494,7 +517,8 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
     int rc = launch_gemm<128, false, true, __nv_bfloat16, false>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
                                                                  p.capacity, n_in, n_out, cu, p.B, p.capacity, 1, n_out,
-                                                                 1, nullptr, d_status, st, "gemm_tc_kernel(dgrad)");
+                                                                 1, nullptr, row_map, accumulate ? 1 : 0, d_status, st,
+                                                                 "gemm_tc_kernel(dgrad)");
     if (rc != SPA_OK) return rc;
   }
   if (dW == nullptr && db == nullptr) return SPA_OK;
@@ -507,12 +531,12 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
     int rc;
     if (db != nullptr)
       rc = launch_gemm<128, true, true, float, true>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity, cu,
-                                                     p.B, p.capacity, 2, sp.k_per_split, sp.splits, part_b, d_status, st,
-                                                     "gemm_tc_kernel(wgrad+colsum)");
+                                                     p.B, p.capacity, 2, sp.k_per_split, sp.splits, part_b, nullptr, 0, d_status,
+                                                     st, "gemm_tc_kernel(wgrad+colsum)");
     else
       rc = launch_gemm<128, true, true, float, false>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity,
-                                                      cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr,
-                                                      d_status, st, "gemm_tc_kernel(wgrad)");
+                                                      cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr, nullptr,
+                                                      0, d_status, st, "gemm_tc_kernel(wgrad)");
     if (rc != SPA_OK) return rc;
     const long long n_b = db != nullptr ? n_out : 0;
     int grid = (int)(((n_w + n_b) / 4 + 255) / 256);

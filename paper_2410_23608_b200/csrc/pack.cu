@@ -227,6 +227,23 @@ int stream_grid(long long total_chunks) {
   return g < 1 ? 1 : (int)g;
 }
 
+// dst = src over `total` 16-byte chunks: the pass-through rows of the unpack step written ahead of
+// time, so that the projection (or the input-gradient product) only has to scatter the selected rows.
+__global__ void __launch_bounds__(kPackThreads)
+copy_chunks_kernel(const uint4* __restrict__ src16, uint4* __restrict__ dst16, long long total) {
+  pdl_entry();
+  const long long stride = (long long)gridDim.x * kPackThreads;
+  for (long long k0 = (long long)blockIdx.x * kPackThreads + threadIdx.x; k0 < total; k0 += stride * kBatch) {
+    uint4 v[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      if (k0 + u * stride < total) v[u] = ld_nc16(src16 + k0 + u * stride);
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      if (k0 + u * stride < total) dst16[k0 + u * stride] = v[u];
+  }
+}
+
 template <typename T> int chunks_per_row(int C) { return C / Vec16<T>::kElems; }
 
 }  // namespace
@@ -299,5 +316,13 @@ int launch_select_pack_bwd(const spa_params& p, const void* dxp, const void* dY,
   return SPA_OK;
 }
 #undef SPA_SCATTER
+
+int launch_copy_tokens(const spa_params& p, const void* src, void* dst, cudaStream_t st) {
+  const int Q = p.dtype == SPA_F32 ? chunks_per_row<float>(p.C) : chunks_per_row<__nv_bfloat16>(p.C);
+  const long long total = (long long)p.B * p.N * Q;
+  launch_pdl(copy_chunks_kernel, stream_grid(total), kPackThreads, 0, st, (const uint4*)src, (uint4*)dst, total);
+  SPA_CUDA_CHECK_LAUNCH("copy_chunks_kernel");
+  return SPA_OK;
+}
 
 }  // namespace spa

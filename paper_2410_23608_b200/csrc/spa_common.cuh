@@ -145,6 +145,7 @@ int launch_unpack_scatter_bwd(const spa_params& p, const void* dY, const int32_t
                               const int32_t* cu, void* dz, void* dX, cudaStream_t st);
 int launch_select_pack_bwd(const spa_params& p, const void* dxp, const void* dY, const int32_t* idx,
                            const int32_t* cu, void* dX, cudaStream_t st);
+int launch_copy_tokens(const spa_params& p, const void* src, void* dst, cudaStream_t st);  // dst[B*N][C] = src
 
 // out[M][n_out] = a[M][n_in] W[n_out][n_in]^T + bias, M = packed rows (device)
 int launch_linear_fwd_simt(const spa_params& p, const void* a, const void* W, const void* bias, int n_in,

@@ -9,11 +9,13 @@ size_t tc_linear_workspace_bytes(const spa_params& p);
 size_t tc_attention_workspace_bytes(const spa_params& p);
 
 bool tc_linear_supported(int n_in, int n_out);
+// row_map (optional): output row i is written to row row_map[i] of `out`, added to its contents if `accumulate`.
 int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
-                         const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st);
+                         const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st,
+                         const int32_t* row_map = nullptr, bool accumulate = false);
 int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
                          const int32_t* cu, void* da, float* dW, float* db, void* workspace, int32_t* d_status,
-                         cudaStream_t st);
+                         cudaStream_t st, const int32_t* row_map = nullptr, bool accumulate = false);
 
 bool tc_attention_fwd_supported(const spa_params& p);
 int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
