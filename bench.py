@@ -78,25 +78,44 @@ def work_model(cfg, cu):
         w[name + ".dW"] = dict(bytes=(Np * n_out + Np * C) * es + 4 * n_out * C, flops=2 * Np * C * n_out)
         w[name + ".db"] = dict(bytes=Np * n_out * es + 4 * n_out, flops=Np * n_out)
     w["pack_bwd"] = dict(bytes=2 * Np * C * es + 4 * Np, flops=0)
+    # fused unpack: the gate also writes y = x; the projection writes to the tokens (idx read per row)
+    w["gate_prefill"] = dict(bytes=2 * BN * C * es + 5 * BN, flops=2 * BN * C)
+    w["proj_scatter"] = dict(bytes=(2 * Np * C + C * C) * es + 4 * Np, flops=2 * Np * C * C)
     return w, Np, S2
 
 
 def call_sequence(L, blk, d, b_g):
-    """The block as (name, thunk) pairs, one per C-ABI call, in execution order."""
+    """The block as (name, thunk) pairs, one per C-ABI call, in the order SpaBlock issues them."""
     p, C = blk.p, blk.C
-    return [
+    head = [
         ("gate", lambda: L.spa_gate(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask)),
         ("select_pack", lambda: L.spa_select_pack(p, d["x"], blk.mask, blk.scores, blk.xp, blk.idx, blk.inv, blk.cu,
                                                   blk.status)),
         ("qkv", lambda: L.spa_packed_qkv(p, blk.xp, d["W_qkv"], d["b_qkv"], blk.cu, blk.qkv, blk.status)),
         ("attn_fwd", lambda: L.spa_packed_attention_fwd(p, blk.qkv, blk.cu, blk.B, blk.ao, blk.lse, blk.status)),
-        ("proj", lambda: L.spa_packed_proj(p, blk.ao, d["W_o"], d["b_o"], blk.cu, blk.z, blk.status)),
-        ("unpack", lambda: L.spa_unpack_scatter(p, blk.z, d["x"], blk.idx, blk.inv, blk.cu, blk.y, blk.status)),
-        ("unpack_bwd", lambda: L.spa_unpack_scatter_bwd(p, d["dY"], blk.idx, blk.inv, blk.cu, blk.dz, blk.dX)),
+    ]
+    mid = [
         ("proj_bwd", lambda: L.spa_packed_linear_bwd(p, blk.ao, d["W_o"], blk.dz, C, C, blk.cu, blk.dao, blk.dW_o,
                                                      blk.db_o, blk.workspace, blk.status)),
         ("attn_bwd", lambda: L.spa_packed_attention_bwd(p, blk.qkv, blk.ao, blk.lse, blk.dao, blk.cu, blk.B, blk.dqkv,
                                                         blk.workspace, blk.status)),
+    ]
+    if blk.fused:
+        head[0] = ("gate", lambda: L.spa_gate_prefill(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask, blk.y))
+        return head + [
+            ("proj_scatter", lambda: L.spa_packed_proj_scatter(p, blk.ao, d["W_o"], d["b_o"], blk.idx, blk.cu, blk.y,
+                                                               blk.status)),
+            ("unpack_bwd", lambda: L.spa_unpack_scatter_bwd(p, d["dY"], blk.idx, blk.inv, blk.cu, blk.dz, blk.dX)),
+        ] + mid + [
+            ("qkv_bwd", lambda: L.spa_packed_linear_bwd_scatter(p, blk.xp, d["W_qkv"], blk.dqkv, C, 3 * C, blk.idx,
+                                                                blk.cu, blk.dX, blk.dW_qkv, blk.db_qkv, blk.workspace,
+                                                                blk.status)),
+        ]
+    return head + [
+        ("proj", lambda: L.spa_packed_proj(p, blk.ao, d["W_o"], d["b_o"], blk.cu, blk.z, blk.status)),
+        ("unpack", lambda: L.spa_unpack_scatter(p, blk.z, d["x"], blk.idx, blk.inv, blk.cu, blk.y, blk.status)),
+        ("unpack_bwd", lambda: L.spa_unpack_scatter_bwd(p, d["dY"], blk.idx, blk.inv, blk.cu, blk.dz, blk.dX)),
+    ] + mid + [
         ("qkv_bwd", lambda: L.spa_packed_linear_bwd(p, blk.xp, d["W_qkv"], blk.dqkv, C, 3 * C, blk.cu, blk.dxp,
                                                     blk.dW_qkv, blk.db_qkv, blk.workspace, blk.status)),
         ("pack_bwd", lambda: L.spa_select_pack_bwd(p, blk.dxp, d["dY"], blk.idx, blk.cu, blk.dX)),
@@ -116,7 +135,9 @@ def timing_units(L, blk, d, b_g):
         ("proj_bwd.da", lin(blk.ao, d["W_o"], blk.dz, C, blk.dao, None, None)),
         ("proj_bwd.dW", lin(blk.ao, d["W_o"], blk.dz, C, None, blk.dW_o, None)),
         ("proj_bwd.db", lin(blk.ao, d["W_o"], blk.dz, C, None, None, blk.db_o)),
-        ("qkv_bwd.da", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, blk.dxp, None, None)),
+        ("qkv_bwd.da", (lambda: L.spa_packed_linear_bwd_scatter(p, blk.xp, d["W_qkv"], blk.dqkv, C, 3 * C, blk.idx, blk.cu,
+                                                                 blk.dX, None, None, None, blk.status))
+         if blk.fused else lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, blk.dxp, None, None)),
         ("qkv_bwd.dW", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, blk.dW_qkv, None)),
         ("qkv_bwd.db", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, None, blk.db_qkv)),
     ]
@@ -234,6 +255,7 @@ def main():
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="issue the weight gradients on the main stream too")
+    ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 2000 and args.warmup == 50:
@@ -270,7 +292,7 @@ def main():
         inp = make_inputs(scaled_config(cfg, seed=cfg.seed + 1000 * s)) if s < 2 else inps[s % 2]
         inps.append(inp)
         d = {n: inp.torch(n, "cuda") for n in names}
-        blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau)
+        blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau, fused=False if args.no_fuse else None)
         sets.append((inp, d, blk, call_sequence(L, blk, d, inp.b_g)))
 
     def capture(fns):
@@ -377,6 +399,8 @@ def main():
         unit_launches[name] = n_l // n_sets
     pk = peaks()
     work, Np0, S2 = work_model(cfg, sets[0][2].cu.cpu().numpy())
+    if sets[0][2].fused:
+        work["gate"] = work["gate_prefill"]
     per_call = {}
     for name, ms_c in call_ms.items():
         wk = work[name]
@@ -395,7 +419,11 @@ def main():
                 "peak_source": pk["source"], "us_per_launch": tr["us"]}
 
     # ---- forward-only time (same rotation), reported beside the headline
-    fwd_graphs = [capture([fn for _, fn in sets[s_][3][:6]])[0] for s_ in range(n_sets)]
+    def forward_only(s_):
+        inp_, d_, blk_, _ = sets[s_]
+        return lambda: blk_.forward(d_["x"], d_["w_g"], inp_.b_g, d_["W_qkv"], d_["b_qkv"], d_["W_o"], d_["b_o"])
+
+    fwd_graphs = [capture([forward_only(s_)])[0] for s_ in range(n_sets)]
     for i in range(n_sets):
         fwd_graphs[i].replay()
     torch.cuda.synchronize()
@@ -413,7 +441,8 @@ def main():
                "sample": f"whole {cfg.name} batch, forward+backward, {len(times)} repetitions "
                          f"({sum(times):.1f} s of CPU work)"}
 
-    useful_flops = sum(work[k]["flops"] for k in work)
+    useful_flops = sum(work[k]["flops"] for k in ("gate", "qkv", "attn_fwd", "proj", "attn_bwd", "proj_bwd.da",
+                                                  "proj_bwd.dW", "proj_bwd.db", "qkv_bwd.da", "qkv_bwd.dW", "qkv_bwd.db"))
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -422,6 +451,8 @@ def main():
                    "selected_tokens": Np_sets[0], "sum_nb_squared": S2, "pass": "forward+backward",
                    "l2_policy": f"{n_sets} rotating buffer sets (x alone {x_bytes * n_sets / 1e6:.0f} MB > L2)",
                    "launch": "one CUDA graph per step",
+                   "unpack": "scatter fused into the projection / input-gradient epilogues" if sets[0][2].fused
+                             else "separate scatter kernels",
                    "replicas": world},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 2 * bytes_io, "d2h_bytes_per_step": 2 * bytes_io},

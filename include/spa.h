@@ -165,8 +165,9 @@ int spa_unpack_scatter(const spa_params* p, const void* z_packed, const void* x,
                        void* stream);
 
 /* Transpose of spa_unpack_scatter:  dz_packed[i][:] = dY[idx[i]][:];  dX[t][:] = dY[t][:] for
- * unselected tokens t.  Selected rows of dX are left for spa_select_pack_bwd.  dX may equal dY
- * (nothing is copied for unselected rows then) or be NULL. */
+ * unselected tokens t.  Selected rows of dX are left for spa_select_pack_bwd (under
+ * SPA_FLAG_RESIDUAL they receive dY too, the term that the residual adds).  dX may equal dY
+ * (nothing is copied then) or be NULL. */
 int spa_unpack_scatter_bwd(const spa_params* p, const void* dY, const int32_t* idx,
                            const int32_t* inv, const int32_t* cu_seqlens, void* dz_packed, void* dX,
                            void* stream);
@@ -194,20 +195,25 @@ int spa_packed_linear_bwd(const spa_params* p, const void* a, const void* W, con
  * whether they apply; otherwise they return SPA_ERR_UNSUPPORTED and the unfused calls must be used. */
 int spa_fused_scatter_supported(const spa_params* p);
 
+/* spa_gate that also writes y[B][N][C] = x while it reads x (nothing is copied when y == x): the
+ * pass-through rows of the fused unpack at no second read of x. */
+int spa_gate_prefill(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up,
+                     float* scores, uint8_t* mask, void* y, void* stream);
+
 /* dst[B][N][C] = src[B][N][C]: writes the pass-through rows ahead of the scatter (y = x in the
  * forward pass, dX = dY in the backward pass).  A no-op when dst == src. */
 int spa_unpack_prefill(const spa_params* p, const void* src, void* dst, void* stream);
 
 /* Output projection with the unpack scatter in its epilogue:  y[idx[i]][:] = b_o + W_o a[i][:]
  * (added to y[idx[i]][:] under SPA_FLAG_RESIDUAL).  y: T[B][N][C] must already hold x
- * (spa_unpack_prefill, or y aliasing x); rows of unselected tokens are not touched. */
+ * (spa_gate_prefill, spa_unpack_prefill, or y aliasing x); rows of unselected tokens are not touched. */
 int spa_packed_proj_scatter(const spa_params* p, const void* a, const void* W_o, const void* b_o,
                             const int32_t* idx, const int32_t* cu_seqlens, void* y, int32_t* d_status,
                             void* stream);
 
 /* spa_packed_linear_bwd with the transpose of the pack gather in the epilogue of the input gradient:
  * dX[idx[i]][:] = dout[i][:] W  (added to dX[idx[i]][:] under SPA_FLAG_RESIDUAL, where dX must
- * already hold dY).  n_in must equal C; dW, db and workspace as in spa_packed_linear_bwd. */
+ * already hold dY: spa_unpack_scatter_bwd copies those rows too when the flag is set).  n_in must equal C; dW, db and workspace as in spa_packed_linear_bwd. */
 int spa_packed_linear_bwd_scatter(const spa_params* p, const void* a, const void* W, const void* dout,
                                   int32_t n_in, int32_t n_out, const int32_t* idx,
                                   const int32_t* cu_seqlens, void* dX, float* dW, float* db,

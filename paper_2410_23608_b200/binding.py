@@ -27,7 +27,7 @@ EXPORTS = (
     "spa_packed_attention_bwd", "spa_packed_proj", "spa_unpack_scatter", "spa_unpack_scatter_bwd",
     "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
     "spa_last_cuda_error", "spa_launch_count", "spa_packed_attention_bwd_static",
-    "spa_fused_scatter_supported", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
+    "spa_fused_scatter_supported", "spa_gate_prefill", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
 )
 
 
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         L.spa_select_pack_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp]
         L.spa_packed_linear_bwd.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.spa_fused_scatter_supported.argtypes = [pp]
+        L.spa_gate_prefill.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp, vp]
         L.spa_unpack_prefill.argtypes = [pp, vp, vp, vp]
         L.spa_packed_proj_scatter.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_packed_linear_bwd_scatter.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -182,6 +183,11 @@ def spa_packed_linear_bwd(p, a, W, dout, n_in, n_out, cu_seqlens, da, dW, db, wo
 
 def spa_fused_scatter_supported(p) -> bool:
     return bool(lib().spa_fused_scatter_supported(C.byref(p)))
+
+
+def spa_gate_prefill(p, x, w_g, b_g, s_up, scores, mask, y, stream=None):
+    _check(lib().spa_gate_prefill(C.byref(p), _ptr(x), _ptr(w_g), float(b_g), _ptr(s_up), _ptr(scores), _ptr(mask),
+                                  _ptr(y), _stream(stream)), "spa_gate_prefill")
 
 
 def spa_unpack_prefill(p, src, dst, stream=None):

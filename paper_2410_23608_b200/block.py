@@ -53,8 +53,7 @@ class SpaBlock:
         self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if ws > 0 else None
         # the weight gradients do not feed the rest of the backward chain: they run on a second stream,
         # with a scratch area of their own, beside the attention backward and the input gradients
-        self.side_stream = torch.cuda.Stream(device=dev) if (backward or self.fused) else None
-        self._prefilled = torch.cuda.Event() if self.fused else None
+        self.side_stream = torch.cuda.Stream(device=dev) if backward else None
         self.workspace_side = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if (ws > 0 and backward) else None
         if backward:
             self.dz = e(cap, C)
@@ -74,19 +73,16 @@ class SpaBlock:
         y = self.y if y is None else y
         inplace = bool(p.flags & L.SPA_FLAG_INPLACE)
         if self.fused and not inplace:
-            # the pass-through rows do not depend on anything the block computes: y = x runs beside the chain
-            main, side = torch.cuda.current_stream(), self.side_stream
-            side.wait_stream(main)
-            L.spa_unpack_prefill(p, x, y, stream=side)
-        L.spa_gate(p, x, w_g, b_g, s_up, self.scores, self.mask)
+            # the pass-through rows y = x are written by the gate, which reads all of x anyway
+            L.spa_gate_prefill(p, x, w_g, b_g, s_up, self.scores, self.mask, y)
+        else:
+            L.spa_gate(p, x, w_g, b_g, s_up, self.scores, self.mask)
         L.spa_select_pack(p, x, self.mask, self.scores, self.xp, self.idx, self.inv, self.cu, self.status)
         L.spa_packed_qkv(p, self.xp, W_qkv, b_qkv, self.cu, self.qkv, self.status)
         L.spa_packed_attention_fwd(p, self.qkv, self.cu, self.B, self.ao, self.lse, self.status)
         if self.fused:
             if inplace:
                 y = x
-            else:
-                main.wait_stream(side)
             L.spa_packed_proj_scatter(p, self.ao, W_o, b_o, self.idx, self.cu, y, self.status)
         else:
             L.spa_packed_proj(p, self.ao, W_o, b_o, self.cu, self.z, self.status)
@@ -109,21 +105,9 @@ class SpaBlock:
         C = self.C
         main = torch.cuda.current_stream()
         side = self.side_stream if (overlap and self.side_stream is not None) else None
-        if self.fused:
-            # dX = dY ahead of time (beside the chain when there is a second stream); the QKV input gradient
-            # then scatters its rows to the selected tokens itself, and dz is a plain gather
-            prefill_on_side = False
-            if dX is not dY and dX.data_ptr() != dY.data_ptr():
-                if side is not None:
-                    prefill_on_side = True
-                    side.wait_stream(main)
-                    L.spa_unpack_prefill(p, dY, dX, stream=side)
-                    self._prefilled.record(side)
-                else:
-                    L.spa_unpack_prefill(p, dY, dX)
-            L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, None)
-        else:
-            L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
+        # dz = gather of dY; dX = dY on the tokens that passed through (fused path: the QKV input gradient
+        # scatters its rows to the selected tokens itself, so no packed dx and no scatter kernel follow)
+        L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
         if side is None:
             L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
                                     self.workspace, self.status)
@@ -143,8 +127,6 @@ class SpaBlock:
                 side.wait_stream(main)
                 L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, None, self.dW_qkv,
                                         self.db_qkv, self.workspace_side, self.status, stream=side)
-                if prefill_on_side:
-                    main.wait_event(self._prefilled)
                 L.spa_packed_linear_bwd_scatter(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.idx, self.cu, dX,
                                                 None, None, None, self.status)
                 main.wait_stream(side)

@@ -70,7 +70,15 @@ int spa_gate(const spa_params* p, const void* x, const void* w_g, float b_g, con
   int rc = check_params(p);
   if (rc != SPA_OK) return rc;
   SPA_PTR(x); SPA_PTR(w_g); SPA_PTR(scores); SPA_PTR(mask); SPA_OPT_PTR(s_up);
-  return launch_gate(*p, x, w_g, b_g, s_up, scores, mask, (cudaStream_t)stream);
+  return launch_gate(*p, x, w_g, b_g, s_up, scores, mask, nullptr, (cudaStream_t)stream);
+}
+
+int spa_gate_prefill(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up, float* scores,
+                     uint8_t* mask, void* y, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(w_g); SPA_PTR(scores); SPA_PTR(mask); SPA_PTR(y); SPA_OPT_PTR(s_up);
+  return launch_gate(*p, x, w_g, b_g, s_up, scores, mask, y == x ? nullptr : y, (cudaStream_t)stream);
 }
 
 int spa_select_pack(const spa_params* p, const void* x, const uint8_t* mask, const float* scores, void* x_packed,

@@ -1,7 +1,8 @@
 // Gate GEMV fused with the hard threshold (Sec. 3.2, Eq. 4 and the deterministic form of Eq. 6).
 //
 // HBM-bound: every element of x is read exactly once with 16-byte streaming loads; the only
-// writes are 4 B (score) + 1 B (mask) per token.  One warp owns kGateRows token rows at a time so
+// writes are 4 B (score) + 1 B (mask) per token - plus, on request, the copy y = x that the fused
+// unpack needs for the tokens that pass through, which costs no second read of x.  One warp owns kGateRows token rows at a time so
 // that several independent 16-byte loads per lane are in flight; w_g sits in shared memory as fp32.
 #include "spa_common.cuh"
 
@@ -14,7 +15,7 @@ constexpr int kGateRows = 2;  // rows per warp per iteration
 template <typename T>
 __global__ void __launch_bounds__(kGateThreads)
 gate_kernel(const T* __restrict__ x, const T* __restrict__ w_g, float b_g, const float* __restrict__ s_up,
-            float tau, int rows, int C, float* __restrict__ scores, uint8_t* __restrict__ mask) {
+            float tau, int rows, int C, float* __restrict__ scores, uint8_t* __restrict__ mask, uint4* __restrict__ y16) {
   pdl_entry();
   constexpr int E = Vec16<T>::kElems;
   extern __shared__ float w_s[];
@@ -37,6 +38,11 @@ gate_kernel(const T* __restrict__ x, const T* __restrict__ w_g, float b_g, const
 #pragma unroll
       for (int k = 0; k < kGateRows; ++k)
         if (r0 + k < rows) v[k] = ld_nc16(x16 + (size_t)(r0 + k) * Q + q);
+      if (y16 != nullptr) {  // pass-through copy y = x rides on the one read of x
+#pragma unroll
+        for (int k = 0; k < kGateRows; ++k)
+          if (r0 + k < rows) y16[(size_t)(r0 + k) * Q + q] = v[k];
+      }
       const float4* wq = reinterpret_cast<const float4*>(w_s + q * E);
       float w[E];
 #pragma unroll
@@ -70,7 +76,7 @@ gate_kernel(const T* __restrict__ x, const T* __restrict__ w_g, float b_g, const
 }  // namespace
 
 int launch_gate(const spa_params& p, const void* x, const void* w_g, float b_g, const float* s_up,
-                float* scores, uint8_t* mask, cudaStream_t st) {
+                float* scores, uint8_t* mask, void* y, cudaStream_t st) {
   const int rows = p.B * p.N;
   if (rows == 0) return SPA_OK;
   const int warps = kGateThreads / 32;
@@ -79,10 +85,10 @@ int launch_gate(const spa_params& p, const void* x, const void* w_g, float b_g, 
   const size_t smem = (size_t)p.C * sizeof(float);
   if (p.dtype == SPA_F32)
     launch_pdl(gate_kernel<float>, grid, kGateThreads, smem, st, (const float*)x, (const float*)w_g, b_g, s_up, p.tau,
-                                                         rows, p.C, scores, mask);
+                                                         rows, p.C, scores, mask, (uint4*)y);
   else
     launch_pdl(gate_kernel<__nv_bfloat16>, grid, kGateThreads, smem, st, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_g,
-                                                                 b_g, s_up, p.tau, rows, p.C, scores, mask);
+                                                                 b_g, s_up, p.tau, rows, p.C, scores, mask, (uint4*)y);
   SPA_CUDA_CHECK_LAUNCH("gate_kernel");
   return SPA_OK;
 }

@@ -191,7 +191,7 @@ row_scatter_kernel(const uint4* __restrict__ src16, const uint4* addp, const int
 __global__ void __launch_bounds__(kPackThreads)
 unpack_scatter_bwd_kernel(const uint4* __restrict__ dY16, const int32_t* __restrict__ inv,
                           const int32_t* __restrict__ cu, int B, int capacity, long long total, int Q,
-                          uint4* __restrict__ dz16, uint4* dX16, bool copy_pass_through) {
+                          uint4* __restrict__ dz16, uint4* dX16, bool copy_pass_through, bool copy_selected) {
   pdl_entry();
   const int Np = packed_rows(cu, B, capacity);
   const long long stride = (long long)gridDim.x * kPackThreads;
@@ -214,8 +214,12 @@ unpack_scatter_bwd_kernel(const uint4* __restrict__ dY16, const int32_t* __restr
 #pragma unroll
     for (int u = 0; u < kBatch; ++u) {
       const long long k = k0 + u * stride;
-      if (o[u] >= 0) dz16[o[u]] = v[u];
-      else if (o[u] == -1) dX16[k] = v[u];
+      if (o[u] >= 0) {
+        dz16[o[u]] = v[u];
+        if (copy_selected) dX16[k] = v[u];
+      } else if (o[u] == -1) {
+        dX16[k] = v[u];
+      }
     }
   }
 }
@@ -299,7 +303,8 @@ int launch_unpack_scatter_bwd(const spa_params& p, const void* dY, const int32_t
   const long long total = (long long)p.B * p.N * Q;
   const bool copy = dX != nullptr && dX != dY;
   launch_pdl(unpack_scatter_bwd_kernel, stream_grid(total), kPackThreads, 0, st, (const uint4*)dY, inv, cu, p.B, p.capacity,
-                                                                        total, Q, (uint4*)dz, (uint4*)dX, copy);
+                                                                        total, Q, (uint4*)dz, (uint4*)dX, copy,
+                                                                        copy && (p.flags & SPA_FLAG_RESIDUAL) != 0);
   SPA_CUDA_CHECK_LAUNCH("unpack_scatter_bwd_kernel");
   return SPA_OK;
 }

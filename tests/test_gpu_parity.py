@@ -162,6 +162,52 @@ def test_residual_and_inplace_flags(ci, fused, flags):
     assert blk.read_status() == 0
 
 
+def test_fused_calls_on_oracle_upstream():
+    """spa_unpack_prefill + spa_packed_proj_scatter, and spa_packed_linear_bwd_scatter, each fed the oracle's
+    own upstream tensors."""
+    from paper_2410_23608_b200 import binding as L
+    cfg, inp, fwd, bwd = problem(2)
+    dt = cfg.dtype
+    d = device_inputs(cfg, inp)
+    blk = make_block(cfg)
+    p, C, cap = blk.p, cfg.C, blk.cap
+    assert L.spa_fused_scatter_supported(p)
+    Np = int(fwd["cu_seqlens"][-1])
+    cu = torch.from_numpy(fwd["cu_seqlens"]).cuda()
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    idx[:Np] = torch.from_numpy(fwd["idx"]).cuda()
+
+    def padded(a, cols):
+        buf = np.zeros((cap, cols))
+        buf[:Np] = a
+        return buf
+
+    # forward: y = x, then the projection writes the selected rows
+    y = torch.empty_like(d["x"])
+    L.spa_unpack_prefill(p, d["x"], y)
+    assert torch.equal(y, d["x"])
+    ao_r = round_to(fwd["ao"], dt)
+    L.spa_packed_proj_scatter(p, dev(padded(ao_r, C), dt), d["W_o"], d["b_o"], idx, cu, y, blk.status)
+    y_ref = O.unpack_scatter(O.linear(ao_r, inp.W_o, inp.b_o), inp.x, fwd["idx"])
+    assert_close(host(y), y_ref, dt, "y")
+    unsel = ~fwd["mask"]
+    assert np.array_equal(host(y)[unsel], inp.x[unsel])
+    # backward: dX = dY, then the input gradient of the QKV layer writes the selected rows
+    dX = torch.empty_like(d["dY"])
+    L.spa_unpack_prefill(p, d["dY"], dX)
+    dqkv_r = round_to(bwd["dqkv"], dt)
+    da_ref, dW_ref, db_ref = O.linear_bwd(fwd["xp"], inp.W_qkv, dqkv_r)
+    L.spa_packed_linear_bwd_scatter(p, dev(padded(fwd["xp"], C), dt), d["W_qkv"], dev(padded(dqkv_r, 3 * C), dt), C,
+                                    3 * C, idx, cu, dX, blk.dW_qkv, blk.db_qkv, blk.workspace, blk.status)
+    dX_ref = O.select_pack_bwd(da_ref, fwd["idx"], O.unpack_scatter_bwd(inp.dY, fwd["idx"])[1])
+    assert_close(host(dX), dX_ref, dt, "dX", scale_max_abs=True)
+    assert np.array_equal(host(dX)[unsel], inp.dY[unsel])
+    assert_close(host(blk.dW_qkv), dW_ref, dt, "dW_qkv", scale_max_abs=True)
+    assert_close(host(blk.db_qkv), db_ref, dt, "db_qkv", scale_max_abs=True)
+    torch.cuda.synchronize()
+    assert blk.read_status() == 0
+
+
 def test_fused_scatter_matches_separate_kernels_bitwise():
     """The fused calls round exactly as the separate projection + scatter kernels do."""
     cfg, inp, fwd, bwd = problem(2, True)
