@@ -295,3 +295,93 @@ def mac_count(B, N, C, cu_seqlens):
     S2 = int((n * n).sum())
     return dict(gate=B * N * C, qkv=3 * Np * C * C, attn=2 * C * S2, proj=Np * C * C,
                 Np=Np, S2=S2)
+
+
+# --------------------------------------------------------------------------- trainable selection
+# Multi-scale supervised selection (Sec. 3.2) and the selection loss (Sec. 3.3, Eq. 10), with the
+# gradients that make the gate trainable when the sigmoid scaling of Eq. 5 is on.  Readings fixed
+# here: the up-scale scores reach the current scale by a 2x2 max-pool (each stage halves the grid);
+# the loss is the sum over all B*N tokens of one block; "Max" in Eq. 4 passes its gradient to the
+# larger argument (to s_up on a tie); the hard selection itself has no gradient.
+
+def score_pool(scores_prev, B, rows, cols):
+    """Scores of the previous (finer) stage, [B, 2*rows, 2*cols], max-pooled 2x2 to this stage's
+    grid: s_up [B, rows*cols] (Sec. 3.2: scores from up-scaled features, adjusted via max-pooling)."""
+    s = np.asarray(scores_prev, F64).reshape(B, rows, 2, cols, 2)
+    return s.max(axis=(2, 4)).reshape(B, rows * cols)
+
+
+def sigmoid(s):
+    return 1.0 / (1.0 + np.exp(-np.asarray(s, F64)))
+
+
+def select_loss(s, labels):
+    """Selection loss of one block, Eq. 10: -sum(y log p + (1-y) log(1-p)), p = Sigmoid(s).
+
+    Returns the loss and its gradient with respect to the logits s (p - y)."""
+    s = np.asarray(s, F64)
+    y = np.asarray(labels, F64)
+    p = sigmoid(s)
+    # log p and log(1-p) written through softplus so that large |s| does not overflow
+    log_p = -np.logaddexp(0.0, -s)
+    log_1mp = -np.logaddexp(0.0, s)
+    loss = -(y * log_p + (1.0 - y) * log_1mp).sum()
+    return loss, p - y
+
+
+def pack_rows_bwd(dxp, x, s, idx, gate_scale=False):
+    """Backward of pack_rows: gradient to the gathered rows of x and, with the sigmoid scaling of
+    Eq. 5, to the logits of the selected tokens.
+
+    xp_i = Sigmoid(s_t) x_t (t = idx[i])  =>  dx_t = Sigmoid(s_t) dxp_i,
+    ds_t = Sigmoid'(s_t) (dxp_i . x_t) with Sigmoid' = p (1 - p)."""
+    dxp = np.asarray(dxp, F64)
+    x2 = np.asarray(x, F64).reshape(-1, np.shape(x)[-1])
+    ds = np.zeros(x2.shape[0], F64)
+    if not gate_scale:
+        return dxp.copy(), ds
+    p = sigmoid(np.asarray(s, F64).reshape(-1)[idx])
+    ds[idx] = p * (1.0 - p) * (dxp * x2[idx]).sum(axis=1)
+    return dxp * p[:, None], ds
+
+
+def gate_bwd(ds, x, w_g, s, s_up=None):
+    """Backward of gate(): ds [B*N] is the gradient with respect to the logits s = Max(f_g(r), s_up).
+
+    Where the linear layer supplied the maximum (always, without s_up) the gradient goes to it:
+    dx_t += ds_t w_g, dw_g = sum_t ds_t x_t, db_g = sum_t ds_t; elsewhere it goes to s_up."""
+    x2 = np.asarray(x, F64).reshape(-1, np.shape(x)[-1])
+    ds = np.asarray(ds, F64).reshape(-1)
+    if s_up is None:
+        lin = np.ones(ds.shape, bool)
+    else:
+        lin = np.asarray(s, F64).reshape(-1) > np.asarray(s_up, F64).reshape(-1)
+    ds_lin = np.where(lin, ds, 0.0)
+    dx = ds_lin[:, None] * np.asarray(w_g, F64)[None, :]
+    dw_g = ds_lin @ x2
+    db_g = ds_lin.sum()
+    ds_up = np.where(lin, 0.0, ds)
+    return dx.reshape(np.shape(x)), dw_g, db_g, ds_up
+
+
+def block_bwd_trainable(fwd, dY, x, w_g, W_qkv, W_o, H, labels=None, alpha=1.0, s_up=None, residual=False,
+                        gate_scale=True, scale=None):
+    """Backward of block_fwd(..., gate_scale=...) for the total alpha * select_loss + <y, dY>:
+    block_bwd plus the gradient through the sigmoid scaling (Eq. 5), the selection loss (Eq. 10)
+    and the gate's linear layer (Eq. 4).  Returns block_bwd's dict extended by ds (gradient at the
+    logits), dw_g, db_g, ds_up, loss."""
+    idx = fwd["idx"]
+    dz, dX = unpack_scatter_bwd(dY, idx, residual)
+    dao, dW_o, db_o = linear_bwd(fwd["ao"], W_o, dz)
+    dqkv = attention_bwd(fwd["qkv"], fwd["ao"], fwd["lse"], dao, fwd["seg"], H, scale)
+    dxp, dW_qkv, db_qkv = linear_bwd(fwd["xp"], W_qkv, dqkv)
+    dx_sel, ds = pack_rows_bwd(dxp, x, fwd["scores"], idx, gate_scale)
+    dX = select_pack_bwd(dx_sel, idx, dX)
+    loss = 0.0
+    if labels is not None:
+        loss, dl = select_loss(fwd["scores"].reshape(-1), np.asarray(labels, F64).reshape(-1))
+        ds = ds + alpha * dl
+    dx_gate, dw_g, db_g, ds_up = gate_bwd(ds, x, w_g, fwd["scores"], s_up)
+    dX = dX + dx_gate
+    return dict(dz=dz, dao=dao, dqkv=dqkv, dxp=dxp, dX=dX, dW_o=dW_o, db_o=db_o, dW_qkv=dW_qkv, db_qkv=db_qkv,
+                ds=ds, dw_g=dw_g, db_g=db_g, ds_up=ds_up, loss=loss)

@@ -355,3 +355,104 @@ def test_full_config_shapes_run():
     fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
     frac = fwd["mask"].mean(axis=1)
     assert np.all(np.abs(frac - inp.keep_target) < 0.08)
+
+
+# ------------------------------------------------------------------ trainable selection (Eq. 4-6 with scaling, Eq. 10)
+def test_score_pool_against_loops():
+    rng = np.random.default_rng(40)
+    B, rows, cols = 2, 3, 4
+    prev = rng.normal(size=(B, 2 * rows, 2 * cols))
+    got = O.score_pool(prev, B, rows, cols)
+    for b in range(B):
+        for i in range(rows):
+            for j in range(cols):
+                want = max(prev[b, 2 * i + di, 2 * j + dj] for di in (0, 1) for dj in (0, 1))
+                assert got[b, i * cols + j] == want
+
+
+def test_select_loss_closed_forms():
+    # all logits zero: every token contributes ln 2, whatever its label; gradient is 1/2 - y
+    y = np.array([0.0, 1.0, 1.0, 0.0, 1.0])
+    loss, g = O.select_loss(np.zeros(5), y)
+    assert abs(loss - 5 * np.log(2.0)) < 1e-14
+    np.testing.assert_allclose(g, 0.5 - y, atol=1e-15)
+    # one token, logit = ln 3 => p = 3/4: loss -ln(3/4) for y = 1, -ln(1/4) for y = 0
+    l1, g1 = O.select_loss(np.array([np.log(3.0)]), np.array([1.0]))
+    l0, g0 = O.select_loss(np.array([np.log(3.0)]), np.array([0.0]))
+    assert abs(l1 + np.log(0.75)) < 1e-14 and abs(l0 + np.log(0.25)) < 1e-14
+    assert abs(g1[0] + 0.25) < 1e-14 and abs(g0[0] - 0.75) < 1e-14
+    # against the library's binary cross entropy on logits, and no overflow far from zero
+    rng = np.random.default_rng(41)
+    s = rng.normal(size=50) * 30
+    yy = (rng.uniform(size=50) > 0.5).astype(np.float64)
+    ref = torch.nn.functional.binary_cross_entropy_with_logits(torch.from_numpy(s), torch.from_numpy(yy), reduction="sum")
+    loss, _ = O.select_loss(s, yy)
+    assert np.isfinite(loss) and abs(loss - float(ref)) <= 1e-10 * max(1.0, abs(float(ref)))
+
+
+def _trainable_total(p, G, labels, alpha, s_up, residual):
+    fwd = O.block_fwd(**p, s_up=s_up, residual=residual, gate_scale=True)
+    loss, _ = O.select_loss(fwd["scores"].reshape(-1), labels.reshape(-1))
+    return float((fwd["y"] * G).sum()) + alpha * loss, fwd
+
+
+@pytest.mark.parametrize("residual", [False, True])
+def test_trainable_backward_against_central_differences(residual):
+    """Total = <y, G> + alpha * selection loss with the sigmoid scaling on and an up-scale score map:
+    gradients to x, w_g, b_g and s_up (and the layer weights) against central differences.  The
+    perturbations are far smaller than the distance of every logit from the threshold and from
+    s_up, so neither the selection nor the winner of Max changes."""
+    p = tiny_problem(seed=42, B=2, N=8, C=6, H=2, keep=0.6)
+    p["b_g"] += 0.037   # tiny_problem puts one logit exactly on the threshold
+    rng = np.random.default_rng(43)
+    G = rng.normal(size=p["x"].shape)
+    labels = (rng.uniform(size=(2, 8)) > 0.5).astype(np.float64)
+    s_lin = O.gate(p["x"], p["w_g"], p["b_g"])
+    s_up = s_lin + rng.choice([-0.7, 0.9], size=s_lin.shape)   # wins on some tokens, loses on others
+    alpha = 0.3
+    _, fwd = _trainable_total(p, G, labels, alpha, s_up, residual)
+    assert 2 < fwd["idx"].size < 16
+    assert np.abs(fwd["scores"] - p["tau"]).min() > 1e-3
+    bwd = O.block_bwd_trainable(fwd, G, p["x"], p["w_g"], p["W_qkv"], p["W_o"], p["H"], labels=labels, alpha=alpha,
+                                s_up=s_up, residual=residual, gate_scale=True)
+    h = 1e-6
+    grads = {"x": bwd["dX"], "w_g": bwd["dw_g"], "W_qkv": bwd["dW_qkv"], "W_o": bwd["dW_o"], "b_o": bwd["db_o"]}
+    for name, grad in grads.items():
+        base = p[name]
+        num = np.zeros_like(base)
+        it = np.nditer(base, flags=["multi_index"])
+        for _ in it:
+            i = it.multi_index
+            pp = dict(p); a = base.copy(); a[i] += h; pp[name] = a
+            pm = dict(p); c = base.copy(); c[i] -= h; pm[name] = c
+            num[i] = (_trainable_total(pp, G, labels, alpha, s_up, residual)[0] -
+                      _trainable_total(pm, G, labels, alpha, s_up, residual)[0]) / (2 * h)
+        assert np.abs(num - grad).max() / max(np.abs(num).max(), 1e-12) <= 1e-6, name
+    # scalar bias of the gate
+    pp = dict(p); pp["b_g"] = p["b_g"] + h
+    pm = dict(p); pm["b_g"] = p["b_g"] - h
+    num_b = (_trainable_total(pp, G, labels, alpha, s_up, residual)[0] -
+             _trainable_total(pm, G, labels, alpha, s_up, residual)[0]) / (2 * h)
+    assert abs(num_b - bwd["db_g"]) <= 1e-6 * max(abs(num_b), 1e-12)
+    # the up-scale scores
+    num_up = np.zeros_like(s_up)
+    for i in np.ndindex(*s_up.shape):
+        a = s_up.copy(); a[i] += h
+        c = s_up.copy(); c[i] -= h
+        num_up[i] = (_trainable_total(p, G, labels, alpha, a, residual)[0] -
+                     _trainable_total(p, G, labels, alpha, c, residual)[0]) / (2 * h)
+    assert np.abs(num_up.reshape(-1) - bwd["ds_up"]).max() <= 1e-6 * max(np.abs(num_up).max(), 1e-12)
+    # where s_up wins the linear layer gets nothing, and the other way round
+    lin = (fwd["scores"] > s_up).reshape(-1)
+    assert np.all(bwd["ds_up"][lin] == 0.0) and np.all(bwd["ds_up"][~lin] == bwd["ds"][~lin])
+
+
+def test_trainable_backward_reduces_to_plain_backward():
+    """Scaling off, no labels, no s_up: nothing reaches the gate and dX equals block_bwd's."""
+    p = tiny_problem(seed=44, B=2, N=9)
+    rng = np.random.default_rng(45)
+    G = rng.normal(size=p["x"].shape)
+    fwd = O.block_fwd(**p)
+    a = O.block_bwd(fwd, G, p["x"], p["W_qkv"], p["W_o"], p["H"])
+    b = O.block_bwd_trainable(fwd, G, p["x"], p["w_g"], p["W_qkv"], p["W_o"], p["H"], gate_scale=False)
+    assert np.array_equal(a["dX"], b["dX"]) and np.all(b["ds"] == 0) and np.all(b["dw_g"] == 0) and b["db_g"] == 0
