@@ -219,6 +219,39 @@ int spa_packed_linear_bwd_scatter(const spa_params* p, const void* a, const void
                                   const int32_t* cu_seqlens, void* dX, float* dW, float* db,
                                   void* workspace, int32_t* d_status, void* stream);
 
+/* ---- Trainable selection (Sec. 3.2 multi-scale supervised selection, Eq. 4-5; Sec. 3.3 Eq. 10) ---------
+ * With SPA_FLAG_GATE_SCALE the packed rows are Sigmoid(s) x (Eq. 5) and a gradient reaches the gate.  The hard
+ * selection itself has no gradient.  Order of the calls in a backward pass: spa_select_loss (writes ds),
+ * ..., spa_select_pack_bwd_gated (adds to ds), spa_gate_bwd (consumes ds).  All buffers are device memory. */
+
+/* Bytes of scratch that spa_select_loss and spa_gate_bwd need (per-CTA partial sums). */
+size_t spa_train_workspace_bytes(const spa_params* p);
+
+/* Scores of the previous, finer stage, float[B][2*rows][2*cols], max-pooled 2x2 to this stage's grid:
+ * s_up float[B][rows*cols], the second argument of Max in Eq. 4. */
+int spa_score_pool(const float* scores_prev, int32_t B, int32_t rows, int32_t cols, float* s_up, void* stream);
+
+/* Selection loss of one block, Eq. 10: loss = -sum_t (y_t log p_t + (1 - y_t) log(1 - p_t)), p = Sigmoid(scores),
+ * y = labels (uint8 0/1, [B*N]).  Writes ds[t] = alpha (p_t - y_t) for every token and, if loss != NULL, the
+ * unweighted sum to *loss (device float).  labels == NULL: ds = 0 and loss = 0 (clears ds for the calls below). */
+int spa_select_loss(const spa_params* p, const float* scores, const uint8_t* labels, float alpha, float* ds,
+                    float* loss, void* workspace, void* stream);
+
+/* Transpose of the pack gather under SPA_FLAG_GATE_SCALE:  dX[idx[i]][:] = Sigmoid(s) dx_packed[i][:]
+ * (+ dY[idx[i]][:] under SPA_FLAG_RESIDUAL) and  ds[idx[i]] += Sigmoid'(s) (dx_packed[i] . x[idx[i]]),
+ * s = scores[idx[i]].  Replaces spa_select_pack_bwd. */
+int spa_select_pack_bwd_gated(const spa_params* p, const void* dx_packed, const void* x, const float* scores,
+                              const void* dY, const int32_t* idx, const int32_t* cu_seqlens, void* dX,
+                              float* ds, void* stream);
+
+/* Backward of spa_gate given ds = gradient at the stored (post-Max) scores.  Where the linear layer supplied
+ * the maximum (scores > s_up, or s_up == NULL):  dX[t][:] += ds[t] w_g,  dw_g = sum_t ds[t] x[t][:]  (float[C]),
+ * db_g = sum_t ds[t] (device float, may be NULL); elsewhere ds_up[t] = ds[t] (float[B*N], may be NULL; zero where
+ * the linear layer won).  Sums over tokens run in a fixed order.  (C + 8 (C + 1)) floats must fit 48 KB. */
+int spa_gate_bwd(const spa_params* p, const void* x, const void* w_g, const float* scores, const float* s_up,
+                 const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace,
+                 void* stream);
+
 /* Blocking read of the device status word: synchronises `stream` and returns its value. */
 int spa_read_status(const int32_t* d_status, void* stream);
 

@@ -28,6 +28,7 @@ EXPORTS = (
     "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
     "spa_last_cuda_error", "spa_launch_count", "spa_packed_attention_bwd_static",
     "spa_fused_scatter_supported", "spa_gate_prefill", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
+    "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
 )
 
 
@@ -80,9 +81,16 @@ def lib() -> C.CDLL:
         L.spa_unpack_prefill.argtypes = [pp, vp, vp, vp]
         L.spa_packed_proj_scatter.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_packed_linear_bwd_scatter.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_train_workspace_bytes.restype = C.c_size_t
+        L.spa_train_workspace_bytes.argtypes = [pp]
+        L.spa_score_pool.argtypes = [vp, i32, i32, i32, vp, vp]
+        L.spa_select_loss.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp]
+        L.spa_select_pack_bwd_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_gate_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
-            if name not in ("spa_workspace_bytes", "spa_status_string", "spa_last_cuda_error", "spa_launch_count"):
+            if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_status_string", "spa_last_cuda_error",
+                            "spa_launch_count"):
                 getattr(L, name).restype = C.c_int
         L.spa_status_string.restype = C.c_char_p
         L.spa_status_string.argtypes = [C.c_int]
@@ -205,6 +213,31 @@ def spa_packed_linear_bwd_scatter(p, a, W, dout, n_in, n_out, idx, cu_seqlens, d
                                                _ptr(idx), _ptr(cu_seqlens), _ptr(dX), _ptr(dW), _ptr(db),
                                                _ptr(workspace), _ptr(d_status), _stream(stream)),
            "spa_packed_linear_bwd_scatter")
+
+
+def spa_train_workspace_bytes(p) -> int:
+    return int(lib().spa_train_workspace_bytes(C.byref(p)))
+
+
+def spa_score_pool(scores_prev, B, rows, cols, s_up, stream=None):
+    _check(lib().spa_score_pool(_ptr(scores_prev), int(B), int(rows), int(cols), _ptr(s_up), _stream(stream)),
+           "spa_score_pool")
+
+
+def spa_select_loss(p, scores, labels, alpha, ds, loss, workspace, stream=None):
+    _check(lib().spa_select_loss(C.byref(p), _ptr(scores), _ptr(labels), float(alpha), _ptr(ds), _ptr(loss),
+                                 _ptr(workspace), _stream(stream)), "spa_select_loss")
+
+
+def spa_select_pack_bwd_gated(p, dx_packed, x, scores, dY, idx, cu_seqlens, dX, ds, stream=None):
+    _check(lib().spa_select_pack_bwd_gated(C.byref(p), _ptr(dx_packed), _ptr(x), _ptr(scores), _ptr(dY), _ptr(idx),
+                                           _ptr(cu_seqlens), _ptr(dX), _ptr(ds), _stream(stream)),
+           "spa_select_pack_bwd_gated")
+
+
+def spa_gate_bwd(p, x, w_g, scores, s_up, ds, dX, dw_g, db_g, ds_up, workspace, stream=None):
+    _check(lib().spa_gate_bwd(C.byref(p), _ptr(x), _ptr(w_g), _ptr(scores), _ptr(s_up), _ptr(ds), _ptr(dX), _ptr(dw_g),
+                              _ptr(db_g), _ptr(ds_up), _ptr(workspace), _stream(stream)), "spa_gate_bwd")
 
 
 def spa_read_status(d_status, stream=None) -> int:

@@ -145,6 +145,38 @@ class SpaBlock:
             main.wait_stream(side)
         return dX
 
+    def backward_trainable(self, dY, x, w_g, labels=None, alpha: float = 1.0, s_up=None, dX=None):
+        """backward() extended by the gradient that reaches the gate (Sec. 3.2 Eq. 4-5, Sec. 3.3 Eq. 10): the
+        selection loss alpha * BCE(Sigmoid(scores), labels) when `labels` (uint8 [B, N]) is given, and, under
+        SPA_FLAG_GATE_SCALE, the path through the sigmoid scaling of the packed rows.  `s_up` must be the
+        tensor given to forward().  Returns dX; also fills dw_g, db_g, ds_up (fp32), ds and loss."""
+        p, C = self.p, self.C
+        W_qkv, W_o = self._saved
+        dX = self.dX if dX is None else dX
+        if not hasattr(self, "ds"):
+            dev = self.scores.device
+            n = max(self.B * self.N, 1)
+            self.ds = torch.empty(n, dtype=torch.float32, device=dev)
+            self.ds_up = torch.empty(n, dtype=torch.float32, device=dev)
+            self.dw_g = torch.empty(C, dtype=torch.float32, device=dev)
+            self.db_g = torch.empty(1, dtype=torch.float32, device=dev)
+            self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+            self.train_ws = torch.empty(max(L.spa_train_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
+        L.spa_select_loss(p, self.scores, labels, alpha, self.ds, self.loss, self.train_ws)
+        L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
+        L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
+                                self.workspace, self.status)
+        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self.cu, self.B, self.dqkv,
+                                   self.workspace, self.status)
+        L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv,
+                                self.db_qkv, self.workspace, self.status)
+        if p.flags & L.SPA_FLAG_GATE_SCALE:
+            L.spa_select_pack_bwd_gated(p, self.dxp, x, self.scores, dY, self.idx, self.cu, dX, self.ds)
+        else:
+            L.spa_select_pack_bwd(p, self.dxp, dY, self.idx, self.cu, dX)
+        L.spa_gate_bwd(p, x, w_g, self.scores, s_up, self.ds, dX, self.dw_g, self.db_g, self.ds_up, self.train_ws)
+        return dX
+
     def read_status(self) -> int:
         """Blocking: the device status word (0 = ok)."""
         return L.spa_read_status(self.status)

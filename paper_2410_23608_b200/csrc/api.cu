@@ -250,6 +250,46 @@ int spa_packed_linear_bwd_scatter(const spa_params* p, const void* a, const void
                               (cudaStream_t)stream, idx, (p->flags & SPA_FLAG_RESIDUAL) != 0);
 }
 
+size_t spa_train_workspace_bytes(const spa_params* p) {
+  if (check_params(p) != SPA_OK) return 0;
+  return train_workspace_bytes(*p);
+}
+
+int spa_score_pool(const float* scores_prev, int32_t B, int32_t rows, int32_t cols, float* s_up, void* stream) {
+  if (B < 0 || rows <= 0 || cols <= 0 || (long long)B * rows * cols > (1LL << 28)) return SPA_ERR_INVALID_ARG;
+  if (scores_prev == nullptr || s_up == nullptr) return SPA_ERR_INVALID_ARG;
+  return launch_score_pool(scores_prev, B, rows, cols, s_up, (cudaStream_t)stream);
+}
+
+int spa_select_loss(const spa_params* p, const float* scores, const uint8_t* labels, float alpha, float* ds,
+                    float* loss, void* workspace, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  if (scores == nullptr || ds == nullptr || workspace == nullptr) return SPA_ERR_INVALID_ARG;
+  return launch_select_loss(*p, scores, labels, alpha, ds, loss, workspace, (cudaStream_t)stream);
+}
+
+int spa_select_pack_bwd_gated(const spa_params* p, const void* dx_packed, const void* x, const float* scores,
+                              const void* dY, const int32_t* idx, const int32_t* cu_seqlens, void* dX, float* ds,
+                              void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dx_packed); SPA_PTR(x); SPA_PTR(idx); SPA_PTR(cu_seqlens); SPA_PTR(dX);
+  if (scores == nullptr || ds == nullptr) return SPA_ERR_INVALID_ARG;
+  if (p->flags & SPA_FLAG_RESIDUAL) SPA_PTR(dY);
+  if (p->B == 0) return SPA_OK;
+  return launch_pack_bwd_gated(*p, dx_packed, x, scores, dY, idx, cu_seqlens, dX, ds, (cudaStream_t)stream);
+}
+
+int spa_gate_bwd(const spa_params* p, const void* x, const void* w_g, const float* scores, const float* s_up,
+                 const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(w_g); SPA_PTR(dX);
+  if (scores == nullptr || ds == nullptr || dw_g == nullptr || workspace == nullptr) return SPA_ERR_INVALID_ARG;
+  return launch_gate_bwd(*p, x, w_g, scores, s_up, ds, dX, dw_g, db_g, ds_up, workspace, (cudaStream_t)stream);
+}
+
 int spa_read_status(const int32_t* d_status, void* stream) {
   if (d_status == nullptr) return SPA_ERR_INVALID_ARG;
   int32_t v = 0;

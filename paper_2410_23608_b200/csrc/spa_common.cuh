@@ -145,6 +145,16 @@ int launch_unpack_scatter_bwd(const spa_params& p, const void* dY, const int32_t
                               const int32_t* cu, void* dz, void* dX, cudaStream_t st);
 int launch_select_pack_bwd(const spa_params& p, const void* dxp, const void* dY, const int32_t* idx,
                            const int32_t* cu, void* dX, cudaStream_t st);
+// trainable selection (select_train.cu)
+size_t train_workspace_bytes(const spa_params& p);
+int launch_score_pool(const float* prev, int B, int rows, int cols, float* s_up, cudaStream_t st);
+int launch_select_loss(const spa_params& p, const float* scores, const uint8_t* labels, float alpha, float* ds,
+                       float* loss, void* workspace, cudaStream_t st);
+int launch_pack_bwd_gated(const spa_params& p, const void* dxp, const void* x, const float* scores, const void* dY,
+                          const int32_t* idx, const int32_t* cu, void* dX, float* ds, cudaStream_t st);
+int launch_gate_bwd(const spa_params& p, const void* x, const void* w_g, const float* scores, const float* s_up,
+                    const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace,
+                    cudaStream_t st);
 int launch_copy_tokens(const spa_params& p, const void* src, void* dst, cudaStream_t st);  // dst[B*N][C] = src
 
 // out[M][n_out] = a[M][n_in] W[n_out][n_in]^T + bias, M = packed rows (device)
