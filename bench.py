@@ -255,6 +255,7 @@ def main():
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="issue the weight gradients on the main stream too")
+    ap.add_argument("--train", action="store_true", help="also time the trainable-selection calls (loss, gated pack backward, gate backward)")
     ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -410,6 +411,47 @@ def main():
         ach = wk["flops"] / (ms_c * 1e-3) / 1e12 if bound == "tensor" else wk["bytes"] / (ms_c * 1e-3) / 1e9
         per_call[name] = dict(us=round(ms_c * 1e3, 2), bound=bound, achieved=round(ach, 2),
                               frac=round(ach / pk[bound], 4), kernels=unit_launches[name])
+    train = None
+    if args.train:
+        # trainable selection (Eq. 4-5, Eq. 10): timed like the other units, reported beside them
+        BN = cfg.B * cfg.N
+        extra = []
+        for inp_, d_, blk_, _ in sets:
+            t = dict(ds=torch.zeros(BN, dtype=torch.float32, device="cuda"), ds_up=torch.empty(BN, dtype=torch.float32, device="cuda"),
+                     dw=torch.empty(cfg.C, dtype=torch.float32, device="cuda"), db=torch.empty(1, dtype=torch.float32, device="cuda"),
+                     loss=torch.empty(1, dtype=torch.float32, device="cuda"),
+                     lab=(torch.rand(BN, device="cuda") < 0.4).to(torch.uint8),
+                     ws=torch.empty(max(L.spa_train_workspace_bytes(blk_.p), 256), dtype=torch.uint8, device="cuda"))
+            extra.append(t)
+        def train_units(k):
+            inp_, d_, blk_, _ = sets[k]; t = extra[k]; p_ = blk_.p
+            return {
+                "select_loss": lambda: L.spa_select_loss(p_, blk_.scores, t["lab"], 0.5, t["ds"], t["loss"], t["ws"]),
+                "pack_bwd_gated": lambda: L.spa_select_pack_bwd_gated(p_, blk_.dxp, d_["x"], blk_.scores, d_["dY"], blk_.idx,
+                                                                      blk_.cu, blk_.dX, t["ds"]),
+                "gate_bwd": lambda: L.spa_gate_bwd(p_, d_["x"], d_["w_g"], blk_.scores, None, t["ds"], blk_.dX, t["dw"],
+                                                   t["db"], t["ds_up"], t["ws"]),
+            }
+        tu = [train_units(k) for k in range(n_sets)]
+        es_ = cfg.elem_size
+        tw = {"select_loss": 9 * BN, "pack_bwd_gated": 3 * Np0 * cfg.C * es_ + 12 * Np0, "gate_bwd": 3 * BN * cfg.C * es_ + 12 * BN}
+        train = {}
+        for name in ("select_loss", "pack_bwd_gated", "gate_bwd"):
+            for u in tu:
+                u[name]()
+            g, n_l = capture([u[name] for u in tu])
+            for _ in range(2):
+                g.replay()
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms_c = e0.elapsed_time(e1) / (reps * n_sets)
+            ach = tw[name] / (ms_c * 1e-3) / 1e9
+            train[name] = dict(us=round(ms_c * 1e3, 2), bound="hbm", achieved=round(ach, 2), frac=round(ach / pk["hbm"], 4),
+                               kernels=n_l // n_sets)
     top = max(call_ms, key=call_ms.get)
     tr = per_call[top]
     roofline = {"kernel": top, "bound": tr["bound"], "achieved": tr["achieved"], "peak": pk[tr["bound"]],
@@ -464,6 +506,8 @@ def main():
         "useful_tflops": useful_flops / (ms_per_step * 1e-3) / 1e12,
         "per_call": per_call,
     }
+    if train is not None:
+        line["trainable_selection"] = train
     print(json.dumps(line))
     replicas.shutdown()
 

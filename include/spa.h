@@ -247,7 +247,8 @@ int spa_select_pack_bwd_gated(const spa_params* p, const void* dx_packed, const 
 /* Backward of spa_gate given ds = gradient at the stored (post-Max) scores.  Where the linear layer supplied
  * the maximum (scores > s_up, or s_up == NULL):  dX[t][:] += ds[t] w_g,  dw_g = sum_t ds[t] x[t][:]  (float[C]),
  * db_g = sum_t ds[t] (device float, may be NULL); elsewhere ds_up[t] = ds[t] (float[B*N], may be NULL; zero where
- * the linear layer won).  Sums over tokens run in a fixed order.  (C + 8 (C + 1)) floats must fit 48 KB. */
+ * the linear layer won).  Sums over tokens run in a fixed order.  C is limited to 128 16-byte chunks per row
+ * (1024 bf16 or 512 fp32 channels); beyond that the call returns SPA_ERR_UNSUPPORTED. */
 int spa_gate_bwd(const spa_params* p, const void* x, const void* w_g, const float* scores, const float* s_up,
                  const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace,
                  void* stream);

@@ -60,15 +60,21 @@ select_loss_kernel(const float* __restrict__ scores, const uint8_t* __restrict__
   }
 }
 
-// out[j] = sum over blocks (in order) of part[block * stride + j], j < n_out
+// out[j] = sum over blocks of part[block * stride + j] for j < n_out (out2[0] takes column n_out when given).
+// One warp per column: lane l adds blocks l, l + 32, ... in order, then the lanes combine in a fixed tree.
 __global__ void __launch_bounds__(kTrainThreads)
-partial_sum_kernel(const float* __restrict__ part, int n_blocks, int stride, int n_out, float* __restrict__ out) {
+partial_sum_kernel(const float* __restrict__ part, int n_blocks, int stride, int n_out, float* __restrict__ out,
+                   float* __restrict__ out2) {
   pdl_entry();
-  const int j = blockIdx.x * kTrainThreads + threadIdx.x;
-  if (j >= n_out) return;
+  const int j = blockIdx.x * (kTrainThreads / 32) + (threadIdx.x >> 5);
+  const int n_cols = n_out + (out2 != nullptr ? 1 : 0);
+  if (j >= n_cols) return;
   float s = 0.f;
-  for (int b = 0; b < n_blocks; ++b) s += part[(long long)b * stride + j];
-  out[j] = s;
+  for (int b = threadIdx.x & 31; b < n_blocks; b += 32) s += part[(long long)b * stride + j];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) {
+    if (j < n_out) out[j] = s; else out2[0] = s;
+  }
 }
 
 // One warp per packed row i (token t = idx[i]):  dX_t = Sigmoid(s_t) dxp_i (+ dY_t with the residual),
@@ -111,9 +117,13 @@ pack_bwd_gated_kernel(const uint4* __restrict__ dxp16, const uint4* __restrict__
   }
 }
 
-// Backward of the gate.  A warp walks rows t; where the linear layer supplied the maximum
-// (g = ds_t) it adds g w_g to dX_t and g x_t to its running dw_g, g to its db_g; elsewhere ds_t goes
-// to ds_up.  Per CTA the eight warps' sums are combined in warp order into part[blockIdx][C + 1].
+// Backward of the gate.  A warp walks rows t, two at a time; where the linear layer supplied the maximum
+// (g = ds_t) it adds g w_g to dX_t and g x_t to its running dw_g (registers: a lane owns the same columns of
+// every row), g to its db_g; elsewhere ds_t goes to ds_up.  Per CTA the eight warps' sums are combined in
+// warp order into part[blockIdx][C + 1].
+constexpr int kGbRows = 2;     // rows in flight per warp
+constexpr int kGbChunks = 4;   // 16-byte chunks of a row per lane: C <= 128 chunks
+
 template <typename T>
 __global__ void __launch_bounds__(kTrainThreads)
 gate_bwd_kernel(const uint4* __restrict__ x16, const T* __restrict__ w_g, const float* __restrict__ scores,
@@ -125,38 +135,72 @@ gate_bwd_kernel(const uint4* __restrict__ x16, const T* __restrict__ w_g, const 
   float* w_s = sm;
   float* acc_s = sm + C;
   for (int c = threadIdx.x; c < C; c += kTrainThreads) w_s[c] = to_f32<T>(w_g[c]);
-  for (int c = threadIdx.x; c < (kTrainThreads / 32) * (C + 1); c += kTrainThreads) acc_s[c] = 0.f;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int Q = C / E;
-  float* my_acc = acc_s + warp * (C + 1);
+  float acc[kGbChunks][E];
+#pragma unroll
+  for (int k = 0; k < kGbChunks; ++k)
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[k][e] = 0.f;
   float db = 0.f;
   const int warps = gridDim.x * (kTrainThreads / 32);
-  for (int t = blockIdx.x * (kTrainThreads / 32) + warp; t < rows; t += warps) {
-    const float d = ds[t];
-    const bool lin = s_up == nullptr || scores[t] > s_up[t];
-    if (ds_up != nullptr && lane == 0) ds_up[t] = lin ? 0.f : d;
-    if (!lin || d == 0.f) continue;  // warp-uniform
-    db += d;
-    for (int q = lane; q < Q; q += 32) {
-      float fx[E], fd[E];
-      Vec16<T>::to_float(ld_nc16(x16 + (long long)t * Q + q), fx);
-      Vec16<T>::to_float(dX16[(long long)t * Q + q], fd);
+  for (int t0 = (blockIdx.x * (kTrainThreads / 32) + warp) * kGbRows; t0 < rows; t0 += warps * kGbRows) {
+    float d[kGbRows];
 #pragma unroll
-      for (int e = 0; e < E; ++e) {
-        my_acc[q * E + e] = fmaf(d, fx[e], my_acc[q * E + e]);  // this lane alone owns columns q*E .. q*E+E-1 of its warp's row
-        fd[e] = fmaf(d, w_s[q * E + e], fd[e]);
+    for (int r = 0; r < kGbRows; ++r) {
+      const int t = t0 + r;
+      d[r] = 0.f;
+      if (t < rows) {
+        const float dv = ds[t];
+        const bool lin = s_up == nullptr || scores[t] > s_up[t];
+        if (ds_up != nullptr && lane == 0) ds_up[t] = lin ? 0.f : dv;
+        d[r] = lin ? dv : 0.f;
+        db += d[r];
       }
-      dX16[(long long)t * Q + q] = Vec16<T>::from_float(fd);
+    }
+#pragma unroll
+    for (int k = 0; k < kGbChunks; ++k) {
+      const int q = lane + 32 * k;
+      if (q >= Q) break;
+      uint4 xv[kGbRows], gv[kGbRows];
+#pragma unroll
+      for (int r = 0; r < kGbRows; ++r)
+        if (d[r] != 0.f) {  // warp-uniform
+          xv[r] = ld_nc16(x16 + (long long)(t0 + r) * Q + q);
+          gv[r] = dX16[(long long)(t0 + r) * Q + q];
+        }
+#pragma unroll
+      for (int r = 0; r < kGbRows; ++r)
+        if (d[r] != 0.f) {
+          float fx[E], fd[E];
+          Vec16<T>::to_float(xv[r], fx);
+          Vec16<T>::to_float(gv[r], fd);
+#pragma unroll
+          for (int e = 0; e < E; ++e) {
+            acc[k][e] = fmaf(d[r], fx[e], acc[k][e]);
+            fd[e] = fmaf(d[r], w_s[q * E + e], fd[e]);
+          }
+          dX16[(long long)(t0 + r) * Q + q] = Vec16<T>::from_float(fd);
+        }
+    }
+  }
+  float* my_acc = acc_s + warp * (C + 1);
+#pragma unroll
+  for (int k = 0; k < kGbChunks; ++k) {
+    const int q = lane + 32 * k;
+    if (q < Q) {
+#pragma unroll
+      for (int e = 0; e < E; ++e) my_acc[q * E + e] = acc[k][e];
     }
   }
   if (lane == 0) my_acc[C] = db;
   __syncthreads();
   for (int c = threadIdx.x; c <= C; c += kTrainThreads) {
-    float s = 0.f;
+    float s2 = 0.f;
 #pragma unroll
-    for (int w = 0; w < kTrainThreads / 32; ++w) s += acc_s[w * (C + 1) + c];
-    part[(long long)blockIdx.x * (C + 1) + c] = s;
+    for (int w = 0; w < kTrainThreads / 32; ++w) s2 += acc_s[w * (C + 1) + c];
+    part[(long long)blockIdx.x * (C + 1) + c] = s2;
   }
 }
 
@@ -166,8 +210,8 @@ int loss_grid(long long total) {
   return g < 1 ? 1 : (int)g;
 }
 int gate_bwd_grid(int rows) {
-  int g = (rows + 63) / 64;  // at least eight rows per warp
-  if (g > kNumSMs * 2) g = kNumSMs * 2;
+  int g = (rows + 31) / 32;  // at least four rows per warp
+  if (g > kNumSMs * 4) g = kNumSMs * 4;
   return g < 1 ? 1 : g;
 }
 
@@ -196,7 +240,7 @@ int launch_select_loss(const spa_params& p, const float* scores, const uint8_t* 
   launch_pdl(select_loss_kernel, grid, kTrainThreads, 0, st, scores, labels, alpha, total, ds, part);
   SPA_CUDA_CHECK_LAUNCH("select_loss_kernel");
   if (loss != nullptr) {
-    launch_pdl(partial_sum_kernel, 1, kTrainThreads, 0, st, (const float*)part, grid, 1, 1, loss);
+    launch_pdl(partial_sum_kernel, 1, kTrainThreads, 0, st, (const float*)part, grid, 1, 1, loss, (float*)nullptr);
     SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel(loss)");
   }
   return SPA_OK;
@@ -225,7 +269,7 @@ int launch_gate_bwd(const spa_params& p, const void* x, const void* w_g, const f
   const int grid = gate_bwd_grid(rows);
   float* part = reinterpret_cast<float*>(workspace);
   const size_t smem = ((size_t)p.C + (kTrainThreads / 32) * (p.C + 1)) * sizeof(float);
-  if (smem > 48 * 1024) return SPA_ERR_UNSUPPORTED;
+  if (smem > 48 * 1024 || p.C / (p.dtype == SPA_F32 ? 4 : 8) > 32 * kGbChunks) return SPA_ERR_UNSUPPORTED;
   if (p.dtype == SPA_F32)
     launch_pdl(gate_bwd_kernel<float>, grid, kTrainThreads, smem, st, (const uint4*)x, (const float*)w_g, scores, s_up, ds,
                rows, p.C, (uint4*)dX, ds_up, part);
@@ -233,15 +277,11 @@ int launch_gate_bwd(const spa_params& p, const void* x, const void* w_g, const f
     launch_pdl(gate_bwd_kernel<__nv_bfloat16>, grid, kTrainThreads, smem, st, (const uint4*)x, (const __nv_bfloat16*)w_g,
                scores, s_up, ds, rows, p.C, (uint4*)dX, ds_up, part);
   SPA_CUDA_CHECK_LAUNCH("gate_bwd_kernel");
-  // dw_g[0..C) and db_g: one pass over the per-CTA sums, in CTA order
-  launch_pdl(partial_sum_kernel, (p.C + kTrainThreads - 1) / kTrainThreads, kTrainThreads, 0, st, (const float*)part, grid,
-             p.C + 1, p.C, dw_g);
-  SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel(dw_g)");
-  if (db_g != nullptr) {
-    // column C of the partials is the bias gradient: same kernel, one output, offset input
-    launch_pdl(partial_sum_kernel, 1, kTrainThreads, 0, st, (const float*)part + p.C, grid, p.C + 1, 1, db_g);
-    SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel(db_g)");
-  }
+  // dw_g[0..C) and db_g (column C of the partials) in one pass over the per-CTA sums
+  const int cols = p.C + (db_g != nullptr ? 1 : 0);
+  launch_pdl(partial_sum_kernel, (cols + kTrainThreads / 32 - 1) / (kTrainThreads / 32), kTrainThreads, 0, st,
+             (const float*)part, grid, p.C + 1, p.C, dw_g, db_g);
+  SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel(dw_g, db_g)");
   return SPA_OK;
 }
 
