@@ -89,3 +89,32 @@ def test_select_loss_without_labels_clears_ds():
     scores = torch.randn(n, dtype=torch.float32, device="cuda")
     L.spa_select_loss(blk.p, scores, None, 1.0, ds, loss, ws)
     assert float(ds.abs().max()) == 0.0 and float(loss.item()) == 0.0
+
+
+@pytest.mark.parametrize("tau", [float("inf"), float("-inf")])
+def test_trainable_block_none_and_all_selected(tau):
+    """Nothing selected: only the selection loss reaches the gate.  Everything selected: every token carries the
+    sigmoid-scaling path."""
+    from paper_2410_23608_b200 import binding as L
+    from paper_2410_23608_b200.block import SpaBlock
+    from spa_workloads import scaled_config
+    cfg = scaled_config(get_config(2), B=3)
+    inp = make_inputs(cfg)
+    rng = np.random.default_rng(5)
+    labels = rng.uniform(size=(cfg.B, cfg.N)) < 0.5
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H, gate_scale=True)
+    bwd = O.block_bwd_trainable(fwd, inp.dY, inp.x, inp.w_g, inp.W_qkv, inp.W_o, cfg.H, labels=labels, alpha=1.0,
+                                gate_scale=True)
+    dt = cfg.dtype
+    d = {n: dev(getattr(inp, n), dt) for n in ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")}
+    blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, dt, tau=tau, flags=L.SPA_FLAG_GATE_SCALE)
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    dX = blk.backward_trainable(d["dY"], d["x"], d["w_g"], labels=torch.from_numpy(labels.astype(np.uint8)).cuda())
+    torch.cuda.synchronize()
+    assert blk.read_status() == 0
+    assert int(blk.cu[-1].item()) == (0 if tau > 0 else cfg.B * cfg.N)
+    assert_close(host(y), fwd["y"], dt, "y")
+    assert_close(host(dX), bwd["dX"], dt, "dX", scale_max_abs=True)
+    assert_close(blk.dw_g.cpu().numpy().astype(np.float64), bwd["dw_g"], dt, "dw_g", scale_max_abs=True)
+    assert abs(float(blk.loss.item()) - bwd["loss"]) <= 1e-4 * max(1.0, abs(bwd["loss"]))
+    assert not blk.ds_up.any()   # no up-scale scores were given: nothing goes to them
