@@ -53,7 +53,8 @@ enum {
   SPA_FLAG_RESIDUAL = 1,  /* selected rows: y = x + z instead of y = z                     */
   SPA_FLAG_INPLACE = 2,   /* spa_unpack_scatter: y aliases x, only selected rows written   */
   SPA_FLAG_GATE_SCALE = 4,/* Eq. 5: packed rows are scaled by sigmoid(score)               */
-  SPA_FLAG_SIMT_ONLY = 8  /* bf16 only: run the fp32-FMA kernels instead of the tensor-core ones */
+  SPA_FLAG_SIMT_ONLY = 8, /* bf16 only: run the fp32-FMA kernels instead of the tensor-core ones */
+  SPA_FLAG_NO_CTA_PAIRS = 16 /* wide linear layers: keep the one-CTA tensor-core kernels (no CTA pairs) */
 };
 
 typedef struct spa_params {

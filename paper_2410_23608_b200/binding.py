@@ -20,7 +20,7 @@ SPA_OK, SPA_ERR_INVALID_ARG, SPA_ERR_UNSUPPORTED, SPA_ERR_CAPACITY, SPA_ERR_CUDA
 SPA_ERR_SCRATCH = -6
 SPA_STATIC_SCRATCH_BYTES = 4 << 20
 SPA_F32, SPA_BF16 = 0, 1
-SPA_FLAG_RESIDUAL, SPA_FLAG_INPLACE, SPA_FLAG_GATE_SCALE, SPA_FLAG_SIMT_ONLY = 1, 2, 4, 8
+SPA_FLAG_RESIDUAL, SPA_FLAG_INPLACE, SPA_FLAG_GATE_SCALE, SPA_FLAG_SIMT_ONLY, SPA_FLAG_NO_CTA_PAIRS = 1, 2, 4, 8, 16
 
 EXPORTS = (
     "spa_workspace_bytes", "spa_gate", "spa_select_pack", "spa_packed_qkv", "spa_packed_attention_fwd",

@@ -494,6 +494,8 @@ size_t tc_linear_workspace_bytes(const spa_params& p) {
 int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
                          const int32_t* cu, void* out, int32_t* d_status, cudaStream_t st, const int32_t* row_map,
                          bool accumulate) {
+  if (tc_pair_linear_supported(p, n_in, n_out))
+    return launch_linear_fwd_pair(p, a, W, bias, n_in, n_out, cu, out, d_status, st, row_map, accumulate);
   CUtensorMap tmA, tmB;
   if (!make_tmap_bf16_2d(&tmA, a, n_in, p.capacity, (uint64_t)n_in * 2, BK, BM) ||
       !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, BK, 128))
@@ -514,7 +516,11 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   if (dW != nullptr && (!make_tmap_bf16_2d(&tmA2, dout, n_out, p.capacity, (uint64_t)n_out * 2, 64, BK) ||
                         !make_tmap_bf16_2d(&tmB2, a, n_in, p.capacity, (uint64_t)n_in * 2, 64, BK)))
     return SPA_ERR_UNSUPPORTED;
-  if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
+  const bool pair_dgrad = da != nullptr && tc_pair_linear_supported(p, n_in, n_out);
+  if (pair_dgrad) {
+    int rc = launch_linear_dgrad_pair(p, W, dout, n_in, n_out, cu, da, d_status, st, row_map, accumulate);
+    if (rc != SPA_OK) return rc;
+  } else if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
     int rc = launch_gemm<128, false, true, __nv_bfloat16, false>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
                                                                  p.capacity, n_in, n_out, cu, p.B, p.capacity, 1, n_out,
                                                                  1, nullptr, row_map, accumulate ? 1 : 0, d_status, st,
