@@ -516,7 +516,11 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   if (dW != nullptr && (!make_tmap_bf16_2d(&tmA2, dout, n_out, p.capacity, (uint64_t)n_out * 2, 64, BK) ||
                         !make_tmap_bf16_2d(&tmB2, a, n_in, p.capacity, (uint64_t)n_in * 2, 64, BK)))
     return SPA_ERR_UNSUPPORTED;
-  const bool pair_dgrad = da != nullptr && tc_pair_linear_supported(p, n_in, n_out);
+  // A pair CTA owns its SM (all 512 TMEM columns, 175 KB of shared memory).  A call that asks for da alone is
+  // the pattern of a caller that runs the weight gradients beside it on another stream: there the one-CTA
+  // kernel, which shares an SM with them, gives the shorter step; a call that computes everything in
+  // sequence takes the pair kernel for da.
+  const bool pair_dgrad = da != nullptr && (dW != nullptr || db != nullptr) && tc_pair_linear_supported(p, n_in, n_out);
   if (pair_dgrad) {
     int rc = launch_linear_dgrad_pair(p, W, dout, n_in, n_out, cu, da, d_status, st, row_map, accumulate);
     if (rc != SPA_OK) return rc;
