@@ -51,11 +51,22 @@ def select(s, tau):
     return (np.asarray(s, F64) > F64(tau))
 
 
-def pack_indices(mask):
+def shift_order(rows, cols, shift_r, shift_c):
+    """Order in which the tokens of an image are visited when its feature map is shifted cyclically
+    by (shift_r, shift_c) before packing (Sec. 1: the feature maps are shifted every two blocks so that
+    the token pairs that share a container vary).  order[j] is the original raster index of the token
+    that sits at raster position j of the shifted map."""
+    i = (np.arange(rows)[:, None] + shift_r) % rows
+    j = (np.arange(cols)[None, :] + shift_c) % cols
+    return (i * cols + j).reshape(-1).astype(np.int32)
+
+
+def pack_indices(mask, order=None):
     """Token packing, index part ("Token Packing" paragraph).
 
     mask [B,N] bool -> cu_seqlens int32 [B+1], idx int32 [N_p], inv int32 [B*N].
-    Selected tokens keep batch order then raster order; idx[i] is the flat position
+    Selected tokens keep batch order then raster order (or, with `order` [N], the order in which
+    order[0], order[1], ... visits each image's tokens); idx[i] is the flat position
     b*N+n of packed row i; inv is its inverse with -1 at unselected positions.
     """
     mask = np.asarray(mask, bool)
@@ -63,7 +74,11 @@ def pack_indices(mask):
     cu = np.zeros(B + 1, dtype=np.int64)
     idx = []
     for b in range(B):
-        pos = np.nonzero(mask[b])[0]
+        if order is None:
+            pos = np.nonzero(mask[b])[0]
+        else:
+            o = np.asarray(order, np.int64)
+            pos = o[np.nonzero(mask[b][o])[0]]
         cu[b + 1] = cu[b] + pos.size
         idx.append(b * N + pos)
     idx = np.concatenate(idx) if idx else np.zeros(0, np.int64)
@@ -183,11 +198,12 @@ def unpack_scatter(z, x, idx, residual=False):
 
 
 def block_fwd(x, w_g, b_g, tau, W_qkv, b_qkv, W_o, b_o, H, s_up=None, residual=False,
-              gate_scale=False, scale=None, container_len=None):
-    """One SPA block: gate -> select -> pack -> QKV -> same-image attention -> projection -> unpack."""
+              gate_scale=False, scale=None, container_len=None, order=None):
+    """One SPA block: gate -> select -> pack -> QKV -> same-image attention -> projection -> unpack.
+    `order` packs each image's tokens in a given order (a shifted feature map) instead of raster order."""
     s = gate(x, w_g, b_g, s_up)
     mask = select(s, tau)
-    cu, idx, inv = pack_indices(mask)
+    cu, idx, inv = pack_indices(mask, order)
     xp = pack_rows(x, idx, s, gate_scale)
     qkv = linear(xp, W_qkv, b_qkv)
     seg = cu if container_len is None else container_cuts(cu, container_len)

@@ -456,3 +456,41 @@ def test_trainable_backward_reduces_to_plain_backward():
     a = O.block_bwd(fwd, G, p["x"], p["W_qkv"], p["W_o"], p["H"])
     b = O.block_bwd_trainable(fwd, G, p["x"], p["w_g"], p["W_qkv"], p["W_o"], p["H"], gate_scale=False)
     assert np.array_equal(a["dX"], b["dX"]) and np.all(b["ds"] == 0) and np.all(b["dw_g"] == 0) and b["db_g"] == 0
+
+
+# ------------------------------------------------------------------ shifted feature map before packing
+def test_shift_order_is_a_cyclic_roll():
+    rows, cols = 3, 5
+    grid = np.arange(rows * cols).reshape(rows, cols)
+    o = O.shift_order(rows, cols, 1, 2)
+    np.testing.assert_array_equal(o.reshape(rows, cols), np.roll(grid, shift=(-1, -2), axis=(0, 1)))
+    np.testing.assert_array_equal(O.shift_order(rows, cols, 0, 0), np.arange(rows * cols))
+    assert sorted(o.tolist()) == list(range(rows * cols))
+
+
+def test_ordered_packing_invariants_and_effect():
+    """Packing in a shifted order permutes each image's packed rows and nothing else: without containers the
+    block output is unchanged (attention inside an image does not depend on the order of its tokens); with
+    containers of length L the output changes, because other token pairs share a container."""
+    p = tiny_problem(seed=50, B=3, N=12, C=8, H=2, keep=0.7)
+    order = O.shift_order(3, 4, 1, 1)
+    a = O.block_fwd(**p)
+    b = O.block_fwd(**p, order=order)
+    # indices: same counts, idx a permutation inside each image, visited in the given order
+    np.testing.assert_array_equal(a["cu_seqlens"], b["cu_seqlens"])
+    mask = a["mask"]
+    for img in range(3):
+        lo, hi = a["cu_seqlens"][img], a["cu_seqlens"][img + 1]
+        assert sorted(b["idx"][lo:hi].tolist()) == a["idx"][lo:hi].tolist()
+        want = [img * 12 + t for t in order if mask[img, t]]        # push-back in visiting order
+        assert b["idx"][lo:hi].tolist() == want
+    assert np.array_equal(b["inv"][b["idx"]], np.arange(b["idx"].size))
+    np.testing.assert_allclose(b["y"], a["y"], rtol=0, atol=1e-12)
+    c = O.block_fwd(**p, container_len=4)
+    d = O.block_fwd(**p, container_len=4, order=order)
+    assert np.abs(c["y"] - d["y"]).max() > 1e-3
+    # and the ordered, containerised block equals the plain one applied to the explicitly permuted input
+    inv_o = np.argsort(order)
+    pp = dict(p); pp["x"] = p["x"][:, order, :]
+    e = O.block_fwd(**pp, container_len=4)
+    np.testing.assert_allclose(d["y"], e["y"][:, inv_o, :], rtol=0, atol=1e-12)
