@@ -94,6 +94,15 @@ int spa_select_pack(const spa_params* p, const void* x, const uint8_t* mask, con
                     void* x_packed, int32_t* idx, int32_t* inv, int32_t* cu_seqlens,
                     int32_t* d_status, void* stream);
 
+/* spa_select_pack with each image's tokens visited in the order order[0], order[1], ... (int32[N], a
+ * permutation of 0..N-1; the same for every image) instead of raster order: the cyclic shift of the feature
+ * map that the paper applies every two blocks so that other tokens share a container (Sec. 1).  mask, scores,
+ * idx and inv stay indexed by the original token, so every later call is unchanged; only the order of the
+ * packed rows inside each image differs.  The order array is read on the device. */
+int spa_select_pack_ordered(const spa_params* p, const void* x, const uint8_t* mask, const float* scores,
+                            const int32_t* order, void* x_packed, int32_t* idx, int32_t* inv,
+                            int32_t* cu_seqlens, int32_t* d_status, void* stream);
+
 /* QKV projection on the packed tokens (the 3LC^2 term of Eq. 9):
  *   qkv[i][j] = b_qkv[j] + sum_c W_qkv[j][c] * x_packed[i][c],  i < N_p, j < 3C.
  * W_qkv: T[3C][C]; b_qkv: T[3C] or NULL; qkv: T[capacity][3C] out. */

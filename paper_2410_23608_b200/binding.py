@@ -28,7 +28,7 @@ EXPORTS = (
     "spa_select_pack_bwd", "spa_packed_linear_bwd", "spa_read_status", "spa_status_string",
     "spa_last_cuda_error", "spa_launch_count", "spa_packed_attention_bwd_static",
     "spa_fused_scatter_supported", "spa_gate_prefill", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
-    "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
+    "spa_select_pack_ordered", "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
 )
 
 
@@ -81,6 +81,7 @@ def lib() -> C.CDLL:
         L.spa_unpack_prefill.argtypes = [pp, vp, vp, vp]
         L.spa_packed_proj_scatter.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_packed_linear_bwd_scatter.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_select_pack_ordered.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_train_workspace_bytes.restype = C.c_size_t
         L.spa_train_workspace_bytes.argtypes = [pp]
         L.spa_score_pool.argtypes = [vp, i32, i32, i32, vp, vp]
@@ -213,6 +214,12 @@ def spa_packed_linear_bwd_scatter(p, a, W, dout, n_in, n_out, idx, cu_seqlens, d
                                                _ptr(idx), _ptr(cu_seqlens), _ptr(dX), _ptr(dW), _ptr(db),
                                                _ptr(workspace), _ptr(d_status), _stream(stream)),
            "spa_packed_linear_bwd_scatter")
+
+
+def spa_select_pack_ordered(p, x, mask, scores, order, x_packed, idx, inv, cu_seqlens, d_status=None, stream=None):
+    _check(lib().spa_select_pack_ordered(C.byref(p), _ptr(x), _ptr(mask), _ptr(scores), _ptr(order), _ptr(x_packed),
+                                         _ptr(idx), _ptr(inv), _ptr(cu_seqlens), _ptr(d_status), _stream(stream)),
+           "spa_select_pack_ordered")
 
 
 def spa_train_workspace_bytes(p) -> int:

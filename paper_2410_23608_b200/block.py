@@ -66,9 +66,13 @@ class SpaBlock:
             self.dW_o = e(C, C, dt=torch.float32)
             self.db_o = e(C, dt=torch.float32)
         self._saved = None
+        self._seg = (self.cu, B)   # attention segments: the images, unless forward() is given others
 
     # ------------------------------------------------------------------ forward
-    def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None):
+    def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None, order=None, seg_offsets=None):
+        """`order` (int32 [N] on the device): visiting order of each image's tokens for the packing (a shifted
+        feature map); `seg_offsets` (int32, ascending, ending at N_p): attention segments other than the images,
+        e.g. the container cut; the backward pass uses the same segments."""
         p = self.p
         y = self.y if y is None else y
         inplace = bool(p.flags & L.SPA_FLAG_INPLACE)
@@ -77,9 +81,14 @@ class SpaBlock:
             L.spa_gate_prefill(p, x, w_g, b_g, s_up, self.scores, self.mask, y)
         else:
             L.spa_gate(p, x, w_g, b_g, s_up, self.scores, self.mask)
-        L.spa_select_pack(p, x, self.mask, self.scores, self.xp, self.idx, self.inv, self.cu, self.status)
+        if order is None:
+            L.spa_select_pack(p, x, self.mask, self.scores, self.xp, self.idx, self.inv, self.cu, self.status)
+        else:
+            L.spa_select_pack_ordered(p, x, self.mask, self.scores, order, self.xp, self.idx, self.inv, self.cu,
+                                      self.status)
         L.spa_packed_qkv(p, self.xp, W_qkv, b_qkv, self.cu, self.qkv, self.status)
-        L.spa_packed_attention_fwd(p, self.qkv, self.cu, self.B, self.ao, self.lse, self.status)
+        self._seg = (self.cu, self.B) if seg_offsets is None else (seg_offsets, int(seg_offsets.numel()) - 1)
+        L.spa_packed_attention_fwd(p, self.qkv, self._seg[0], self._seg[1], self.ao, self.lse, self.status)
         if self.fused:
             if inplace:
                 y = x
@@ -117,7 +126,7 @@ class SpaBlock:
                                     self.workspace_side, self.status, stream=side)
             L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, None, None,
                                     self.workspace, self.status)
-        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self.cu, self.B, self.dqkv,
+        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self._seg[0], self._seg[1], self.dqkv,
                                    self.workspace, self.status)
         if self.fused:
             if side is None:
@@ -166,7 +175,7 @@ class SpaBlock:
         L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
         L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
                                 self.workspace, self.status)
-        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self.cu, self.B, self.dqkv,
+        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self._seg[0], self._seg[1], self.dqkv,
                                    self.workspace, self.status)
         L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv,
                                 self.db_qkv, self.workspace, self.status)

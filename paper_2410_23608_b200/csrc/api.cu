@@ -92,7 +92,23 @@ int spa_select_pack(const spa_params* p, const void* x, const uint8_t* mask, con
     if (e != cudaSuccess) { set_cuda_error(e, "spa_select_pack"); return SPA_ERR_CUDA; }
     return SPA_OK;
   }
-  return launch_select_pack(*p, x, mask, scores, x_packed, idx, inv, cu_seqlens, d_status, (cudaStream_t)stream);
+  return launch_select_pack(*p, x, mask, scores, nullptr, x_packed, idx, inv, cu_seqlens, d_status, (cudaStream_t)stream);
+}
+
+int spa_select_pack_ordered(const spa_params* p, const void* x, const uint8_t* mask, const float* scores,
+                            const int32_t* order, void* x_packed, int32_t* idx, int32_t* inv, int32_t* cu_seqlens,
+                            int32_t* d_status, void* stream) {
+  if (order == nullptr) return SPA_ERR_INVALID_ARG;
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(mask); SPA_PTR(x_packed); SPA_PTR(idx); SPA_PTR(cu_seqlens); SPA_OPT_PTR(inv);
+  if (p->flags & SPA_FLAG_GATE_SCALE) SPA_PTR(scores);
+  if (p->B == 0) {
+    cudaError_t e = cudaMemsetAsync(cu_seqlens, 0, sizeof(int32_t), (cudaStream_t)stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "spa_select_pack_ordered"); return SPA_ERR_CUDA; }
+    return SPA_OK;
+  }
+  return launch_select_pack(*p, x, mask, scores, order, x_packed, idx, inv, cu_seqlens, d_status, (cudaStream_t)stream);
 }
 
 int spa_packed_qkv(const spa_params* p, const void* x_packed, const void* W_qkv, const void* b_qkv,

@@ -40,16 +40,20 @@ __device__ __forceinline__ uint4 add16(uint4 a, uint4 b) {
 }
 
 // ------------------------------------------------------------------------------ select + pack
-template <typename T, bool kGateScale>
+// kOrdered: the tokens of every image are visited in the order order[0], order[1], ... (a cyclically shifted
+// feature map) instead of raster order.  Flat position t = b*N + j of the visiting order then stands for
+// token b*N + order[j]; mask, scores, idx and inv stay indexed by the original token.
+template <typename T, bool kGateScale, bool kOrdered>
 __global__ void __launch_bounds__(kPackThreads)
 select_pack_kernel(const uint4* __restrict__ x16, const uint8_t* __restrict__ mask, const float* __restrict__ scores,
-                   int rows, int N, int B, int Q, int tile, int capacity, uint4* __restrict__ xp16,
+                   const int32_t* __restrict__ order, int rows, int N, int B, int Q, int tile, int capacity,
+                   uint4* __restrict__ xp16,
                    int32_t* __restrict__ idx, int32_t* __restrict__ inv, int32_t* __restrict__ cu,
                    int32_t* d_status) {
   pdl_entry();
   __shared__ int warp_cnt[kPackThreads / 32];
   __shared__ int warp_sel[kPackThreads / 32];
-  __shared__ int sel_tok[kPackThreads];   // tile-local offsets of the selected tokens, in order
+  __shared__ int sel_tok[kPackThreads];   // flat indices of the tile's selected tokens, in order
   __shared__ float sel_scale[kPackThreads];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int tile_start = blockIdx.x * tile;  // multiple of 16
@@ -57,14 +61,25 @@ select_pack_kernel(const uint4* __restrict__ x16, const uint8_t* __restrict__ ma
   // 1. number of selected tokens before this tile
   int cnt = 0;
   const uint4* mask16 = reinterpret_cast<const uint4*>(mask);
-  for (int k = tid; k < (tile_start >> 4); k += kPackThreads) cnt += count_nonzero_bytes(__ldg(mask16 + k));
+  if (!kOrdered) {
+    for (int k = tid; k < (tile_start >> 4); k += kPackThreads) cnt += count_nonzero_bytes(__ldg(mask16 + k));
+  } else {
+    // whole images before the tile's first image: any order visits the same bytes; then the positions of
+    // that image which the given order visits before the tile
+    const int img0 = (tile_start / N) * N;
+    for (int k = tid; k < (img0 >> 4); k += kPackThreads) cnt += count_nonzero_bytes(__ldg(mask16 + k));
+    for (int k = (img0 & ~15) + tid; k < img0; k += kPackThreads) cnt += mask[k] != 0;
+    for (int j = tid; j < tile_start - img0; j += kPackThreads) cnt += mask[img0 + __ldg(order + j)] != 0;
+  }
   cnt = (int)__reduce_add_sync(0xffffffffu, (unsigned)cnt);
   if (lane == 0) warp_cnt[wid] = cnt;
 
   // 2. ranks inside the tile
   const int t = tile_start + tid;
   const bool in_tile = tid < tile && t < rows;
-  const bool sel = in_tile && mask[t] != 0;
+  int tok = t;  // the token that position t of the visiting order stands for
+  if (kOrdered && in_tile) tok = (t / N) * N + __ldg(order + t % N);
+  const bool sel = in_tile && mask[tok] != 0;
   const unsigned ballot = __ballot_sync(0xffffffffu, sel);
   if (lane == 0) warp_sel[wid] = __popc(ballot);
   __syncthreads();
@@ -79,13 +94,13 @@ select_pack_kernel(const uint4* __restrict__ x16, const uint8_t* __restrict__ ma
   const int dst = base + local;
   if (in_tile) {
     if (t % N == 0) cu[t / N] = dst;  // exclusive prefix at an image's first token
-    if (inv != nullptr) inv[t] = (sel && dst < capacity) ? dst : -1;
+    if (inv != nullptr) inv[tok] = (sel && dst < capacity) ? dst : -1;
   }
   if (sel) {
     if (dst < capacity) {
-      idx[dst] = t;
-      sel_tok[local] = tid;
-      if (kGateScale) sel_scale[local] = 1.f / (1.f + __expf(-scores[t]));
+      idx[dst] = tok;
+      sel_tok[local] = tok;
+      if (kGateScale) sel_scale[local] = 1.f / (1.f + __expf(-scores[tok]));
     } else {
       record_status(d_status, SPA_ERR_CAPACITY);
     }
@@ -106,7 +121,7 @@ select_pack_kernel(const uint4* __restrict__ x16, const uint8_t* __restrict__ ma
       if (k < total) {
         r[u] = k / Q;
         q[u] = k - r[u] * Q;
-        v[u] = ld_nc16(x16 + (size_t)(tile_start + sel_tok[r[u]]) * Q + q[u]);
+        v[u] = ld_nc16(x16 + (size_t)sel_tok[r[u]] * Q + q[u]);
       }
     }
 #pragma unroll
@@ -252,19 +267,21 @@ template <typename T> int chunks_per_row(int C) { return C / Vec16<T>::kElems; }
 
 }  // namespace
 
-int launch_select_pack(const spa_params& p, const void* x, const uint8_t* mask, const float* scores, void* xp,
-                       int32_t* idx, int32_t* inv, int32_t* cu, int32_t* d_status, cudaStream_t st) {
+int launch_select_pack(const spa_params& p, const void* x, const uint8_t* mask, const float* scores,
+                       const int32_t* order, void* xp, int32_t* idx, int32_t* inv, int32_t* cu, int32_t* d_status,
+                       cudaStream_t st) {
   const int rows = p.B * p.N;
   int tile = 256;
   while (tile > 32 && (rows + tile - 1) / tile < 2 * kNumSMs) tile >>= 1;
   const int grid = (rows + tile - 1) / tile;
   const bool gs = (p.flags & SPA_FLAG_GATE_SCALE) != 0;
-#define SPA_PACK_LAUNCH(T, GS)                                                                              \
-  launch_pdl(select_pack_kernel<T, GS>, grid, kPackThreads, 0, st, (const uint4*)x, mask, scores, rows, p.N, p.B,    \
-                                                          chunks_per_row<T>(p.C), tile, p.capacity,         \
-                                                          (uint4*)xp, idx, inv, cu, d_status)
-  if (p.dtype == SPA_F32) { if (gs) SPA_PACK_LAUNCH(float, true); else SPA_PACK_LAUNCH(float, false); }
-  else { if (gs) SPA_PACK_LAUNCH(__nv_bfloat16, true); else SPA_PACK_LAUNCH(__nv_bfloat16, false); }
+#define SPA_PACK_LAUNCH(T, GS, ORD)                                                                              \
+  launch_pdl(select_pack_kernel<T, GS, ORD>, grid, kPackThreads, 0, st, (const uint4*)x, mask, scores, order, rows, p.N, \
+             p.B, chunks_per_row<T>(p.C), tile, p.capacity, (uint4*)xp, idx, inv, cu, d_status)
+#define SPA_PACK_ORD(T, GS) do { if (order != nullptr) SPA_PACK_LAUNCH(T, GS, true); else SPA_PACK_LAUNCH(T, GS, false); } while (0)
+  if (p.dtype == SPA_F32) { if (gs) SPA_PACK_ORD(float, true); else SPA_PACK_ORD(float, false); }
+  else { if (gs) SPA_PACK_ORD(__nv_bfloat16, true); else SPA_PACK_ORD(__nv_bfloat16, false); }
+#undef SPA_PACK_ORD
 #undef SPA_PACK_LAUNCH
   SPA_CUDA_CHECK_LAUNCH("select_pack_kernel");
   return SPA_OK;

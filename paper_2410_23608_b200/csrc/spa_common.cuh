@@ -138,7 +138,8 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
 int launch_gate(const spa_params& p, const void* x, const void* w_g, float b_g, const float* s_up,
                 float* scores, uint8_t* mask, void* y, cudaStream_t st);
 int launch_select_pack(const spa_params& p, const void* x, const uint8_t* mask, const float* scores,
-                       void* xp, int32_t* idx, int32_t* inv, int32_t* cu, int32_t* d_status, cudaStream_t st);
+                       const int32_t* order, void* xp, int32_t* idx, int32_t* inv, int32_t* cu, int32_t* d_status,
+                       cudaStream_t st);
 int launch_unpack_scatter(const spa_params& p, const void* z, const void* x, const int32_t* idx,
                           const int32_t* inv, const int32_t* cu, void* y, cudaStream_t st);
 int launch_unpack_scatter_bwd(const spa_params& p, const void* dY, const int32_t* idx, const int32_t* inv,

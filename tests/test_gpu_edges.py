@@ -193,3 +193,35 @@ def test_invalid_arguments_are_rejected_on_the_host():
     with pytest.raises(lib.SpaError) as e:
         lib.spa_gate(lib.make_params(2, 16, 64, 2, "f32", capacity=33), x, w, 0.0, None, sc, mk)  # capacity > B*N
     assert e.value.status == lib.SPA_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("ci,fused", [(1, False), (2, False), (2, True)])
+def test_shifted_packing_order_with_containers(ci, fused):
+    """Tokens packed in the order of a cyclically shifted feature map, attention cut into containers of 49 tokens
+    (the paper's own batching): indices bit for bit, forward and backward against the oracle."""
+    cfg = scaled_config(get_config(ci), B=5)
+    inp = make_inputs(cfg)
+    rows, cols = cfg.grid
+    order = O.shift_order(rows, cols, 3, 5)
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H,
+                      container_len=49, order=order)
+    bwd = O.block_bwd(fwd, inp.dY, inp.x, inp.W_qkv, inp.W_o, cfg.H)
+    plain = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H, container_len=49)
+    assert np.abs(plain["y"] - fwd["y"]).max() > 1e-2   # the shift changes which tokens meet
+    d = {n: dev(getattr(inp, n), cfg.dtype) for n in ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")}
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, fused=fused)
+    seg = torch.from_numpy(fwd["seg"].astype(np.int32)).cuda()
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"],
+                    order=torch.from_numpy(order).cuda(), seg_offsets=seg)
+    dX = blk.backward(d["dY"])
+    torch.cuda.synchronize()
+    assert blk.read_status() == 0
+    Np = int(fwd["cu_seqlens"][-1])
+    assert np.array_equal(blk.cu.cpu().numpy(), fwd["cu_seqlens"])
+    assert np.array_equal(blk.idx.cpu().numpy()[:Np], fwd["idx"])
+    assert np.array_equal(blk.inv.cpu().numpy(), fwd["inv"])
+    assert np.array_equal(host(blk.xp)[:Np], fwd["xp"])
+    assert_close(host(y), fwd["y"], cfg.dtype, "y")
+    assert_close(host(dX), bwd["dX"], cfg.dtype, "dX", scale_max_abs=True)
+    for name in ("dW_qkv", "db_qkv", "dW_o", "db_o"):
+        assert_close(host(getattr(blk, name)), bwd[name], cfg.dtype, name, scale_max_abs=True)
