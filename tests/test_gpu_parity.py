@@ -237,3 +237,33 @@ def test_run_to_run_determinism():
         outs.append([t.clone() for t in (y, dX, blk.dW_qkv, blk.db_qkv, blk.dW_o, blk.db_o, blk.dqkv[:Np])])
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("ci", [2, 4])
+def test_graph_replay_is_stable_and_reproducible(ci):
+    """The whole step as one CUDA graph (second stream, programmatic dependent launches), replayed many times:
+    no device-side wait may expire and every replay must give the same bits as the first."""
+    cfg, inp, fwd, bwd = problem(ci)
+    d = device_inputs(cfg, inp)
+    blk = make_block(cfg)
+
+    def step():
+        blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+        blk.backward(d["dY"])
+
+    step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    g.replay()
+    torch.cuda.synchronize()
+    outs = (blk.y, blk.dX, blk.dW_qkv, blk.db_qkv, blk.dW_o, blk.db_o)
+    first = [t.clone() for t in outs]
+    for _ in range(300):
+        g.replay()
+    torch.cuda.synchronize()
+    assert blk.read_status() == 0
+    for a, b in zip(first, outs):
+        assert torch.equal(a, b)
+    assert_close(host(blk.y), fwd["y"], cfg.dtype, "y")
