@@ -401,3 +401,83 @@ def block_bwd_trainable(fwd, dY, x, w_g, W_qkv, W_o, H, labels=None, alpha=1.0, 
     dX = dX + dx_gate
     return dict(dz=dz, dao=dao, dqkv=dqkv, dxp=dxp, dX=dX, dW_o=dW_o, db_o=db_o, dW_qkv=dW_qkv, db_qkv=db_qkv,
                 ds=ds, dw_g=dw_g, db_g=db_g, ds_up=ds_up, loss=loss)
+
+
+# --------------------------------------------------------------------------- the rest of the transformer block
+# Pre-norm block around SPA (Sec. 3.2: selected tokens go through attention, the others are passed on to the
+# feed-forward network): y1 = x + scatter(SPA(LN1(x))), out = y1 + FFN(LN2(y1)), FFN = W2 gelu(W1 t + b1) + b2.
+# Readings fixed here (the paper's block figure is not in the text we have): LayerNorm with eps = 1e-5 over the
+# channels, exact (erf) GELU, hidden width 4C, the gate reads the normalised tokens, the residual base of the
+# selected tokens is x itself, and unselected tokens receive no attention update.
+
+def layer_norm(x, gamma, beta, eps=1e-5):
+    """y = (x - mean) / sqrt(var + eps) * gamma + beta over the last axis; also returns mean and rstd."""
+    x = np.asarray(x, F64)
+    mean = x.mean(axis=-1, keepdims=True)
+    var = ((x - mean) ** 2).mean(axis=-1, keepdims=True)
+    rstd = 1.0 / np.sqrt(var + eps)
+    return (x - mean) * rstd * np.asarray(gamma, F64) + np.asarray(beta, F64), mean[..., 0], rstd[..., 0]
+
+
+def layer_norm_bwd(dy, x, gamma, mean, rstd):
+    """Gradients of layer_norm: dx, dgamma, dbeta."""
+    dy = np.asarray(dy, F64)
+    x = np.asarray(x, F64)
+    xh = (x - mean[..., None]) * rstd[..., None]
+    g = dy * np.asarray(gamma, F64)
+    C = x.shape[-1]
+    dx = (g - g.mean(axis=-1, keepdims=True) - xh * (g * xh).mean(axis=-1, keepdims=True)) * rstd[..., None]
+    red = tuple(range(dy.ndim - 1))
+    return dx, (dy * xh).sum(axis=red), dy.sum(axis=red)
+
+
+def gelu(u):
+    """Exact GELU: u Phi(u), Phi the standard normal distribution function."""
+    from math import erf, sqrt
+    u = np.asarray(u, F64)
+    return 0.5 * u * (1.0 + np.vectorize(erf)(u / sqrt(2.0)))
+
+
+def gelu_grad(u):
+    """d gelu / du = Phi(u) + u phi(u)."""
+    from math import erf, sqrt, pi
+    u = np.asarray(u, F64)
+    return 0.5 * (1.0 + np.vectorize(erf)(u / sqrt(2.0))) + u * np.exp(-0.5 * u * u) / sqrt(2.0 * pi)
+
+
+def layer_fwd(x, prm, H, tau=0.0, eps=1e-5):
+    """One pre-norm block.  prm: dict with g1, be1, w_g, b_g, W_qkv, b_qkv, W_o, b_o, g2, be2, W1, b1, W2, b2."""
+    x = np.asarray(x, F64)
+    z, m1, r1 = layer_norm(x, prm["g1"], prm["be1"], eps)
+    spa = block_fwd(z, prm["w_g"], prm["b_g"], tau, prm["W_qkv"], prm["b_qkv"], prm["W_o"], prm["b_o"], H)
+    y1 = x.reshape(-1, x.shape[-1]).copy()
+    y1[spa["idx"]] += spa["z"]                      # residual on the selected tokens only
+    y1 = y1.reshape(x.shape)
+    t, m2, r2 = layer_norm(y1, prm["g2"], prm["be2"], eps)
+    u = linear(t.reshape(-1, x.shape[-1]), prm["W1"], prm["b1"])
+    h = gelu(u)
+    out = y1 + linear(h, prm["W2"], prm["b2"]).reshape(x.shape)
+    return dict(z=z, m1=m1, r1=r1, spa=spa, y1=y1, t=t, m2=m2, r2=r2, u=u, h=h, out=out)
+
+
+def layer_bwd(f, d_out, x, prm, H):
+    """Backward of layer_fwd: gradient to x and to every parameter except the gate (hard selection)."""
+    x = np.asarray(x, F64)
+    C = x.shape[-1]
+    d_out = np.asarray(d_out, F64)
+    dh, dW2, db2 = linear_bwd(f["h"], prm["W2"], d_out.reshape(-1, C))
+    du = dh * gelu_grad(f["u"])
+    dt, dW1, db1 = linear_bwd(f["t"].reshape(-1, C), prm["W1"], du)
+    dy1_ln, dg2, dbe2 = layer_norm_bwd(dt.reshape(x.shape), f["y1"], prm["g2"], f["m2"], f["r2"])
+    dy1 = d_out + dy1_ln
+    spa = f["spa"]
+    idx = spa["idx"]
+    dz_packed = dy1.reshape(-1, C)[idx]
+    dao, dW_o, db_o = linear_bwd(spa["ao"], prm["W_o"], dz_packed)
+    dqkv = attention_bwd(spa["qkv"], spa["ao"], spa["lse"], dao, spa["seg"], H)
+    dxp, dW_qkv, db_qkv = linear_bwd(spa["xp"], prm["W_qkv"], dqkv)
+    dZ = np.zeros((x.size // C, C), F64)
+    dZ[idx] = dxp
+    dx_ln, dg1, dbe1 = layer_norm_bwd(dZ.reshape(x.shape), x, prm["g1"], f["m1"], f["r1"])
+    return dict(dX=dy1 + dx_ln, dg1=dg1, dbe1=dbe1, dg2=dg2, dbe2=dbe2, dW1=dW1, db1=db1, dW2=dW2, db2=db2,
+                dW_qkv=dW_qkv, db_qkv=db_qkv, dW_o=dW_o, db_o=db_o, dy1=dy1, du=du, dt=dt, dZ=dZ)

@@ -494,3 +494,67 @@ def test_ordered_packing_invariants_and_effect():
     pp = dict(p); pp["x"] = p["x"][:, order, :]
     e = O.block_fwd(**pp, container_len=4)
     np.testing.assert_allclose(d["y"], e["y"][:, inv_o, :], rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------------ LayerNorm, GELU, feed-forward, whole block
+def test_layer_norm_and_gelu_against_library():
+    rng = np.random.default_rng(60)
+    x = rng.normal(size=(3, 5, 16)) * 2 + 0.5
+    g, b = rng.normal(size=16), rng.normal(size=16)
+    y, mean, rstd = O.layer_norm(x, g, b)
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(x), (16,), torch.from_numpy(g), torch.from_numpy(b), 1e-5)
+    np.testing.assert_allclose(y, ref.numpy(), rtol=0, atol=1e-12)
+    xt = torch.from_numpy(x).requires_grad_(True)
+    gt = torch.from_numpy(g).requires_grad_(True)
+    bt = torch.from_numpy(b).requires_grad_(True)
+    dy = rng.normal(size=x.shape)
+    torch.nn.functional.layer_norm(xt, (16,), gt, bt, 1e-5).backward(torch.from_numpy(dy))
+    dx, dg, db = O.layer_norm_bwd(dy, x, g, mean, rstd)
+    np.testing.assert_allclose(dx, xt.grad.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dg, gt.grad.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(db, bt.grad.numpy(), rtol=0, atol=1e-12)
+    u = rng.normal(size=200) * 3
+    np.testing.assert_allclose(O.gelu(u), torch.nn.functional.gelu(torch.from_numpy(u)).numpy(), rtol=0, atol=1e-14)
+    h = 1e-6
+    np.testing.assert_allclose(O.gelu_grad(u), (O.gelu(u + h) - O.gelu(u - h)) / (2 * h), rtol=0, atol=1e-8)
+    assert O.gelu(np.array([0.0]))[0] == 0.0 and abs(O.gelu_grad(np.array([0.0]))[0] - 0.5) < 1e-15
+
+
+def _layer_params(rng, C, Hd):
+    s = 1.0 / np.sqrt(C)
+    return dict(g1=1 + 0.1 * rng.normal(size=C), be1=0.1 * rng.normal(size=C), w_g=rng.normal(size=C) * s, b_g=0.03,
+                W_qkv=rng.normal(size=(3 * C, C)) * s, b_qkv=0.1 * rng.normal(size=3 * C), W_o=rng.normal(size=(C, C)) * s,
+                b_o=0.1 * rng.normal(size=C), g2=1 + 0.1 * rng.normal(size=C), be2=0.1 * rng.normal(size=C),
+                W1=rng.normal(size=(Hd, C)) * s, b1=0.1 * rng.normal(size=Hd), W2=rng.normal(size=(C, Hd)) / np.sqrt(Hd),
+                b2=0.1 * rng.normal(size=C))
+
+
+def test_layer_backward_against_central_differences():
+    rng = np.random.default_rng(61)
+    B, N, C, H = 2, 6, 8, 2
+    prm = _layer_params(rng, C, 4 * C)
+    x = rng.normal(size=(B, N, C))
+    G = rng.normal(size=x.shape)
+    f = O.layer_fwd(x, prm, H)
+    assert 2 < f["spa"]["idx"].size < B * N and np.abs(f["spa"]["scores"]).min() > 1e-3
+    bwd = O.layer_bwd(f, G, x, prm, H)
+    # unselected tokens receive no attention update
+    unsel = ~f["spa"]["mask"]
+    assert np.array_equal(f["y1"][unsel], x[unsel])
+    total = lambda xx, pp: float((O.layer_fwd(xx, pp, H)["out"] * G).sum())
+    h = 1e-6
+    num = np.zeros_like(x)
+    for i in np.ndindex(*x.shape):
+        a = x.copy(); a[i] += h
+        c = x.copy(); c[i] -= h
+        num[i] = (total(a, prm) - total(c, prm)) / (2 * h)
+    assert np.abs(num - bwd["dX"]).max() / np.abs(num).max() <= 1e-6
+    for name, gname in (("g1", "dg1"), ("be1", "dbe1"), ("g2", "dg2"), ("be2", "dbe2"), ("W1", "dW1"), ("b1", "db1"),
+                        ("W2", "dW2"), ("b2", "db2"), ("W_qkv", "dW_qkv"), ("b_o", "db_o")):
+        base = prm[name]
+        numg = np.zeros_like(base)
+        for i in np.ndindex(*base.shape):
+            pa = dict(prm); a = base.copy(); a[i] += h; pa[name] = a
+            pc = dict(prm); c = base.copy(); c[i] -= h; pc[name] = c
+            numg[i] = (total(x, pa) - total(x, pc)) / (2 * h)
+        assert np.abs(numg - bwd[gname]).max() / max(np.abs(numg).max(), 1e-12) <= 1e-6, name
