@@ -234,7 +234,7 @@ int spa_packed_linear_bwd_scatter(const spa_params* p, const void* a, const void
  * selection itself has no gradient.  Order of the calls in a backward pass: spa_select_loss (writes ds),
  * ..., spa_select_pack_bwd_gated (adds to ds), spa_gate_bwd (consumes ds).  All buffers are device memory. */
 
-/* Bytes of scratch that spa_select_loss and spa_gate_bwd need (per-CTA partial sums). */
+/* Bytes of scratch that spa_select_loss, spa_gate_bwd and spa_layer_norm_bwd need (per-CTA partial sums). */
 size_t spa_train_workspace_bytes(const spa_params* p);
 
 /* Scores of the previous, finer stage, float[B][2*rows][2*cols], max-pooled 2x2 to this stage's grid:
@@ -262,6 +262,32 @@ int spa_select_pack_bwd_gated(const spa_params* p, const void* dx_packed, const 
 int spa_gate_bwd(const spa_params* p, const void* x, const void* w_g, const float* scores, const float* s_up,
                  const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace,
                  void* stream);
+
+/* ---- The rest of the pre-norm transformer block around SPA (Sec. 3.2: selected tokens go through attention,
+ * the others straight to the feed-forward network).  The paper prints no formula for these standard parts;
+ * they are: LayerNorm over the channels, linear layers over all tokens, the exact (erf) GELU. --------------- */
+
+/* out[i][:] = b + W a[i][:] for the rows that cu_seqlens[B] counts (W: T[n_out][n_in], b: T[n_out] or NULL,
+ * a: T[capacity][n_in], out: T[capacity][n_out]).  accumulate != 0 adds the result to what out holds (a residual
+ * branch).  With cu_seqlens[b] = b*N the layer runs over every token.  spa_packed_linear_bwd is its backward. */
+int spa_packed_linear(const spa_params* p, const void* a, const void* W, const void* b, int32_t n_in,
+                      int32_t n_out, const int32_t* cu_seqlens, void* out, int32_t accumulate,
+                      int32_t* d_status, void* stream);
+
+/* y = (x - mean) * rstd * gamma + beta over the C channels of each of the B*N tokens; mean, rstd: float[B*N] out
+ * (saved for the backward).  C is limited to 128 16-byte chunks per row (else SPA_ERR_UNSUPPORTED). */
+int spa_layer_norm(const spa_params* p, const void* x, const void* gamma, const void* beta, float eps, void* y,
+                   float* mean, float* rstd, void* stream);
+
+/* Backward of spa_layer_norm: dx (+ add[t][:] if add != NULL: the gradient of a residual branch), dgamma and
+ * dbeta (float[C], sums over tokens in a fixed order).  workspace: spa_train_workspace_bytes. */
+int spa_layer_norm_bwd(const spa_params* p, const void* dy, const void* x, const void* gamma, const float* mean,
+                       const float* rstd, const void* add, void* dx, float* dgamma, float* dbeta,
+                       void* workspace, void* stream);
+
+/* h = gelu(u) = u Phi(u) and du = dh * gelu'(u) over T[B*N][n_cols]; du may alias dh. */
+int spa_gelu(const spa_params* p, const void* u, int32_t n_cols, void* h, void* stream);
+int spa_gelu_bwd(const spa_params* p, const void* dh, const void* u, int32_t n_cols, void* du, void* stream);
 
 /* Blocking read of the device status word: synchronises `stream` and returns its value. */
 int spa_read_status(const int32_t* d_status, void* stream);

@@ -29,6 +29,7 @@ EXPORTS = (
     "spa_last_cuda_error", "spa_launch_count", "spa_packed_attention_bwd_static",
     "spa_fused_scatter_supported", "spa_gate_prefill", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
     "spa_select_pack_ordered", "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
+    "spa_packed_linear", "spa_layer_norm", "spa_layer_norm_bwd", "spa_gelu", "spa_gelu_bwd",
 )
 
 
@@ -88,6 +89,11 @@ def lib() -> C.CDLL:
         L.spa_select_loss.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp]
         L.spa_select_pack_bwd_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_gate_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_packed_linear.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]
+        L.spa_layer_norm.argtypes = [pp, vp, vp, vp, f32, vp, vp, vp, vp]
+        L.spa_layer_norm_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_gelu.argtypes = [pp, vp, i32, vp, vp]
+        L.spa_gelu_bwd.argtypes = [pp, vp, vp, i32, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
             if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_status_string", "spa_last_cuda_error",
@@ -245,6 +251,29 @@ def spa_select_pack_bwd_gated(p, dx_packed, x, scores, dY, idx, cu_seqlens, dX, 
 def spa_gate_bwd(p, x, w_g, scores, s_up, ds, dX, dw_g, db_g, ds_up, workspace, stream=None):
     _check(lib().spa_gate_bwd(C.byref(p), _ptr(x), _ptr(w_g), _ptr(scores), _ptr(s_up), _ptr(ds), _ptr(dX), _ptr(dw_g),
                               _ptr(db_g), _ptr(ds_up), _ptr(workspace), _stream(stream)), "spa_gate_bwd")
+
+
+def spa_packed_linear(p, a, W, b, n_in, n_out, cu_seqlens, out, accumulate=False, d_status=None, stream=None):
+    _check(lib().spa_packed_linear(C.byref(p), _ptr(a), _ptr(W), _ptr(b), int(n_in), int(n_out), _ptr(cu_seqlens), _ptr(out),
+                                   1 if accumulate else 0, _ptr(d_status), _stream(stream)), "spa_packed_linear")
+
+
+def spa_layer_norm(p, x, gamma, beta, eps, y, mean, rstd, stream=None):
+    _check(lib().spa_layer_norm(C.byref(p), _ptr(x), _ptr(gamma), _ptr(beta), float(eps), _ptr(y), _ptr(mean), _ptr(rstd),
+                                _stream(stream)), "spa_layer_norm")
+
+
+def spa_layer_norm_bwd(p, dy, x, gamma, mean, rstd, add, dx, dgamma, dbeta, workspace, stream=None):
+    _check(lib().spa_layer_norm_bwd(C.byref(p), _ptr(dy), _ptr(x), _ptr(gamma), _ptr(mean), _ptr(rstd), _ptr(add), _ptr(dx),
+                                    _ptr(dgamma), _ptr(dbeta), _ptr(workspace), _stream(stream)), "spa_layer_norm_bwd")
+
+
+def spa_gelu(p, u, n_cols, h, stream=None):
+    _check(lib().spa_gelu(C.byref(p), _ptr(u), int(n_cols), _ptr(h), _stream(stream)), "spa_gelu")
+
+
+def spa_gelu_bwd(p, dh, u, n_cols, du, stream=None):
+    _check(lib().spa_gelu_bwd(C.byref(p), _ptr(dh), _ptr(u), int(n_cols), _ptr(du), _stream(stream)), "spa_gelu_bwd")
 
 
 def spa_read_status(d_status, stream=None) -> int:

@@ -306,6 +306,58 @@ int spa_gate_bwd(const spa_params* p, const void* x, const void* w_g, const floa
   return launch_gate_bwd(*p, x, w_g, scores, s_up, ds, dX, dw_g, db_g, ds_up, workspace, (cudaStream_t)stream);
 }
 
+int spa_packed_linear(const spa_params* p, const void* a, const void* W, const void* b, int32_t n_in, int32_t n_out,
+                      const int32_t* cu_seqlens, void* out, int32_t accumulate, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(a); SPA_PTR(W); SPA_PTR(cu_seqlens); SPA_PTR(out); SPA_OPT_PTR(b);
+  SPA_REQUIRE(n_in > 0 && n_out > 0, SPA_ERR_INVALID_ARG);
+  const int es = p->dtype == SPA_F32 ? 4 : 2;
+  SPA_REQUIRE((n_in * es) % 16 == 0 && (n_out * es) % 16 == 0, SPA_ERR_UNSUPPORTED);
+  if (use_tc(p) && tc_linear_supported(n_in, n_out)) {
+    rc = launch_linear_fwd_tc(*p, a, W, b, n_in, n_out, cu_seqlens, out, d_status, (cudaStream_t)stream, nullptr,
+                              accumulate != 0);
+    if (rc != SPA_ERR_UNSUPPORTED) return rc;
+  }
+  return launch_linear_fwd_simt(*p, a, W, b, n_in, n_out, cu_seqlens, out, (cudaStream_t)stream, accumulate != 0);
+}
+
+int spa_layer_norm(const spa_params* p, const void* x, const void* gamma, const void* beta, float eps, void* y,
+                   float* mean, float* rstd, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(gamma); SPA_PTR(beta); SPA_PTR(y);
+  if (mean == nullptr || rstd == nullptr || !(eps > 0.f)) return SPA_ERR_INVALID_ARG;
+  return launch_layer_norm(*p, x, gamma, beta, eps, y, mean, rstd, (cudaStream_t)stream);
+}
+
+int spa_layer_norm_bwd(const spa_params* p, const void* dy, const void* x, const void* gamma, const float* mean,
+                       const float* rstd, const void* add, void* dx, float* dgamma, float* dbeta, void* workspace,
+                       void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dy); SPA_PTR(x); SPA_PTR(gamma); SPA_PTR(dx); SPA_OPT_PTR(add);
+  if (mean == nullptr || rstd == nullptr || dgamma == nullptr || dbeta == nullptr || workspace == nullptr)
+    return SPA_ERR_INVALID_ARG;
+  return launch_layer_norm_bwd(*p, dy, x, gamma, mean, rstd, add, dx, dgamma, dbeta, workspace, (cudaStream_t)stream);
+}
+
+int spa_gelu(const spa_params* p, const void* u, int32_t n_cols, void* h, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(u); SPA_PTR(h);
+  SPA_REQUIRE(n_cols > 0 && (n_cols * (p->dtype == SPA_F32 ? 4 : 2)) % 16 == 0, SPA_ERR_INVALID_ARG);
+  return launch_gelu(*p, u, nullptr, n_cols, h, (cudaStream_t)stream);
+}
+
+int spa_gelu_bwd(const spa_params* p, const void* dh, const void* u, int32_t n_cols, void* du, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(dh); SPA_PTR(u); SPA_PTR(du);
+  SPA_REQUIRE(n_cols > 0 && (n_cols * (p->dtype == SPA_F32 ? 4 : 2)) % 16 == 0, SPA_ERR_INVALID_ARG);
+  return launch_gelu(*p, u, dh, n_cols, du, (cudaStream_t)stream);
+}
+
 int spa_read_status(const int32_t* d_status, void* stream) {
   if (d_status == nullptr) return SPA_ERR_INVALID_ARG;
   int32_t v = 0;

@@ -17,7 +17,7 @@ template <typename T, typename TO>
 __global__ void __launch_bounds__(kThreads)
 gemm_simt_kernel(const T* __restrict__ A, long long sAm, long long sAk, const T* __restrict__ Bm, long long sBn,
                  long long sBk, const T* __restrict__ bias, TO* __restrict__ out, long long ldo, int M, int N, int K,
-                 const int32_t* __restrict__ cu, int n_seg, int capacity, int dyn_which) {
+                 const int32_t* __restrict__ cu, int n_seg, int capacity, int dyn_which, int accumulate) {
   pdl_entry();
   if (dyn_which != 0) {
     const int rows = packed_rows(cu, n_seg, capacity);
@@ -71,6 +71,7 @@ gemm_simt_kernel(const T* __restrict__ A, long long sAm, long long sAk, const T*
       if (n >= N) continue;
       float v = acc[i][j];
       if (bias != nullptr) v += to_f32<T>(bias[n]);
+      if (accumulate) v += to_f32<TO>(out[(long long)m * ldo + n]);  // residual: the product joins what the row holds
       out[(long long)m * ldo + n] = from_f32<TO>(v);
     }
   }
@@ -97,17 +98,17 @@ colsum_kernel(const T* __restrict__ dout, int n_out, const int32_t* __restrict__
 template <typename T, typename TO>
 void launch_gemm(const T* A, long long sAm, long long sAk, const T* Bm, long long sBn, long long sBk, const T* bias,
                  TO* out, long long ldo, int M, int N, int K, const int32_t* cu, int n_seg, int capacity,
-                 int dyn_which, cudaStream_t st) {
+                 int dyn_which, cudaStream_t st, int accumulate = 0) {
   dim3 grid((N + kTile - 1) / kTile, (M + kTile - 1) / kTile);
   launch_pdl(gemm_simt_kernel<T, TO>, grid, kThreads, 0, st, A, sAm, sAk, Bm, sBn, sBk, bias, out, ldo, M, N, K, cu, n_seg,
-                                                    capacity, dyn_which);
+                                                    capacity, dyn_which, accumulate);
 }
 
 template <typename T>
 int linear_fwd(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
-               const int32_t* cu, void* out, cudaStream_t st) {
+               const int32_t* cu, void* out, cudaStream_t st, bool accumulate) {
   launch_gemm<T, T>((const T*)a, n_in, 1, (const T*)W, n_in, 1, (const T*)bias, (T*)out, n_out, p.capacity, n_out,
-                    n_in, cu, p.B, p.capacity, 1, st);
+                    n_in, cu, p.B, p.capacity, 1, st, accumulate ? 1 : 0);
   SPA_CUDA_CHECK_LAUNCH("gemm_simt_kernel(fwd)");
   return SPA_OK;
 }
@@ -135,9 +136,9 @@ int linear_bwd(const spa_params& p, const void* a, const void* W, const void* do
 }  // namespace
 
 int launch_linear_fwd_simt(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
-                           const int32_t* cu, void* out, cudaStream_t st) {
-  return p.dtype == SPA_F32 ? linear_fwd<float>(p, a, W, bias, n_in, n_out, cu, out, st)
-                            : linear_fwd<__nv_bfloat16>(p, a, W, bias, n_in, n_out, cu, out, st);
+                           const int32_t* cu, void* out, cudaStream_t st, bool accumulate) {
+  return p.dtype == SPA_F32 ? linear_fwd<float>(p, a, W, bias, n_in, n_out, cu, out, st, accumulate)
+                            : linear_fwd<__nv_bfloat16>(p, a, W, bias, n_in, n_out, cu, out, st, accumulate);
 }
 
 int launch_linear_bwd_simt(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,

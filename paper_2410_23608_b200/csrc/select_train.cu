@@ -217,10 +217,20 @@ int gate_bwd_grid(int rows) {
 
 }  // namespace
 
+int launch_partial_sum(const float* part, int n_blocks, int stride, int n_out, float* out, float* out2, cudaStream_t st) {
+  const int cols = n_out + (out2 != nullptr ? 1 : 0);
+  launch_pdl(partial_sum_kernel, (cols + kTrainThreads / 32 - 1) / (kTrainThreads / 32), kTrainThreads, 0, st, part, n_blocks,
+             stride, n_out, out, out2);
+  SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel");
+  return SPA_OK;
+}
+
 size_t train_workspace_bytes(const spa_params& p) {
   const size_t a = (size_t)gate_bwd_grid(p.B * p.N) * (p.C + 1) * sizeof(float);
   const size_t b = (size_t)loss_grid((long long)p.B * p.N) * sizeof(float);
-  return ((a > b ? a : b) + 255) & ~(size_t)255;
+  const size_t c = layer_norm_workspace_bytes(p);
+  const size_t m = a > b ? (a > c ? a : c) : (b > c ? b : c);
+  return (m + 255) & ~(size_t)255;
 }
 
 int launch_score_pool(const float* prev, int B, int rows, int cols, float* s_up, cudaStream_t st) {

@@ -156,11 +156,22 @@ int launch_pack_bwd_gated(const spa_params& p, const void* dxp, const void* x, c
 int launch_gate_bwd(const spa_params& p, const void* x, const void* w_g, const float* scores, const float* s_up,
                     const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace,
                     cudaStream_t st);
+// out[j] = sum over blocks (fixed order) of part[block * stride + j], j < n_out; out2[0] = column n_out if given
+int launch_partial_sum(const float* part, int n_blocks, int stride, int n_out, float* out, float* out2, cudaStream_t st);
+// the rest of the transformer block (block_rest.cu)
+size_t layer_norm_workspace_bytes(const spa_params& p);
+bool layer_norm_supported(const spa_params& p);
+int launch_layer_norm(const spa_params& p, const void* x, const void* gamma, const void* beta, float eps, void* y,
+                      float* mean, float* rstd, cudaStream_t st);
+int launch_layer_norm_bwd(const spa_params& p, const void* dy, const void* x, const void* gamma, const float* mean,
+                          const float* rstd, const void* add, void* dx, float* dgamma, float* dbeta, void* workspace,
+                          cudaStream_t st);
+int launch_gelu(const spa_params& p, const void* u, const void* dh, int n_cols, void* out, cudaStream_t st);
 int launch_copy_tokens(const spa_params& p, const void* src, void* dst, cudaStream_t st);  // dst[B*N][C] = src
 
 // out[M][n_out] = a[M][n_in] W[n_out][n_in]^T + bias, M = packed rows (device)
 int launch_linear_fwd_simt(const spa_params& p, const void* a, const void* W, const void* bias, int n_in,
-                           int n_out, const int32_t* cu, void* out, cudaStream_t st);
+                           int n_out, const int32_t* cu, void* out, cudaStream_t st, bool accumulate = false);
 int launch_linear_bwd_simt(const spa_params& p, const void* a, const void* W, const void* dout, int n_in,
                            int n_out, const int32_t* cu, void* da, float* dW, float* db, cudaStream_t st);
 int launch_attention_fwd_simt(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao,
