@@ -256,6 +256,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="issue the weight gradients on the main stream too")
     ap.add_argument("--train", action="store_true", help="also time the trainable-selection calls (loss, gated pack backward, gate backward)")
+    ap.add_argument("--layer", action="store_true", help="also time the whole pre-norm block (LayerNorm, SPA, feed-forward) and its new calls")
     ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -452,6 +453,62 @@ def main():
             ach = tw[name] / (ms_c * 1e-3) / 1e9
             train[name] = dict(us=round(ms_c * 1e3, 2), bound="hbm", achieved=round(ach, 2), frac=round(ach / pk["hbm"], 4),
                                kernels=n_l // n_sets)
+    layer = None
+    if args.layer:
+        # the pre-norm block around SPA: whole forward + backward as one graph per buffer set, and its new calls alone
+        from paper_2410_23608_b200.layer import SpaLayer
+        n_l = min(n_sets, 6)
+        Hd = 4 * cfg.C
+        lays = []
+        for k in range(n_l):
+            inp_, d_, blk_, _ = sets[k]
+            rp = lambda *sh: (torch.randn(*sh, device="cuda") * 0.05).to(blk_.tdtype)
+            prm = dict(g1=(1 + rp(cfg.C)), be1=rp(cfg.C), g2=(1 + rp(cfg.C)), be2=rp(cfg.C), W1=rp(Hd, cfg.C), b1=rp(Hd),
+                       W2=rp(cfg.C, Hd), b2=rp(cfg.C), w_g=d_["w_g"], b_g=0.0, W_qkv=d_["W_qkv"], b_qkv=d_["b_qkv"],
+                       W_o=d_["W_o"], b_o=d_["b_o"])
+            lays.append((SpaLayer(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype), prm, d_))
+        def timed(fns):
+            for f_ in fns:
+                f_()
+            torch.cuda.synchronize()
+            g_, n_k = capture(fns)
+            for _ in range(2):
+                g_.replay()
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                g_.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / (reps * len(fns)), n_k // len(fns)
+        def whole(k):
+            lay, prm, d_ = lays[k]
+            def run():
+                lay.forward(d_["x"], prm)
+                lay.backward(d_["dY"])
+            return run
+        ms_l, k_l = timed([whole(k) for k in range(n_l)])
+        BNr, es_ = cfg.B * cfg.N, cfg.elem_size
+        units = {
+            "layer_norm": (lambda lay, prm, d_: (lambda: L.spa_layer_norm(lay.p, d_["x"], prm["g1"], prm["be1"], 1e-5, lay.z, lay.m1, lay.r1)),
+                           2 * BNr * cfg.C * es_, 0),
+            "layer_norm_bwd": (lambda lay, prm, d_: (lambda: L.spa_layer_norm_bwd(lay.p, lay.dt, lay.y1, prm["g2"], lay.m2, lay.r2, d_["dY"], lay.dy1,
+                                                                                    lay.dg2, lay.dbe2, lay.workspace)), 4 * BNr * cfg.C * es_, 0),
+            "gelu": (lambda lay, prm, d_: (lambda: L.spa_gelu(lay.p, lay.u, Hd, lay.h)), 2 * BNr * Hd * es_, 0),
+            "gelu_bwd": (lambda lay, prm, d_: (lambda: L.spa_gelu_bwd(lay.p, lay.dh, lay.u, Hd, lay.dh)), 3 * BNr * Hd * es_, 0),
+            "ffn1": (lambda lay, prm, d_: (lambda: L.spa_packed_linear(lay.p, lay.t, prm["W1"], prm["b1"], cfg.C, Hd, lay.cu_all, lay.u, False,
+                                                                        lay.blk.status)), (BNr * cfg.C + Hd * cfg.C + BNr * Hd) * es_, 2 * BNr * cfg.C * Hd),
+            "ffn2": (lambda lay, prm, d_: (lambda: L.spa_packed_linear(lay.p, lay.h, prm["W2"], prm["b2"], Hd, cfg.C, lay.cu_all, lay.out, True,
+                                                                        lay.blk.status)), (BNr * Hd + Hd * cfg.C + 2 * BNr * cfg.C) * es_, 2 * BNr * cfg.C * Hd),
+        }
+        layer = {"ms_per_step": ms_l, "kernels_per_step": k_l, "tokens_per_s": cfg.B * cfg.N / (ms_l * 1e-3), "per_call": {}}
+        for name, (mk, nbytes, nflops) in units.items():
+            ms_c, n_k = timed([mk(*lays[k]) for k in range(n_l)])
+            t_b, t_f = nbytes / (pk["hbm"] * 1e9), nflops / (pk["tensor"] * 1e12)
+            bound = "tensor" if (t_f > t_b and cfg.dtype == "bf16") else "hbm"
+            ach = nflops / (ms_c * 1e-3) / 1e12 if bound == "tensor" else nbytes / (ms_c * 1e-3) / 1e9
+            layer["per_call"][name] = dict(us=round(ms_c * 1e3, 2), bound=bound, achieved=round(ach, 2), frac=round(ach / pk[bound], 4),
+                                           kernels=n_k)
     top = max(call_ms, key=call_ms.get)
     tr = per_call[top]
     roofline = {"kernel": top, "bound": tr["bound"], "achieved": tr["achieved"], "peak": pk[tr["bound"]],
@@ -508,6 +565,8 @@ def main():
     }
     if train is not None:
         line["trainable_selection"] = train
+    if layer is not None:
+        line["pre_norm_block"] = layer
     print(json.dumps(line))
     replicas.shutdown()
 

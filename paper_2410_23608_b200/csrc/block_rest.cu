@@ -157,7 +157,14 @@ gelu_kernel(const uint4* __restrict__ u16, const uint4* dh16, long long total, u
   }
 }
 
+// Both kernels are bound by the latency of a row rather than by bandwidth: the forward takes two rows per
+// warp; the backward four, because every extra CTA is another line of partial sums to combine (measured).
 int ln_grid(int rows) {
+  int g = (rows + 15) / 16;
+  if (g > kNumSMs * 6) g = kNumSMs * 6;
+  return g < 1 ? 1 : g;
+}
+int ln_bwd_grid(int rows) {
   int g = (rows + 31) / 32;
   if (g > kNumSMs * 4) g = kNumSMs * 4;
   return g < 1 ? 1 : g;
@@ -165,7 +172,7 @@ int ln_grid(int rows) {
 
 }  // namespace
 
-size_t layer_norm_workspace_bytes(const spa_params& p) { return (size_t)ln_grid(p.B * p.N) * 2 * p.C * sizeof(float) + 256; }
+size_t layer_norm_workspace_bytes(const spa_params& p) { return (size_t)ln_bwd_grid(p.B * p.N) * 2 * p.C * sizeof(float) + 256; }
 
 bool layer_norm_supported(const spa_params& p) { return p.C / (p.dtype == SPA_F32 ? 4 : 8) <= 32 * kLnChunks; }
 
@@ -190,7 +197,7 @@ int launch_layer_norm_bwd(const spa_params& p, const void* dy, const void* x, co
   const int rows = p.B * p.N;
   if (rows == 0) return SPA_OK;
   if (!layer_norm_supported(p)) return SPA_ERR_UNSUPPORTED;
-  const int grid = ln_grid(rows);
+  const int grid = ln_bwd_grid(rows);
   const size_t smem = (size_t)(kRestThreads / 32) * 2 * p.C * sizeof(float);
   float* part = reinterpret_cast<float*>(workspace);
   static bool attr_set = false;
