@@ -57,7 +57,9 @@ layer_norm_kernel(const uint4* __restrict__ x16, const T* __restrict__ gamma, co
 
 // dx = rstd (g - mean(g) - xh mean(g xh)), g = dy gamma, xh = (x - mean) rstd; optionally + add (the residual
 // branch's gradient).  Per-CTA sums of dy xh (dgamma) and dy (dbeta) go to part[blockIdx][2C].
-template <typename T>
+// kCh = 16-byte chunks of a row per lane (ceil(C / (32 chunks))): sized exactly, so that narrow rows do not
+// carry the registers of wide ones and several CTAs share an SM.
+template <typename T, int kCh>
 __global__ void __launch_bounds__(kRestThreads)
 layer_norm_bwd_kernel(const uint4* __restrict__ dy16, const uint4* __restrict__ x16, const T* __restrict__ gamma,
                       const float* __restrict__ mean, const float* __restrict__ rstd, const uint4* add16, int rows,
@@ -66,18 +68,18 @@ layer_norm_bwd_kernel(const uint4* __restrict__ dy16, const uint4* __restrict__ 
   constexpr int E = Vec16<T>::kElems;
   extern __shared__ float acc_s[];  // [8 warps][2C]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, Q = C / E;
-  float ag[kLnChunks][E], ab[kLnChunks][E];
+  float ag[kCh][E], ab[kCh][E];
 #pragma unroll
-  for (int k = 0; k < kLnChunks; ++k)
+  for (int k = 0; k < kCh; ++k)
 #pragma unroll
     for (int e = 0; e < E; ++e) { ag[k][e] = 0.f; ab[k][e] = 0.f; }
   const int warps = gridDim.x * (kRestThreads / 32);
   for (int t = blockIdx.x * (kRestThreads / 32) + warp; t < rows; t += warps) {
     const float mu = mean[t], rs = rstd[t];
-    float g[kLnChunks][E], xh[kLnChunks][E];
+    float g[kCh][E], xh[kCh][E];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-    for (int k = 0; k < kLnChunks; ++k) {
+    for (int k = 0; k < kCh; ++k) {
       const int q = lane + 32 * k;
       if (q < Q) {
         float dy[E], xv[E];
@@ -96,7 +98,7 @@ layer_norm_bwd_kernel(const uint4* __restrict__ dy16, const uint4* __restrict__ 
     }
     const float m1 = warp_sum(s1) / C, m2 = warp_sum(s2) / C;
 #pragma unroll
-    for (int k = 0; k < kLnChunks; ++k) {
+    for (int k = 0; k < kCh; ++k) {
       const int q = lane + 32 * k;
       if (q < Q) {
         float o[E];
@@ -114,7 +116,7 @@ layer_norm_bwd_kernel(const uint4* __restrict__ dy16, const uint4* __restrict__ 
   }
   float* mine = acc_s + warp * 2 * C;
 #pragma unroll
-  for (int k = 0; k < kLnChunks; ++k) {
+  for (int k = 0; k < kCh; ++k) {
     const int q = lane + 32 * k;
     if (q < Q) {
 #pragma unroll
@@ -200,20 +202,26 @@ int launch_layer_norm_bwd(const spa_params& p, const void* dy, const void* x, co
   const int grid = ln_bwd_grid(rows);
   const size_t smem = (size_t)(kRestThreads / 32) * 2 * p.C * sizeof(float);
   float* part = reinterpret_cast<float*>(workspace);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(layer_norm_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(layer_norm_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-    if (e != cudaSuccess) { set_cuda_error(e, "layer_norm_bwd_kernel"); return SPA_ERR_CUDA; }
-    attr_set = true;
-  }
-  if (p.dtype == SPA_F32)
-    launch_pdl(layer_norm_bwd_kernel<float>, grid, kRestThreads, smem, st, (const uint4*)dy, (const uint4*)x,
-               (const float*)gamma, mean, rstd, (const uint4*)add, rows, p.C, (uint4*)dx, part);
-  else
-    launch_pdl(layer_norm_bwd_kernel<__nv_bfloat16>, grid, kRestThreads, smem, st, (const uint4*)dy, (const uint4*)x,
-               (const __nv_bfloat16*)gamma, mean, rstd, (const uint4*)add, rows, p.C, (uint4*)dx, part);
+  const int chunks = (p.C / (p.dtype == SPA_F32 ? 4 : 8) + 31) / 32;  // 1..4 (layer_norm_supported)
+  cudaError_t e = cudaSuccess;
+#define SPA_LN_BWD(T, CH)                                                                                             \
+  do {                                                                                                                \
+    auto kern = layer_norm_bwd_kernel<T, CH>;                                                                         \
+    static bool attr_set = false;                                                                                     \
+    if (!attr_set) { e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); attr_set = e == cudaSuccess; } \
+    if (e == cudaSuccess)                                                                                             \
+      launch_pdl(kern, grid, kRestThreads, smem, st, (const uint4*)dy, (const uint4*)x, (const T*)gamma, mean, rstd, \
+                 (const uint4*)add, rows, p.C, (uint4*)dx, part);                                                     \
+  } while (0)
+#define SPA_LN_BWD_T(T)                                                                                               \
+  do {                                                                                                                \
+    if (chunks <= 1) SPA_LN_BWD(T, 1); else if (chunks == 2) SPA_LN_BWD(T, 2); else if (chunks == 3) SPA_LN_BWD(T, 3); \
+    else SPA_LN_BWD(T, 4);                                                                                            \
+  } while (0)
+  if (p.dtype == SPA_F32) SPA_LN_BWD_T(float); else SPA_LN_BWD_T(__nv_bfloat16);
+#undef SPA_LN_BWD_T
+#undef SPA_LN_BWD
+  if (e != cudaSuccess) { set_cuda_error(e, "layer_norm_bwd_kernel"); return SPA_ERR_CUDA; }
   SPA_CUDA_CHECK_LAUNCH("layer_norm_bwd_kernel");
   // dgamma = columns [0, C) of the per-CTA sums, dbeta = columns [C, 2C)
   int rc = launch_partial_sum(part, grid, 2 * p.C, p.C, dgamma, nullptr, st);
