@@ -223,10 +223,8 @@ int launch_layer_norm_bwd(const spa_params& p, const void* dy, const void* x, co
 #undef SPA_LN_BWD
   if (e != cudaSuccess) { set_cuda_error(e, "layer_norm_bwd_kernel"); return SPA_ERR_CUDA; }
   SPA_CUDA_CHECK_LAUNCH("layer_norm_bwd_kernel");
-  // dgamma = columns [0, C) of the per-CTA sums, dbeta = columns [C, 2C)
-  int rc = launch_partial_sum(part, grid, 2 * p.C, p.C, dgamma, nullptr, st);
-  if (rc != SPA_OK) return rc;
-  return launch_partial_sum(part + p.C, grid, 2 * p.C, p.C, dbeta, nullptr, st);
+  // dgamma = columns [0, C) of the per-CTA sums, dbeta = columns [C, 2C): one reduction launch for both
+  return launch_partial_sum(part, grid, 2 * p.C, p.C, dgamma, p.C, dbeta, st);
 }
 
 int launch_gelu(const spa_params& p, const void* u, const void* dh, int n_cols, void* out, cudaStream_t st) {

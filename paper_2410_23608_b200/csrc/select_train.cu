@@ -60,20 +60,19 @@ select_loss_kernel(const float* __restrict__ scores, const uint8_t* __restrict__
   }
 }
 
-// out[j] = sum over blocks of part[block * stride + j] for j < n_out (out2[0] takes column n_out when given).
+// out[j] = sum over blocks of part[block * stride + j] for j < n_out; columns n_out .. n_out + n_out2 - 1 go to out2.
 // One warp per column: lane l adds blocks l, l + 32, ... in order, then the lanes combine in a fixed tree.
 __global__ void __launch_bounds__(kTrainThreads)
-partial_sum_kernel(const float* __restrict__ part, int n_blocks, int stride, int n_out, float* __restrict__ out,
+partial_sum_kernel(const float* __restrict__ part, int n_blocks, int stride, int n_out, float* __restrict__ out, int n_out2,
                    float* __restrict__ out2) {
   pdl_entry();
   const int j = blockIdx.x * (kTrainThreads / 32) + (threadIdx.x >> 5);
-  const int n_cols = n_out + (out2 != nullptr ? 1 : 0);
-  if (j >= n_cols) return;
+  if (j >= n_out + n_out2) return;
   float s = 0.f;
   for (int b = threadIdx.x & 31; b < n_blocks; b += 32) s += part[(long long)b * stride + j];
   s = warp_sum(s);
   if ((threadIdx.x & 31) == 0) {
-    if (j < n_out) out[j] = s; else out2[0] = s;
+    if (j < n_out) out[j] = s; else out2[j - n_out] = s;
   }
 }
 
@@ -217,10 +216,12 @@ int gate_bwd_grid(int rows) {
 
 }  // namespace
 
-int launch_partial_sum(const float* part, int n_blocks, int stride, int n_out, float* out, float* out2, cudaStream_t st) {
-  const int cols = n_out + (out2 != nullptr ? 1 : 0);
+int launch_partial_sum(const float* part, int n_blocks, int stride, int n_out, float* out, int n_out2, float* out2,
+                       cudaStream_t st) {
+  if (out2 == nullptr) n_out2 = 0;
+  const int cols = n_out + n_out2;
   launch_pdl(partial_sum_kernel, (cols + kTrainThreads / 32 - 1) / (kTrainThreads / 32), kTrainThreads, 0, st, part, n_blocks,
-             stride, n_out, out, out2);
+             stride, n_out, out, n_out2, out2);
   SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel");
   return SPA_OK;
 }
@@ -250,8 +251,8 @@ int launch_select_loss(const spa_params& p, const float* scores, const uint8_t* 
   launch_pdl(select_loss_kernel, grid, kTrainThreads, 0, st, scores, labels, alpha, total, ds, part);
   SPA_CUDA_CHECK_LAUNCH("select_loss_kernel");
   if (loss != nullptr) {
-    launch_pdl(partial_sum_kernel, 1, kTrainThreads, 0, st, (const float*)part, grid, 1, 1, loss, (float*)nullptr);
-    SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel(loss)");
+    const int rc = launch_partial_sum(part, grid, 1, 1, loss, 0, nullptr, st);
+    if (rc != SPA_OK) return rc;
   }
   return SPA_OK;
 }
@@ -288,10 +289,8 @@ int launch_gate_bwd(const spa_params& p, const void* x, const void* w_g, const f
                scores, s_up, ds, rows, p.C, (uint4*)dX, ds_up, part);
   SPA_CUDA_CHECK_LAUNCH("gate_bwd_kernel");
   // dw_g[0..C) and db_g (column C of the partials) in one pass over the per-CTA sums
-  const int cols = p.C + (db_g != nullptr ? 1 : 0);
-  launch_pdl(partial_sum_kernel, (cols + kTrainThreads / 32 - 1) / (kTrainThreads / 32), kTrainThreads, 0, st,
-             (const float*)part, grid, p.C + 1, p.C, dw_g, db_g);
-  SPA_CUDA_CHECK_LAUNCH("partial_sum_kernel(dw_g, db_g)");
+  const int rc = launch_partial_sum(part, grid, p.C + 1, p.C, dw_g, 1, db_g, st);
+  if (rc != SPA_OK) return rc;
   return SPA_OK;
 }
 

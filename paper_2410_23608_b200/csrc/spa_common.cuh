@@ -156,8 +156,9 @@ int launch_pack_bwd_gated(const spa_params& p, const void* dxp, const void* x, c
 int launch_gate_bwd(const spa_params& p, const void* x, const void* w_g, const float* scores, const float* s_up,
                     const float* ds, void* dX, float* dw_g, float* db_g, float* ds_up, void* workspace,
                     cudaStream_t st);
-// out[j] = sum over blocks (fixed order) of part[block * stride + j], j < n_out; out2[0] = column n_out if given
-int launch_partial_sum(const float* part, int n_blocks, int stride, int n_out, float* out, float* out2, cudaStream_t st);
+// out[j] = sum over blocks (fixed order) of part[block * stride + j], j < n_out; the next n_out2 columns go to out2
+int launch_partial_sum(const float* part, int n_blocks, int stride, int n_out, float* out, int n_out2, float* out2,
+                       cudaStream_t st);
 // the rest of the transformer block (block_rest.cu)
 size_t layer_norm_workspace_bytes(const spa_params& p);
 bool layer_norm_supported(const spa_params& p);
