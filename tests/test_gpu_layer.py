@@ -105,3 +105,47 @@ def test_layer_norm_and_gelu_calls_alone():
     du = dev(dh, dt)
     L.spa_gelu_bwd(blk.p, du, dev(u, dt), 4 * C, du)      # in place
     assert_close(host(du), dh * O.gelu_grad(u), dt, "gelu_bwd")
+
+
+def test_two_blocks_in_one_graph():
+    """A stage of two blocks with its own selection in each, captured as one CUDA graph and replayed: the second
+    block's gate sees the first block's output, nothing returns to the host in between."""
+    from paper_2410_23608_b200.layer import SpaLayer
+    cfg, inp, x, prm, f1 = layer_problem(2, 3)
+    dt = cfg.dtype
+    dprm = {k_: (dev(v, dt) if isinstance(v, np.ndarray) else v) for k_, v in prm.items()}
+    a, b = SpaLayer(cfg.B, cfg.N, cfg.C, cfg.H, dt), SpaLayer(cfg.B, cfg.N, cfg.C, cfg.H, dt)
+    xd = dev(x, dt)
+    a.forward(xd, dprm)
+    torch.cuda.synchronize()
+    assert_close(host(a.out), f1["out"], dt, "block 1", scale_max_abs=True)
+    # the oracle's second block reads the very bits the device's first block wrote (runs are reproducible), with
+    # the threshold of the second gate placed in the widest gap of its scores
+    x2 = host(a.out)
+    z2, _, _ = O.layer_norm(x2, prm["g1"], prm["be1"])
+    srt = np.sort(z2.reshape(-1, cfg.C) @ prm["w_g"])
+    lo, hi = len(srt) // 3, 2 * len(srt) // 3
+    k = int(np.argmax(np.diff(srt)[lo:hi])) + lo
+    assert srt[k + 1] - srt[k] > 2e-3
+    prm2 = dict(prm)
+    prm2["b_g"] = float(np.float32(-(srt[k] + srt[k + 1]) / 2))
+    f2 = O.layer_fwd(x2, prm2, cfg.H)
+    dprm2 = dict(dprm)
+    dprm2["b_g"] = prm2["b_g"]
+
+    def stage():
+        return b.forward(a.forward(xd, dprm), dprm2)
+
+    stage()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        out = stage()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    assert a.read_status() == 0 and b.read_status() == 0
+    assert np.array_equal(host(a.out), x2)                      # block 1 reproduced bit for bit inside the graph
+    assert np.array_equal(b.blk.mask.cpu().numpy().astype(bool), f2["spa"]["mask"].reshape(-1))
+    assert 0 < int(b.blk.cu[-1].item()) < cfg.B * cfg.N
+    assert_close(host(out), f2["out"], dt, "block 2", scale_max_abs=True)
