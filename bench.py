@@ -352,26 +352,44 @@ def main():
     value, ms_total = replicas.whole_job_rate(tokens_per_step * args.steps, ms, "cuda")
     ms_per_step = ms_total / args.steps
 
-    # ---- end to end: pinned host inputs in, results out, every step
+    # ---- end to end: pinned host inputs in, results out, every step.  A three-stage pipeline over the rotating
+    # buffer sets: the inputs of a step are copied in on one stream while the previous step computes on the main
+    # stream and the step before that is copied out on a third (PCIe carries both directions at once); every
+    # step still pays for all four copies, and the timed region ends when the last result has reached the host.
     hx = [inp.torch("x").pin_memory() for inp in inps[:2]]
     hdy = [inp.torch("dY").pin_memory() for inp in inps[:2]]
-    hy = torch.empty_like(hx[0]).pin_memory()
-    hdx = torch.empty_like(hx[0]).pin_memory()
+    hy = [torch.empty_like(hx[0]).pin_memory() for _ in range(2)]
+    hdx = [torch.empty_like(hx[0]).pin_memory() for _ in range(2)]
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(n_sets)]
+    ev_done = [torch.cuda.Event() for _ in range(n_sets)]
+    ev_out = [torch.cuda.Event() for _ in range(n_sets)]
 
     def e2e_step(i):
-        inp, d, blk, seq = sets[i % n_sets]
-        d["x"].copy_(hx[(i % n_sets) % 2], non_blocking=True)
-        d["dY"].copy_(hdy[(i % n_sets) % 2], non_blocking=True)
+        k = i % n_sets
+        inp, d, blk, seq = sets[k]
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_out[k])               # the set's previous results have left the device (no-op at first use)
+            d["x"].copy_(hx[k % 2], non_blocking=True)
+            d["dY"].copy_(hdy[k % 2], non_blocking=True)
+            ev_in[k].record(s_in)
+        stream.wait_event(ev_in[k])
         step(i)
-        hy.copy_(blk.y, non_blocking=True)
-        hdx.copy_(blk.dX, non_blocking=True)
+        ev_done[k].record(stream)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_done[k])
+            hy[i % 2].copy_(blk.y, non_blocking=True)
+            hdx[i % 2].copy_(blk.dX, non_blocking=True)
+            ev_out[k].record(s_out)
 
-    for i in range(3):
+    for i in range(min(3, n_sets)):
         e2e_step(i)
+    torch.cuda.synchronize()
     barrier()
     e0.record(stream)
     for i in range(args.steps):
         e2e_step(i)
+    stream.wait_stream(s_out)
     e1.record(stream)
     barrier()
     e2e_value, e2e_total = replicas.whole_job_rate(tokens_per_step * args.steps, e0.elapsed_time(e1), "cuda")
