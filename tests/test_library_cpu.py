@@ -53,3 +53,30 @@ def test_host_side_validation_needs_no_gpu(lib):
 
 def test_params_struct_layout_matches_header(lib):
     assert ctypes.sizeof(lib.SpaParams) == 36
+
+
+def test_later_entry_points_validate_on_the_host(lib):
+    """Fused, trainable-selection, ordered-packing and block calls: bad arguments come back as a status before
+    anything touches a device."""
+    L = lib.lib()
+    p = lib.make_params(2, 16, 64, 2, "bf16")
+    pp = ctypes.byref(p)
+    inv, uns = lib.SPA_ERR_INVALID_ARG, lib.SPA_ERR_UNSUPPORTED
+    assert L.spa_gate_prefill(pp, None, None, 0.0, None, None, None, None, None) == inv
+    assert L.spa_unpack_prefill(pp, None, None, None) == inv
+    assert L.spa_packed_proj_scatter(pp, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_packed_linear_bwd_scatter(pp, None, None, None, 64, 192, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_select_pack_ordered(pp, None, None, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_score_pool(None, 1, 2, 2, None, None) == inv
+    assert L.spa_select_loss(pp, None, None, 1.0, None, None, None, None) == inv
+    assert L.spa_select_pack_bwd_gated(pp, None, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_gate_bwd(pp, None, None, None, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_packed_linear(pp, None, None, None, 64, 256, None, None, 0, None, None) == inv
+    assert L.spa_layer_norm(pp, None, None, None, 1e-5, None, None, None, None) == inv
+    assert L.spa_layer_norm_bwd(pp, None, None, None, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_gelu(pp, None, 256, None, None) == inv
+    assert L.spa_gelu_bwd(pp, None, None, 256, None, None) == inv
+    f32 = lib.make_params(2, 16, 64, 2, "f32")
+    assert L.spa_fused_scatter_supported(ctypes.byref(f32)) == 0          # tensor-core problems only
+    assert L.spa_packed_proj_scatter(ctypes.byref(f32), None, None, None, None, None, None, None, None) in (inv, uns)
+    assert L.spa_train_workspace_bytes(pp) > 0 and L.spa_train_workspace_bytes(None) == 0
