@@ -225,3 +225,59 @@ def test_shifted_packing_order_with_containers(ci, fused):
     assert_close(host(dX), bwd["dX"], cfg.dtype, "dX", scale_max_abs=True)
     for name in ("dW_qkv", "db_qkv", "dW_o", "db_o"):
         assert_close(host(getattr(blk, name)), bwd[name], cfg.dtype, name, scale_max_abs=True)
+
+
+@pytest.mark.parametrize("dtype,n_in,n_out,rows,flags", [
+    ("f32", 96, 200, 300, 0),          # fp32-FMA kernel, ragged tiles
+    ("bf16", 128, 200, 700, 0),        # one-CTA tensor-core kernel, last N tile partly outside
+    ("bf16", 512, 640, 4500, 0),       # CTA pairs: 2.5 tiles of 256 columns, rows not a multiple of 256
+    ("bf16", 512, 640, 4500, 16),      # the same problem on the one-CTA kernel
+])
+def test_general_linear_layer_ragged_sizes_and_accumulation(dtype, n_in, n_out, rows, flags):
+    """spa_packed_linear on sizes that are no multiple of any tile, plain and accumulating, rows counted on the device;
+    rows past the count must stay untouched."""
+    rng = np.random.default_rng(n_out + rows)
+    cap = rows + 37
+    p = L().make_params(1, cap, n_in, 1, dtype, cap, flags)
+    a = round_to(rng.normal(size=(cap, n_in)), dtype)
+    W = round_to(rng.normal(size=(n_out, n_in)) / np.sqrt(n_in), dtype)
+    b = round_to(rng.normal(size=n_out) * 0.1, dtype)
+    base = round_to(rng.normal(size=(cap, n_out)), dtype)
+    cu = torch.tensor([0, rows], dtype=torch.int32, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    ref = O.linear(a[:rows], W, b)
+    for accumulate in (False, True):
+        out = dev(base, dtype)
+        L().spa_packed_linear(p, dev(a, dtype), dev(W, dtype), dev(b, dtype), n_in, n_out, cu, out, accumulate, status)
+        torch.cuda.synchronize()
+        assert L().spa_read_status(status) == 0
+        got = host(out)
+        assert_close(got[:rows], ref + (base[:rows] if accumulate else 0.0), dtype, "out", scale_max_abs=True)
+        assert np.array_equal(got[rows:], base[rows:])
+
+
+@pytest.mark.parametrize("n_in,n_out,rows,flags", [(128, 200, 700, 0), (512, 640, 4500, 0), (512, 640, 4500, 16)])
+def test_general_linear_backward_ragged_sizes(n_in, n_out, rows, flags):
+    """spa_packed_linear_bwd (input gradient, weight gradient, bias gradient in one call: on wide layers the input
+    gradient then runs on CTA pairs) on sizes that are no multiple of any tile."""
+    dtype = "bf16"
+    rng = np.random.default_rng(n_in + rows)
+    cap = rows + 37
+    p = L().make_params(1, cap, n_in, 1, dtype, cap, flags)
+    a = round_to(rng.normal(size=(cap, n_in)), dtype)
+    W = round_to(rng.normal(size=(n_out, n_in)) / np.sqrt(n_in), dtype)
+    dout = round_to(rng.normal(size=(cap, n_out)), dtype)
+    cu = torch.tensor([0, rows], dtype=torch.int32, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    da = torch.full((cap, n_in), 7.0, dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty(n_out, n_in, dtype=torch.float32, device="cuda")
+    db = torch.empty(n_out, dtype=torch.float32, device="cuda")
+    ws = torch.empty(32 * n_out * n_in * 4 + 32 * n_out * 4 + 1024, dtype=torch.uint8, device="cuda")
+    L().spa_packed_linear_bwd(p, dev(a, dtype), dev(W, dtype), dev(dout, dtype), n_in, n_out, cu, da, dW, db, ws, status)
+    torch.cuda.synchronize()
+    assert L().spa_read_status(status) == 0
+    da_ref, dW_ref, db_ref = O.linear_bwd(a[:rows], W, dout[:rows])
+    assert_close(host(da)[:rows], da_ref, dtype, "da", scale_max_abs=True)
+    assert bool((da[rows:] == 7.0).all())
+    assert_close(host(dW), dW_ref, dtype, "dW", scale_max_abs=True)
+    assert_close(host(db), db_ref, dtype, "db", scale_max_abs=True)
