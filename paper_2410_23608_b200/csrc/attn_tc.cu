@@ -25,7 +25,9 @@ namespace {
 
 constexpr int kQ = 128;        // query rows per CTA = TMEM lanes
 constexpr int kKV = 128;       // keys per tile
-constexpr int kFwdThreads = 256;  // two threads per query row: each owns half of the key columns and half of d
+constexpr int kSoftmaxThreads = 256;  // two threads per query row: each owns half of the key columns and half of d
+constexpr int kFwdThreads = kSoftmaxThreads + 32;  // and one warp whose first lane issues every copy and product
+constexpr float kRescaleGap = 8.f;  // log2 units by which a row's maximum may outgrow the one its P and O refer to
 constexpr uint32_t kTmemCols = 256;  // S: 128 fp32 columns, P: 64 (bf16 pairs), O tile: up to 64
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
 
@@ -87,17 +89,18 @@ template <int D> __host__ __device__ constexpr int fwd_smem_bytes() {
 }
 
 template <int D>
-__global__ void __launch_bounds__(kFwdThreads)
+__global__ void __launch_bounds__(kFwdThreads, 2)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __restrict__ seg, int n_seg, int capacity,
                    int C, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
                    int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
   const int q0 = blockIdx.y * kQ;  // grid = (heads, tiles): CTAs past the last valid tile are dispatched last
-  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
+  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool is_softmax = warp < kSoftmaxThreads / 32;  // warps 0-7; warp 8 issues the copies and the products
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 query rows and split
   // the work of each row (key columns of S and P, head dimensions of O) in two halves
-  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
+  const int quarter = warp & 3, half = (warp >> 2) & 1, rl = quarter * 32 + lane;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -107,11 +110,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   auto v_s = [&](int st) { return smem_base + kTile * (2 + 2 * st); };
   const uint32_t bar_base = smem_base + 5 * kTile;
   const uint32_t bar_q = bar_base, bar_s = bar_base + 40, bar_o = bar_base + 48;
+  const uint32_t bar_sfree = bar_base + 56;   // 8 arrivals: every softmax warp holds its part of S_t in registers
+  const uint32_t bar_pready = bar_base + 64;  // 8 arrivals: every softmax warp has written its part of P_t
   auto bar_k = [&](int st) { return bar_base + 8 + 8 * st; };
   auto bar_v = [&](int st) { return bar_base + 24 + 8 * st; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 5 * kTile + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 68);
-  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 72);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + 5 * kTile + 72);
+  volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 76);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 80);
+  // [2 tile parities][4 quarters]: written by the two warps of a quarter before their barrier, read after it
+  volatile int* abort_pair = reinterpret_cast<volatile int*>(smem_al + 5 * kTile + 88);
   float* xch = reinterpret_cast<float*>(smem_al + 5 * kTile + 128);  // [2 tile parities][2 halves][128 rows]
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + 5 * kTile + 128 + 2048);  // [kSegStage + 1]
 
@@ -122,7 +129,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     for (int s = 0; s < 2; ++s) { ptx::mbar_init(bar_k(s), 1); ptx::mbar_init(bar_v(s), 1); }
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_o, 1);
-    *abort_flag = 0;
+    ptx::mbar_init(bar_sfree, kSoftmaxThreads / 32);
+    ptx::mbar_init(bar_pready, kSoftmaxThreads / 32);
+    *abort_any = 0;
+    for (int i = 0; i < 8; ++i) abort_pair[i] = 0;
     ptx::fence_mbar_init();
   }
   pdl_entry();
@@ -131,7 +141,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     for (int i = tid; i <= n_seg; i += kFwdThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
   if (q0 >= Np) return;
-  if (tid == 0) {  // the Q tile depends only on q0: fetch it under the segment search
+  if (tid == kSoftmaxThreads) {  // the Q tile depends only on q0: fetch it under the segment search
     ptx::mbar_expect_tx(bar_q, kTile);
     ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
   }
@@ -142,14 +152,18 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   const uint32_t tmem = *tmem_slot;
 
   const int row = q0 + rl;
-  const RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
-  if (half == 0) {
-    const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
-    if (row == q0) range[0] = mine.lo;
-    if (row == last) range[1] = mine.hi;
+  RowSeg mine{0, 0};
+  if (is_softmax) {
+    mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+    if (half == 0) {
+      const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
+      if (row == q0) range[0] = mine.lo;
+      if (row == last) range[1] = mine.hi;
+    }
   }
   __syncthreads();
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;  // TMEM lanes this warp may touch
+  float lse_m = 0.f;
   constexpr int kCols = kKV / 2;  // key columns of each tile owned by this thread
   constexpr int kDh = D / 2;      // head dimensions of O owned by this thread
   const int col0 = half * kCols;
@@ -159,182 +173,222 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(kQ, kKV, false, false);
   constexpr uint32_t kIdescO = ptx::idesc_bf16_f32(kQ, D, false, true);
 
-  auto load_k = [&](int t) {
-    ptx::mbar_expect_tx(bar_k(t & 1), kTile);
-    ptx::tma_load_2d(k_s(t & 1), &tm, bar_k(t & 1), C + h * D, kv_lo + t * kKV);
-  };
-  auto load_v = [&](int t) {
-    ptx::mbar_expect_tx(bar_v(t & 1), kTile);
-    ptx::tma_load_2d(v_s(t & 1), &tm, bar_v(t & 1), 2 * C + h * D, kv_lo + t * kKV);
-  };
-  auto issue_qk = [&](int t) {  // S = Q K_t^T into TMEM; bar_s completes when it is done
-    bool ok = (t > 0) || ptx::mbar_wait(bar_q, 0);
-    ok = ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1) && ok;
-    if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; return; }
-    ptx::tc_fence_after_sync();
-#pragma unroll
-    for (int k = 0; k < D / 16; ++k)
-      ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(k_s(t & 1), k), kIdescS, k != 0 ? 1u : 0u);
-    ptx::mma_commit(bar_s);
-  };
-  int loads_k = 0, loads_v = 0;  // tiles whose loads thread 0 has issued
-  if (tid == 0) {
-    load_k(0);
-    load_v(0);
-    loads_k = loads_v = 1;
-    if (n_tiles > 1) { load_k(1); loads_k = 2; }
-    issue_qk(0);
-  }
-
-  float o[kDh];
-#pragma unroll
-  for (int e = 0; e < kDh; ++e) o[e] = 0.f;
-  float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
-  const unsigned span = (unsigned)(mine.hi - mine.lo);
-
-  // O = alpha O + (P V of tile t_prev), read from TMEM once that product has completed
-  auto fold_o = [&](int t_prev) {
-    if (!ptx::mbar_wait(bar_o, t_prev & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-    ptx::tc_fence_after_sync();
-    uint32_t r[kDh];
-    if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + kColO + half * kDh, r);
-    else ptx::tmem_ld_32x16(tmem + lane_base + kColO + half * kDh, r);
-    ptx::tmem_ld_wait();
-#pragma unroll
-    for (int e = 0; e < kDh; ++e) o[e] = fmaf(o[e], alpha_prev, __uint_as_float(r[e]));
-  };
-
-  for (int t = 0; t < n_tiles; ++t) {
-    const int st = t & 1;
-    const int kv0 = kv_lo + t * kKV;
-    // ---- fold in the previous tile's P V (it was issued after this tile's S, so both are complete by then)
-    if (t > 0) fold_o(t - 1);
-    if (tid == 0 && t + 1 < n_tiles) { load_v(t + 1); loads_v = t + 2; }  // V stage of tile t-1 is free
-    // ---- S_t into registers: four TMEM loads in flight, one wait
-    if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-    ptx::tc_fence_after_sync();
-    uint32_t s[kCols];
-#pragma unroll
-    for (int c = 0; c < kCols / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColS + col0 + c * 32, s + c * 32);
-    ptx::tmem_ld_wait();
-    // Which of this thread's groups of 32 key columns meet its row's segment at all (the others take no
-    // arithmetic: their P is zero); the mask is applied only where a boundary of the segment crosses a group.
-    // This half's row maximum is handed to the partner thread through shared memory.
-    const int kc0 = kv0 + col0;
-    bool need[kCols / 32];
-#pragma unroll
-    for (int c = 0; c < kCols / 32; ++c) {
-      const int g0 = kc0 + c * 32;
-      need[c] = g0 < mine.hi && g0 + 32 > mine.lo;
-      if (need[c] && !(g0 >= mine.lo && g0 + 32 <= mine.hi)) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if ((unsigned)(g0 + j - mine.lo) >= span) s[c * 32 + j] = 0xff800000u;  // -inf
-      }
+  // Bounded wait that also gives up as soon as any thread of the CTA has reported a failure.
+  auto wait = [&](uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < ptx::kWaitLimit; ++i) {
+      if (ptx::mbar_try_wait(bar, parity)) return true;
+      if ((i & 255u) == 255u && *abort_any) return false;
     }
-    float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+    return false;
+  };
+
+  if (!is_softmax) {
+    // ---------------------------------------------------------------- copies and products: one thread
+    if (lane == 0) {
+      auto load_k = [&](int t) {
+        ptx::mbar_expect_tx(bar_k(t & 1), kTile);
+        ptx::tma_load_2d(k_s(t & 1), &tm, bar_k(t & 1), C + h * D, kv_lo + t * kKV);
+      };
+      auto load_v = [&](int t) {
+        ptx::mbar_expect_tx(bar_v(t & 1), kTile);
+        ptx::tma_load_2d(v_s(t & 1), &tm, bar_v(t & 1), 2 * C + h * D, kv_lo + t * kKV);
+      };
+      auto issue_qk = [&](int t) {  // S = Q K_t^T into TMEM; bar_s completes when it is done
+        if (!wait(bar_k(t & 1), (t >> 1) & 1)) return false;
+        ptx::tc_fence_after_sync();
 #pragma unroll
-    for (int c = 0; c < kCols / 32; ++c) {
-      if (need[c]) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c * 32 + j + u]));
+        for (int k = 0; k < D / 16; ++k)
+          ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(k_s(t & 1), k), kIdescS, k != 0 ? 1u : 0u);
+        ptx::mma_commit(bar_s);
+        return true;
+      };
+      int loads_k = 0, loads_v = 0;  // tiles whose loads have been issued
+      bool ok = true;
+      if (n_tiles > 0) {
+        load_k(0);
+        load_v(0);
+        loads_k = loads_v = 1;
+        if (n_tiles > 1) { load_k(1); loads_k = 2; }
+        ok = wait(bar_q, 0) && issue_qk(0);
+      }
+      for (int t = 0; ok && t < n_tiles; ++t) {
+        // every softmax thread holds its S_t columns: the S columns and K stage t & 1 are free
+        if (!(ok = wait(bar_sfree, t & 1))) break;
+        if (t + 1 < n_tiles) {
+          if (!(ok = issue_qk(t + 1))) break;  // runs on the tensor core under the softmax of tile t
+          if (t + 2 < n_tiles) { load_k(t + 2); loads_k = t + 3; }
         }
-      }
-    }
-    float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-    xch[((t & 1) * 2 + half) * 128 + rl] = mt;
-    if (tid == 0 && t + 2 < n_tiles) { load_k(t + 2); loads_k = t + 3; }  // K stage st is free: S_t is complete
-    ptx::tc_fence_before_sync();
-    __syncthreads();  // A: every thread holds its S row and has consumed the previous O tile
-    if (*abort_flag) break;
-    if (tid == 0 && t + 1 < n_tiles) issue_qk(t + 1);  // runs on the tensor core under the softmax below
-
-    // ---- online softmax of this half row (exp2 domain): one fma, one ex2 and one add per key
-    mt = fmaxf(mt, xch[((t & 1) * 2 + (half ^ 1)) * 128 + rl]);
-    const float m_new = fmaxf(m, mt * scale_log2e);  // the scale is positive: max commutes with it
-    const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
-    const float alpha = ptx::ex2_approx(m - m_use);
-    float rs0 = 0.f, rs1 = 0.f;
-#pragma unroll
-    for (int c = 0; c < kCols / 32; ++c) {
-      uint32_t pk[16];
-      if (need[c]) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j]), scale_log2e, -m_use));  // -inf -> 0
-          const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j + 1]), scale_log2e, -m_use));
-          rs0 += p0;
-          rs1 += p1;
-          __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
-          pk[j >> 1] = *reinterpret_cast<uint32_t*>(&b);
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) pk[j] = 0u;
-      }
-      ptx::tmem_st_32x16(tmem + lane_base + kColP + (col0 >> 1) + c * 16, pk);
-    }
-    const float rs = rs0 + rs1;
-    ptx::tmem_st_wait();
-    l = l * alpha + rs;
-    m = m_new;
-    alpha_prev = alpha;
-    // ---- V lines past the last valid packed row must not reach the product
-    if (kv0 + kKV > Np) {
-      if (!ptx::mbar_wait(bar_v(st), (t >> 1) & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-      const int first = Np - kv0;  // >= 1
-      constexpr int kChunks = HT::kRowBytes / 16;
-      for (int c = tid; c < (kKV - first) * kChunks; c += kFwdThreads)
-        *reinterpret_cast<uint4*>(smem_al + kTile * (2 + 2 * st) + (first + c / kChunks) * HT::kRowBytes +
-                                  (c % kChunks) * 16) = make_uint4(0, 0, 0, 0);
-      ptx::fence_proxy_async_smem();
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();  // B: P_t is complete in TMEM
-    if (*abort_flag) break;
-    if (tid == 0) {
-      if (ptx::mbar_wait(bar_v(st), (t >> 1) & 1)) {
+        // P_t is in TMEM, O has been rescaled where needed, and the previous P V product has completed
+        if (!(ok = wait(bar_pready, t & 1))) break;
+        if (!(ok = wait(bar_v(t & 1), (t >> 1) & 1))) break;
         ptx::tc_fence_after_sync();
 #pragma unroll
         for (int k = 0; k < kKV / 16; ++k)
-          ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(v_s(st), k), kIdescO, k != 0 ? 1u : 0u);
+          ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(v_s(t & 1), k), kIdescO,
+                           (k != 0 || t > 0) ? 1u : 0u);
         ptx::mma_commit(bar_o);
-      } else {
+        if (t + 1 < n_tiles) { load_v(t + 1); loads_v = t + 2; }  // its stage held V of tile t - 1
+      }
+      if (!ok) {
         record_status(d_status, SPA_ERR_TIMEOUT);
-        *abort_flag = 1;
+        *abort_any = 1;
+        // let outstanding loads land before shared memory is released
+        for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
+        for (int t = loads_v > 2 ? loads_v - 2 : 0; t < loads_v; ++t) ptx::mbar_wait(bar_v(t & 1), (t >> 1) & 1);
+        ptx::mbar_wait(bar_q, 0);
       }
     }
-  }
-  if (!*abort_flag && n_tiles > 0) fold_o(n_tiles - 1);
+  } else {
+    // ---------------------------------------------------------------- online softmax: two threads per query row
+    float m = -CUDART_INF_F, l = 0.f;  // m: the maximum the stored P and O refer to (may lag the true one by kRescaleGap)
+    const unsigned span = (unsigned)(mine.hi - mine.lo);
+    auto fail = [&](int slot) {
+      record_status(d_status, SPA_ERR_TIMEOUT);
+      abort_pair[slot * 4 + quarter] = 1;
+      *abort_any = 1;
+    };
+    for (int t = 0; t < n_tiles; ++t) {
+      const int st = t & 1;
+      const int kv0 = kv_lo + t * kKV;
+      // ---- S_t into registers: TMEM loads in flight together, one wait
+      if (!wait(bar_s, t & 1)) fail(t & 1);
+      ptx::tc_fence_after_sync();
+      uint32_t s[kCols];
+#pragma unroll
+      for (int c = 0; c < kCols / 32; ++c) ptx::tmem_ld_32x32(tmem + lane_base + kColS + col0 + c * 32, s + c * 32);
+      ptx::tmem_ld_wait();
+      // Which of this thread's groups of 32 key columns meet its row's segment at all (the others take no
+      // arithmetic: their P is zero); the mask is applied only where a boundary of the segment crosses a group.
+      // This half's row maximum is handed to the partner thread through shared memory.
+      const int kc0 = kv0 + col0;
+      bool need[kCols / 32];
+#pragma unroll
+      for (int c = 0; c < kCols / 32; ++c) {
+        const int g0 = kc0 + c * 32;
+        need[c] = g0 < mine.hi && g0 + 32 > mine.lo;
+        if (need[c] && !(g0 >= mine.lo && g0 + 32 <= mine.hi)) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if ((unsigned)(g0 + j - mine.lo) >= span) s[c * 32 + j] = 0xff800000u;  // -inf
+        }
+      }
+      float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+      for (int c = 0; c < kCols / 32; ++c) {
+        if (need[c]) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c * 32 + j + u]));
+          }
+        }
+      }
+      float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      xch[((t & 1) * 2 + half) * 128 + rl] = mt;
+      ptx::tc_fence_before_sync();
+      ptx::named_barrier(1 + quarter, 64);  // the two warps that share these 32 rows
+      if (abort_pair[(t & 1) * 4 + quarter]) break;
+      if (lane == 0) ptx::mbar_arrive(bar_sfree);
 
-  // the two halves of a row share the running max but kept separate sums: combine them
-  xch[half * 128 + rl] = l;
-  __syncthreads();  // nobody sets the flag from here on: the branch below is taken by all threads or by none
-  if (!*abort_flag) {
+      // ---- this half row's P (exp2 domain): one fma, one ex2 and one add per key.  The maximum that P and O
+      // refer to is raised only when the true one has grown by more than kRescaleGap, so O (accumulated in
+      // TMEM over all tiles) is rescaled rarely; sums and outputs are exact for any such reference value.
+      mt = fmaxf(mt, xch[((t & 1) * 2 + (half ^ 1)) * 128 + rl]);
+      const float m_cand = fmaxf(m, mt * scale_log2e);  // the scale is positive: max commutes with it
+      const bool raise = m_cand > m + kRescaleGap;      // also the first tile that has a key of this row
+      const float m_new = raise ? m_cand : m;
+      const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
+      const float alpha = raise ? ptx::ex2_approx(m - m_use) : 1.f;
+      float rs0 = 0.f, rs1 = 0.f;
+      uint32_t pk[kCols / 2];
+#pragma unroll
+      for (int c = 0; c < kCols / 32; ++c) {
+        if (need[c]) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j]), scale_log2e, -m_use));  // -inf -> 0
+            const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(s[c * 32 + j + 1]), scale_log2e, -m_use));
+            rs0 += p0;
+            rs1 += p1;
+            __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);  // low half = even key
+            pk[c * 16 + (j >> 1)] = *reinterpret_cast<uint32_t*>(&b);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) pk[c * 16 + j] = 0u;
+        }
+      }
+      // ---- the previous P V product must have completed before P is overwritten or O rescaled
+      if (t > 0) {
+        if (!wait(bar_o, (t - 1) & 1)) fail((t + 1) & 1);
+        ptx::tc_fence_after_sync();
+        if (__any_sync(0xffffffffu, raise)) {
+          uint32_t r[kDh];
+          if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + kColO + half * kDh, r);
+          else ptx::tmem_ld_32x16(tmem + lane_base + kColO + half * kDh, r);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < kDh; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+          if (kDh == 32) ptx::tmem_st_32x32(tmem + lane_base + kColO + half * kDh, r);
+          else ptx::tmem_st_32x16(tmem + lane_base + kColO + half * kDh, r);
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < kCols / 32; ++c)
+        ptx::tmem_st_32x16(tmem + lane_base + kColP + (col0 >> 1) + c * 16, pk + c * 16);
+      ptx::tmem_st_wait();
+      l = l * alpha + (rs0 + rs1);
+      m = m_new;
+      // ---- V lines past the last valid packed row must not reach the product
+      if (kv0 + kKV > Np) {
+        if (!wait(bar_v(st), (t >> 1) & 1)) fail((t + 1) & 1);
+        const int first = Np - kv0;  // >= 1
+        constexpr int kChunks = HT::kRowBytes / 16;
+        for (int c = tid; c < (kKV - first) * kChunks; c += kSoftmaxThreads)
+          *reinterpret_cast<uint4*>(smem_al + kTile * (2 + 2 * st) + (first + c / kChunks) * HT::kRowBytes +
+                                    (c % kChunks) * 16) = make_uint4(0, 0, 0, 0);
+        ptx::fence_proxy_async_smem();
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_pready);
+    }
+    // the last product completes O
+    if (n_tiles > 0 && !*abort_any && !wait(bar_o, (n_tiles - 1) & 1)) fail(0);
+    xch[half * 128 + rl] = l;  // the two halves of a row share the reference maximum but kept separate sums
+    lse_m = m;
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // nobody reports a failure from here on: the branches below are taken by all threads or by none
+  ptx::tc_fence_after_sync();
+  const bool failed = *abort_any != 0;
+  if (!failed && is_softmax) {
     // normalised rows go to the Q tile's shared memory (idle now: every product has completed) as bf16 and
     // leave from there as whole lines
-    const float l_row = l + xch[(half ^ 1) * 128 + rl];
+    uint32_t r[kDh];
+    if (n_tiles > 0) {
+      if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + kColO + half * kDh, r);
+      else ptx::tmem_ld_32x16(tmem + lane_base + kColO + half * kDh, r);
+      ptx::tmem_ld_wait();
+    } else {
+#pragma unroll
+      for (int e = 0; e < kDh; ++e) r[e] = 0u;
+    }
+    const float l_row = xch[half * 128 + rl] + xch[(half ^ 1) * 128 + rl];
     const float inv_l = row < Np ? 1.f / l_row : 0.f;
     const int rot = chunk_rot<D>(rl);
 #pragma unroll
     for (int c = 0; c < kDh / 8; ++c) {
       float v[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = o[c * 8 + e] * inv_l;
+      for (int e = 0; e < 8; ++e) v[e] = row < Np ? __uint_as_float(r[c * 8 + e]) * inv_l : 0.f;
       *reinterpret_cast<uint4*>(smem_al + rl * HT::kRowBytes + (((half * (kDh / 8) + c) ^ rot) << 4)) =
           Vec16<__nv_bfloat16>::from_float(v);
     }
-    if (half == 0 && row < Np) lse[(long long)h * capacity + row] = (m + log2f(l_row)) * 0.6931471805599453f;
-    __syncthreads();
-    copy_tile_out<D, kFwdThreads>(smem_al, ao + h * D, C, q0, Np, tid);
+    if (half == 0 && row < Np) lse[(long long)h * capacity + row] = (lse_m + log2f(l_row)) * 0.6931471805599453f;
   }
-  if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
-    for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
-    for (int t = loads_v > 2 ? loads_v - 2 : 0; t < loads_v; ++t) ptx::mbar_wait(bar_v(t & 1), (t >> 1) & 1);
-    ptx::mbar_wait(bar_q, 0);
-  }
+  __syncthreads();
+  if (!failed) copy_tile_out<D, kFwdThreads>(smem_al, ao + h * D, C, q0, Np, tid);
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) {
