@@ -122,8 +122,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   float* xch = reinterpret_cast<float*>(smem_al + 5 * kTile + 128);  // [2 tile parities][2 halves][128 rows]
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + 5 * kTile + 128 + 2048);  // [kSegStage + 1]
 
-  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
-  if (tid == 0) {
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail.  The thread
+  // that sets the barriers up is the one that later issues the copies counted on them (program order: no copy
+  // can meet a barrier that is not initialised yet).
+  if (tid == kSoftmaxThreads) {
     ptx::prefetch_tensormap(&tm);
     ptx::mbar_init(bar_q, 1);
     for (int s = 0; s < 2; ++s) { ptx::mbar_init(bar_k(s), 1); ptx::mbar_init(bar_v(s), 1); }
@@ -247,11 +249,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       abort_pair[slot * 4 + quarter] = 1;
       *abort_any = 1;
     };
+    // every lane polls (measured faster than one lane polling for the warp); the warp takes one answer
+    auto wait_w = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, wait(bar, parity)) != 0; };
     for (int t = 0; t < n_tiles; ++t) {
       const int st = t & 1;
       const int kv0 = kv_lo + t * kKV;
       // ---- S_t into registers: TMEM loads in flight together, one wait
-      if (!wait(bar_s, t & 1)) fail(t & 1);
+      if (!wait_w(bar_s, t & 1)) fail(t & 1);
       ptx::tc_fence_after_sync();
       uint32_t s[kCols];
 #pragma unroll
@@ -320,7 +324,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       }
       // ---- the previous P V product must have completed before P is overwritten or O rescaled
       if (t > 0) {
-        if (!wait(bar_o, (t - 1) & 1)) fail((t + 1) & 1);
+        if (!wait_w(bar_o, (t - 1) & 1)) fail((t + 1) & 1);
         ptx::tc_fence_after_sync();
         if (__any_sync(0xffffffffu, raise)) {
           uint32_t r[kDh];
@@ -354,7 +358,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       if (lane == 0) ptx::mbar_arrive(bar_pready);
     }
     // the last product completes O
-    if (n_tiles > 0 && !*abort_any && !wait(bar_o, (n_tiles - 1) & 1)) fail(0);
+    const bool gave_up = __shfl_sync(0xffffffffu, *abort_any, 0) != 0;  // one answer per warp
+    if (n_tiles > 0 && !gave_up && !wait_w(bar_o, (n_tiles - 1) & 1)) fail(0);
     xch[half * 128 + rl] = l;  // the two halves of a row share the reference maximum but kept separate sums
     lse_m = m;
   }
@@ -406,30 +411,417 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 //   kDQ = false: a CTA owns 128 key rows j; per streamed tile of 64 queries  S^T = K Q^T, dP^T = V dO^T,
 //                P^T and dS^T written to TMEM as bf16,        dV += P^T dO,  dK += dS^T Q.
 // The footprint is kept to 256 TMEM columns and about 80 KB of shared memory so that two CTAs share an
-// SM: one CTA's arithmetic runs under the other's MMA round trips and prologue.  To fit, the streamed
-// tiles are 64 rows, and the bf16 operands (P^T, dS) are written over the first half of the fp32 tiles
-// they were computed from - after a barrier, once every thread holds its fp32 columns in registers.
-// MMAs execute in issue order, so the next tile's fp32 products (which overwrite those columns) are
-// simply issued behind the accumulating products that read them.
-constexpr int kBwdThreads = 256;   // two threads per TMEM lane (row): each owns 32 of the 64 streamed columns
+// SM.  Warps 0-7 do the arithmetic (two threads per row, 32 of the 64 streamed columns each); the first
+// lane of warp 8 issues every copy and product and is told through mbarriers when the others hold a tile's
+// fp32 values in registers and when its bf16 operands are in TMEM.
+// The bf16 operands have TMEM columns of their own, so the next tile's fp32 products are issued as soon as
+// the current ones are in registers and run under the arithmetic.  That needs room in TMEM: this kernel serves
+// the dQ pass and the dK/dV pass at d = 32; the dK/dV pass at d = 64 is attn_bwd_kv_aliased_kernel below.
+constexpr int kBwdMath = 256;      // arithmetic threads: two per TMEM lane (row)
+constexpr int kBwdThreads = kBwdMath + 32;
 constexpr int kBwdY = 64;          // rows of a streamed tile
 constexpr int kBwdStages = 3;      // streamed tiles in shared memory
 constexpr uint32_t kBwdTmemCols = 256;
-constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;  // operands alias S1 / S2 columns [0, 32)
+constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;
+constexpr int kBwdStatBytes = 3 * 2 * kBwdY * 4;  // three tiles' worth of lse_i and D_i of the streamed queries
 
 template <int D, bool kDQ> __host__ __device__ constexpr int bwd_smem_bytes() {
   // own tiles (the dQ pass also holds the O tile), streamed tiles, alignment slack, statistics, barriers, segment offsets
-  return (kDQ ? 3 : 2) * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64;
+  return (kDQ ? 3 : 2) * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64;
 }
 
 template <int D, bool kDQ>
-__global__ void __launch_bounds__(kBwdThreads)
+__global__ void __launch_bounds__(kBwdThreads, 2)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
                    int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
   using HT = HeadTile<D>;
+  constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
+  constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
+  constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
+  constexpr float kLog2e = 1.4426950408889634f;
+  // the bf16 operands have TMEM columns of their own, so the next fp32 products need not wait for the accumulating ones
+  static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_aliased_kernel");
+  constexpr uint32_t kColOpP = 160u;                // P^T (dK/dV pass only)
+  constexpr uint32_t kColOpDS = kDQ ? 192u : 224u;  // dS or dS^T
+  const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
+  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool is_math = warp < kBwdMath / 32;
+  // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
+  const int quarter = warp & 3, half = (warp >> 2) & 1, rl = quarter * 32 + lane;
+  const float scale_log2e = scale * kLog2e;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  const uint32_t x1_s = smem_base, x2_s = smem_base + kTile, x3_s = smem_base + 2 * kTile;
+  constexpr int kYBase = kOwn * kTile;
+  auto y1_off = [&](int st) { return kYBase + kYTile * (2 * st); };
+  auto y2_off = [&](int st) { return kYBase + kYTile * (2 * st + 1); };
+  constexpr int kStatBase = kYBase + kBwdStages * 2 * kYTile;
+  float* stat_lse = reinterpret_cast<float*>(smem_al + kStatBase);  // [3][64] lse_i * log2e of the staged query tile
+  float* stat_D = stat_lse + 3 * kBwdY;                              // [3][64] D_i
+  constexpr int kBarBase = kStatBase + kBwdStatBytes;
+  const uint32_t bar_base = smem_base + kBarBase;
+  const uint32_t bar_x = bar_base, bar_s = bar_base + 32, bar_acc = bar_base + 40;
+  const uint32_t bar_sfree = bar_base + 48;    // 8 arrivals: every arithmetic warp holds the fp32 values of tile t
+  const uint32_t bar_opready = bar_base + 56;  // 8 arrivals: every arithmetic warp has written the operands of tile t
+  auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kBarBase + 64);
+  volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + kBarBase + 68);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + kBarBase + 72);
+  int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kBarBase + 128);  // [kSegStage + 1]
+
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail.  The thread
+  // that sets the barriers up is the one that later issues the copies counted on them.
+  if (tid == kBwdMath) {
+    ptx::prefetch_tensormap(&tm_qkv);
+    ptx::prefetch_tensormap(&tm_do);
+    ptx::prefetch_tensormap(&tm_qkv_y);
+    ptx::prefetch_tensormap(&tm_do_y);
+    if (kDQ) ptx::prefetch_tensormap(&tm_o);
+    ptx::mbar_init(bar_x, 1);
+    for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_acc, 1);
+    ptx::mbar_init(bar_sfree, kBwdMath / 32);
+    ptx::mbar_init(bar_opready, kBwdMath / 32);
+    *abort_any = 0;
+    ptx::fence_mbar_init();
+  }
+  pdl_entry();
+  const bool staged = n_seg < kSegStage;
+  if (staged)
+    for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  if (r0 >= Np) return;
+  const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
+  if (tid == kBwdMath) {  // the own tiles depend only on r0: fetch them under the segment search
+    ptx::mbar_expect_tx(bar_x, kOwn * kTile);
+    ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
+    if (kDQ) {
+      ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                  // dO
+      ptx::tma_load_2d(x3_s, &tm_o, bar_x, h * D, r0);                   // O, for D_i = dO_i . O_i
+    } else {
+      ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
+    }
+  }
+  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // barriers, TMEM address and staged offsets are visible
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+
+  const int row = r0 + rl;
+  RowSeg mine{0, 0};
+  if (is_math) {
+    mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+    if (half == 0) {
+      const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
+      if (row == r0) range[0] = mine.lo;
+      if (row == last) range[1] = mine.hi;
+    }
+  }
+  __syncthreads();
+  const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
+  const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
+
+  const int y1_col = (kDQ ? C : 0) + h * D;           // streamed operand inside qkv: K | Q
+  auto load_other = [&](int t_) {  // streamed tile t_ into stage t_ mod kBwdStages
+    const int st = t_ % kBwdStages, y0 = o_lo + t_ * kBwdY;
+    ptx::mbar_expect_tx(bar_y(st), 2 * kYTile);
+    ptx::tma_load_2d(smem_base + y1_off(st), &tm_qkv_y, bar_y(st), y1_col, y0);
+    if (kDQ) ptx::tma_load_2d(smem_base + y2_off(st), &tm_qkv_y, bar_y(st), 2 * C + h * D, y0);   // V
+    else ptx::tma_load_2d(smem_base + y2_off(st), &tm_do_y, bar_y(st), h * D, y0);                // dO
+  };
+  int issued = 0;  // streamed tiles whose loads have been issued (kept by the issuing thread)
+  if (tid == kBwdMath) {
+    for (int t_ = 0; t_ < n_tiles && t_ < 2; ++t_) load_other(t_);
+    issued = n_tiles < 2 ? n_tiles : 2;
+  }
+
+  // Bounded wait that also gives up as soon as any thread of the CTA has reported a failure.
+  auto wait = [&](uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < ptx::kWaitLimit; ++i) {
+      if (ptx::mbar_try_wait(bar, parity)) return true;
+      if ((i & 255u) == 255u && *abort_any) return false;
+    }
+    return false;
+  };
+  // every lane polls; the warp takes one answer, so that a whole warp gives up or none of it
+  auto wait_w = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, wait(bar, parity)) != 0; };
+
+  // per-row statistics of the query side
+  float my_lse = 0.f, my_D = 0.f;   // kDQ: this thread's query row
+  float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next streamed query tile, row rl < 64
+  if (is_math) {
+    if (kDQ) {
+      if (row < Np) my_lse = lse[(long long)h * capacity + row] * kLog2e;
+    } else if (half == 0 && rl < kBwdY) {
+      const int i = o_lo + rl;
+      if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
+    }
+  }
+
+  constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, kBwdY, false, false);
+  constexpr uint32_t kIdescAcc = ptx::idesc_bf16_f32(128, D, false, true);
+  const unsigned span = (unsigned)(mine.hi - mine.lo);
+
+  // Make streamed tile t_ ready for the products (arithmetic warps): its load has landed, lines past the last
+  // valid packed row are zeroed (they are unspecified memory and would be summed over), its query statistics
+  // are staged.  Returns false when the wait for the load gave up.
+  auto prep = [&](int t_) {
+    const int st = t_ % kBwdStages;
+    bool ok = wait_w(bar_y(st), (t_ / kBwdStages) & 1);
+    if (t_ == 0) ok = wait_w(bar_x, 0) && ok;
+    const int y0 = o_lo + t_ * kBwdY;
+    if (y0 + kBwdY > Np) {
+      const int first = Np - y0;
+      constexpr int kChunks = HT::kRowBytes / 16;
+      for (int c = tid; c < (kBwdY - first) * kChunks; c += kBwdMath) {
+        const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
+        *reinterpret_cast<uint4*>(smem_al + y1_off(st) + off) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(smem_al + y2_off(st) + off) = make_uint4(0, 0, 0, 0);
+      }
+      ptx::fence_proxy_async_smem();
+    }
+    if (!kDQ && half == 0 && rl < kBwdY) {
+      stat_lse[(t_ % 3) * kBwdY + rl] = nxt_lse;
+      stat_D[(t_ % 3) * kBwdY + rl] = nxt_D;
+      const int i = y0 + kBwdY + rl;
+      nxt_lse = 0.f; nxt_D = 0.f;
+      if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
+    }
+    return ok;
+  };
+
+  if (is_math && !prep(0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // tile 0 is ready; a failure so far is seen by all threads or by none
+  const bool failed_early = *abort_any != 0;
+
+  if (!is_math) {
+    // ---------------------------------------------------------------- copies and products: one thread
+    if (lane == 0 && !failed_early) {
+      auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
+        const int st = t_ % kBwdStages;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(smem_base + y1_off(st), k), kIdescS, k != 0 ? 1u : 0u);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(smem_base + y2_off(st), k), kIdescS, k != 0 ? 1u : 0u);
+        ptx::mma_commit(bar_s);
+      };
+      bool ok = true;
+      ptx::tc_fence_after_sync();
+      if (n_tiles > 0) issue_s(0);
+      for (int t = 0; ok && t < n_tiles; ++t) {
+        const int st = t % kBwdStages;
+        if (t + 1 < n_tiles) {
+          // the fp32 values of tile t are in registers and tile t + 1 is ready: its products run under the arithmetic
+          if (!(ok = wait(bar_sfree, t & 1))) break;
+          ptx::tc_fence_after_sync();
+          issue_s(t + 1);
+        }
+        // the stage of tile t - 1 is free once its accumulating products have completed
+        if (t + 2 < n_tiles) {
+          if (t > 0 && !(ok = wait(bar_acc, (t - 1) & 1))) break;
+          load_other(t + 2);
+          issued = t + 3;
+        }
+        if (!(ok = wait(bar_opready, t & 1))) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t acc = (t != 0) ? 1u : 0u;
+        const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
+        if (kDQ) {
+#pragma unroll
+          for (int k = 0; k < kBwdY / 16; ++k)   // dQ += dS K
+            ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpDS + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+        } else {
+#pragma unroll
+          for (int k = 0; k < kBwdY / 16; ++k)   // dV += P^T dO
+            ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpP + k * 8, HT::mnmajor(y2a, k), kIdescAcc, acc | (k != 0));
+#pragma unroll
+          for (int k = 0; k < kBwdY / 16; ++k)   // dK += dS^T Q
+            ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColOpDS + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+        }
+        ptx::mma_commit(bar_acc);
+      }
+      if (!ok) {
+        record_status(d_status, SPA_ERR_TIMEOUT);
+        *abort_any = 1;
+      }
+    }
+  } else if (!failed_early) {
+    // ---------------------------------------------------------------- arithmetic: two threads per row
+    if (kDQ && row < Np) {
+      // D_i = dO_i . O_i from the two staged tiles (their load has completed: prep(0) waited for it).  Both
+      // carry the same swizzle, so equal positions hold equal columns and the order of the chunks is free:
+      // each row starts at a different chunk to keep 8 neighbouring rows off one bank.
+      constexpr int kChunks = HT::kRowBytes / 16;
+      const uint8_t* po = smem_al + 2 * kTile + rl * HT::kRowBytes;
+      const uint8_t* pg = smem_al + kTile + rl * HT::kRowBytes;
+      const int rot = chunk_rot<D>(rl);
+#pragma unroll
+      for (int c = 0; c < kChunks; ++c) {
+        float a[8], b[8];
+        Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(po + ((c ^ rot) << 4)), a);
+        Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(pg + ((c ^ rot) << 4)), b);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
+      }
+      if (half == 0) delta[(long long)h * capacity + row] = my_D;
+    }
+
+    constexpr int kPc = kBwdY / 2;  // fp32 columns of each tile owned by this thread
+    const int col0 = half * kPc;
+    // no barrier joins the arithmetic warps inside the loop, so a warp whose wait gave up may leave it alone: the
+    // others see the flag in their own waits
+    auto fail = [&]() {
+      record_status(d_status, SPA_ERR_TIMEOUT);
+      *abort_any = 1;
+    };
+    for (int t = 0; t < n_tiles; ++t) {
+      const int y0 = o_lo + t * kBwdY;
+      // ---- this thread's columns of both fp32 tiles into registers
+      bool ok = wait_w(bar_s, t & 1);
+      ptx::tc_fence_after_sync();
+      uint32_t rs[kPc], rp[kPc];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0, rs);
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0, rp);
+      ptx::tmem_ld_wait();
+      if (ok && t + 1 < n_tiles) ok = prep(t + 1);
+      // the statistics of tile t were staged by other warps before they announced tile t - 1 (that phase has
+      // completed; it is waited for, before this warp's own arrival for tile t, to order the reads below)
+      if (ok && !kDQ && t > 0) ok = wait_w(bar_sfree, (t - 1) & 1);
+      if (!ok) { fail(); break; }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_sfree);
+
+      // ---- P = 2^(S - lse), dS = P (dP - D).  A thread whose 32 columns lie wholly outside its row's segment
+      // writes zeros without doing the arithmetic; the mask costs something only where a boundary crosses.
+      const int yc0 = y0 + col0;
+      uint32_t pk_p[kPc / 2], pk_ds[kPc / 2];
+      if (yc0 < mine.hi && yc0 + kPc > mine.lo) {
+        if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {
+#pragma unroll
+          for (int j = 0; j < kPc; ++j)
+            if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
+        }
+        const float* sl = stat_lse + (t % 3) * kBwdY + col0;
+        const float* sd = stat_D + (t % 3) * kBwdY + col0;
+#pragma unroll
+        for (int j = 0; j < kPc; j += 2) {
+          float pv[2], dsv[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const float l2 = kDQ ? my_lse : sl[j + u];
+            const float Dv = kDQ ? my_D : sd[j + u];
+            pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + u]), scale_log2e, -l2));
+            dsv[u] = pv[u] * (__uint_as_float(rp[j + u]) - Dv);
+          }
+          __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
+          pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
+          __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
+          pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < kPc / 2; ++j) { pk_p[j] = 0u; pk_ds[j] = 0u; }
+      }
+      // the accumulating products of tile t - 1 must have read the operand columns
+      if (t > 0) {
+        if (!wait_w(bar_acc, (t - 1) & 1)) { fail(); break; }
+        ptx::tc_fence_after_sync();
+      }
+      if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColOpP + (col0 >> 1), pk_p);
+      ptx::tmem_st_32x16(tmem + lane_base + kColOpDS + (col0 >> 1), pk_ds);
+      ptx::tmem_st_wait();
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_opready);
+    }
+    // the last accumulating products complete the outputs
+    const bool gave_up = __shfl_sync(0xffffffffu, *abort_any, 0) != 0;  // one answer per warp
+    if (n_tiles > 0 && !gave_up && !wait_w(bar_acc, (n_tiles - 1) & 1)) fail();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // nobody reports a failure from here on: the branches below are taken by all threads or by none
+  ptx::tc_fence_after_sync();
+  const bool failed = *abort_any != 0;
+
+  if (!failed && n_tiles > 0) {
+    // Each thread drains d/2 columns of its row of the accumulators into the own tiles' shared memory (idle
+    // now: every product has completed), from where whole rows go out as full lines.
+    constexpr int kDh = D / 2;
+    auto stage_acc = [&](uint32_t acc_col, uint8_t* tile, float mul) {
+      uint32_t r[kDh];
+      if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + acc_col + half * kDh, r);
+      else ptx::tmem_ld_32x16(tmem + lane_base + acc_col + half * kDh, r);
+      ptx::tmem_ld_wait();
+      const int rot = chunk_rot<D>(rl);
+#pragma unroll
+      for (int g = 0; g < kDh / 8; ++g) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul;
+        *reinterpret_cast<uint4*>(tile + rl * HT::kRowBytes + (((half * (kDh / 8) + g) ^ rot) << 4)) =
+            Vec16<__nv_bfloat16>::from_float(v);
+      }
+    };
+    const long long ld = 3LL * C;
+    if (kDQ) {
+      if (is_math) stage_acc(kColAcc1, smem_al, scale);
+      __syncthreads();
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
+    } else {
+      if (is_math) {
+        stage_acc(kColAcc1, smem_al, 1.f);             // dV
+        stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
+      }
+      __syncthreads();
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
+    }
+  }
+  if (failed && tid == kBwdMath) {  // let outstanding loads land before shared memory is released
+    for (int t = issued > kBwdStages ? issued - kBwdStages : 0; t < issued; ++t)
+      ptx::mbar_wait(bar_y(t % kBwdStages), (t / kBwdStages) & 1);
+    ptx::mbar_wait(bar_x, 0);
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem, kBwdTmemCols);
+  }
+}
+
+// The dK / dV pass where TMEM has no room for the bf16 operands beside the fp32 tiles (d = 64: S^T, dP^T, dV and dK
+// fill all 256 columns).  P^T and dS^T are written over the first half of the fp32 tiles they were computed from -
+// after a barrier, once every thread holds its fp32 columns in registers - and the next tile's fp32 products are
+// queued behind the accumulating products that read them (MMAs execute in issue order).  Eight warps, no issuing
+// warp: with nothing to run under the arithmetic, thread 0 issues the copies and products between the barriers.
+constexpr int kAliasedThreads = 256;   // two threads per TMEM lane (row): each owns 32 of the 64 streamed columns
+template <int D> __host__ __device__ constexpr int aliased_smem_bytes() {
+  // own tiles, streamed tiles, alignment slack, statistics, barriers, segment offsets
+  return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAliasedThreads)
+attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
+                   const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
+                   const __grid_constant__ CUtensorMap tm_o,
+                   const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
+                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
+  using HT = HeadTile<D>;
+  constexpr bool kDQ = false;  // this kernel is the dK / dV pass only
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
   constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
@@ -475,7 +867,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   pdl_entry();
   const bool staged = n_seg < kSegStage;
   if (staged)
-    for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
+    for (int i = tid; i <= n_seg; i += kAliasedThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
   if (r0 >= Np) return;
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
@@ -545,7 +937,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     if (y0 + kBwdY > Np) {
       const int first = Np - y0;
       constexpr int kChunks = HT::kRowBytes / 16;
-      for (int c = tid; c < (kBwdY - first) * kChunks; c += kBwdThreads) {
+      for (int c = tid; c < (kBwdY - first) * kChunks; c += kAliasedThreads) {
         const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
         *reinterpret_cast<uint4*>(smem_al + y1_off(st) + off) = make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4*>(smem_al + y2_off(st) + off) = make_uint4(0, 0, 0, 0);
@@ -700,13 +1092,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     if (kDQ) {
       stage_acc(kColAcc1, smem_al, scale);
       __syncthreads();
-      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
     } else {
       stage_acc(kColAcc1, smem_al, 1.f);             // dV
       stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
       __syncthreads();
-      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
-      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
     }
   }
   if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
@@ -722,6 +1114,19 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   }
 }
 
+
+// Which kernel runs the dK / dV pass for head dimension D.
+template <int D> struct kv_pass {
+  static constexpr int kThreads = kBwdThreads;
+  static constexpr int kSmem = bwd_smem_bytes<D, false>();
+  static auto kernel() { return attn_bwd_tc_kernel<D, false>; }
+};
+template <> struct kv_pass<64> {
+  static constexpr int kThreads = kAliasedThreads;
+  static constexpr int kSmem = aliased_smem_bytes<64>();
+  static auto kernel() { return attn_bwd_kv_aliased_kernel<64>; }
+};
+
 template <int D>
 int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st) {
@@ -733,12 +1138,12 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
       !make_tmap_bf16_2d(&tm_o, ao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2))
     return SPA_ERR_UNSUPPORTED;
   auto kq = attn_bwd_tc_kernel<D, true>;
-  auto kkv = attn_bwd_tc_kernel<D, false>;
+  auto kkv = kv_pass<D>::kernel();
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, true>());
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, false>());
+      e = cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_pass<D>::kSmem);
     if (e != cudaSuccess) { set_cuda_error(e, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
     attr_set = true;
   }
@@ -748,7 +1153,7 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
   launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D, true>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
              n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
-  launch_pdl(kkv, grid, kBwdThreads, bwd_smem_bytes<D, false>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
+  launch_pdl(kkv, grid, kv_pass<D>::kThreads, kv_pass<D>::kSmem, st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
              n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
   return SPA_OK;
