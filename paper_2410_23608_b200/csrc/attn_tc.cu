@@ -425,9 +425,12 @@ constexpr uint32_t kBwdTmemCols = 256;
 constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;
 constexpr int kBwdStatBytes = 3 * 2 * kBwdY * 4;  // three tiles' worth of lse_i and D_i of the streamed queries
 
+// Streamed tiles in shared memory.  In the dQ pass the first of them is the memory of the O tile, which is only
+// needed for D_i before the loop starts.  A stage is as large as an own tile (two 64-row tiles).
+template <int D, bool kDQ> __host__ __device__ constexpr int bwd_stages() { return D == 32 ? 6 : (kDQ ? 4 : 3); }
 template <int D, bool kDQ> __host__ __device__ constexpr int bwd_smem_bytes() {
-  // own tiles (the dQ pass also holds the O tile), streamed tiles, alignment slack, statistics, barriers, segment offsets
-  return (kDQ ? 3 : 2) * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64;
+  // two own tiles, streamed stages, alignment slack, statistics, barriers, segment offsets
+  return (2 + bwd_stages<D, kDQ>()) * 128 * D * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64;
 }
 
 template <int D, bool kDQ>
@@ -440,7 +443,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
-  constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
+  constexpr int kStages = bwd_stages<D, kDQ>();     // streamed stages; in the dQ pass stage 0 first holds the O tile
+  constexpr int kShift = kDQ ? 1 : 0;               // tile t lives in stage (t + kShift) mod kStages
+  static_assert(2 * kYTile == kTile, "a stage is as large as an own tile");
   constexpr float kLog2e = 1.4426950408889634f;
   // the bf16 operands have TMEM columns of their own, so the next fp32 products need not wait for the accumulating ones
   static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_aliased_kernel");
@@ -457,21 +462,23 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   const uint32_t x1_s = smem_base, x2_s = smem_base + kTile, x3_s = smem_base + 2 * kTile;
-  constexpr int kYBase = kOwn * kTile;
+  constexpr int kYBase = 2 * kTile;
   auto y1_off = [&](int st) { return kYBase + kYTile * (2 * st); };
   auto y2_off = [&](int st) { return kYBase + kYTile * (2 * st + 1); };
-  constexpr int kStatBase = kYBase + kBwdStages * 2 * kYTile;
+  auto stage_of = [&](int t_) { return (t_ + kShift) % kStages; };
+  auto use_of = [&](int t_) { return (uint32_t)(((t_ + kShift) / kStages) & 1); };  // parity of that stage's barrier
+  constexpr int kStatBase = kYBase + kStages * 2 * kYTile;
   float* stat_lse = reinterpret_cast<float*>(smem_al + kStatBase);  // [3][64] lse_i * log2e of the staged query tile
   float* stat_D = stat_lse + 3 * kBwdY;                              // [3][64] D_i
   constexpr int kBarBase = kStatBase + kBwdStatBytes;
   const uint32_t bar_base = smem_base + kBarBase;
-  const uint32_t bar_x = bar_base, bar_s = bar_base + 32, bar_acc = bar_base + 40;
-  const uint32_t bar_sfree = bar_base + 48;    // 8 arrivals: every arithmetic warp holds the fp32 values of tile t
-  const uint32_t bar_opready = bar_base + 56;  // 8 arrivals: every arithmetic warp has written the operands of tile t
-  auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kBarBase + 64);
-  volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + kBarBase + 68);
-  volatile int* range = reinterpret_cast<volatile int*>(smem_al + kBarBase + 72);
+  const uint32_t bar_x = bar_base, bar_s = bar_base + 56, bar_acc = bar_base + 64;
+  const uint32_t bar_sfree = bar_base + 72;    // 8 arrivals: every arithmetic warp holds the fp32 values of tile t
+  const uint32_t bar_opready = bar_base + 80;  // 8 arrivals: every arithmetic warp has written the operands of tile t
+  auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };  // up to six stages
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kBarBase + 88);
+  volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + kBarBase + 92);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + kBarBase + 96);
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kBarBase + 128);  // [kSegStage + 1]
 
   // everything up to the wait touches no global memory, so it runs under the previous kernel's tail.  The thread
@@ -483,7 +490,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     ptx::prefetch_tensormap(&tm_do_y);
     if (kDQ) ptx::prefetch_tensormap(&tm_o);
     ptx::mbar_init(bar_x, 1);
-    for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
+    for (int s3 = 0; s3 < kStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_acc, 1);
     ptx::mbar_init(bar_sfree, kBwdMath / 32);
@@ -499,11 +506,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   if (r0 >= Np) return;
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
   if (tid == kBwdMath) {  // the own tiles depend only on r0: fetch them under the segment search
-    ptx::mbar_expect_tx(bar_x, kOwn * kTile);
+    ptx::mbar_expect_tx(bar_x, 2 * kTile);
     ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
     if (kDQ) {
       ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                  // dO
-      ptx::tma_load_2d(x3_s, &tm_o, bar_x, h * D, r0);                   // O, for D_i = dO_i . O_i
+      ptx::mbar_expect_tx(bar_y(0), kTile);                              // first use of stage 0:
+      ptx::tma_load_2d(x3_s, &tm_o, bar_y(0), h * D, r0);                // O, for D_i = dO_i . O_i
     } else {
       ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
     }
@@ -530,8 +538,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
 
   const int y1_col = (kDQ ? C : 0) + h * D;           // streamed operand inside qkv: K | Q
-  auto load_other = [&](int t_) {  // streamed tile t_ into stage t_ mod kBwdStages
-    const int st = t_ % kBwdStages, y0 = o_lo + t_ * kBwdY;
+  auto load_other = [&](int t_) {  // streamed tile t_ into its stage
+    const int st = stage_of(t_), y0 = o_lo + t_ * kBwdY;
     ptx::mbar_expect_tx(bar_y(st), 2 * kYTile);
     ptx::tma_load_2d(smem_base + y1_off(st), &tm_qkv_y, bar_y(st), y1_col, y0);
     if (kDQ) ptx::tma_load_2d(smem_base + y2_off(st), &tm_qkv_y, bar_y(st), 2 * C + h * D, y0);   // V
@@ -539,8 +547,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   };
   int issued = 0;  // streamed tiles whose loads have been issued (kept by the issuing thread)
   if (tid == kBwdMath) {
-    for (int t_ = 0; t_ < n_tiles && t_ < 2; ++t_) load_other(t_);
-    issued = n_tiles < 2 ? n_tiles : 2;
+    for (int t_ = 0; t_ < n_tiles && t_ < kStages - 1; ++t_) load_other(t_);  // the stages that are free at the start
+    issued = n_tiles < kStages - 1 ? n_tiles : kStages - 1;
   }
 
   // Bounded wait that also gives up as soon as any thread of the CTA has reported a failure.
@@ -574,9 +582,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   // valid packed row are zeroed (they are unspecified memory and would be summed over), its query statistics
   // are staged.  Returns false when the wait for the load gave up.
   auto prep = [&](int t_) {
-    const int st = t_ % kBwdStages;
-    bool ok = wait_w(bar_y(st), (t_ / kBwdStages) & 1);
-    if (t_ == 0) ok = wait_w(bar_x, 0) && ok;
+    const int st = stage_of(t_);
+    bool ok = wait_w(bar_y(st), use_of(t_));
+    if (t_ == 0) {
+      ok = wait_w(bar_x, 0) && ok;
+      if (kDQ) ok = wait_w(bar_y(0), 0) && ok;  // the O tile
+    }
     const int y0 = o_lo + t_ * kBwdY;
     if (y0 + kBwdY > Np) {
       const int first = Np - y0;
@@ -607,7 +618,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     // ---------------------------------------------------------------- copies and products: one thread
     if (lane == 0 && !failed_early) {
       auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
-        const int st = t_ % kBwdStages;
+        const int st = stage_of(t_);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
           ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(smem_base + y1_off(st), k), kIdescS, k != 0 ? 1u : 0u);
@@ -620,18 +631,20 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       ptx::tc_fence_after_sync();
       if (n_tiles > 0) issue_s(0);
       for (int t = 0; ok && t < n_tiles; ++t) {
-        const int st = t % kBwdStages;
+        const int st = stage_of(t);
         if (t + 1 < n_tiles) {
           // the fp32 values of tile t are in registers and tile t + 1 is ready: its products run under the arithmetic
           if (!(ok = wait(bar_sfree, t & 1))) break;
           ptx::tc_fence_after_sync();
           issue_s(t + 1);
         }
-        // the stage of tile t - 1 is free once its accumulating products have completed
-        if (t + 2 < n_tiles) {
+        // the stage of tile t - 1 is free once its accumulating products have completed; at t = 0 the stage that
+        // is filled is the last one, or in the dQ pass the O tile's memory, which the arithmetic warps have finished
+        // with before they announce tile 0 (waited for above: a tile to prefetch implies a tile t + 1)
+        if (t + kStages - 1 < n_tiles) {
           if (t > 0 && !(ok = wait(bar_acc, (t - 1) & 1))) break;
-          load_other(t + 2);
-          issued = t + 3;
+          load_other(t + kStages - 1);
+          issued = t + kStages;
         }
         if (!(ok = wait(bar_opready, t & 1))) break;
         ptx::tc_fence_after_sync();
@@ -790,8 +803,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     }
   }
   if (failed && tid == kBwdMath) {  // let outstanding loads land before shared memory is released
-    for (int t = issued > kBwdStages ? issued - kBwdStages : 0; t < issued; ++t)
-      ptx::mbar_wait(bar_y(t % kBwdStages), (t / kBwdStages) & 1);
+    for (int t = issued > kStages ? issued - kStages : 0; t < issued; ++t) ptx::mbar_wait(bar_y(stage_of(t)), use_of(t));
+    if (kDQ && issued < kStages) ptx::mbar_wait(bar_y(0), 0);  // the O tile, if no streamed tile followed it there
     ptx::mbar_wait(bar_x, 0);
   }
   ptx::tc_fence_before_sync();
