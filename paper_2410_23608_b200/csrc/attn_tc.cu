@@ -583,12 +583,16 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   // are staged.  Returns false when the wait for the load gave up.
   auto prep = [&](int t_) {
     const int st = stage_of(t_);
-    bool ok = wait_w(bar_y(st), use_of(t_));
+    bool ok = true;
+    const int y0 = o_lo + t_ * kBwdY;
+    // the issuing thread waits for the load itself; the arithmetic warps need it only where they touch the tile
     if (t_ == 0) {
+      ok = wait_w(bar_y(st), use_of(t_));
       ok = wait_w(bar_x, 0) && ok;
       if (kDQ) ok = wait_w(bar_y(0), 0) && ok;  // the O tile
+    } else if (y0 + kBwdY > Np) {
+      ok = wait_w(bar_y(st), use_of(t_));
     }
-    const int y0 = o_lo + t_ * kBwdY;
     if (y0 + kBwdY > Np) {
       const int first = Np - y0;
       constexpr int kChunks = HT::kRowBytes / 16;
@@ -635,6 +639,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
         if (t + 1 < n_tiles) {
           // the fp32 values of tile t are in registers and tile t + 1 is ready: its products run under the arithmetic
           if (!(ok = wait(bar_sfree, t & 1))) break;
+          if (!(ok = wait(bar_y(stage_of(t + 1)), use_of(t + 1)))) break;
           ptx::tc_fence_after_sync();
           issue_s(t + 1);
         }
@@ -747,7 +752,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
 #pragma unroll
         for (int j = 0; j < kPc / 2; ++j) { pk_p[j] = 0u; pk_ds[j] = 0u; }
       }
-      // the accumulating products of tile t - 1 must have read the operand columns
+      // The accumulating products of tile t - 1 must have read the operand columns.  (Two operand copies in the dQ
+      // pass, written without this wait on the grounds that the fp32 products of tile t were committed after the
+      // accumulating products of tile t - 2, gave sporadic non-finite dQ at d = 32: the wait stays.)
       if (t > 0) {
         if (!wait_w(bar_acc, (t - 1) & 1)) { fail(); break; }
         ptx::tc_fence_after_sync();
