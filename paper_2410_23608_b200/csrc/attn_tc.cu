@@ -420,7 +420,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 constexpr int kBwdMath = 256;      // arithmetic threads: two per TMEM lane (row)
 constexpr int kBwdThreads = kBwdMath + 32;
 constexpr int kBwdY = 64;          // rows of a streamed tile
-constexpr int kBwdStages = 3;      // streamed tiles in shared memory
+constexpr int kBwdStages = 4;      // streamed tiles in shared memory of the aliased dK / dV kernel
 constexpr uint32_t kBwdTmemCols = 256;
 constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;
 constexpr int kBwdStatBytes = 3 * 2 * kBwdY * 4;  // three tiles' worth of lse_i and D_i of the streamed queries
@@ -929,8 +929,8 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   };
   int issued = 0;  // streamed tiles whose loads thread 0 has issued
   if (tid == 0) {
-    for (int t_ = 0; t_ < n_tiles && t_ < 2; ++t_) load_other(t_);
-    issued = n_tiles < 2 ? n_tiles : 2;
+    for (int t_ = 0; t_ < n_tiles && t_ < kBwdStages - 1; ++t_) load_other(t_);
+    issued = n_tiles < kBwdStages - 1 ? n_tiles : kBwdStages - 1;
   }
   // per-row statistics of the query side
   float my_lse = 0.f, my_D = 0.f;   // kDQ: this thread's query row
@@ -1016,7 +1016,7 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
     // products of tile t-1 (commits are in issue order), so its streamed stage is free again.
     if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
     ptx::tc_fence_after_sync();
-    if (tid == 0 && t + 2 < n_tiles) { load_other(t + 2); issued = t + 3; }
+    if (tid == 0 && t + kBwdStages - 1 < n_tiles) { load_other(t + kBwdStages - 1); issued = t + kBwdStages; }  // stage of tile t - 1
     uint32_t rs[kPc], rp[kPc];
     ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0, rs);
     ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0, rp);
