@@ -37,6 +37,8 @@ int check_params(const spa_params* p) {
   if (p->C % p->H != 0) return SPA_ERR_INVALID_ARG;
   const int es = p->dtype == SPA_F32 ? 4 : 2;
   if ((p->C * es) % 16 != 0 || p->C > 8192) return SPA_ERR_UNSUPPORTED;
+  // the kernels take row maxima before scaling, which needs a scale that is positive (0 selects 1/sqrt(d))
+  if (!(p->softmax_scale >= 0.f) || !(p->softmax_scale <= 3.0e38f)) return SPA_ERR_INVALID_ARG;
   return SPA_OK;
 }
 
@@ -168,6 +170,25 @@ int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* a
   }
   return launch_attention_bwd_simt(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv,
                                    (cudaStream_t)stream);
+}
+
+int spa_packed_attention_bwd_static(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
+                                    const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg, void* dqkv,
+                                    int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  rc = check_heads(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(qkv); SPA_PTR(attn_out); SPA_PTR(lse); SPA_PTR(d_attn_out); SPA_PTR(seg_offsets); SPA_PTR(dqkv);
+  SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
+  if (!use_tc(p) || !tc_attention_bwd_supported(*p)) return SPA_ERR_UNSUPPORTED;
+  if ((unsigned long long)p->H * (unsigned long long)p->capacity * sizeof(float) > SPA_STATIC_SCRATCH_BYTES)
+    return SPA_ERR_SCRATCH;
+  void* scratch = nullptr;  // the array inside the library image: nothing is allocated here
+  rc = static_attention_scratch(&scratch);
+  if (rc != SPA_OK) return rc;
+  return launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, scratch, d_status,
+                                 (cudaStream_t)stream);
 }
 
 int spa_unpack_scatter(const spa_params* p, const void* z_packed, const void* x, const int32_t* idx,

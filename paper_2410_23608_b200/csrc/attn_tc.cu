@@ -1159,14 +1159,12 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
     return SPA_ERR_UNSUPPORTED;
   auto kq = attn_bwd_tc_kernel<D, true>;
   auto kkv = kv_pass<D>::kernel();
-  static bool attr_set = false;
-  if (!attr_set) {
+  static DeviceOnce attr;
+  cudaError_t ea = attr.run([&] {
     cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, true>());
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_pass<D>::kSmem);
-    if (e != cudaSuccess) { set_cuda_error(e, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
-    attr_set = true;
-  }
+    return e != cudaSuccess ? e : cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_pass<D>::kSmem);
+  });
+  if (ea != cudaSuccess) { set_cuda_error(ea, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
   dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
@@ -1185,12 +1183,9 @@ int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_s
   CUtensorMap tm;
   if (!make_tmap_bf16_2d(&tm, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2)) return SPA_ERR_UNSUPPORTED;
   auto kern = attn_fwd_tc_kernel<D>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem_bytes<D>());
-    if (e != cudaSuccess) { set_cuda_error(e, "attn_fwd_tc_kernel"); return SPA_ERR_CUDA; }
-    attr_set = true;
-  }
+  static DeviceOnce attr;
+  cudaError_t ea = attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem_bytes<D>()); });
+  if (ea != cudaSuccess) { set_cuda_error(ea, "attn_fwd_tc_kernel"); return SPA_ERR_CUDA; }
   dim3 grid(p.H, (p.capacity + kQ - 1) / kQ);
   launch_pdl(kern, grid, kFwdThreads, fwd_smem_bytes<D>(), st, tm, seg, n_seg, p.capacity, p.C,
                                                       softmax_scale_of(p) * 1.4426950408889634f,
@@ -1229,30 +1224,32 @@ int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t*
 }  // namespace spa
 
 // ------------------------------------------------------------------------------------------------
-// Attention backward without caller scratch.  The D_i values (one float per head and packed row)
-// that the dQ pass hands to the dK/dV pass live in this array, which is part of the library image:
-// a caller that may not allocate device memory still gets the tensor-core backward.  Host code must
-// not pass the symbol itself to a kernel - on the host it only stands for the array - so the device
-// address is looked up once per device and cached.
+// Scratch of spa_packed_attention_bwd_static, the attention backward for callers that cannot allocate.
+// The D_i values (one float per head and packed row) that the dQ pass hands to the dK/dV pass live in
+// this array, which is part of the library image.  Host code must not pass the symbol itself to a
+// kernel - on the host it only stands for the array - so the device address is looked up once per
+// device, with that device current, and cached.
 static __device__ __align__(256) unsigned char g_static_scratch[SPA_STATIC_SCRATCH_BYTES];
 
+namespace spa {
 namespace {
 constexpr int kMaxDevices = 64;
 std::mutex g_scratch_mutex;
 void* g_scratch_ptr[kMaxDevices] = {};
+}  // namespace
 
 // Device address of g_static_scratch on the current device (looked up on first use).
-int static_scratch_address(void** out) {
+int static_attention_scratch(void** out) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) { spa::set_cuda_error(e, "spa_packed_attention_bwd_static: cudaGetDevice"); return SPA_ERR_CUDA; }
+  if (e != cudaSuccess) { set_cuda_error(e, "spa_packed_attention_bwd_static: cudaGetDevice"); return SPA_ERR_CUDA; }
   if (dev < 0 || dev >= kMaxDevices) return SPA_ERR_UNSUPPORTED;
   std::lock_guard<std::mutex> lock(g_scratch_mutex);
   if (g_scratch_ptr[dev] == nullptr) {
     void* ptr = nullptr;
     e = cudaGetSymbolAddress(&ptr, g_static_scratch);
     if (e != cudaSuccess || ptr == nullptr) {
-      spa::set_cuda_error(e, "spa_packed_attention_bwd_static: cudaGetSymbolAddress");
+      set_cuda_error(e, "spa_packed_attention_bwd_static: cudaGetSymbolAddress");
       return SPA_ERR_CUDA;
     }
     g_scratch_ptr[dev] = ptr;
@@ -1260,25 +1257,5 @@ int static_scratch_address(void** out) {
   *out = g_scratch_ptr[dev];
   return SPA_OK;
 }
-}  // namespace
 
-extern "C" int spa_packed_attention_bwd_static(const spa_params* p, const void* qkv, const void* attn_out,
-                                               const float* lse, const void* d_attn_out, const int32_t* seg_offsets,
-                                               int32_t n_seg, void* dqkv, int32_t* d_status, void* stream) {
-  auto misaligned = [](const void* q) { return q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
-  if (p == nullptr || p->B < 0 || p->N <= 0 || p->C <= 0 || p->H <= 0 || p->C % p->H != 0 || n_seg < 0 ||
-      p->capacity < 1 || (long long)p->capacity > (long long)(p->B > 0 ? p->B : 1) * p->N)
-    return SPA_ERR_INVALID_ARG;
-  if (misaligned(qkv) || misaligned(attn_out) || misaligned(lse) || misaligned(d_attn_out) ||
-      misaligned(seg_offsets) || misaligned(dqkv))
-    return SPA_ERR_INVALID_ARG;
-  if ((long long)p->B * p->N > (1LL << 20) || (p->flags & SPA_FLAG_SIMT_ONLY) || !spa::tc_attention_bwd_supported(*p))
-    return SPA_ERR_UNSUPPORTED;
-  if ((unsigned long long)p->H * (unsigned long long)p->capacity * sizeof(float) > SPA_STATIC_SCRATCH_BYTES)
-    return SPA_ERR_SCRATCH;
-  void* scratch = nullptr;
-  const int rc = static_scratch_address(&scratch);
-  if (rc != SPA_OK) return rc;
-  return spa::launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, scratch, d_status,
-                                      (cudaStream_t)stream);
-}
+}  // namespace spa

@@ -207,8 +207,8 @@ int launch_layer_norm_bwd(const spa_params& p, const void* dy, const void* x, co
 #define SPA_LN_BWD(T, CH)                                                                                             \
   do {                                                                                                                \
     auto kern = layer_norm_bwd_kernel<T, CH>;                                                                         \
-    static bool attr_set = false;                                                                                     \
-    if (!attr_set) { e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); attr_set = e == cudaSuccess; } \
+    static DeviceOnce attr;                                                                                           \
+    e = attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); }); \
     if (e == cudaSuccess)                                                                                             \
       launch_pdl(kern, grid, kRestThreads, smem, st, (const uint4*)dy, (const uint4*)x, (const T*)gamma, mean, rstd, \
                  (const uint4*)add, rows, p.C, (uint4*)dx, part);                                                     \

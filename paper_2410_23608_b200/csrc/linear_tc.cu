@@ -462,12 +462,9 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
                 int k_per_split, int splits, float* colsum_part, const int32_t* row_map, int accumulate,
                 int32_t* d_status, cudaStream_t st, const char* what) {
   auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT, kColSum>;
-  static bool attr_set = false;  // per instantiation
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes<BN>());
-    if (e != cudaSuccess) { set_cuda_error(e, what); return SPA_ERR_CUDA; }
-    attr_set = true;
-  }
+  static DeviceOnce attr;  // per instantiation and device
+  cudaError_t ea = attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes<BN>()); });
+  if (ea != cudaSuccess) { set_cuda_error(ea, what); return SPA_ERR_CUDA; }
   // persistent grid: two CTAs per SM (99 KB of shared memory and 256 TMEM columns each), never more
   // CTAs than there are tiles when every allocated row is in use
   long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * splits;

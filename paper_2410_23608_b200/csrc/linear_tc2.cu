@@ -297,12 +297,9 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
                 int N, int K, const int32_t* cu, int n_seg, int capacity, const int32_t* row_map, int accumulate,
                 int32_t* d_status, cudaStream_t st, const char* what) {
   auto kern = gemm_pair_kernel<kBMn>;
-  static bool attr_set = false;  // per instantiation
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem);
-    if (e != cudaSuccess) { set_cuda_error(e, what); return SPA_ERR_CUDA; }
-    attr_set = true;
-  }
+  static DeviceOnce smem_attr;  // per instantiation and device
+  cudaError_t ea = smem_attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem); });
+  if (ea != cudaSuccess) { set_cuda_error(ea, what); return SPA_ERR_CUDA; }
   const long long tiles = (long long)((N + PN - 1) / PN) * ((capacity + 2 * PM - 1) / (2 * PM));
   const int pairs = (int)(tiles < kMaxPairs ? (tiles < 1 ? 1 : tiles) : kMaxPairs);
   cudaLaunchConfig_t cfg = {};

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "spa.h"
 
 namespace spa {
@@ -115,6 +117,25 @@ void count_launch();  // one more kernel of this library was enqueued (host-side
     if (e__ != cudaSuccess) { ::spa::set_cuda_error(e__, where); return SPA_ERR_CUDA; } \
     ::spa::count_launch();                                             \
   } while (0)
+
+// Set-up that a kernel needs once on every device that runs it (the opt-in to more than 48 KB of dynamic shared
+// memory is a per-device attribute of the function).  run(fn) calls fn with the current device the first time that
+// device is seen and never again once fn has returned cudaSuccess; safe to call from several host threads.
+class DeviceOnce {
+ public:
+  template <typename F> cudaError_t run(F&& fn) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (done_.load(std::memory_order_acquire) & bit) return cudaSuccess;
+    e = fn();
+    if (e == cudaSuccess) done_.fetch_or(bit, std::memory_order_release);
+    return e;
+  }
+ private:
+  std::atomic<unsigned long long> done_{0};
+};
 
 bool pdl_enabled();  // programmatic dependent launch is on unless the environment sets SPA_PDL=0
 

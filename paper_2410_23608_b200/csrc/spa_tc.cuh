@@ -32,5 +32,7 @@ bool tc_attention_bwd_supported(const spa_params& p);
 int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                             const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
                             cudaStream_t st);
+// Device address, on the current device, of the SPA_STATIC_SCRATCH_BYTES array built into the library.
+int static_attention_scratch(void** out);
 
 }  // namespace spa

@@ -193,6 +193,50 @@ def test_invalid_arguments_are_rejected_on_the_host():
     with pytest.raises(lib.SpaError) as e:
         lib.spa_gate(lib.make_params(2, 16, 64, 2, "f32", capacity=33), x, w, 0.0, None, sc, mk)  # capacity > B*N
     assert e.value.status == lib.SPA_ERR_INVALID_ARG
+    for bad_scale in (-0.125, float("nan"), float("inf")):     # the kernels need a positive, finite softmax scale
+        with pytest.raises(lib.SpaError) as e:
+            lib.spa_gate(lib.make_params(2, 16, 64, 2, "f32", softmax_scale=bad_scale), x, w, 0.0, None, sc, mk)
+        assert e.value.status == lib.SPA_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("C,H", [(128, 2), (128, 4)])   # head dimension 64 and 32
+def test_attention_with_more_segments_than_the_kernels_stage(C, H):
+    """600 segments of 1-40 rows: above 512 segments the attention kernels search the offsets in global memory
+    instead of their shared-memory copy.  Forward and backward against the oracle fed the same rounded bits."""
+    lib = L()
+    dt = "bf16"
+    rng = np.random.default_rng(77 + H)
+    counts = rng.integers(1, 41, size=600)
+    counts[[0, 17, 599]] = 1
+    counts[300] = 40
+    cu_np = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    n_seg, Np = len(counts), int(cu_np[-1])
+    B, N = 24, 1024                     # capacity B*N >= Np; the segments are not images here
+    assert Np <= B * N
+    blk = block(B, N, C, H, dt)
+    p, cap = blk.p, blk.cap
+
+    def padded(a, cols):
+        buf = np.zeros((cap, cols))
+        buf[:Np] = a
+        return buf
+
+    qkv_r = round_to(rng.normal(size=(Np, 3 * C)), dt)
+    ao_ref, lse_ref = O.attention_fwd(qkv_r, cu_np, H)
+    seg = torch.from_numpy(cu_np).cuda()
+    qkv = dev(padded(qkv_r, 3 * C), dt)
+    lib.spa_packed_attention_fwd(p, qkv, seg, n_seg, blk.ao, blk.lse, blk.status)
+    assert_close(host(blk.ao)[:Np], ao_ref, dt, "attn_out")
+    assert np.abs(host(blk.lse)[:, :Np] - lse_ref).max() <= TOL[dt]["lse"]
+    ao_r = round_to(ao_ref, dt)
+    dao_r = round_to(rng.normal(size=(Np, C)), dt)
+    lse_t = torch.zeros(H, cap, dtype=torch.float32, device="cuda")
+    lse_t[:, :Np] = torch.from_numpy(lse_ref).float().cuda()
+    ref = O.attention_bwd(qkv_r, ao_r, lse_t[:, :Np].double().cpu().numpy(), dao_r, cu_np, H)
+    lib.spa_packed_attention_bwd(p, qkv, dev(padded(ao_r, C), dt), lse_t, dev(padded(dao_r, C), dt), seg, n_seg,
+                                 blk.dqkv, blk.workspace, blk.status)
+    assert_close(host(blk.dqkv)[:Np], ref, dt, "dqkv", scale_max_abs=True)
+    assert blk.read_status() == 0
 
 
 @pytest.mark.parametrize("ci,fused", [(1, False), (2, False), (2, True)])

@@ -37,7 +37,9 @@ def layer_problem(ci, B):
     return cfg, inp, x, prm, f
 
 
-@pytest.mark.parametrize("ci,B", [(1, 3), (2, 4)])
+# C = 96, 384, 256 and 768: every row-width instantiation of the LayerNorm backward; (4, 8) has 4 608 tokens, so its
+# 768 -> 3072 -> 768 feed-forward products and their input gradients run on CTA pairs
+@pytest.mark.parametrize("ci,B", [(1, 3), (2, 4), (3, 1), (4, 8)])
 def test_layer_forward_backward(ci, B):
     from paper_2410_23608_b200.layer import SpaLayer
     cfg, inp, x, prm, f = layer_problem(ci, B)
@@ -67,11 +69,12 @@ def test_layer_forward_backward(ci, B):
         assert_close(host(getattr(lay.blk, name)), bwd[name], dt, name, scale_max_abs=True)
 
 
-def test_layer_norm_and_gelu_calls_alone():
+@pytest.mark.parametrize("ci", [2, 3, 4])   # C = 384, 256, 768
+def test_layer_norm_and_gelu_calls_alone(ci):
     """Each new call on its own inputs: LayerNorm forward / backward (with and without the added branch), GELU."""
     from paper_2410_23608_b200 import binding as L
     from paper_2410_23608_b200.block import SpaBlock
-    cfg = scaled_config(get_config(2), B=2)
+    cfg = scaled_config(get_config(ci), B=2 if ci != 3 else 1)
     dt = cfg.dtype
     rng = np.random.default_rng(9)
     B, N, C = cfg.B, cfg.N, cfg.C

@@ -21,8 +21,9 @@ def test_score_pool_exact():
     assert np.array_equal(out.cpu().numpy(), O.score_pool(prev, B, rows, cols).astype(np.float32))
 
 
-def _problem(ci, residual):
-    cfg = get_config(ci)
+def _problem(ci, residual, B=None):
+    from spa_workloads import scaled_config
+    cfg = get_config(ci) if B is None else scaled_config(get_config(ci), B=B)
     inp = make_inputs(cfg)
     rng = np.random.default_rng(100 + ci)
     s_lin = O.gate(inp.x, inp.w_g, inp.b_g)
@@ -38,11 +39,14 @@ def _problem(ci, residual):
     return cfg, inp, s_up, labels, fwd
 
 
-@pytest.mark.parametrize("ci,residual", [(1, False), (2, False), (2, True)])
-def test_trainable_block_against_oracle(ci, residual):
+# configs 3-5 (C = 256 and 768: the widest rows of the gate backward and of the gated pack transpose) on a slice
+# of their batch
+@pytest.mark.parametrize("ci,residual,B", [(1, False, None), (2, False, None), (2, True, None), (3, False, 2),
+                                            (4, True, 4), (5, False, 12)])
+def test_trainable_block_against_oracle(ci, residual, B):
     from paper_2410_23608_b200 import binding as L
     from paper_2410_23608_b200.block import SpaBlock
-    cfg, inp, s_up, labels, fwd = _problem(ci, residual)
+    cfg, inp, s_up, labels, fwd = _problem(ci, residual, B)
     alpha = 0.25
     bwd = O.block_bwd_trainable(fwd, inp.dY, inp.x, inp.w_g, inp.W_qkv, inp.W_o, cfg.H, labels=labels, alpha=alpha,
                                 s_up=s_up, residual=residual, gate_scale=True)

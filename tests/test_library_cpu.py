@@ -55,6 +55,14 @@ def test_params_struct_layout_matches_header(lib):
     assert ctypes.sizeof(lib.SpaParams) == 36
 
 
+def test_binding_constants_match_header(lib):
+    text = open(os.path.join(ROOT, "include", "spa.h")).read()
+    m = re.search(r"#define\s+SPA_STATIC_SCRATCH_BYTES\s+\((\d+)u\s*<<\s*(\d+)\)", text)
+    assert m and lib.SPA_STATIC_SCRATCH_BYTES == int(m.group(1)) << int(m.group(2))
+    for name, val in re.findall(r"\b(SPA_(?:ERR_[A-Z_]+|OK|FLAG_[A-Z_]+|F32|BF16))\s*=\s*(-?\d+)", text):
+        assert getattr(lib, name) == int(val), name
+
+
 def test_later_entry_points_validate_on_the_host(lib):
     """Fused, trainable-selection, ordered-packing and block calls: bad arguments come back as a status before
     anything touches a device."""

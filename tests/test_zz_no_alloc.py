@@ -6,7 +6,8 @@ that is being recorded for replay, inside a runtime whose memory pool is frozen 
 someone else, or they are handed only their inputs and outputs.  For them the library carries its
 scratch inside its own image.  This test calls that entry point through the C boundary twice in a
 row, on different data, and checks each result against the regular entry point (which takes caller
-scratch) within the tolerance of the other parity tests; it also checks that a problem larger than
+scratch): both run the same deterministic kernels, so the results must agree bit for bit, which is
+inside every tolerance the other parity tests use.  It also checks that a problem larger than
 the built-in array is refused with its own status.  It is collected last so that a failure here
 cannot hide the result of any other test.
 """
@@ -50,6 +51,7 @@ def test_static_scratch_entry_matches_regular_entry_twice(C, H):
         assert L.spa_read_status(status) == 0
         assert np.abs(host(ref)[:Np]).max() > 0
         assert_close(host(got)[:Np], host(ref)[:Np], "bf16", "dqkv (static scratch)", scale_max_abs=True)
+        assert torch.equal(got[:Np], ref[:Np])
 
 
 def test_static_scratch_entry_refuses_what_does_not_fit():
