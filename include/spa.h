@@ -54,7 +54,9 @@ enum {
   SPA_FLAG_INPLACE = 2,   /* spa_unpack_scatter: y aliases x, only selected rows written   */
   SPA_FLAG_GATE_SCALE = 4,/* Eq. 5: packed rows are scaled by sigmoid(score)               */
   SPA_FLAG_SIMT_ONLY = 8, /* bf16 only: run the fp32-FMA kernels instead of the tensor-core ones */
-  SPA_FLAG_NO_CTA_PAIRS = 16 /* wide linear layers: keep the one-CTA tensor-core kernels (no CTA pairs) */
+  SPA_FLAG_NO_CTA_PAIRS = 16,/* wide linear layers: keep the one-CTA tensor-core kernels (no CTA pairs) */
+  SPA_FLAG_UNFUSED = 32   /* spa_block_fwd / spa_block_bwd: separate projection, scatter and gather kernels even
+                             where the fused calls apply                                                      */
 };
 
 typedef struct spa_params {
@@ -288,6 +290,98 @@ int spa_layer_norm_bwd(const spa_params* p, const void* dy, const void* x, const
 /* h = gelu(u) = u Phi(u) and du = dh * gelu'(u) over T[B*N][n_cols]; du may alias dh. */
 int spa_gelu(const spa_params* p, const void* u, int32_t n_cols, void* h, void* stream);
 int spa_gelu_bwd(const spa_params* p, const void* dh, const void* u, int32_t n_cols, void* du, void* stream);
+
+/* ---- The block as one unit (Sec. 3.2: gate -> select and pack -> attention on the packed tokens -> unpack; Eq. 9
+ * counts it as one).  spa_block_fwd and spa_block_bwd issue the calls above in order on `stream`; they choose the
+ * fused calls where spa_fused_scatter_supported() allows (unless SPA_FLAG_UNFUSED), and spa_block_bwd runs the two
+ * weight-gradient products on a second stream beside the attention backward when `overlap` is given.  Nothing
+ * synchronises with the host, so both can be recorded into one CUDA graph.
+ *
+ * All pointers are device memory owned by the caller and sized as in the single calls (packed buffers: `capacity`
+ * rows).  Which fields may be NULL:
+ *   s_up, order, seg_offsets (NULL: the images are the attention segments), b_qkv, b_o;
+ *   z, dx_packed            when the fused calls apply (the products write y and dX rows themselves);
+ *   every backward field    for spa_block_fwd;
+ *   labels .. train_workspace unless `trainable` is non-zero.
+ * The forward pass leaves scores, mask, cu_seqlens, idx, inv, x_packed, qkv, attn_out, lse for the backward pass. */
+typedef struct spa_overlap spa_overlap;  /* a second stream and the two events that fork to it and join it */
+
+typedef struct spa_block_buffers {
+  /* inputs of the forward pass */
+  const void* x;              /* T[B][N][C]                                                          */
+  const void* w_g;            /* T[C]                                                                */
+  float b_g;
+  const float* s_up;          /* float[B*N] or NULL (Eq. 4)                                          */
+  const void* W_qkv;          /* T[3C][C]                                                            */
+  const void* b_qkv;          /* T[3C] or NULL                                                       */
+  const void* W_o;            /* T[C][C]                                                             */
+  const void* b_o;            /* T[C] or NULL                                                        */
+  const int32_t* order;       /* int32[N] packing order of each image's tokens, or NULL (raster)     */
+  const int32_t* seg_offsets; /* int32[n_seg+1] attention segments, or NULL (cu_seqlens, B)          */
+  int32_t n_seg;
+  /* results and intermediates of the forward pass */
+  float* scores;              /* float[B*N]                                                          */
+  uint8_t* mask;              /* uint8[B*N]                                                          */
+  int32_t* cu_seqlens;        /* int32[B+1]                                                          */
+  int32_t* idx;               /* int32[capacity]                                                     */
+  int32_t* inv;               /* int32[B*N]                                                          */
+  void* x_packed;             /* T[capacity][C]                                                      */
+  void* qkv;                  /* T[capacity][3C]                                                     */
+  void* attn_out;             /* T[capacity][C]                                                      */
+  float* lse;                 /* float[H][capacity]                                                  */
+  void* z;                    /* T[capacity][C]; unfused path only                                   */
+  void* y;                    /* T[B][N][C]; equal to x under SPA_FLAG_INPLACE                       */
+  /* backward pass */
+  const void* dY;             /* T[B][N][C]                                                          */
+  void* dz;                   /* T[capacity][C]                                                      */
+  void* d_attn_out;           /* T[capacity][C]                                                      */
+  void* dqkv;                 /* T[capacity][3C]                                                     */
+  void* dx_packed;            /* T[capacity][C]; unfused path only                                   */
+  void* dX;                   /* T[B][N][C]                                                          */
+  float* dW_qkv;              /* float[3C][C]                                                        */
+  float* db_qkv;              /* float[3C]                                                           */
+  float* dW_o;                /* float[C][C]                                                         */
+  float* db_o;                /* float[C]                                                            */
+  void* workspace;            /* spa_workspace_bytes()                                               */
+  void* workspace_side;       /* a second area of that size; needed when `overlap` is given          */
+  spa_overlap* overlap;       /* spa_overlap_create(), or NULL: everything on `stream`               */
+  int32_t* d_status;          /* device status word or NULL                                          */
+  /* trainable selection (Eq. 4-5, Eq. 10): gradient to the gate */
+  int32_t trainable;          /* non-zero: spa_block_bwd also runs the four calls of that section    */
+  const uint8_t* labels;      /* uint8[B*N] or NULL (no selection loss)                              */
+  float alpha;                /* weight of the selection loss                                        */
+  float* ds;                  /* float[B*N]                                                          */
+  float* ds_up;               /* float[B*N] or NULL                                                  */
+  float* dw_g;                /* float[C]                                                            */
+  float* db_g;                /* float[1] or NULL                                                    */
+  float* loss;                /* float[1] or NULL                                                    */
+  void* train_workspace;      /* spa_train_workspace_bytes()                                         */
+} spa_block_buffers;
+
+/* A non-blocking stream and two events on the current device (host-side objects, no device memory).  Create one
+ * per block that runs concurrently; destroy it when no work that uses it is in flight. */
+int spa_overlap_create(spa_overlap** out);
+int spa_overlap_destroy(spa_overlap* ov);
+
+/* Forward pass of one block: y = x on unselected tokens, the projected attention output (plus x under
+ * SPA_FLAG_RESIDUAL) on selected ones. */
+int spa_block_fwd(const spa_params* p, const spa_block_buffers* b, void* stream);
+
+/* Backward pass for the last spa_block_fwd on the same buffers: dX, dW_qkv, db_qkv, dW_o, db_o (and, when
+ * `trainable`, ds, ds_up, dw_g, db_g, loss).  When it returns, every piece of work it enqueued, on either stream,
+ * is ordered before whatever is enqueued on `stream` next. */
+int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream);
+
+/* ---- Diagnostics (the paper has no counterpart) ----------------------------------------------------------------
+ * spa_probe_exp2: n_ctas CTAs of 512 threads evaluate base-2 exponentials with the instruction the softmax kernels
+ * use, 8 * iters per thread; *n_exp (host, may be NULL) receives the total count.  Timed by the caller, it gives the
+ * exponential throughput that bounds attention at head dimension 32 (Eq. 9's 2L^2C term costs one exponential per
+ * 4d flops).  sink: float[n_ctas], never written in practice.
+ * spa_probe_wait_expiry: one warp waits on a barrier that nobody arrives at and gives up after `limit` polls
+ * (<= 2^20): d_status receives SPA_ERR_TIMEOUT and *polls_done (device int32, may be NULL) the polls made.  Shows,
+ * without any fault or hang, what every bounded wait of the kernels does when it runs out. */
+int spa_probe_exp2(int32_t n_ctas, int32_t iters, float* sink, unsigned long long* n_exp, void* stream);
+int spa_probe_wait_expiry(int32_t limit, int32_t* d_status, int32_t* polls_done, void* stream);
 
 /* Blocking read of the device status word: synchronises `stream` and returns its value. */
 int spa_read_status(const int32_t* d_status, void* stream);

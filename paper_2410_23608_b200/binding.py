@@ -21,6 +21,7 @@ SPA_ERR_SCRATCH = -6
 SPA_STATIC_SCRATCH_BYTES = 4 << 20
 SPA_F32, SPA_BF16 = 0, 1
 SPA_FLAG_RESIDUAL, SPA_FLAG_INPLACE, SPA_FLAG_GATE_SCALE, SPA_FLAG_SIMT_ONLY, SPA_FLAG_NO_CTA_PAIRS = 1, 2, 4, 8, 16
+SPA_FLAG_UNFUSED = 32
 
 EXPORTS = (
     "spa_workspace_bytes", "spa_gate", "spa_select_pack", "spa_packed_qkv", "spa_packed_attention_fwd",
@@ -30,6 +31,8 @@ EXPORTS = (
     "spa_fused_scatter_supported", "spa_gate_prefill", "spa_unpack_prefill", "spa_packed_proj_scatter", "spa_packed_linear_bwd_scatter",
     "spa_select_pack_ordered", "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
     "spa_packed_linear", "spa_layer_norm", "spa_layer_norm_bwd", "spa_gelu", "spa_gelu_bwd",
+    "spa_overlap_create", "spa_overlap_destroy", "spa_block_fwd", "spa_block_bwd",
+    "spa_probe_exp2", "spa_probe_wait_expiry",
 )
 
 
@@ -45,6 +48,23 @@ class SpaError(RuntimeError):
 class SpaParams(C.Structure):
     _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("C", C.c_int32), ("H", C.c_int32), ("dtype", C.c_int32),
                 ("flags", C.c_int32), ("capacity", C.c_int32), ("tau", C.c_float), ("softmax_scale", C.c_float)]
+
+
+class SpaBlockBuffers(C.Structure):
+    """spa_block_buffers of include/spa.h, field for field."""
+    _fields_ = [("x", C.c_void_p), ("w_g", C.c_void_p), ("b_g", C.c_float), ("s_up", C.c_void_p),
+                ("W_qkv", C.c_void_p), ("b_qkv", C.c_void_p), ("W_o", C.c_void_p), ("b_o", C.c_void_p),
+                ("order", C.c_void_p), ("seg_offsets", C.c_void_p), ("n_seg", C.c_int32),
+                ("scores", C.c_void_p), ("mask", C.c_void_p), ("cu_seqlens", C.c_void_p), ("idx", C.c_void_p),
+                ("inv", C.c_void_p), ("x_packed", C.c_void_p), ("qkv", C.c_void_p), ("attn_out", C.c_void_p),
+                ("lse", C.c_void_p), ("z", C.c_void_p), ("y", C.c_void_p),
+                ("dY", C.c_void_p), ("dz", C.c_void_p), ("d_attn_out", C.c_void_p), ("dqkv", C.c_void_p),
+                ("dx_packed", C.c_void_p), ("dX", C.c_void_p), ("dW_qkv", C.c_void_p), ("db_qkv", C.c_void_p),
+                ("dW_o", C.c_void_p), ("db_o", C.c_void_p), ("workspace", C.c_void_p), ("workspace_side", C.c_void_p),
+                ("overlap", C.c_void_p), ("d_status", C.c_void_p),
+                ("trainable", C.c_int32), ("labels", C.c_void_p), ("alpha", C.c_float), ("ds", C.c_void_p),
+                ("ds_up", C.c_void_p), ("dw_g", C.c_void_p), ("db_g", C.c_void_p), ("loss", C.c_void_p),
+                ("train_workspace", C.c_void_p)]
 
 
 def make_params(B, N, Cc, H, dtype, capacity=None, flags=0, tau=0.0, softmax_scale=0.0) -> SpaParams:
@@ -94,6 +114,12 @@ def lib() -> C.CDLL:
         L.spa_layer_norm_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_gelu.argtypes = [pp, vp, i32, vp, vp]
         L.spa_gelu_bwd.argtypes = [pp, vp, vp, i32, vp, vp]
+        L.spa_overlap_create.argtypes = [C.POINTER(vp)]
+        L.spa_overlap_destroy.argtypes = [vp]
+        L.spa_block_fwd.argtypes = [pp, C.POINTER(SpaBlockBuffers), vp]
+        L.spa_block_bwd.argtypes = [pp, C.POINTER(SpaBlockBuffers), vp]
+        L.spa_probe_exp2.argtypes = [i32, i32, vp, C.POINTER(C.c_ulonglong), vp]
+        L.spa_probe_wait_expiry.argtypes = [i32, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
             if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_status_string", "spa_last_cuda_error",
@@ -274,6 +300,49 @@ def spa_gelu(p, u, n_cols, h, stream=None):
 
 def spa_gelu_bwd(p, dh, u, n_cols, du, stream=None):
     _check(lib().spa_gelu_bwd(C.byref(p), _ptr(dh), _ptr(u), int(n_cols), _ptr(du), _stream(stream)), "spa_gelu_bwd")
+
+
+def spa_overlap_create() -> int:
+    """Handle of a second stream plus fork / join events, for spa_block_buffers.overlap."""
+    h = C.c_void_p()
+    _check(lib().spa_overlap_create(C.byref(h)), "spa_overlap_create")
+    return h.value
+
+
+def spa_overlap_destroy(handle) -> None:
+    if handle:
+        _check(lib().spa_overlap_destroy(C.c_void_p(handle)), "spa_overlap_destroy")
+
+
+def block_buffers(**fields) -> SpaBlockBuffers:
+    """A spa_block_buffers filled from tensors (device pointers), scalars and None (NULL)."""
+    b = SpaBlockBuffers()
+    for name, v in fields.items():
+        if isinstance(v, torch.Tensor):
+            p = _ptr(v)
+            v = p.value if p is not None else None
+        setattr(b, name, v)
+    return b
+
+
+def spa_block_fwd(p, bufs: SpaBlockBuffers, stream=None):
+    _check(lib().spa_block_fwd(C.byref(p), C.byref(bufs), _stream(stream)), "spa_block_fwd")
+
+
+def spa_block_bwd(p, bufs: SpaBlockBuffers, stream=None):
+    _check(lib().spa_block_bwd(C.byref(p), C.byref(bufs), _stream(stream)), "spa_block_bwd")
+
+
+def spa_probe_exp2(n_ctas, iters, sink, stream=None) -> int:
+    """Enqueue the exponential-throughput probe; returns the number of exponentials it evaluates."""
+    n = C.c_ulonglong(0)
+    _check(lib().spa_probe_exp2(int(n_ctas), int(iters), _ptr(sink), C.byref(n), _stream(stream)), "spa_probe_exp2")
+    return int(n.value)
+
+
+def spa_probe_wait_expiry(limit, d_status, polls_done=None, stream=None):
+    _check(lib().spa_probe_wait_expiry(int(limit), _ptr(d_status), _ptr(polls_done), _stream(stream)),
+           "spa_probe_wait_expiry")
 
 
 def spa_read_status(d_status, stream=None) -> int:

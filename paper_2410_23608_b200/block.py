@@ -1,8 +1,9 @@
-"""One SPA block as a sequence of library calls.
+"""One SPA block: the device buffers, handed to the library's two block calls.
 
-`SpaBlock` owns the device buffers of one block (allocated once through PyTorch) and issues the
-C-ABI calls in order on the current stream.  It computes nothing itself: every step runs in the
-CUDA library.  Nothing here synchronises; N_p stays on the device.
+`SpaBlock` owns the buffers of one block (allocated once through PyTorch) and calls `spa_block_fwd` /
+`spa_block_bwd` on the current stream.  The order of the kernels, the choice between fused and separate
+scatter calls and the second stream for the weight gradients all live in the library; nothing here
+computes or sequences.  Nothing synchronises; N_p stays on the device.
 """
 from __future__ import annotations
 
@@ -14,8 +15,8 @@ from . import binding as L
 
 
 class SpaBlock:
-    """Buffers + call sequence for gate -> select/pack -> QKV -> attention -> projection -> unpack
-    (paper Sec. 3.2) and the matching backward pass."""
+    """Buffers for gate -> select/pack -> QKV -> attention -> projection -> unpack (paper Sec. 3.2) and the
+    matching backward pass."""
 
     def __init__(self, B: int, N: int, C: int, H: int, dtype: str, tau: float = 0.0, flags: int = 0,
                  capacity: Optional[int] = None, backward: bool = True, device: str = "cuda",
@@ -26,14 +27,16 @@ class SpaBlock:
         self.B, self.N, self.C, self.H = B, N, C, H
         self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
         cap = capacity if capacity is not None else max(B * N, 1)
-        self.p = L.make_params(B, N, C, H, dtype, cap, flags, tau)
-        self.cap = cap
         # fused unpack: the projection and the QKV input gradient scatter their rows to the tokens themselves
         # (tensor-core problems only); None = use it where the library offers it
-        can_fuse = L.spa_fused_scatter_supported(self.p)
+        can_fuse = L.spa_fused_scatter_supported(L.make_params(B, N, C, H, dtype, cap, flags, tau))
         if fused and not can_fuse:
             raise ValueError("the fused scatter calls do not apply to this problem (needs bf16 tensor-core sizes)")
         self.fused = can_fuse if fused is None else bool(fused)
+        if not self.fused:
+            flags |= L.SPA_FLAG_UNFUSED
+        self.p = L.make_params(B, N, C, H, dtype, cap, flags, tau)
+        self.cap = cap
         dev = torch.device(device)
         T = self.tdtype
         e = lambda *s, dt=T: torch.empty(*s, dtype=dt, device=dev)
@@ -51,10 +54,9 @@ class SpaBlock:
         self.status = torch.zeros(4, dtype=torch.int32, device=dev)
         ws = L.spa_workspace_bytes(self.p)
         self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if ws > 0 else None
-        # the weight gradients do not feed the rest of the backward chain: they run on a second stream,
-        # with a scratch area of their own, beside the attention backward and the input gradients
-        self.side_stream = torch.cuda.Stream(device=dev) if backward else None
+        # the weight gradients run on a second stream (owned by the library handle), with a scratch area of their own
         self.workspace_side = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if (ws > 0 and backward) else None
+        self._overlap = L.spa_overlap_create() if backward else None
         if backward:
             self.dz = e(cap, C)
             self.dao = e(cap, C)
@@ -65,93 +67,55 @@ class SpaBlock:
             self.db_qkv = e(3 * C, dt=torch.float32)
             self.dW_o = e(C, C, dt=torch.float32)
             self.db_o = e(C, dt=torch.float32)
-        self._saved = None
-        self._seg = (self.cu, B)   # attention segments: the images, unless forward() is given others
+        self._saved = None            # (W_qkv, W_o) of the last forward()
+        self._seg = (self.cu, B)      # attention segments: the images, unless forward() is given others
+        self._keep = None             # tensors of the last call that the enqueued work still reads
+
+    def __del__(self):
+        try:
+            if getattr(self, "_overlap", None):
+                torch.cuda.synchronize()
+                L.spa_overlap_destroy(self._overlap)
+                self._overlap = None
+        except Exception:
+            pass
+
+    def _buffers(self, **extra):
+        seg, n_seg = self._seg
+        f = dict(scores=self.scores, mask=self.mask, cu_seqlens=self.cu, idx=self.idx, inv=self.inv, x_packed=self.xp,
+                 qkv=self.qkv, attn_out=self.ao, lse=self.lse, z=self.z, workspace=self.workspace, d_status=self.status,
+                 seg_offsets=None if seg is self.cu else seg, n_seg=n_seg)
+        f.update(extra)
+        return L.block_buffers(**f)
 
     # ------------------------------------------------------------------ forward
     def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None, order=None, seg_offsets=None):
         """`order` (int32 [N] on the device): visiting order of each image's tokens for the packing (a shifted
         feature map); `seg_offsets` (int32, ascending, ending at N_p): attention segments other than the images,
         e.g. the container cut; the backward pass uses the same segments."""
-        p = self.p
-        y = self.y if y is None else y
-        inplace = bool(p.flags & L.SPA_FLAG_INPLACE)
-        if self.fused and not inplace:
-            # the pass-through rows y = x are written by the gate, which reads all of x anyway
-            L.spa_gate_prefill(p, x, w_g, b_g, s_up, self.scores, self.mask, y)
-        else:
-            L.spa_gate(p, x, w_g, b_g, s_up, self.scores, self.mask)
-        if order is None:
-            L.spa_select_pack(p, x, self.mask, self.scores, self.xp, self.idx, self.inv, self.cu, self.status)
-        else:
-            L.spa_select_pack_ordered(p, x, self.mask, self.scores, order, self.xp, self.idx, self.inv, self.cu,
-                                      self.status)
-        L.spa_packed_qkv(p, self.xp, W_qkv, b_qkv, self.cu, self.qkv, self.status)
+        inplace = bool(self.p.flags & L.SPA_FLAG_INPLACE)
+        y = x if inplace else (self.y if y is None else y)
         self._seg = (self.cu, self.B) if seg_offsets is None else (seg_offsets, int(seg_offsets.numel()) - 1)
-        L.spa_packed_attention_fwd(p, self.qkv, self._seg[0], self._seg[1], self.ao, self.lse, self.status)
-        if self.fused:
-            if inplace:
-                y = x
-            L.spa_packed_proj_scatter(p, self.ao, W_o, b_o, self.idx, self.cu, y, self.status)
-        else:
-            L.spa_packed_proj(p, self.ao, W_o, b_o, self.cu, self.z, self.status)
-            if inplace:
-                L.spa_unpack_scatter(p, self.z, None, self.idx, self.inv, self.cu, x, self.status)
-                y = x
-            else:
-                L.spa_unpack_scatter(p, self.z, x, self.idx, self.inv, self.cu, y, self.status)
         self._saved = (W_qkv, W_o)
+        self._keep = (x, w_g, W_qkv, b_qkv, W_o, b_o, s_up, order, seg_offsets, y)
+        L.spa_block_fwd(self.p, self._buffers(x=x, w_g=w_g, b_g=float(b_g), s_up=s_up, W_qkv=W_qkv, b_qkv=b_qkv, W_o=W_o,
+                                              b_o=b_o, order=order, y=y))
         return y
 
     # ------------------------------------------------------------------ backward
+    def _backward_fields(self, dY, dX):
+        W_qkv, W_o = self._saved
+        return dict(W_qkv=W_qkv, W_o=W_o, dY=dY, dz=self.dz, d_attn_out=self.dao, dqkv=self.dqkv, dx_packed=self.dxp,
+                    dX=dX, dW_qkv=self.dW_qkv, db_qkv=self.db_qkv, dW_o=self.dW_o, db_o=self.db_o,
+                    workspace_side=self.workspace_side)
+
     def backward(self, dY, dX=None, overlap=True):
         """Gradients for the last forward(): returns dX; parameter gradients land in dW_qkv, db_qkv,
         dW_o, db_o (fp32).  No gradient reaches the gate (hard threshold).  With overlap=True the two
-        weight-gradient calls are issued on a second stream and joined before returning."""
-        p = self.p
-        W_qkv, W_o = self._saved
+        weight-gradient products run on the library's second stream and are joined before the call returns."""
         dX = self.dX if dX is None else dX
-        C = self.C
-        main = torch.cuda.current_stream()
-        side = self.side_stream if (overlap and self.side_stream is not None) else None
-        # dz = gather of dY; dX = dY on the tokens that passed through (fused path: the QKV input gradient
-        # scatters its rows to the selected tokens itself, so no packed dx and no scatter kernel follow)
-        L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
-        if side is None:
-            L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
-                                    self.workspace, self.status)
-        else:
-            side.wait_stream(main)
-            L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, None, self.dW_o, self.db_o,
-                                    self.workspace_side, self.status, stream=side)
-            L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, None, None,
-                                    self.workspace, self.status)
-        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self._seg[0], self._seg[1], self.dqkv,
-                                   self.workspace, self.status)
-        if self.fused:
-            if side is None:
-                L.spa_packed_linear_bwd_scatter(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.idx, self.cu, dX,
-                                                self.dW_qkv, self.db_qkv, self.workspace, self.status)
-            else:
-                side.wait_stream(main)
-                L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, None, self.dW_qkv,
-                                        self.db_qkv, self.workspace_side, self.status, stream=side)
-                L.spa_packed_linear_bwd_scatter(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.idx, self.cu, dX,
-                                                None, None, None, self.status)
-                main.wait_stream(side)
-            return dX
-        if side is None:
-            L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv,
-                                    self.db_qkv, self.workspace, self.status)
-        else:
-            side.wait_stream(main)
-            L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, None, self.dW_qkv, self.db_qkv,
-                                    self.workspace_side, self.status, stream=side)
-            L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, None, None,
-                                    self.workspace, self.status)
-        L.spa_select_pack_bwd(p, self.dxp, dY, self.idx, self.cu, dX)
-        if side is not None:
-            main.wait_stream(side)
+        L.spa_block_bwd(self.p, self._buffers(overlap=self._overlap if overlap else None,
+                                              **self._backward_fields(dY, dX)))
         return dX
 
     def backward_trainable(self, dY, x, w_g, labels=None, alpha: float = 1.0, s_up=None, dX=None):
@@ -159,31 +123,20 @@ class SpaBlock:
         selection loss alpha * BCE(Sigmoid(scores), labels) when `labels` (uint8 [B, N]) is given, and, under
         SPA_FLAG_GATE_SCALE, the path through the sigmoid scaling of the packed rows.  `s_up` must be the
         tensor given to forward().  Returns dX; also fills dw_g, db_g, ds_up (fp32), ds and loss."""
-        p, C = self.p, self.C
-        W_qkv, W_o = self._saved
         dX = self.dX if dX is None else dX
         if not hasattr(self, "ds"):
             dev = self.scores.device
             n = max(self.B * self.N, 1)
             self.ds = torch.empty(n, dtype=torch.float32, device=dev)
             self.ds_up = torch.empty(n, dtype=torch.float32, device=dev)
-            self.dw_g = torch.empty(C, dtype=torch.float32, device=dev)
+            self.dw_g = torch.empty(self.C, dtype=torch.float32, device=dev)
             self.db_g = torch.empty(1, dtype=torch.float32, device=dev)
             self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
-            self.train_ws = torch.empty(max(L.spa_train_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
-        L.spa_select_loss(p, self.scores, labels, alpha, self.ds, self.loss, self.train_ws)
-        L.spa_unpack_scatter_bwd(p, dY, self.idx, self.inv, self.cu, self.dz, dX)
-        L.spa_packed_linear_bwd(p, self.ao, W_o, self.dz, C, C, self.cu, self.dao, self.dW_o, self.db_o,
-                                self.workspace, self.status)
-        L.spa_packed_attention_bwd(p, self.qkv, self.ao, self.lse, self.dao, self._seg[0], self._seg[1], self.dqkv,
-                                   self.workspace, self.status)
-        L.spa_packed_linear_bwd(p, self.xp, W_qkv, self.dqkv, C, 3 * C, self.cu, self.dxp, self.dW_qkv,
-                                self.db_qkv, self.workspace, self.status)
-        if p.flags & L.SPA_FLAG_GATE_SCALE:
-            L.spa_select_pack_bwd_gated(p, self.dxp, x, self.scores, dY, self.idx, self.cu, dX, self.ds)
-        else:
-            L.spa_select_pack_bwd(p, self.dxp, dY, self.idx, self.cu, dX)
-        L.spa_gate_bwd(p, x, w_g, self.scores, s_up, self.ds, dX, self.dw_g, self.db_g, self.ds_up, self.train_ws)
+            self.train_ws = torch.empty(max(L.spa_train_workspace_bytes(self.p), 256), dtype=torch.uint8, device=dev)
+        L.spa_block_bwd(self.p, self._buffers(x=x, w_g=w_g, s_up=s_up, trainable=1, labels=labels, alpha=float(alpha),
+                                              ds=self.ds, ds_up=self.ds_up, dw_g=self.dw_g, db_g=self.db_g,
+                                              loss=self.loss, train_workspace=self.train_ws,
+                                              **self._backward_fields(dY, dX)))
         return dX
 
     def read_status(self) -> int:

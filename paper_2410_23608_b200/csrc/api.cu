@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <new>
 
 #include "spa_common.cuh"
 #include "spa_tc.cuh"
@@ -378,6 +379,157 @@ int spa_gelu_bwd(const spa_params* p, const void* dh, const void* u, int32_t n_c
   SPA_REQUIRE(n_cols > 0 && (n_cols * (p->dtype == SPA_F32 ? 4 : 2)) % 16 == 0, SPA_ERR_INVALID_ARG);
   return launch_gelu(*p, u, dh, n_cols, du, (cudaStream_t)stream);
 }
+
+// ---- the block as one unit: sequencing only ------------------------------------------------------------------
+struct spa_overlap {
+  cudaStream_t side;
+  cudaEvent_t fork, join;
+};
+
+int spa_overlap_create(spa_overlap** out) {
+  if (out == nullptr) return SPA_ERR_INVALID_ARG;
+  spa_overlap* ov = new (std::nothrow) spa_overlap{nullptr, nullptr, nullptr};
+  if (ov == nullptr) return SPA_ERR_INVALID_ARG;
+  cudaError_t e = cudaStreamCreateWithFlags(&ov->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ov->fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ov->join, cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    set_cuda_error(e, "spa_overlap_create");
+    spa_overlap_destroy(ov);
+    return SPA_ERR_CUDA;
+  }
+  *out = ov;
+  return SPA_OK;
+}
+
+int spa_overlap_destroy(spa_overlap* ov) {
+  if (ov == nullptr) return SPA_OK;
+  if (ov->join != nullptr) cudaEventDestroy(ov->join);
+  if (ov->fork != nullptr) cudaEventDestroy(ov->fork);
+  if (ov->side != nullptr) cudaStreamDestroy(ov->side);
+  delete ov;
+  return SPA_OK;
+}
+
+namespace {
+inline bool block_fused(const spa_params* p) {
+  return !(p->flags & SPA_FLAG_UNFUSED) && spa_fused_scatter_supported(p) != 0;
+}
+// the second stream starts after everything enqueued on the main stream so far
+inline int fork_side(const spa_overlap* ov, cudaStream_t main) {
+  cudaError_t e = cudaEventRecord(ov->fork, main);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ov->side, ov->fork, 0);
+  if (e != cudaSuccess) { set_cuda_error(e, "spa_block_bwd: fork"); return SPA_ERR_CUDA; }
+  return SPA_OK;
+}
+inline int join_side(const spa_overlap* ov, cudaStream_t main) {
+  cudaError_t e = cudaEventRecord(ov->join, ov->side);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(main, ov->join, 0);
+  if (e != cudaSuccess) { set_cuda_error(e, "spa_block_bwd: join"); return SPA_ERR_CUDA; }
+  return SPA_OK;
+}
+#define SPA_STEP(call) do { rc = (call); if (rc != SPA_OK) return rc; } while (0)
+}  // namespace
+
+int spa_block_fwd(const spa_params* p, const spa_block_buffers* b, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  if (b == nullptr) return SPA_ERR_INVALID_ARG;
+  const bool inplace = (p->flags & SPA_FLAG_INPLACE) != 0;
+  const bool fused = block_fused(p);
+  void* y = inplace ? const_cast<void*>(b->x) : b->y;
+  SPA_REQUIRE(!inplace || b->y == nullptr || b->y == b->x, SPA_ERR_INVALID_ARG);
+  // gate (Eq. 4) and hard selection; on the fused path it also writes the pass-through rows y = x
+  if (fused && !inplace) SPA_STEP(spa_gate_prefill(p, b->x, b->w_g, b->b_g, b->s_up, b->scores, b->mask, y, stream));
+  else SPA_STEP(spa_gate(p, b->x, b->w_g, b->b_g, b->s_up, b->scores, b->mask, stream));
+  // token packing
+  if (b->order == nullptr)
+    SPA_STEP(spa_select_pack(p, b->x, b->mask, b->scores, b->x_packed, b->idx, b->inv, b->cu_seqlens, b->d_status, stream));
+  else
+    SPA_STEP(spa_select_pack_ordered(p, b->x, b->mask, b->scores, b->order, b->x_packed, b->idx, b->inv, b->cu_seqlens,
+                                     b->d_status, stream));
+  SPA_STEP(spa_packed_qkv(p, b->x_packed, b->W_qkv, b->b_qkv, b->cu_seqlens, b->qkv, b->d_status, stream));
+  const int32_t* seg = b->seg_offsets != nullptr ? b->seg_offsets : b->cu_seqlens;
+  const int32_t n_seg = b->seg_offsets != nullptr ? b->n_seg : p->B;
+  SPA_STEP(spa_packed_attention_fwd(p, b->qkv, seg, n_seg, b->attn_out, b->lse, b->d_status, stream));
+  if (fused) return spa_packed_proj_scatter(p, b->attn_out, b->W_o, b->b_o, b->idx, b->cu_seqlens, y, b->d_status, stream);
+  SPA_STEP(spa_packed_proj(p, b->attn_out, b->W_o, b->b_o, b->cu_seqlens, b->z, b->d_status, stream));
+  return spa_unpack_scatter(p, b->z, inplace ? nullptr : b->x, b->idx, b->inv, b->cu_seqlens, y, b->d_status, stream);
+}
+
+int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  if (b == nullptr) return SPA_ERR_INVALID_ARG;
+  const int C = p->C;
+  cudaStream_t main = (cudaStream_t)stream;
+  // the weight gradients feed nothing downstream: with `overlap` they run on the second stream, with a scratch
+  // area of their own, beside the attention backward and the input gradients.  The trainable path keeps one stream.
+  const spa_overlap* ov = b->trainable ? nullptr : b->overlap;
+  SPA_REQUIRE(ov == nullptr || b->workspace_side != nullptr || spa_workspace_bytes(p) == 0, SPA_ERR_INVALID_ARG);
+  const bool fused = block_fused(p) && !b->trainable;
+  const int32_t* seg = b->seg_offsets != nullptr ? b->seg_offsets : b->cu_seqlens;
+  const int32_t n_seg = b->seg_offsets != nullptr ? b->n_seg : p->B;
+  void* side = ov != nullptr ? (void*)ov->side : nullptr;
+
+  if (b->trainable)
+    SPA_STEP(spa_select_loss(p, b->scores, b->labels, b->alpha, b->ds, b->loss, b->train_workspace, stream));
+  // dz = rows of dY at the selected tokens; dX = dY on the tokens that passed through
+  SPA_STEP(spa_unpack_scatter_bwd(p, b->dY, b->idx, b->inv, b->cu_seqlens, b->dz, b->dX, stream));
+  bool forked = false;
+  int rc_side = SPA_OK;
+  if (ov == nullptr) {
+    SPA_STEP(spa_packed_linear_bwd(p, b->attn_out, b->W_o, b->dz, C, C, b->cu_seqlens, b->d_attn_out, b->dW_o, b->db_o,
+                                   b->workspace, b->d_status, stream));
+  } else {
+    SPA_STEP(fork_side(ov, main));
+    forked = true;
+    rc_side = spa_packed_linear_bwd(p, b->attn_out, b->W_o, b->dz, C, C, b->cu_seqlens, nullptr, b->dW_o, b->db_o,
+                                    b->workspace_side, b->d_status, side);
+    rc = spa_packed_linear_bwd(p, b->attn_out, b->W_o, b->dz, C, C, b->cu_seqlens, b->d_attn_out, nullptr, nullptr,
+                               b->workspace, b->d_status, stream);
+  }
+  if (rc == SPA_OK && rc_side == SPA_OK)
+    rc = spa_packed_attention_bwd(p, b->qkv, b->attn_out, b->lse, b->d_attn_out, seg, n_seg, b->dqkv, b->workspace,
+                                  b->d_status, stream);
+  if (rc == SPA_OK && rc_side == SPA_OK) {
+    if (ov != nullptr) {
+      // the second stream's next call reads dqkv: it waits for the attention backward
+      rc_side = fork_side(ov, main);
+      if (rc_side == SPA_OK)
+        rc_side = spa_packed_linear_bwd(p, b->x_packed, b->W_qkv, b->dqkv, C, 3 * C, b->cu_seqlens, nullptr, b->dW_qkv,
+                                        b->db_qkv, b->workspace_side, b->d_status, side);
+    }
+    float* dW = ov != nullptr ? nullptr : b->dW_qkv;
+    float* db = ov != nullptr ? nullptr : b->db_qkv;
+    void* ws = ov != nullptr ? nullptr : b->workspace;
+    if (fused) {
+      // the input gradient scatters its rows to the selected tokens itself: no packed dx, no scatter kernel
+      rc = spa_packed_linear_bwd_scatter(p, b->x_packed, b->W_qkv, b->dqkv, C, 3 * C, b->idx, b->cu_seqlens, b->dX, dW,
+                                         db, ws, b->d_status, stream);
+    } else {
+      rc = spa_packed_linear_bwd(p, b->x_packed, b->W_qkv, b->dqkv, C, 3 * C, b->cu_seqlens, b->dx_packed, dW, db,
+                                 ov != nullptr ? b->workspace : ws, b->d_status, stream);
+      if (rc == SPA_OK) {
+        if (b->trainable && (p->flags & SPA_FLAG_GATE_SCALE))
+          rc = spa_select_pack_bwd_gated(p, b->dx_packed, b->x, b->scores, b->dY, b->idx, b->cu_seqlens, b->dX, b->ds,
+                                         stream);
+        else
+          rc = spa_select_pack_bwd(p, b->dx_packed, b->dY, b->idx, b->cu_seqlens, b->dX, stream);
+      }
+    }
+  }
+  if (forked) {  // joined on every path, so that a recording stream is never left forked
+    const int rj = join_side(ov, main);
+    if (rc == SPA_OK) rc = rc_side != SPA_OK ? rc_side : rj;
+  }
+  if (rc != SPA_OK) return rc;
+  if (b->trainable)
+    SPA_STEP(spa_gate_bwd(p, b->x, b->w_g, b->scores, b->s_up, b->ds, b->dX, b->dw_g, b->db_g, b->ds_up,
+                          b->train_workspace, stream));
+  return SPA_OK;
+}
+#undef SPA_STEP
 
 int spa_read_status(const int32_t* d_status, void* stream) {
   if (d_status == nullptr) return SPA_ERR_INVALID_ARG;

@@ -325,3 +325,28 @@ def test_general_linear_backward_ragged_sizes(n_in, n_out, rows, flags):
     assert bool((da[rows:] == 7.0).all())
     assert_close(host(dW), dW_ref, dtype, "dW", scale_max_abs=True)
     assert_close(host(db), db_ref, dtype, "db", scale_max_abs=True)
+
+
+def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
+    """A device-side wait that can never be satisfied (a barrier nobody arrives at, polled 1 024 times) ends by
+    itself: the kernel returns, the status word reads SPA_ERR_TIMEOUT, and the next ordinary call is correct."""
+    lib = L()
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    polls = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lib.spa_probe_wait_expiry(1024, status, polls)
+    torch.cuda.synchronize()
+    assert lib.spa_read_status(status) == lib.SPA_ERR_TIMEOUT
+    assert int(polls.item()) == 1024
+    assert "wait" in lib.lib().spa_status_string(lib.SPA_ERR_TIMEOUT).decode()
+    # first error wins: a later, different condition does not overwrite it; a zeroed word is clean again
+    lib.spa_probe_wait_expiry(16, status, polls)
+    assert lib.spa_read_status(status) == lib.SPA_ERR_TIMEOUT
+    status.zero_()
+    cfg = get_config(1)
+    inp = make_inputs(cfg)
+    blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau)
+    d = {n: dev(getattr(inp, n), cfg.dtype) for n in ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o")}
+    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+    fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
+    assert_close(host(y), fwd["y"], cfg.dtype, "y after an expired wait")
+    assert blk.read_status() == 0 and lib.spa_read_status(status) == 0

@@ -267,3 +267,76 @@ def test_graph_replay_is_stable_and_reproducible(ci):
     for a, b in zip(first, outs):
         assert torch.equal(a, b)
     assert_close(host(blk.y), fwd["y"], cfg.dtype, "y")
+
+
+CANARY = 0x5A
+
+
+def guarded(shape, dtype, guard_rows=2):
+    """A device buffer with `guard_rows` extra rows before and after it, every byte set to a fixed pattern; returns
+    (the inner view, a function that checks that the guard rows still hold the pattern)."""
+    rows = shape[0] if len(shape) > 1 else 1
+    row_elems = int(np.prod(shape[1:])) if len(shape) > 1 else int(shape[0])
+    # a guard row is one row of the buffer, rounded up so that the inner view stays 256-byte aligned
+    esz = torch.empty(0, dtype=dtype).element_size()
+    g = ((guard_rows * row_elems * esz + 255) // 256) * 256
+    inner_bytes = rows * row_elems * esz
+    raw = torch.full((g + inner_bytes + g,), CANARY, dtype=torch.uint8, device="cuda")
+    inner = raw[g:g + inner_bytes].view(dtype).view(*shape)
+
+    def intact():
+        return bool((raw[:g] == CANARY).all()) and bool((raw[g + inner_bytes:] == CANARY).all())
+
+    return inner, intact
+
+
+@pytest.mark.parametrize("ci,flags", [(1, 0), (2, 0), (2, 32), (2, 1)])   # 32: separate scatter kernels; 1: residual
+def test_block_calls_alone_with_guard_bands(ci, flags):
+    """One forward and one backward pass through nothing but spa_block_fwd / spa_block_bwd (no Python class in
+    between), every buffer the library writes framed by guard rows that must come back untouched."""
+    from paper_2410_23608_b200 import binding as L
+    cfg, inp, fwd, bwd = problem(ci, residual=bool(flags & 1))
+    d = device_inputs(cfg, inp)
+    B, N, C, H, dt = cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype
+    T = torch.float32 if dt == "f32" else torch.bfloat16
+    cap = B * N
+    p = L.make_params(B, N, C, H, dt, cap, flags, cfg.tau)
+    f32, i32, u8 = torch.float32, torch.int32, torch.uint8
+    spec = dict(scores=((cap,), f32), mask=((cap,), u8), cu_seqlens=((B + 1,), i32), idx=((cap,), i32),
+                inv=((cap,), i32), x_packed=((cap, C), T), qkv=((cap, 3 * C), T), attn_out=((cap, C), T),
+                lse=((H, cap), f32), z=((cap, C), T), y=((B * N, C), T), dz=((cap, C), T), d_attn_out=((cap, C), T),
+                dqkv=((cap, 3 * C), T), dx_packed=((cap, C), T), dX=((B * N, C), T), dW_qkv=((3 * C, C), f32),
+                db_qkv=((3 * C,), f32), dW_o=((C, C), f32), db_o=((C,), f32))
+    buf, checks = {}, {}
+    for name, (shape, dtype) in spec.items():
+        buf[name], checks[name] = guarded(shape, dtype)
+    ws_bytes = max(L.spa_workspace_bytes(p), 256)
+    buf["workspace"], checks["workspace"] = guarded((ws_bytes,), u8)
+    buf["workspace_side"], checks["workspace_side"] = guarded((ws_bytes,), u8)
+    status = torch.zeros(4, dtype=i32, device="cuda")
+    ov = L.spa_overlap_create()
+    try:
+        bufs = L.block_buffers(x=d["x"], w_g=d["w_g"], b_g=float(inp.b_g), W_qkv=d["W_qkv"], b_qkv=d["b_qkv"],
+                               W_o=d["W_o"], b_o=d["b_o"], dY=d["dY"], overlap=ov, d_status=status, **buf)
+        L.spa_block_fwd(p, bufs)
+        L.spa_block_bwd(p, bufs)
+        torch.cuda.synchronize()
+    finally:
+        L.spa_overlap_destroy(ov)
+    assert L.spa_read_status(status) == 0
+    touched = [name for name, ok in checks.items() if not ok()]
+    assert not touched, f"writes outside the buffer: {touched}"
+    Np = int(fwd["cu_seqlens"][-1])
+    assert np.array_equal(buf["cu_seqlens"].cpu().numpy(), fwd["cu_seqlens"])
+    assert np.array_equal(buf["idx"].cpu().numpy()[:Np], fwd["idx"])
+    assert np.array_equal(buf["inv"].cpu().numpy(), fwd["inv"])
+    assert np.array_equal(buf["mask"].cpu().numpy().astype(bool), fwd["mask"].reshape(-1))
+    yh, dXh = host(buf["y"]).reshape(B, N, C), host(buf["dX"]).reshape(B, N, C)
+    assert_close(yh, fwd["y"], dt, "y")
+    assert_close(dXh, bwd["dX"], dt, "dX", scale_max_abs=True)
+    unsel = ~fwd["mask"]
+    assert np.array_equal(yh[unsel], inp.x[unsel])
+    if not flags & 1:
+        assert np.array_equal(dXh[unsel], inp.dY[unsel])
+    for name in ("dW_qkv", "db_qkv", "dW_o", "db_o"):
+        assert_close(host(buf[name]), bwd[name], dt, name, scale_max_abs=True)

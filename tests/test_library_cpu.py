@@ -84,6 +84,12 @@ def test_later_entry_points_validate_on_the_host(lib):
     assert L.spa_layer_norm_bwd(pp, None, None, None, None, None, None, None, None, None, None, None) == inv
     assert L.spa_gelu(pp, None, 256, None, None) == inv
     assert L.spa_gelu_bwd(pp, None, None, 256, None, None) == inv
+    empty = lib.SpaBlockBuffers()
+    assert L.spa_block_fwd(pp, None, None) == inv and L.spa_block_bwd(pp, None, None) == inv
+    assert L.spa_block_fwd(pp, ctypes.byref(empty), None) == inv      # no inputs: refused by the first call
+    assert L.spa_block_bwd(pp, ctypes.byref(empty), None) == inv
+    assert L.spa_block_fwd(None, ctypes.byref(empty), None) == inv
+    assert L.spa_overlap_create(None) == inv and L.spa_overlap_destroy(None) == 0
     f32 = lib.make_params(2, 16, 64, 2, "f32")
     assert L.spa_fused_scatter_supported(ctypes.byref(f32)) == 0          # tensor-core problems only
     assert L.spa_packed_proj_scatter(ctypes.byref(f32), None, None, None, None, None, None, None, None) in (inv, uns)
