@@ -100,13 +100,18 @@ def timing_units(L, blk, d, b_g):
     p, C = blk.p, blk.C
     fused = blk.fused
     units = []
-    if fused:
-        units.append(("gate", lambda: L.spa_gate_prefill(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask, blk.y)))
+    if blk.one_pass:
+        units.append(("gate_pack", lambda: L.spa_gate_select_pack(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask,
+                                                                  blk.y if fused else None, blk.xp, blk.idx, blk.inv,
+                                                                  blk.cu, blk.pack_state, blk.status)))
     else:
-        units.append(("gate", lambda: L.spa_gate(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask)))
+        if fused:
+            units.append(("gate", lambda: L.spa_gate_prefill(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask, blk.y)))
+        else:
+            units.append(("gate", lambda: L.spa_gate(p, d["x"], d["w_g"], b_g, None, blk.scores, blk.mask)))
+        units.append(("select_pack", lambda: L.spa_select_pack(p, d["x"], blk.mask, blk.scores, blk.xp, blk.idx, blk.inv,
+                                                               blk.cu, blk.status)))
     units += [
-        ("select_pack", lambda: L.spa_select_pack(p, d["x"], blk.mask, blk.scores, blk.xp, blk.idx, blk.inv, blk.cu,
-                                                  blk.status)),
         ("qkv", lambda: L.spa_packed_qkv(p, blk.xp, d["W_qkv"], d["b_qkv"], blk.cu, blk.qkv, blk.status)),
         ("attn_fwd", lambda: L.spa_packed_attention_fwd(p, blk.qkv, blk.cu, blk.B, blk.ao, blk.lse, blk.status)),
     ]
@@ -268,7 +273,7 @@ def run_reference(args):
 class Workload:
     """Rotating buffer sets of one workload, its whole-step graphs and its per-unit timings."""
 
-    def __init__(self, torch, L, cfg, no_fuse=False, sets=0):
+    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=True):
         from paper_2410_23608_b200.block import SpaBlock
         from spa_workloads import make_inputs, scaled_config
         self.torch, self.L, self.cfg = torch, L, cfg
@@ -282,7 +287,7 @@ class Workload:
             inp = make_inputs(scaled_config(cfg, seed=cfg.seed + 1000 * s)) if s < 2 else self.inps[s % 2]
             self.inps.append(inp)
             d = {n: inp.torch(n, "cuda") for n in names}
-            blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau, fused=False if no_fuse else None)
+            blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau, fused=False if no_fuse else None, one_pass=one_pass)
             self.sets.append((inp, d, blk))
         self.stream = torch.cuda.current_stream()
         for s in range(self.n_sets):     # eager pass: first-use set-up (attributes, tensor maps) outside capture
@@ -366,6 +371,7 @@ class Workload:
         work, Np0, S2 = work_model(cfg, self.sets[0][2].cu.cpu().numpy())
         if self.sets[0][2].fused:
             work["gate"] = work["gate_prefill"]
+            work["gate_pack"] = work["gate_pack_prefill"]
         out = {}
         for name in per_set[0]:
             g, n_l = self.capture([u[name] for u in per_set])
@@ -443,6 +449,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="time the headline workload only")
     ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
+    ap.add_argument("--two-kernel-pack", action="store_true", help="gate and packing as two kernels instead of the one-pass call")
     ap.add_argument("--train", action="store_true", help="also time the trainable-selection calls (loss, gated pack backward, gate backward)")
     ap.add_argument("--layer", action="store_true", help="also time the whole pre-norm block (LayerNorm, SPA, feed-forward) and its new calls")
     args = ap.parse_args()
@@ -471,7 +478,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     cfg = get_config(args.config)
-    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets)
+    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=not args.two_kernel_pack)
     stream = wl.stream
     n_sets = wl.n_sets
     wl.warm(args.warmup)
@@ -644,7 +651,7 @@ def main():
     if not args.no_cpu_baseline:
         cpu = cpu_baseline(cfg, wl.inps[0], make_inputs, scaled_config)
 
-    flop_units = ("gate", "qkv", "attn_fwd", "proj", "attn_bwd", "proj_bwd.da", "proj_bwd.dW", "proj_bwd.db",
+    flop_units = ("gate_pack" if wl.sets[0][2].one_pass else "gate", "qkv", "attn_fwd", "proj", "attn_bwd", "proj_bwd.da", "proj_bwd.dW", "proj_bwd.db",
                   "qkv_bwd.da", "qkv_bwd.dW", "qkv_bwd.db")
     useful_flops = sum(work[k]["flops"] for k in flop_units)
     Np_head = wl.Np_sets[0]
@@ -665,7 +672,7 @@ def main():
             if ci == args.config:
                 continue
             c2 = get_config(ci)
-            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse)
+            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=not args.two_kernel_pack)
             w2.warm(20)
             steps2 = 200
             ms2 = w2.time_steps(steps2) / steps2

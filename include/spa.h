@@ -105,6 +105,20 @@ int spa_select_pack_ordered(const spa_params* p, const void* x, const uint8_t* m
                             const int32_t* order, void* x_packed, int32_t* idx, int32_t* inv,
                             int32_t* cu_seqlens, int32_t* d_status, void* stream);
 
+/* spa_gate (or spa_gate_prefill when y != NULL) and spa_select_pack in one pass over x (Sec. 3.2, Eq. 4, Eq. 6,
+ * "Token Packing"): x is read once, the selected rows go from registers to x_packed.  Same outputs, bit for bit, as
+ * the two calls.  Rows of at most 128 16-byte chunks (1024 bf16 or 512 fp32 channels): spa_gate_select_pack_supported
+ * says whether the call applies, else it returns SPA_ERR_UNSUPPORTED.
+ * pack_state: spa_pack_state_bytes() bytes of device memory that must be ZERO when the call starts; the kernel
+ * leaves it zero again (also after an error), so the caller clears it once, after allocating it.  Two calls that
+ * share one pack_state must not overlap on the GPU.  Tiles of tokens exchange their selected counts through it;
+ * every wait on it is bounded (SPA_ERR_TIMEOUT in d_status when one runs out; the packed outputs are then undefined). */
+size_t spa_pack_state_bytes(const spa_params* p);
+int spa_gate_select_pack_supported(const spa_params* p);
+int spa_gate_select_pack(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up,
+                         float* scores, uint8_t* mask, void* y, void* x_packed, int32_t* idx, int32_t* inv,
+                         int32_t* cu_seqlens, void* pack_state, int32_t* d_status, void* stream);
+
 /* QKV projection on the packed tokens (the 3LC^2 term of Eq. 9):
  *   qkv[i][j] = b_qkv[j] + sum_c W_qkv[j][c] * x_packed[i][c],  i < N_p, j < 3C.
  * W_qkv: T[3C][C]; b_qkv: T[3C] or NULL; qkv: T[capacity][3C] out. */
@@ -299,7 +313,7 @@ int spa_gelu_bwd(const spa_params* p, const void* dh, const void* u, int32_t n_c
  *
  * All pointers are device memory owned by the caller and sized as in the single calls (packed buffers: `capacity`
  * rows).  Which fields may be NULL:
- *   s_up, order, seg_offsets (NULL: the images are the attention segments), b_qkv, b_o;
+ *   s_up, order, seg_offsets (NULL: the images are the attention segments), b_qkv, b_o, pack_state;
  *   z, dx_packed            when the fused calls apply (the products write y and dX rows themselves);
  *   every backward field    for spa_block_fwd;
  *   labels .. train_workspace unless `trainable` is non-zero.
@@ -344,6 +358,8 @@ typedef struct spa_block_buffers {
   float* db_o;                /* float[C]                                                            */
   void* workspace;            /* spa_workspace_bytes()                                               */
   void* workspace_side;       /* a second area of that size; needed when `overlap` is given          */
+  void* pack_state;           /* spa_pack_state_bytes(), zeroed once by the caller, or NULL: gate and
+                                 packing then run as two kernels                                     */
   spa_overlap* overlap;       /* spa_overlap_create(), or NULL: everything on `stream`               */
   int32_t* d_status;          /* device status word or NULL                                          */
   /* trainable selection (Eq. 4-5, Eq. 10): gradient to the gate */

@@ -32,7 +32,8 @@ EXPORTS = (
     "spa_select_pack_ordered", "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
     "spa_packed_linear", "spa_layer_norm", "spa_layer_norm_bwd", "spa_gelu", "spa_gelu_bwd",
     "spa_overlap_create", "spa_overlap_destroy", "spa_block_fwd", "spa_block_bwd",
-    "spa_probe_exp2", "spa_probe_wait_expiry",
+    "spa_probe_exp2", "spa_probe_wait_expiry", "spa_pack_state_bytes", "spa_gate_select_pack_supported",
+    "spa_gate_select_pack",
 )
 
 
@@ -61,7 +62,7 @@ class SpaBlockBuffers(C.Structure):
                 ("dY", C.c_void_p), ("dz", C.c_void_p), ("d_attn_out", C.c_void_p), ("dqkv", C.c_void_p),
                 ("dx_packed", C.c_void_p), ("dX", C.c_void_p), ("dW_qkv", C.c_void_p), ("db_qkv", C.c_void_p),
                 ("dW_o", C.c_void_p), ("db_o", C.c_void_p), ("workspace", C.c_void_p), ("workspace_side", C.c_void_p),
-                ("overlap", C.c_void_p), ("d_status", C.c_void_p),
+                ("pack_state", C.c_void_p), ("overlap", C.c_void_p), ("d_status", C.c_void_p),
                 ("trainable", C.c_int32), ("labels", C.c_void_p), ("alpha", C.c_float), ("ds", C.c_void_p),
                 ("ds_up", C.c_void_p), ("dw_g", C.c_void_p), ("db_g", C.c_void_p), ("loss", C.c_void_p),
                 ("train_workspace", C.c_void_p)]
@@ -118,11 +119,15 @@ def lib() -> C.CDLL:
         L.spa_overlap_destroy.argtypes = [vp]
         L.spa_block_fwd.argtypes = [pp, C.POINTER(SpaBlockBuffers), vp]
         L.spa_block_bwd.argtypes = [pp, C.POINTER(SpaBlockBuffers), vp]
+        L.spa_pack_state_bytes.restype = C.c_size_t
+        L.spa_pack_state_bytes.argtypes = [pp]
+        L.spa_gate_select_pack_supported.argtypes = [pp]
+        L.spa_gate_select_pack.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_probe_exp2.argtypes = [i32, i32, vp, C.POINTER(C.c_ulonglong), vp]
         L.spa_probe_wait_expiry.argtypes = [i32, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
-            if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_status_string", "spa_last_cuda_error",
+            if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_pack_state_bytes", "spa_status_string", "spa_last_cuda_error",
                             "spa_launch_count"):
                 getattr(L, name).restype = C.c_int
         L.spa_status_string.restype = C.c_char_p
@@ -162,6 +167,21 @@ def spa_workspace_bytes(p: SpaParams) -> int:
 def spa_gate(p, x, w_g, b_g, s_up, scores, mask, stream=None):
     _check(lib().spa_gate(C.byref(p), _ptr(x), _ptr(w_g), float(b_g), _ptr(s_up), _ptr(scores), _ptr(mask),
                           _stream(stream)), "spa_gate")
+
+
+def spa_pack_state_bytes(p) -> int:
+    return int(lib().spa_pack_state_bytes(C.byref(p)))
+
+
+def spa_gate_select_pack_supported(p) -> bool:
+    return bool(lib().spa_gate_select_pack_supported(C.byref(p)))
+
+
+def spa_gate_select_pack(p, x, w_g, b_g, s_up, scores, mask, y, x_packed, idx, inv, cu_seqlens, pack_state,
+                         d_status=None, stream=None):
+    _check(lib().spa_gate_select_pack(C.byref(p), _ptr(x), _ptr(w_g), float(b_g), _ptr(s_up), _ptr(scores), _ptr(mask),
+                                      _ptr(y), _ptr(x_packed), _ptr(idx), _ptr(inv), _ptr(cu_seqlens), _ptr(pack_state),
+                                      _ptr(d_status), _stream(stream)), "spa_gate_select_pack")
 
 
 def spa_select_pack(p, x, mask, scores, x_packed, idx, inv, cu_seqlens, d_status=None, stream=None):

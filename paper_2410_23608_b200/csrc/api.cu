@@ -98,6 +98,32 @@ int spa_select_pack(const spa_params* p, const void* x, const uint8_t* mask, con
   return launch_select_pack(*p, x, mask, scores, nullptr, x_packed, idx, inv, cu_seqlens, d_status, (cudaStream_t)stream);
 }
 
+size_t spa_pack_state_bytes(const spa_params* p) {
+  if (check_params(p) != SPA_OK) return 0;
+  return gate_pack_state_bytes(*p);
+}
+
+int spa_gate_select_pack_supported(const spa_params* p) {
+  return (check_params(p) == SPA_OK && gate_pack_supported(*p)) ? 1 : 0;
+}
+
+int spa_gate_select_pack(const spa_params* p, const void* x, const void* w_g, float b_g, const float* s_up,
+                         float* scores, uint8_t* mask, void* y, void* x_packed, int32_t* idx, int32_t* inv,
+                         int32_t* cu_seqlens, void* pack_state, int32_t* d_status, void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  SPA_PTR(x); SPA_PTR(w_g); SPA_PTR(scores); SPA_PTR(mask); SPA_PTR(x_packed); SPA_PTR(idx); SPA_PTR(cu_seqlens);
+  SPA_PTR(pack_state); SPA_OPT_PTR(s_up); SPA_OPT_PTR(inv); SPA_OPT_PTR(y);
+  if (!gate_pack_supported(*p)) return SPA_ERR_UNSUPPORTED;
+  if (p->B == 0) {
+    cudaError_t e = cudaMemsetAsync(cu_seqlens, 0, sizeof(int32_t), (cudaStream_t)stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "spa_gate_select_pack"); return SPA_ERR_CUDA; }
+    return SPA_OK;
+  }
+  return launch_gate_pack(*p, x, w_g, b_g, s_up, scores, mask, y == x ? nullptr : y, x_packed, idx, inv, cu_seqlens,
+                          pack_state, d_status, (cudaStream_t)stream);
+}
+
 int spa_select_pack_ordered(const spa_params* p, const void* x, const uint8_t* mask, const float* scores,
                             const int32_t* order, void* x_packed, int32_t* idx, int32_t* inv, int32_t* cu_seqlens,
                             int32_t* d_status, void* stream) {
@@ -440,10 +466,15 @@ int spa_block_fwd(const spa_params* p, const spa_block_buffers* b, void* stream)
   void* y = inplace ? const_cast<void*>(b->x) : b->y;
   SPA_REQUIRE(!inplace || b->y == nullptr || b->y == b->x, SPA_ERR_INVALID_ARG);
   // gate (Eq. 4) and hard selection; on the fused path it also writes the pass-through rows y = x
-  if (fused && !inplace) SPA_STEP(spa_gate_prefill(p, b->x, b->w_g, b->b_g, b->s_up, b->scores, b->mask, y, stream));
+  const bool one_pass = b->pack_state != nullptr && b->order == nullptr && gate_pack_supported(*p);
+  if (one_pass)  // gate, selection and packing read x once
+    SPA_STEP(spa_gate_select_pack(p, b->x, b->w_g, b->b_g, b->s_up, b->scores, b->mask, (fused && !inplace) ? y : nullptr,
+                                  b->x_packed, b->idx, b->inv, b->cu_seqlens, b->pack_state, b->d_status, stream));
+  else if (fused && !inplace) SPA_STEP(spa_gate_prefill(p, b->x, b->w_g, b->b_g, b->s_up, b->scores, b->mask, y, stream));
   else SPA_STEP(spa_gate(p, b->x, b->w_g, b->b_g, b->s_up, b->scores, b->mask, stream));
   // token packing
-  if (b->order == nullptr)
+  if (one_pass) {
+  } else if (b->order == nullptr)
     SPA_STEP(spa_select_pack(p, b->x, b->mask, b->scores, b->x_packed, b->idx, b->inv, b->cu_seqlens, b->d_status, stream));
   else
     SPA_STEP(spa_select_pack_ordered(p, b->x, b->mask, b->scores, b->order, b->x_packed, b->idx, b->inv, b->cu_seqlens,

@@ -84,6 +84,11 @@ def test_later_entry_points_validate_on_the_host(lib):
     assert L.spa_layer_norm_bwd(pp, None, None, None, None, None, None, None, None, None, None, None) == inv
     assert L.spa_gelu(pp, None, 256, None, None) == inv
     assert L.spa_gelu_bwd(pp, None, None, 256, None, None) == inv
+    assert L.spa_gate_select_pack(pp, None, None, 0.0, None, None, None, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_pack_state_bytes(pp) >= 16 + 4 and L.spa_pack_state_bytes(None) == 0
+    assert L.spa_gate_select_pack_supported(pp) == 1
+    wide = lib.make_params(2, 16, 2048, 32, "bf16")                 # 256 chunks per row: two-kernel path only
+    assert L.spa_gate_select_pack_supported(ctypes.byref(wide)) == 0
     empty = lib.SpaBlockBuffers()
     assert L.spa_block_fwd(pp, None, None) == inv and L.spa_block_bwd(pp, None, None) == inv
     assert L.spa_block_fwd(pp, ctypes.byref(empty), None) == inv      # no inputs: refused by the first call
