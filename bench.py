@@ -84,8 +84,8 @@ def work_model(cfg, cu):
     w["attn_bwd"] = dict(bytes=(3 + 1 + 1 + 3) * Np * C * es + 4 * H * Np, flops=10 * C * S2, exps=H * S2)
     for name, n_out in (("proj_bwd", C), ("qkv_bwd", 3 * C)):
         w[name + ".da"] = dict(bytes=(Np * n_out + n_out * C + Np * C) * es, flops=2 * Np * C * n_out)
-        w[name + ".dW"] = dict(bytes=(Np * n_out + Np * C) * es + 4 * n_out * C, flops=2 * Np * C * n_out)
-        w[name + ".db"] = dict(bytes=Np * n_out * es + 4 * n_out, flops=Np * n_out)
+        w[name + ".dW"] = dict(bytes=(Np * n_out + Np * C) * es + 4 * n_out * C + 4 * n_out,
+                               flops=2 * Np * C * n_out + Np * n_out)   # dW and db
     w["pack_bwd"] = dict(bytes=2 * Np * C * es + 4 * Np, flops=0)
     # fused unpack: the gate also writes y = x; the projection writes to the tokens (idx read per row)
     w["gate_prefill"] = dict(bytes=2 * BN * C * es + 5 * BN, flops=2 * BN * C)
@@ -95,8 +95,9 @@ def work_model(cfg, cu):
 
 
 def timing_units(L, blk, d, b_g):
-    """The block's calls as (name, thunk) pairs with the linear-layer gradients split into their three
-    products, so that each timed unit is one kernel (dW: the split-K product plus its fixed-order reduction)."""
+    """The block's calls as (name, thunk) pairs with the linear-layer gradients split the way the step issues them:
+    the input gradient, and the weight gradient together with the bias gradient (column sums taken from the tiles
+    that stream through the weight-gradient product; split-K product plus its fixed-order reduction)."""
     p, C = blk.p, blk.C
     fused = blk.fused
     units = []
@@ -130,13 +131,11 @@ def timing_units(L, blk, d, b_g):
 
     units += [
         ("proj_bwd.da", lin(blk.ao, d["W_o"], blk.dz, C, blk.dao, None, None)),
-        ("proj_bwd.dW", lin(blk.ao, d["W_o"], blk.dz, C, None, blk.dW_o, None)),
-        ("proj_bwd.db", lin(blk.ao, d["W_o"], blk.dz, C, None, None, blk.db_o)),
+        ("proj_bwd.dW", lin(blk.ao, d["W_o"], blk.dz, C, None, blk.dW_o, blk.db_o)),
         ("qkv_bwd.da", (lambda: L.spa_packed_linear_bwd_scatter(p, blk.xp, d["W_qkv"], blk.dqkv, C, 3 * C, blk.idx, blk.cu,
                                                                  blk.dX, None, None, None, blk.status))
          if fused else lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, blk.dxp, None, None)),
-        ("qkv_bwd.dW", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, blk.dW_qkv, None)),
-        ("qkv_bwd.db", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, None, blk.db_qkv)),
+        ("qkv_bwd.dW", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, blk.dW_qkv, blk.db_qkv)),
     ]
     if not fused:
         units.append(("pack_bwd", lambda: L.spa_select_pack_bwd(p, blk.dxp, d["dY"], blk.idx, blk.cu, blk.dX)))
@@ -273,7 +272,7 @@ def run_reference(args):
 class Workload:
     """Rotating buffer sets of one workload, its whole-step graphs and its per-unit timings."""
 
-    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=True):
+    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=False):
         from paper_2410_23608_b200.block import SpaBlock
         from spa_workloads import make_inputs, scaled_config
         self.torch, self.L, self.cfg = torch, L, cfg
@@ -449,7 +448,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="time the headline workload only")
     ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
-    ap.add_argument("--two-kernel-pack", action="store_true", help="gate and packing as two kernels instead of the one-pass call")
+    ap.add_argument("--one-pass-pack", action="store_true", help="gate, selection and packing as one kernel (spa_gate_select_pack) instead of two")
     ap.add_argument("--train", action="store_true", help="also time the trainable-selection calls (loss, gated pack backward, gate backward)")
     ap.add_argument("--layer", action="store_true", help="also time the whole pre-norm block (LayerNorm, SPA, feed-forward) and its new calls")
     args = ap.parse_args()
@@ -478,7 +477,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     cfg = get_config(args.config)
-    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=not args.two_kernel_pack)
+    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=args.one_pass_pack)
     stream = wl.stream
     n_sets = wl.n_sets
     wl.warm(args.warmup)
@@ -651,8 +650,8 @@ def main():
     if not args.no_cpu_baseline:
         cpu = cpu_baseline(cfg, wl.inps[0], make_inputs, scaled_config)
 
-    flop_units = ("gate_pack" if wl.sets[0][2].one_pass else "gate", "qkv", "attn_fwd", "proj", "attn_bwd", "proj_bwd.da", "proj_bwd.dW", "proj_bwd.db",
-                  "qkv_bwd.da", "qkv_bwd.dW", "qkv_bwd.db")
+    flop_units = ("gate_pack" if wl.sets[0][2].one_pass else "gate", "qkv", "attn_fwd", "proj", "attn_bwd", "proj_bwd.da", "proj_bwd.dW",
+                  "qkv_bwd.da", "qkv_bwd.dW")
     useful_flops = sum(work[k]["flops"] for k in flop_units)
     Np_head = wl.Np_sets[0]
     fused_head = wl.sets[0][2].fused
@@ -672,7 +671,7 @@ def main():
             if ci == args.config:
                 continue
             c2 = get_config(ci)
-            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=not args.two_kernel_pack)
+            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=args.one_pass_pack)
             w2.warm(20)
             steps2 = 200
             ms2 = w2.time_steps(steps2) / steps2

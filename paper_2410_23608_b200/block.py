@@ -20,7 +20,7 @@ class SpaBlock:
 
     def __init__(self, B: int, N: int, C: int, H: int, dtype: str, tau: float = 0.0, flags: int = 0,
                  capacity: Optional[int] = None, backward: bool = True, device: str = "cuda",
-                 fused: Optional[bool] = None, one_pass: bool = True):
+                 fused: Optional[bool] = None, one_pass: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("SpaBlock needs a CUDA device; there is no CPU path")
         L.lib()
@@ -57,7 +57,8 @@ class SpaBlock:
         # the weight gradients run on a second stream (owned by the library handle), with a scratch area of their own
         self.workspace_side = torch.empty(max(ws, 256), dtype=torch.uint8, device=dev) if (ws > 0 and backward) else None
         self._overlap = L.spa_overlap_create() if backward else None
-        # scratch of the one-pass gate + packing kernel: zeroed once here, the kernel leaves it zero
+        # one_pass: gate, selection and packing as one kernel (measured slower than the two kernels on the five
+        # workloads, so off unless asked for); its scratch is zeroed once here, the kernel leaves it zero
         self.one_pass = one_pass and L.spa_gate_select_pack_supported(self.p)
         self.pack_state = (torch.zeros(max(L.spa_pack_state_bytes(self.p), 256), dtype=torch.uint8, device=dev)
                            if self.one_pass else None)

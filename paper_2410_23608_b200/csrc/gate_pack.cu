@@ -4,14 +4,15 @@
 // A CTA owns a tile of consecutive tokens.  Each warp pulls its rows of x into registers with 16-byte streaming loads
 // (and, on request, writes the pass-through copy y = x from them), forms the gate logits, thresholds them, and the CTA
 // counts its selected tokens.  Where the tile's rows land in the packed buffer depends on the number of selected tokens
-// in all earlier tiles: tiles publish their counts in a small state array and obtain their exclusive prefix by
-// looking back over their predecessors' entries (aggregate of one tile, or inclusive prefix of everything up to it).
-// The selected rows then go from the registers straight to x_packed: x is read from memory exactly once.
+// in all earlier tiles: every tile publishes its count in a small state array as soon as it knows it, and obtains its
+// exclusive prefix by reading the counts of up to kWindow predecessors at once, all threads of the CTA polling in
+// parallel (one round trip to L2 when the others are ready), plus the published inclusive prefix of the tile before
+// that window.  The selected rows then go from the registers straight to x_packed: x is read from memory exactly once.
 //
-// Tiles are handed out by an atomic ticket, so every tile with a smaller number is already running when a tile looks
-// back; no CTA ever waits for one that has not started.  Every poll loop is bounded all the same: when it runs out the
-// kernel records SPA_ERR_TIMEOUT and returns without writing packed rows.  The state array must be zero when the
-// kernel starts; the CTA that finishes last puts it back to zero.
+// A CTA waits only for CTAs with smaller block indices, which the hardware dispatches first, so whatever it waits for
+// is running or done.  Every poll loop is bounded all the same: when one runs out the kernel records SPA_ERR_TIMEOUT
+// and returns without writing packed rows.  The state array must be zero when the kernel starts; the CTA that
+// finishes last puts it back to zero.
 #include "sm100_ptx.cuh"
 #include "spa_common.cuh"
 
@@ -20,10 +21,9 @@ namespace {
 
 constexpr int kGpThreads = 256;
 constexpr int kGpWarps = kGpThreads / 32;
-constexpr uint32_t kFlagAgg = 1u << 30;   // value = selected tokens of this tile
-constexpr uint32_t kFlagIncl = 2u << 30;  // value = selected tokens of this tile and all before it
-constexpr uint32_t kFlagMask = 3u << 30;
-constexpr int kStateHeader = 4;           // words: ticket counter, finished counter, two spare
+constexpr uint32_t kValid = 1u << 31;  // set in a published word; the low bits hold the count
+constexpr int kWindow = 4 * kGpThreads;   // predecessors whose counts a tile sums directly
+constexpr int kStateHeader = 4;           // words: finished counter, three spare; then counts[tiles], prefixes[tiles]
 
 __device__ __forceinline__ uint32_t ld_volatile(const uint32_t* p) {
   uint32_t v;
@@ -50,23 +50,16 @@ gate_pack_kernel(const uint4* __restrict__ x16, const T* __restrict__ w_g, float
                  float tau, int rows, int N, int B, int Q, int capacity, float* __restrict__ scores,
                  uint8_t* __restrict__ mask, uint4* __restrict__ y16, uint4* __restrict__ xp16,
                  int32_t* __restrict__ idx, int32_t* __restrict__ inv, int32_t* __restrict__ cu, uint32_t* state,
-                 int n_tiles, int32_t* d_status) {
+                 int n_tiles, int max_tiles, int32_t* d_status) {
   constexpr int E = Vec16<T>::kElems;
   constexpr int kTile = kGpWarps * kRows;
   __shared__ __align__(16) float w_s[32 * kChunks * E];
-  __shared__ int s_tile, s_base, s_abort, s_last;
-  __shared__ int warp_sel[kGpWarps];
+  __shared__ int s_last;
+  __shared__ int warp_sel[kGpWarps], warp_part[kGpWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_entry();
-  if (tid == 0) {
-    s_tile = (int)atomicAdd(&state[0], 1u);
-    s_abort = 0;
-    s_last = 0;
-  }
-  for (int c = tid; c < 32 * kChunks * E; c += kGpThreads) w_s[c] = c < Q * E ? to_f32<T>(w_g[c]) : 0.f;
-  __syncthreads();
-  const int tile = s_tile;
+  const int tile = blockIdx.x;
   const int row0 = tile * kTile + warp * kRows;
+  pdl_entry();
 
   // ---- this warp's rows into registers (and out again as the pass-through copy)
   uint4 v[kRows][kChunks];
@@ -89,6 +82,8 @@ gate_pack_kernel(const uint4* __restrict__ x16, const T* __restrict__ w_g, float
       }
     }
   }
+  for (int c = tid; c < 32 * kChunks * E; c += kGpThreads) w_s[c] = c < Q * E ? to_f32<T>(w_g[c]) : 0.f;
+  __syncthreads();
   // ---- gate logits (Eq. 4) and the selection
   float acc[kRows];
 #pragma unroll
@@ -135,44 +130,39 @@ gate_pack_kernel(const uint4* __restrict__ x16, const T* __restrict__ w_g, float
     total += warp_sel[w];
   }
 
-  // ---- exclusive prefix of this tile: publish the tile's count, then look back
-  if (warp == 0) {
-    uint32_t* tiles = state + kStateHeader;
-    if (lane == 0) st_volatile(tiles + tile, (tile == 0 ? kFlagIncl : kFlagAgg) | (uint32_t)total);
-    int excl = 0;
-    bool ok = true;
-    for (int j = tile - 1; j >= 0 && ok; j -= 32) {
-      const int t = j - lane;  // lane 0 looks at the nearest predecessor
-      uint32_t wv = kFlagIncl;  // tiles before the first: an inclusive prefix of zero
-      if (t >= 0) {
-        wv = 0u;
-        for (uint32_t i = 0; i < ptx::kWaitLimit; ++i) {
-          wv = ld_volatile(tiles + t);
-          if (wv & kFlagMask) break;
-        }
-      }
-      if (__any_sync(0xffffffffu, (wv & kFlagMask) == 0u)) { ok = false; break; }
-      const unsigned incl = __ballot_sync(0xffffffffu, (wv & kFlagMask) == kFlagIncl);
-      const int stop = incl ? __ffs(incl) - 1 : 31;  // nearest entry that already covers everything before it
-      const int part = lane <= stop ? (int)(wv & ~kFlagMask) : 0;
-      excl += (int)__reduce_add_sync(0xffffffffu, (unsigned)part);
-      if (incl) break;
-    }
-    if (lane == 0) {
-      if (!ok) {
-        record_status(d_status, SPA_ERR_TIMEOUT);
-        s_abort = 1;
-      } else if (tile > 0) {
-        st_volatile(tiles + tile, kFlagIncl | (uint32_t)(excl + total));
-      }
-      s_base = excl;
-    }
+  // ---- exclusive prefix of this tile: publish the tile's count, then sum the predecessors' counts
+  uint32_t* counts = state + kStateHeader;
+  uint32_t* prefixes = counts + max_tiles;
+  if (tid == 0) st_volatile(counts + tile, kValid | (uint32_t)total);
+  const int lo = tile > kWindow ? tile - kWindow : 0;
+  int part = 0;
+  bool ok = true;
+  for (int t = lo + tid; t < tile; t += kGpThreads) {
+    uint32_t wv = 0u;
+    for (uint32_t i = 0; i < ptx::kWaitLimit && !(wv & kValid); ++i) wv = ld_volatile(counts + t);
+    ok = ok && (wv & kValid);
+    part += (int)(wv & ~kValid);
   }
-  __syncthreads();
+  if (lo > 0 && tid == kGpThreads - 1) {  // everything before the window: the inclusive prefix of tile lo - 1
+    uint32_t wv = 0u;
+    for (uint32_t i = 0; i < ptx::kWaitLimit && !(wv & kValid); ++i) wv = ld_volatile(prefixes + lo - 1);
+    ok = ok && (wv & kValid);
+    part += (int)(wv & ~kValid);
+  }
+  part = (int)__reduce_add_sync(0xffffffffu, (unsigned)part);
+  if (lane == 0) warp_part[warp] = part;
+  const bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
+  int excl = 0;
+#pragma unroll
+  for (int w = 0; w < kGpWarps; ++w) excl += warp_part[w];
+  if (tid == 0) {
+    if (all_ok) st_volatile(prefixes + tile, kValid | (uint32_t)(excl + total));
+    else record_status(d_status, SPA_ERR_TIMEOUT);
+  }
 
   // ---- indices, offsets and the packed rows
-  if (!s_abort) {
-    const int base = s_base + before;
+  if (all_ok) {
+    const int base = excl + before;
 #pragma unroll
     for (int k = 0; k < kRows; ++k) {
       const int r = row0 + k;
@@ -197,16 +187,16 @@ gate_pack_kernel(const uint4* __restrict__ x16, const T* __restrict__ w_g, float
         }
       }
     }
-    if (tid == 0 && tile == n_tiles - 1) cu[B] = s_base + total;
+    if (tid == 0 && tile == n_tiles - 1) cu[B] = excl + total;
   }
 
   // ---- the CTA that finishes last leaves the state array zeroed for the next call
   __syncthreads();
-  if (tid == 0) s_last = atomicAdd(&state[1], 1u) == (uint32_t)(n_tiles - 1) ? 1 : 0;
+  if (tid == 0) s_last = atomicAdd(&state[0], 1u) == (uint32_t)(n_tiles - 1) ? 1 : 0;
   __syncthreads();
   if (s_last) {
-    for (int i = tid; i < n_tiles; i += kGpThreads) state[kStateHeader + i] = 0u;
-    if (tid == 0) { state[0] = 0u; state[1] = 0u; }
+    for (int i = tid; i < n_tiles; i += kGpThreads) { counts[i] = 0u; prefixes[i] = 0u; }
+    if (tid == 0) state[0] = 0u;
   }
 }
 
@@ -216,6 +206,9 @@ inline int chunks_per_lane(const spa_params& p) {
   const int Q = p.C * (p.dtype == SPA_F32 ? 4 : 2) / 16;
   return (Q + 31) / 32;
 }
+
+// tiles of the smallest tile size (32 tokens): the length of each of the two arrays in the state
+inline int max_tiles_of(const spa_params& p) { return (int)(((long long)p.B * p.N + 31) / 32); }
 
 template <typename T, int kChunks>
 int launch_one(const spa_params& p, const void* x, const void* w_g, float b_g, const float* s_up, float* scores,
@@ -228,11 +221,11 @@ int launch_one(const spa_params& p, const void* x, const void* w_g, float b_g, c
   if (p.flags & SPA_FLAG_GATE_SCALE)
     launch_pdl(gate_pack_kernel<T, kChunks, kRows, true>, n_tiles, kGpThreads, 0, st, (const uint4*)x, (const T*)w_g, b_g,
                s_up, p.tau, rows, p.N, p.B, Q, p.capacity, scores, mask, (uint4*)y, (uint4*)xp, idx, inv, cu,
-               (uint32_t*)state, n_tiles, d_status);
+               (uint32_t*)state, n_tiles, max_tiles_of(p), d_status);
   else
     launch_pdl(gate_pack_kernel<T, kChunks, kRows, false>, n_tiles, kGpThreads, 0, st, (const uint4*)x, (const T*)w_g, b_g,
                s_up, p.tau, rows, p.N, p.B, Q, p.capacity, scores, mask, (uint4*)y, (uint4*)xp, idx, inv, cu,
-               (uint32_t*)state, n_tiles, d_status);
+               (uint32_t*)state, n_tiles, max_tiles_of(p), d_status);
   SPA_CUDA_CHECK_LAUNCH("gate_pack_kernel");
   return SPA_OK;
 }
@@ -254,10 +247,9 @@ int launch_typed(const spa_params& p, const void* x, const void* w_g, float b_g,
 
 bool gate_pack_supported(const spa_params& p) { return chunks_per_lane(p) <= 4; }
 
-// state words: header + one per tile of the smallest tile size (32 tokens)
+// state words: header, then a count and an inclusive prefix per tile
 size_t gate_pack_state_bytes(const spa_params& p) {
-  const size_t tiles = ((size_t)p.B * p.N + 31) / 32;
-  return ((kStateHeader + tiles) * sizeof(uint32_t) + 255) & ~(size_t)255;
+  return ((kStateHeader + 2 * (size_t)max_tiles_of(p)) * sizeof(uint32_t) + 255) & ~(size_t)255;
 }
 
 int launch_gate_pack(const spa_params& p, const void* x, const void* w_g, float b_g, const float* s_up, float* scores,
