@@ -119,6 +119,17 @@ int spa_gate_select_pack(const spa_params* p, const void* x, const void* w_g, fl
                          float* scores, uint8_t* mask, void* y, void* x_packed, int32_t* idx, int32_t* inv,
                          int32_t* cu_seqlens, void* pack_state, int32_t* d_status, void* stream);
 
+/* Attention segments of the paper's own batching (Sec. 3.2 "Token Packing": the selected tokens fill containers of a
+ * fixed length L = M^2, and the mask keeps a token from attending to tokens of other images): the packed buffer is cut
+ * at every multiple of L and at every image boundary.  seg_offsets (device, int32[spa_container_max_segments() + 1])
+ * receives the distinct cut positions in ascending order - 0 first, N_p last - padded with copies of N_p (empty
+ * segments).  Pass it to the attention calls with n_seg = spa_container_max_segments(p, L) = B + capacity / L: nothing
+ * is read back to the host, so the container variant runs inside the same recorded step as everything else.
+ * B is limited to 4095 images (else SPA_ERR_UNSUPPORTED); L >= 1. */
+int32_t spa_container_max_segments(const spa_params* p, int32_t L);
+int spa_container_offsets(const spa_params* p, const int32_t* cu_seqlens, int32_t L, int32_t* seg_offsets,
+                          void* stream);
+
 /* QKV projection on the packed tokens (the 3LC^2 term of Eq. 9):
  *   qkv[i][j] = b_qkv[j] + sum_c W_qkv[j][c] * x_packed[i][c],  i < N_p, j < 3C.
  * W_qkv: T[3C][C]; b_qkv: T[3C] or NULL; qkv: T[capacity][3C] out. */

@@ -33,7 +33,7 @@ EXPORTS = (
     "spa_packed_linear", "spa_layer_norm", "spa_layer_norm_bwd", "spa_gelu", "spa_gelu_bwd",
     "spa_overlap_create", "spa_overlap_destroy", "spa_block_fwd", "spa_block_bwd",
     "spa_probe_exp2", "spa_probe_wait_expiry", "spa_pack_state_bytes", "spa_gate_select_pack_supported",
-    "spa_gate_select_pack",
+    "spa_gate_select_pack", "spa_container_max_segments", "spa_container_offsets",
 )
 
 
@@ -123,6 +123,8 @@ def lib() -> C.CDLL:
         L.spa_pack_state_bytes.argtypes = [pp]
         L.spa_gate_select_pack_supported.argtypes = [pp]
         L.spa_gate_select_pack.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.spa_container_max_segments.argtypes = [pp, i32]
+        L.spa_container_offsets.argtypes = [pp, vp, i32, vp, vp]
         L.spa_probe_exp2.argtypes = [i32, i32, vp, C.POINTER(C.c_ulonglong), vp]
         L.spa_probe_wait_expiry.argtypes = [i32, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
@@ -182,6 +184,15 @@ def spa_gate_select_pack(p, x, w_g, b_g, s_up, scores, mask, y, x_packed, idx, i
     _check(lib().spa_gate_select_pack(C.byref(p), _ptr(x), _ptr(w_g), float(b_g), _ptr(s_up), _ptr(scores), _ptr(mask),
                                       _ptr(y), _ptr(x_packed), _ptr(idx), _ptr(inv), _ptr(cu_seqlens), _ptr(pack_state),
                                       _ptr(d_status), _stream(stream)), "spa_gate_select_pack")
+
+
+def spa_container_max_segments(p, L) -> int:
+    return int(lib().spa_container_max_segments(C.byref(p), int(L)))
+
+
+def spa_container_offsets(p, cu_seqlens, L, seg_offsets, stream=None):
+    _check(lib().spa_container_offsets(C.byref(p), _ptr(cu_seqlens), int(L), _ptr(seg_offsets), _stream(stream)),
+           "spa_container_offsets")
 
 
 def spa_select_pack(p, x, mask, scores, x_packed, idx, inv, cu_seqlens, d_status=None, stream=None):

@@ -140,6 +140,19 @@ int spa_select_pack_ordered(const spa_params* p, const void* x, const uint8_t* m
   return launch_select_pack(*p, x, mask, scores, order, x_packed, idx, inv, cu_seqlens, d_status, (cudaStream_t)stream);
 }
 
+int32_t spa_container_max_segments(const spa_params* p, int32_t L) {
+  if (check_params(p) != SPA_OK || L < 1) return 0;
+  return p->B + p->capacity / L;
+}
+
+int spa_container_offsets(const spa_params* p, const int32_t* cu_seqlens, int32_t L, int32_t* seg_offsets,
+                          void* stream) {
+  int rc = check_params(p);
+  if (rc != SPA_OK) return rc;
+  if (cu_seqlens == nullptr || seg_offsets == nullptr || L < 1) return SPA_ERR_INVALID_ARG;
+  return launch_container_offsets(*p, cu_seqlens, L, spa_container_max_segments(p, L), seg_offsets, (cudaStream_t)stream);
+}
+
 int spa_packed_qkv(const spa_params* p, const void* x_packed, const void* W_qkv, const void* b_qkv,
                    const int32_t* cu_seqlens, void* qkv, int32_t* d_status, void* stream) {
   int rc = check_params(p);

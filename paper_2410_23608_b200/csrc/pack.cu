@@ -265,7 +265,78 @@ copy_chunks_kernel(const uint4* __restrict__ src16, uint4* __restrict__ dst16, l
 
 template <typename T> int chunks_per_row(int C) { return C / Vec16<T>::kElems; }
 
+
+// ------------------------------------------------------------------------------ container cuts
+// Attention segments of the paper's fixed-length containers (Sec. 3.2 "Token Packing": the packed tokens fill
+// containers of L tokens, and the mask keeps a token from attending to other images): the packed buffer is cut at
+// every multiple of L and at every image boundary.  out receives the distinct cut positions in ascending order,
+// 0 first and N_p last, followed by copies of N_p up to n_max + 1 entries (empty segments, which the attention
+// kernels skip), so that the caller can pass the upper bound n_max as the segment count without reading anything back.
+// A cut position's rank is the number of multiples of L below it plus the number of distinct image boundaries below
+// it that are not multiples of L; one CTA computes the latter as a prefix sum over the B + 1 offsets.
+constexpr int kCutThreads = 1024;
+constexpr int kCutMaxOffsets = 4096;  // B + 1 offsets and their prefix counts are held in shared memory
+
+__global__ void __launch_bounds__(kCutThreads)
+container_offsets_kernel(const int32_t* __restrict__ cu, int B, int L, int n_max, int32_t* __restrict__ out) {
+  pdl_entry();
+  __shared__ int32_t cu_s[kCutMaxOffsets];
+  __shared__ int32_t pre_s[kCutMaxOffsets + 1];  // pre_s[b] = distinct non-multiple offsets among cu[0..b)
+  __shared__ int warp_tot[kCutThreads / 32];
+  __shared__ int carry_s;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int n = B + 1;
+  for (int i = tid; i < n; i += kCutThreads) cu_s[i] = __ldg(cu + i);
+  if (tid == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < n; base += kCutThreads) {
+    const int b = base + tid;
+    const int c = b < n ? cu_s[b] : 0;
+    const int flag = (b < n && c % L != 0 && (b == 0 || c != cu_s[b - 1])) ? 1 : 0;
+    int incl = flag;  // inclusive scan inside the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    int before = carry_s;
+    for (int w = 0; w < wid; ++w) before += warp_tot[w];
+    if (b < n) pre_s[b] = before + incl - flag;
+    __syncthreads();
+    if (tid == kCutThreads - 1) carry_s = before + incl;
+    __syncthreads();
+  }
+  if (tid == 0) pre_s[n] = carry_s;
+  __syncthreads();
+  const int Np = cu_s[B];
+  const int K = Np / L;                 // multiples 0, L, ..., K L
+  const int total = K + 1 + pre_s[n];   // distinct cut positions
+  for (int b = tid; b < n; b += kCutThreads) {
+    const int c = cu_s[b];
+    if (c % L != 0 && (b == 0 || c != cu_s[b - 1])) out[(c + L - 1) / L + pre_s[b]] = c;
+  }
+  for (int k = tid; k <= K; k += kCutThreads) {
+    const int v = k * L;
+    int lo = 0, hi = n;  // first index with cu_s[index] >= v
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (cu_s[mid] < v) lo = mid + 1; else hi = mid;
+    }
+    out[k + pre_s[lo]] = v;
+  }
+  for (int j = total + tid; j <= n_max; j += kCutThreads) out[j] = Np;
+}
+
 }  // namespace
+
+int launch_container_offsets(const spa_params& p, const int32_t* cu, int L, int n_max, int32_t* out, cudaStream_t st) {
+  if (p.B + 1 > kCutMaxOffsets) return SPA_ERR_UNSUPPORTED;
+  launch_pdl(container_offsets_kernel, 1, kCutThreads, 0, st, cu, p.B, L, n_max, out);
+  SPA_CUDA_CHECK_LAUNCH("container_offsets_kernel");
+  return SPA_OK;
+}
 
 int launch_select_pack(const spa_params& p, const void* x, const uint8_t* mask, const float* scores,
                        const int32_t* order, void* xp, int32_t* idx, int32_t* inv, int32_t* cu, int32_t* d_status,

@@ -167,6 +167,7 @@ size_t gate_pack_state_bytes(const spa_params& p);
 int launch_gate_pack(const spa_params& p, const void* x, const void* w_g, float b_g, const float* s_up, float* scores,
                      uint8_t* mask, void* y, void* xp, int32_t* idx, int32_t* inv, int32_t* cu, void* state,
                      int32_t* d_status, cudaStream_t st);
+int launch_container_offsets(const spa_params& p, const int32_t* cu, int L, int n_max, int32_t* out, cudaStream_t st);
 int launch_unpack_scatter(const spa_params& p, const void* z, const void* x, const int32_t* idx,
                           const int32_t* inv, const int32_t* cu, void* y, cudaStream_t st);
 int launch_unpack_scatter_bwd(const spa_params& p, const void* dY, const int32_t* idx, const int32_t* inv,

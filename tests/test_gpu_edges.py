@@ -350,3 +350,36 @@ def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
     fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
     assert_close(host(y), fwd["y"], cfg.dtype, "y after an expired wait")
     assert blk.read_status() == 0 and lib.spa_read_status(status) == 0
+
+
+@pytest.mark.parametrize("L_c,counts", [(49, [0, 1, 49, 48, 50, 98, 0, 0, 147, 5]), (16, [3, 16, 0, 31, 33, 1]),
+                                        (7, [0, 0, 0]), (1, [2, 0, 3]), (64, [197] * 9)])
+def test_container_cuts_on_the_device(L_c, counts):
+    """spa_container_offsets against the oracle's container_cuts: the distinct cuts first, copies of N_p after them,
+    and attention over the padded list (the upper bound given as the segment count) equal to the oracle's."""
+    lib = L()
+    B, N, C, H, dt = len(counts), 200, 128, 2, "bf16"
+    cu_np = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    Np = int(cu_np[-1])
+    blk = block(B, N, C, H, dt)
+    p = blk.p
+    n_max = lib.spa_container_max_segments(p, L_c)
+    assert n_max == B + (B * N) // L_c
+    out = torch.full((n_max + 1,), -5, dtype=torch.int32, device="cuda")
+    lib.spa_container_offsets(p, torch.from_numpy(cu_np).cuda(), L_c, out)
+    got = out.cpu().numpy()
+    ref = O.container_cuts(cu_np, L_c)
+    assert len(ref) <= n_max + 1
+    assert np.array_equal(got[:len(ref)], ref)
+    assert np.all(got[len(ref):] == Np)
+    if Np == 0:
+        return
+    rng = np.random.default_rng(L_c)
+    qkv_r = round_to(rng.normal(size=(Np, 3 * C)), dt)
+    buf = np.zeros((blk.cap, 3 * C))
+    buf[:Np] = qkv_r
+    lib.spa_packed_attention_fwd(p, dev(buf, dt), out, n_max, blk.ao, blk.lse, blk.status)
+    ao_ref, lse_ref = O.attention_fwd(qkv_r, ref, H)
+    assert_close(host(blk.ao)[:Np], ao_ref, dt, "attention over device-built containers")
+    assert np.abs(host(blk.lse)[:, :Np] - lse_ref).max() <= TOL[dt]["lse"]
+    assert blk.read_status() == 0

@@ -290,8 +290,10 @@ def guarded(shape, dtype, guard_rows=2):
     return inner, intact
 
 
-@pytest.mark.parametrize("ci,flags", [(1, 0), (2, 0), (2, 32), (2, 1)])   # 32: separate scatter kernels; 1: residual
-def test_block_calls_alone_with_guard_bands(ci, flags):
+# flags 32: separate scatter kernels; 1: residual.  one_pass: gate, selection and packing as one kernel
+@pytest.mark.parametrize("ci,flags,one_pass", [(1, 0, False), (2, 0, False), (2, 32, False), (2, 1, False),
+                                               (1, 0, True), (2, 0, True), (4, 1, True)])
+def test_block_calls_alone_with_guard_bands(ci, flags, one_pass):
     """One forward and one backward pass through nothing but spa_block_fwd / spa_block_bwd (no Python class in
     between), every buffer the library writes framed by guard rows that must come back untouched."""
     from paper_2410_23608_b200 import binding as L
@@ -313,6 +315,9 @@ def test_block_calls_alone_with_guard_bands(ci, flags):
     ws_bytes = max(L.spa_workspace_bytes(p), 256)
     buf["workspace"], checks["workspace"] = guarded((ws_bytes,), u8)
     buf["workspace_side"], checks["workspace_side"] = guarded((ws_bytes,), u8)
+    if one_pass:
+        buf["pack_state"], checks["pack_state"] = guarded((max(L.spa_pack_state_bytes(p), 256),), u8)
+        buf["pack_state"].zero_()
     status = torch.zeros(4, dtype=i32, device="cuda")
     ov = L.spa_overlap_create()
     try:
@@ -324,6 +329,8 @@ def test_block_calls_alone_with_guard_bands(ci, flags):
     finally:
         L.spa_overlap_destroy(ov)
     assert L.spa_read_status(status) == 0
+    if one_pass:
+        assert not buf["pack_state"].any()          # the kernel leaves its scratch zeroed
     touched = [name for name, ok in checks.items() if not ok()]
     assert not touched, f"writes outside the buffer: {touched}"
     Np = int(fwd["cu_seqlens"][-1])
