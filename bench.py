@@ -298,11 +298,11 @@ class Workload:
             self.step_graphs.append(g)
             self.launches_per_step = n
 
-    def step_fn(self, s, backward, overlap=True):
+    def step_fn(self, s, backward, overlap=True, container_len=0):
         inp, d, blk = self.sets[s]
 
         def run():
-            blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"])
+            blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"], container_len=container_len)
             if backward:
                 blk.backward(d["dY"], overlap=overlap)
         return run
@@ -356,6 +356,16 @@ class Workload:
         torch.cuda.synchronize()
         t = [ev[r].elapsed_time(ev[r + 1]) / calls_per_replay for r in range(replays)]
         return statistics.median(t), min(t)
+
+    def containers_ms(self, container_len, replays):
+        """Whole step (forward + backward) with the paper's own batching: attention limited to containers of
+        `container_len` tokens, their cuts built on the device inside the step.  Median per step in ms."""
+        fns = [self.step_fn(s, True, container_len=container_len) for s in range(self.n_sets)]
+        for f in fns:
+            f()
+        self.torch.cuda.synchronize()
+        g, _ = self.capture(fns)
+        return self.time_graph(g, self.n_sets, max(20, replays // 4))[0]
 
     def forward_only_ms(self, replays):
         fns = [self.step_fn(s, False) for s in range(self.n_sets)]
@@ -558,6 +568,7 @@ def main():
     per_call, work, Np0, S2 = wl.per_call(pk, exp_rate)
     roofline = roofline_of(cfg, per_call, work, pk)
     fwd_ms = wl.forward_only_ms(UNIT_REPLAYS)
+    cont_ms = wl.containers_ms(49, UNIT_REPLAYS) if (args.config in (3, 4) and cfg.dtype == "bf16") else None
     reps = 50
 
     train = None
@@ -663,6 +674,8 @@ def main():
                    kernels_per_step=wl.launches_per_step, dominant_unit=roofline["kernel"],
                    dominant_bound=roofline["bound"], dominant_us=roofline["us_per_launch"], dominant_frac=roofline["frac"],
                    traffic=roofline["traffic"], useful_tflops=useful_flops / (ms_per_step * 1e-3) / 1e12)
+    if cont_ms is not None:   # the paper's containers of L = 7 x 7 tokens (cost linear in N, Eq. 9)
+        summary["containers_L49_ms_per_step"] = cont_ms
     per_config[cfg.name] = summary
     if not args.no_per_config:
         del wl
@@ -679,6 +692,7 @@ def main():
             r2 = roofline_of(c2, pc2, work2, pk)
             f2 = w2.forward_only_ms(UNIT_REPLAYS)
             uf2 = sum(work2[k]["flops"] for k in flop_units)
+            c2_ms = w2.containers_ms(49, UNIT_REPLAYS) if ci in (3, 4) else None
             per_config[c2.name] = dict(
                 ms_per_step=ms2, tokens_per_s=w2.tokens_per_step(steps2) / (ms2 * 1e-3), forward_only_ms=f2,
                 forward_only_tokens_per_s=w2.Np_sets[0] / (f2 * 1e-3), selected_tokens=w2.Np_sets[0],
@@ -686,6 +700,8 @@ def main():
                 dominant_us=r2["us_per_launch"], dominant_frac=r2["frac"], traffic=r2["traffic"],
                 useful_tflops=uf2 / (ms2 * 1e-3) / 1e12, steps=steps2,
                 per_call={k: dict(us=v["us"], bound=v["bound"], frac=v["frac"]) for k, v in pc2.items()})
+            if c2_ms is not None:
+                per_config[c2.name]["containers_L49_ms_per_step"] = c2_ms
             del w2
             torch.cuda.empty_cache()
 

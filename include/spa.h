@@ -383,6 +383,10 @@ typedef struct spa_block_buffers {
   float* db_g;                /* float[1] or NULL                                                    */
   float* loss;                /* float[1] or NULL                                                    */
   void* train_workspace;      /* spa_train_workspace_bytes()                                         */
+  /* the paper's containers (Sec. 3.2 "Token Packing") */
+  int32_t container_len;      /* L > 0: spa_block_fwd fills seg_offsets (which must then be a writable
+                                 int32[spa_container_max_segments(p, L) + 1]) with the container cuts of the
+                                 selection it has just packed and both passes use them; n_seg is ignored */
 } spa_block_buffers;
 
 /* A non-blocking stream and two events on the current device (host-side objects, no device memory).  Create one

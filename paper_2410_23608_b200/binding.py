@@ -65,7 +65,7 @@ class SpaBlockBuffers(C.Structure):
                 ("pack_state", C.c_void_p), ("overlap", C.c_void_p), ("d_status", C.c_void_p),
                 ("trainable", C.c_int32), ("labels", C.c_void_p), ("alpha", C.c_float), ("ds", C.c_void_p),
                 ("ds_up", C.c_void_p), ("dw_g", C.c_void_p), ("db_g", C.c_void_p), ("loss", C.c_void_p),
-                ("train_workspace", C.c_void_p)]
+                ("train_workspace", C.c_void_p), ("container_len", C.c_int32)]
 
 
 def make_params(B, N, Cc, H, dtype, capacity=None, flags=0, tau=0.0, softmax_scale=0.0) -> SpaParams:

@@ -75,6 +75,8 @@ class SpaBlock:
         self._saved = None            # (W_qkv, W_o) of the last forward()
         self._seg = (self.cu, B)      # attention segments: the images, unless forward() is given others
         self._keep = None             # tensors of the last call that the enqueued work still reads
+        self._container_len = 0       # > 0: the library builds the container cuts itself (forward(container_len=L))
+        self.container_seg = None
 
     def __del__(self):
         try:
@@ -89,18 +91,26 @@ class SpaBlock:
         seg, n_seg = self._seg
         f = dict(scores=self.scores, mask=self.mask, cu_seqlens=self.cu, idx=self.idx, inv=self.inv, x_packed=self.xp,
                  qkv=self.qkv, attn_out=self.ao, lse=self.lse, z=self.z, workspace=self.workspace, d_status=self.status,
-                 pack_state=self.pack_state,
+                 pack_state=self.pack_state, container_len=self._container_len,
                  seg_offsets=None if seg is self.cu else seg, n_seg=n_seg)
         f.update(extra)
         return L.block_buffers(**f)
 
     # ------------------------------------------------------------------ forward
-    def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None, order=None, seg_offsets=None):
+    def forward(self, x, w_g, b_g: float, W_qkv, b_qkv, W_o, b_o, s_up=None, y=None, order=None, seg_offsets=None,
+                container_len: int = 0):
         """`order` (int32 [N] on the device): visiting order of each image's tokens for the packing (a shifted
-        feature map); `seg_offsets` (int32, ascending, ending at N_p): attention segments other than the images,
-        e.g. the container cut; the backward pass uses the same segments."""
+        feature map); `seg_offsets` (int32, ascending, ending at N_p): attention segments other than the images;
+        `container_len` = L > 0: the paper's containers, their cuts built on the device by the library (the segment
+        array is owned here).  The backward pass uses the same segments."""
         inplace = bool(self.p.flags & L.SPA_FLAG_INPLACE)
         y = x if inplace else (self.y if y is None else y)
+        self._container_len = int(container_len)
+        if container_len > 0:
+            n_max = L.spa_container_max_segments(self.p, container_len)
+            if self.container_seg is None or self.container_seg.numel() != n_max + 1:
+                self.container_seg = torch.zeros(n_max + 1, dtype=torch.int32, device=self.cu.device)
+            seg_offsets = self.container_seg
         self._seg = (self.cu, self.B) if seg_offsets is None else (seg_offsets, int(seg_offsets.numel()) - 1)
         self._saved = (W_qkv, W_o)
         self._keep = (x, w_g, W_qkv, b_qkv, W_o, b_o, s_up, order, seg_offsets, y)

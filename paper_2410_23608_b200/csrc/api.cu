@@ -492,9 +492,14 @@ int spa_block_fwd(const spa_params* p, const spa_block_buffers* b, void* stream)
   else
     SPA_STEP(spa_select_pack_ordered(p, b->x, b->mask, b->scores, b->order, b->x_packed, b->idx, b->inv, b->cu_seqlens,
                                      b->d_status, stream));
+  if (b->container_len > 0) {  // the paper's containers: cuts built on the device from the selection just packed
+    SPA_REQUIRE(b->seg_offsets != nullptr, SPA_ERR_INVALID_ARG);
+    SPA_STEP(spa_container_offsets(p, b->cu_seqlens, b->container_len, const_cast<int32_t*>(b->seg_offsets), stream));
+  }
   SPA_STEP(spa_packed_qkv(p, b->x_packed, b->W_qkv, b->b_qkv, b->cu_seqlens, b->qkv, b->d_status, stream));
   const int32_t* seg = b->seg_offsets != nullptr ? b->seg_offsets : b->cu_seqlens;
-  const int32_t n_seg = b->seg_offsets != nullptr ? b->n_seg : p->B;
+  const int32_t n_seg = b->container_len > 0 ? spa_container_max_segments(p, b->container_len)
+                                             : (b->seg_offsets != nullptr ? b->n_seg : p->B);
   SPA_STEP(spa_packed_attention_fwd(p, b->qkv, seg, n_seg, b->attn_out, b->lse, b->d_status, stream));
   if (fused) return spa_packed_proj_scatter(p, b->attn_out, b->W_o, b->b_o, b->idx, b->cu_seqlens, y, b->d_status, stream);
   SPA_STEP(spa_packed_proj(p, b->attn_out, b->W_o, b->b_o, b->cu_seqlens, b->z, b->d_status, stream));
@@ -513,7 +518,9 @@ int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream)
   SPA_REQUIRE(ov == nullptr || b->workspace_side != nullptr || spa_workspace_bytes(p) == 0, SPA_ERR_INVALID_ARG);
   const bool fused = block_fused(p) && !b->trainable;
   const int32_t* seg = b->seg_offsets != nullptr ? b->seg_offsets : b->cu_seqlens;
-  const int32_t n_seg = b->seg_offsets != nullptr ? b->n_seg : p->B;
+  const int32_t n_seg = (b->container_len > 0 && b->seg_offsets != nullptr)
+                            ? spa_container_max_segments(p, b->container_len)
+                            : (b->seg_offsets != nullptr ? b->n_seg : p->B);
   void* side = ov != nullptr ? (void*)ov->side : nullptr;
 
   if (b->trainable)

@@ -239,8 +239,10 @@ def test_attention_with_more_segments_than_the_kernels_stage(C, H):
     assert blk.read_status() == 0
 
 
-@pytest.mark.parametrize("ci,fused", [(1, False), (2, False), (2, True)])
-def test_shifted_packing_order_with_containers(ci, fused):
+# device_cuts: the library builds the container cuts itself inside the block call (nothing comes from the host)
+@pytest.mark.parametrize("ci,fused,device_cuts", [(1, False, False), (2, False, False), (2, True, False),
+                                                  (1, False, True), (2, True, True), (4, True, True)])
+def test_shifted_packing_order_with_containers(ci, fused, device_cuts):
     """Tokens packed in the order of a cyclically shifted feature map, attention cut into containers of 49 tokens
     (the paper's own batching): indices bit for bit, forward and backward against the oracle."""
     cfg = scaled_config(get_config(ci), B=5)
@@ -254,13 +256,20 @@ def test_shifted_packing_order_with_containers(ci, fused):
     assert np.abs(plain["y"] - fwd["y"]).max() > 1e-2   # the shift changes which tokens meet
     d = {n: dev(getattr(inp, n), cfg.dtype) for n in ("x", "w_g", "W_qkv", "b_qkv", "W_o", "b_o", "dY")}
     blk = block(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, fused=fused)
-    seg = torch.from_numpy(fwd["seg"].astype(np.int32)).cuda()
-    y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"],
-                    order=torch.from_numpy(order).cuda(), seg_offsets=seg)
+    if device_cuts:
+        y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"],
+                        order=torch.from_numpy(order).cuda(), container_len=49)
+    else:
+        seg = torch.from_numpy(fwd["seg"].astype(np.int32)).cuda()
+        y = blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"],
+                        order=torch.from_numpy(order).cuda(), seg_offsets=seg)
     dX = blk.backward(d["dY"])
     torch.cuda.synchronize()
     assert blk.read_status() == 0
     Np = int(fwd["cu_seqlens"][-1])
+    if device_cuts:
+        got_seg = blk.container_seg.cpu().numpy()
+        assert np.array_equal(got_seg[:len(fwd["seg"])], fwd["seg"]) and np.all(got_seg[len(fwd["seg"]):] == Np)
     assert np.array_equal(blk.cu.cpu().numpy(), fwd["cu_seqlens"])
     assert np.array_equal(blk.idx.cpu().numpy()[:Np], fwd["idx"])
     assert np.array_equal(blk.inv.cpu().numpy(), fwd["inv"])
