@@ -61,11 +61,8 @@ def test_tile_map_covers_every_row_once_with_whole_segments(name):
             assert lo in seg_np and hi in seg_np
     assert np.all(covered == 1)
     # greedy grouping: a group and the first non-empty segment after it never fit into one tile together
-    def seg_len_at(row):
-        k = int(np.searchsorted(seg_np, row, side="right")) - 1
-        return int(seg_np[k + 1] - seg_np[k])
-
-    short_groups = sorted((int(lo), int(hi)) for lo, hi in ent if seg_len_at(lo) <= 128)
+    short_groups = sorted((int(lo), int(hi)) for lo, hi in ent
+                          if seg_np[int(np.searchsorted(seg_np, lo, side="right"))] - lo <= 128)
     for lo, hi in short_groups:
         nxt_end = seg_np[np.searchsorted(seg_np, hi, side="right")] if hi < Np else None
         if nxt_end is not None and nxt_end - hi <= 128:      # the next segment is a short one
