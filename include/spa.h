@@ -159,25 +159,6 @@ int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* a
                              int32_t n_seg, void* dqkv, void* workspace, int32_t* d_status,
                              void* stream);
 
-/* Row tiles that follow the segments (Sec. 3.2: attention never crosses an image, or a container).  The attention
- * kernels work on tiles of up to 128 packed rows; cut at fixed multiples of 128 a tile straddles the boundaries of
- * short segments and must walk the union of their key ranges.  spa_attention_tile_map cuts the rows along the
- * segments instead: a segment longer than 128 rows gets tiles of its own, consecutive shorter ones are grouped while
- * they fit into 128 rows.  Results are those of the plain calls up to the summation order inside a head (the same
- * tolerances apply); with short segments the tiled calls do a fraction of the work.
- *   tiles: device scratch of spa_attention_tiles_bytes(p, n_seg) bytes, written by spa_attention_tile_map and read
- *   by the two _tiled calls, which must be given the same seg_offsets and n_seg.  The map depends on the segments
- *   only: build it once per selection and use it for the forward and the backward pass.
- * n_seg is limited to 4096 segments: beyond that spa_attention_tiles_bytes returns 0, the map call returns
- * SPA_ERR_UNSUPPORTED, and the plain calls must be used.  Tensor-core problems only (bf16, head dimension 32 or 64). */
-size_t spa_attention_tiles_bytes(const spa_params* p, int32_t n_seg);
-int spa_attention_tile_map(const spa_params* p, const int32_t* seg_offsets, int32_t n_seg, void* tiles, void* stream);
-int spa_packed_attention_fwd_tiled(const spa_params* p, const void* qkv, const int32_t* seg_offsets, int32_t n_seg,
-                                   const void* tiles, void* attn_out, float* lse, int32_t* d_status, void* stream);
-int spa_packed_attention_bwd_tiled(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
-                                   const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg,
-                                   const void* tiles, void* dqkv, void* workspace, int32_t* d_status, void* stream);
-
 /* Attention backward for callers that cannot hand over scratch memory.  (The paper has no
  * counterpart: this is a packaging variant of spa_packed_attention_bwd, same arithmetic.)
  *
@@ -402,8 +383,6 @@ typedef struct spa_block_buffers {
   float* db_g;                /* float[1] or NULL                                                    */
   float* loss;                /* float[1] or NULL                                                    */
   void* train_workspace;      /* spa_train_workspace_bytes()                                         */
-  void* attn_tiles;           /* spa_attention_tiles_bytes(p, n_seg of the pass) or NULL: with it, spa_block_fwd
-                                 builds the segment-aligned row tiles and both passes use the tiled attention calls */
   /* the paper's containers (Sec. 3.2 "Token Packing") */
   int32_t container_len;      /* L > 0: spa_block_fwd fills seg_offsets (which must then be a writable
                                  int32[spa_container_max_segments(p, L) + 1]) with the container cuts of the

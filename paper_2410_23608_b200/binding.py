@@ -34,8 +34,6 @@ EXPORTS = (
     "spa_overlap_create", "spa_overlap_destroy", "spa_block_fwd", "spa_block_bwd",
     "spa_probe_exp2", "spa_probe_wait_expiry", "spa_pack_state_bytes", "spa_gate_select_pack_supported",
     "spa_gate_select_pack", "spa_container_max_segments", "spa_container_offsets",
-    "spa_attention_tiles_bytes", "spa_attention_tile_map", "spa_packed_attention_fwd_tiled",
-    "spa_packed_attention_bwd_tiled",
 )
 
 
@@ -67,7 +65,7 @@ class SpaBlockBuffers(C.Structure):
                 ("pack_state", C.c_void_p), ("overlap", C.c_void_p), ("d_status", C.c_void_p),
                 ("trainable", C.c_int32), ("labels", C.c_void_p), ("alpha", C.c_float), ("ds", C.c_void_p),
                 ("ds_up", C.c_void_p), ("dw_g", C.c_void_p), ("db_g", C.c_void_p), ("loss", C.c_void_p),
-                ("train_workspace", C.c_void_p), ("attn_tiles", C.c_void_p), ("container_len", C.c_int32)]
+                ("train_workspace", C.c_void_p), ("container_len", C.c_int32)]
 
 
 def make_params(B, N, Cc, H, dtype, capacity=None, flags=0, tau=0.0, softmax_scale=0.0) -> SpaParams:
@@ -127,16 +125,11 @@ def lib() -> C.CDLL:
         L.spa_gate_select_pack.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.spa_container_max_segments.argtypes = [pp, i32]
         L.spa_container_offsets.argtypes = [pp, vp, i32, vp, vp]
-        L.spa_attention_tiles_bytes.restype = C.c_size_t
-        L.spa_attention_tiles_bytes.argtypes = [pp, i32]
-        L.spa_attention_tile_map.argtypes = [pp, vp, i32, vp, vp]
-        L.spa_packed_attention_fwd_tiled.argtypes = [pp, vp, vp, i32, vp, vp, vp, vp, vp]
-        L.spa_packed_attention_bwd_tiled.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.spa_probe_exp2.argtypes = [i32, i32, vp, C.POINTER(C.c_ulonglong), vp]
         L.spa_probe_wait_expiry.argtypes = [i32, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
-            if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_pack_state_bytes", "spa_attention_tiles_bytes", "spa_status_string", "spa_last_cuda_error",
+            if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_pack_state_bytes", "spa_status_string", "spa_last_cuda_error",
                             "spa_launch_count"):
                 getattr(L, name).restype = C.c_int
         L.spa_status_string.restype = C.c_char_p
@@ -222,28 +215,6 @@ def spa_packed_attention_bwd(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_s
     _check(lib().spa_packed_attention_bwd(C.byref(p), _ptr(qkv), _ptr(attn_out), _ptr(lse), _ptr(d_attn_out),
                                           _ptr(seg_offsets), int(n_seg), _ptr(dqkv), _ptr(workspace), _ptr(d_status),
                                           _stream(stream)), "spa_packed_attention_bwd")
-
-
-def spa_attention_tiles_bytes(p, n_seg) -> int:
-    return int(lib().spa_attention_tiles_bytes(C.byref(p), int(n_seg)))
-
-
-def spa_attention_tile_map(p, seg_offsets, n_seg, tiles, stream=None):
-    _check(lib().spa_attention_tile_map(C.byref(p), _ptr(seg_offsets), int(n_seg), _ptr(tiles), _stream(stream)),
-           "spa_attention_tile_map")
-
-
-def spa_packed_attention_fwd_tiled(p, qkv, seg_offsets, n_seg, tiles, attn_out, lse, d_status=None, stream=None):
-    _check(lib().spa_packed_attention_fwd_tiled(C.byref(p), _ptr(qkv), _ptr(seg_offsets), int(n_seg), _ptr(tiles),
-                                                _ptr(attn_out), _ptr(lse), _ptr(d_status), _stream(stream)),
-           "spa_packed_attention_fwd_tiled")
-
-
-def spa_packed_attention_bwd_tiled(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, tiles, dqkv, workspace,
-                                   d_status=None, stream=None):
-    _check(lib().spa_packed_attention_bwd_tiled(C.byref(p), _ptr(qkv), _ptr(attn_out), _ptr(lse), _ptr(d_attn_out),
-                                                _ptr(seg_offsets), int(n_seg), _ptr(tiles), _ptr(dqkv), _ptr(workspace),
-                                                _ptr(d_status), _stream(stream)), "spa_packed_attention_bwd_tiled")
 
 
 def spa_packed_attention_bwd_static(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, d_status=None,

@@ -20,7 +20,7 @@ class SpaBlock:
 
     def __init__(self, B: int, N: int, C: int, H: int, dtype: str, tau: float = 0.0, flags: int = 0,
                  capacity: Optional[int] = None, backward: bool = True, device: str = "cuda",
-                 fused: Optional[bool] = None, one_pass: bool = False, seg_tiles: bool = True):
+                 fused: Optional[bool] = None, one_pass: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("SpaBlock needs a CUDA device; there is no CPU path")
         L.lib()
@@ -75,10 +75,6 @@ class SpaBlock:
         self._saved = None            # (W_qkv, W_o) of the last forward()
         self._seg = (self.cu, B)      # attention segments: the images, unless forward() is given others
         self._keep = None             # tensors of the last call that the enqueued work still reads
-        # seg_tiles: attention on row tiles cut along the segments (a small map built on the device each forward pass)
-        self.seg_tiles = seg_tiles
-        self._tiles = {}              # n_seg -> scratch of the tile map
-        self._tiles_for = None        # (segment array, n_seg) that the last forward() built the map for
         self._container_len = 0       # > 0: the library builds the container cuts itself (forward(container_len=L))
         self.container_seg = None
 
@@ -91,16 +87,9 @@ class SpaBlock:
         except Exception:
             pass
 
-    def _buffers(self, building_tiles=False, **extra):
+    def _buffers(self, **extra):
         seg, n_seg = self._seg
-        tiles = None
-        if self.seg_tiles and (building_tiles or self._tiles_for == (seg.data_ptr(), n_seg)):
-            nbytes = L.spa_attention_tiles_bytes(self.p, n_seg)
-            if nbytes > 0:
-                if n_seg not in self._tiles:
-                    self._tiles[n_seg] = torch.zeros(nbytes, dtype=torch.uint8, device=self.cu.device)
-                tiles = self._tiles[n_seg]
-        f = dict(attn_tiles=tiles, scores=self.scores, mask=self.mask, cu_seqlens=self.cu, idx=self.idx, inv=self.inv, x_packed=self.xp,
+        f = dict(scores=self.scores, mask=self.mask, cu_seqlens=self.cu, idx=self.idx, inv=self.inv, x_packed=self.xp,
                  qkv=self.qkv, attn_out=self.ao, lse=self.lse, z=self.z, workspace=self.workspace, d_status=self.status,
                  pack_state=self.pack_state, container_len=self._container_len,
                  seg_offsets=None if seg is self.cu else seg, n_seg=n_seg)
@@ -125,8 +114,7 @@ class SpaBlock:
         self._seg = (self.cu, self.B) if seg_offsets is None else (seg_offsets, int(seg_offsets.numel()) - 1)
         self._saved = (W_qkv, W_o)
         self._keep = (x, w_g, W_qkv, b_qkv, W_o, b_o, s_up, order, seg_offsets, y)
-        self._tiles_for = (self._seg[0].data_ptr(), self._seg[1])
-        L.spa_block_fwd(self.p, self._buffers(building_tiles=True, x=x, w_g=w_g, b_g=float(b_g), s_up=s_up, W_qkv=W_qkv, b_qkv=b_qkv, W_o=W_o,
+        L.spa_block_fwd(self.p, self._buffers(x=x, w_g=w_g, b_g=float(b_g), s_up=s_up, W_qkv=W_qkv, b_qkv=b_qkv, W_o=W_o,
                                               b_o=b_o, order=order, y=y))
         return y
 

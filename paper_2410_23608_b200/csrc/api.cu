@@ -212,48 +212,6 @@ int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* a
                                    (cudaStream_t)stream);
 }
 
-size_t spa_attention_tiles_bytes(const spa_params* p, int32_t n_seg) {
-  if (check_params(p) != SPA_OK || check_heads(p) != SPA_OK || !use_tc(p) || !tc_attention_fwd_supported(*p)) return 0;
-  return attention_tiles_bytes(*p, n_seg);
-}
-
-int spa_attention_tile_map(const spa_params* p, const int32_t* seg_offsets, int32_t n_seg, void* tiles, void* stream) {
-  int rc = check_params(p);
-  if (rc != SPA_OK) return rc;
-  SPA_PTR(seg_offsets); SPA_PTR(tiles);
-  SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
-  if (spa_attention_tiles_bytes(p, n_seg) == 0) return SPA_ERR_UNSUPPORTED;
-  return launch_attention_tile_map(*p, seg_offsets, n_seg, (int32_t*)tiles, (cudaStream_t)stream);
-}
-
-int spa_packed_attention_fwd_tiled(const spa_params* p, const void* qkv, const int32_t* seg_offsets, int32_t n_seg,
-                                   const void* tiles, void* attn_out, float* lse, int32_t* d_status, void* stream) {
-  int rc = check_params(p);
-  if (rc != SPA_OK) return rc;
-  rc = check_heads(p);
-  if (rc != SPA_OK) return rc;
-  SPA_PTR(qkv); SPA_PTR(seg_offsets); SPA_PTR(tiles); SPA_PTR(attn_out); SPA_PTR(lse);
-  SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
-  if (spa_attention_tiles_bytes(p, n_seg) == 0) return SPA_ERR_UNSUPPORTED;
-  return launch_attention_fwd_tc(*p, qkv, seg_offsets, n_seg, attn_out, lse, d_status, (cudaStream_t)stream,
-                                 (const int32_t*)tiles);
-}
-
-int spa_packed_attention_bwd_tiled(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
-                                   const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg,
-                                   const void* tiles, void* dqkv, void* workspace, int32_t* d_status, void* stream) {
-  int rc = check_params(p);
-  if (rc != SPA_OK) return rc;
-  rc = check_heads(p);
-  if (rc != SPA_OK) return rc;
-  SPA_PTR(qkv); SPA_PTR(attn_out); SPA_PTR(lse); SPA_PTR(d_attn_out); SPA_PTR(seg_offsets); SPA_PTR(tiles); SPA_PTR(dqkv);
-  SPA_PTR(workspace);
-  SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
-  if (spa_attention_tiles_bytes(p, n_seg) == 0) return SPA_ERR_UNSUPPORTED;
-  return launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace, d_status,
-                                 (cudaStream_t)stream, (const int32_t*)tiles);
-}
-
 int spa_packed_attention_bwd_static(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
                                     const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg, void* dqkv,
                                     int32_t* d_status, void* stream) {
@@ -542,13 +500,7 @@ int spa_block_fwd(const spa_params* p, const spa_block_buffers* b, void* stream)
   const int32_t* seg = b->seg_offsets != nullptr ? b->seg_offsets : b->cu_seqlens;
   const int32_t n_seg = b->container_len > 0 ? spa_container_max_segments(p, b->container_len)
                                              : (b->seg_offsets != nullptr ? b->n_seg : p->B);
-  if (b->attn_tiles != nullptr && spa_attention_tiles_bytes(p, n_seg) != 0) {
-    // row tiles cut along the segments: built once here, used again by the backward pass
-    SPA_STEP(spa_attention_tile_map(p, seg, n_seg, b->attn_tiles, stream));
-    SPA_STEP(spa_packed_attention_fwd_tiled(p, b->qkv, seg, n_seg, b->attn_tiles, b->attn_out, b->lse, b->d_status, stream));
-  } else {
-    SPA_STEP(spa_packed_attention_fwd(p, b->qkv, seg, n_seg, b->attn_out, b->lse, b->d_status, stream));
-  }
+  SPA_STEP(spa_packed_attention_fwd(p, b->qkv, seg, n_seg, b->attn_out, b->lse, b->d_status, stream));
   if (fused) return spa_packed_proj_scatter(p, b->attn_out, b->W_o, b->b_o, b->idx, b->cu_seqlens, y, b->d_status, stream);
   SPA_STEP(spa_packed_proj(p, b->attn_out, b->W_o, b->b_o, b->cu_seqlens, b->z, b->d_status, stream));
   return spa_unpack_scatter(p, b->z, inplace ? nullptr : b->x, b->idx, b->inv, b->cu_seqlens, y, b->d_status, stream);
@@ -588,14 +540,9 @@ int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream)
     rc = spa_packed_linear_bwd(p, b->attn_out, b->W_o, b->dz, C, C, b->cu_seqlens, b->d_attn_out, nullptr, nullptr,
                                b->workspace, b->d_status, stream);
   }
-  if (rc == SPA_OK && rc_side == SPA_OK) {
-    if (b->attn_tiles != nullptr && spa_attention_tiles_bytes(p, n_seg) != 0)
-      rc = spa_packed_attention_bwd_tiled(p, b->qkv, b->attn_out, b->lse, b->d_attn_out, seg, n_seg, b->attn_tiles, b->dqkv,
-                                          b->workspace, b->d_status, stream);
-    else
-      rc = spa_packed_attention_bwd(p, b->qkv, b->attn_out, b->lse, b->d_attn_out, seg, n_seg, b->dqkv, b->workspace,
-                                    b->d_status, stream);
-  }
+  if (rc == SPA_OK && rc_side == SPA_OK)
+    rc = spa_packed_attention_bwd(p, b->qkv, b->attn_out, b->lse, b->d_attn_out, seg, n_seg, b->dqkv, b->workspace,
+                                  b->d_status, stream);
   if (rc == SPA_OK && rc_side == SPA_OK) {
     if (ov != nullptr) {
       // the second stream's next call reads dqkv: it waits for the attention backward

@@ -92,12 +92,10 @@ template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __restrict__ seg, int n_seg, int capacity,
                    int C, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
-                   const int32_t* __restrict__ tiles, int32_t* d_status) {
+                   int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
-  // grid = (heads, tiles): CTAs past the last valid tile are dispatched last.  Without a tile map, tile y covers the
-  // packed rows [128 y, 128 y + 128); with one, the rows that its entry names (whole segments, see attn_tiles.cu).
-  int q0 = blockIdx.y * kQ;
+  const int q0 = blockIdx.y * kQ;  // grid = (heads, tiles): CTAs past the last valid tile are dispatched last
   const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool is_softmax = warp < kSoftmaxThreads / 32;  // warps 0-7; warp 8 issues the copies and the products
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 query rows and split
@@ -140,18 +138,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     ptx::fence_mbar_init();
   }
   pdl_entry();
-  const int Np = packed_rows(seg, n_seg, capacity);
-  int q_end = q0 + kQ < Np ? q0 + kQ : Np;  // rows from q_end on are not this tile's
-  if (tiles != nullptr) {
-    if ((int)blockIdx.y >= __ldg(tiles)) return;
-    q0 = __ldg(tiles + 2 + 2 * blockIdx.y);
-    q_end = __ldg(tiles + 3 + 2 * blockIdx.y);
-  } else if (q0 >= Np) {
-    return;
-  }
   const bool staged = n_seg < kSegStage;
   if (staged)
     for (int i = tid; i <= n_seg; i += kFwdThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  if (q0 >= Np) return;
   if (tid == kSoftmaxThreads) {  // the Q tile depends only on q0: fetch it under the segment search
     ptx::mbar_expect_tx(bar_q, kTile);
     ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
@@ -165,9 +156,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   const int row = q0 + rl;
   RowSeg mine{0, 0};
   if (is_softmax) {
-    if (row < q_end) mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+    mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
     if (half == 0) {
-      const int last = q_end - 1;
+      const int last = (q0 + kQ - 1 < Np - 1) ? q0 + kQ - 1 : Np - 1;
       if (row == q0) range[0] = mine.lo;
       if (row == last) range[1] = mine.hi;
     }
@@ -389,20 +380,20 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       for (int e = 0; e < kDh; ++e) r[e] = 0u;
     }
     const float l_row = xch[half * 128 + rl] + xch[(half ^ 1) * 128 + rl];
-    const float inv_l = row < q_end ? 1.f / l_row : 0.f;
+    const float inv_l = row < Np ? 1.f / l_row : 0.f;
     const int rot = chunk_rot<D>(rl);
 #pragma unroll
     for (int c = 0; c < kDh / 8; ++c) {
       float v[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = row < q_end ? __uint_as_float(r[c * 8 + e]) * inv_l : 0.f;
+      for (int e = 0; e < 8; ++e) v[e] = row < Np ? __uint_as_float(r[c * 8 + e]) * inv_l : 0.f;
       *reinterpret_cast<uint4*>(smem_al + rl * HT::kRowBytes + (((half * (kDh / 8) + c) ^ rot) << 4)) =
           Vec16<__nv_bfloat16>::from_float(v);
     }
-    if (half == 0 && row < q_end) lse[(long long)h * capacity + row] = (lse_m + log2f(l_row)) * 0.6931471805599453f;
+    if (half == 0 && row < Np) lse[(long long)h * capacity + row] = (lse_m + log2f(l_row)) * 0.6931471805599453f;
   }
   __syncthreads();
-  if (!failed) copy_tile_out<D, kFwdThreads>(smem_al, ao + h * D, C, q0, q_end, tid);
+  if (!failed) copy_tile_out<D, kFwdThreads>(smem_al, ao + h * D, C, q0, Np, tid);
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) {
@@ -448,8 +439,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
-                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, const int32_t* __restrict__ tiles,
-                   int32_t* d_status) {
+                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
@@ -461,7 +451,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_aliased_kernel");
   constexpr uint32_t kColOpP = 160u;                // P^T (dK/dV pass only)
   constexpr uint32_t kColOpDS = kDQ ? 192u : 224u;  // dS or dS^T
-  int r0 = blockIdx.y * 128;  // grid = (heads, tiles); rows of tile y: [128 y, 128 y + 128), or what the tile map says
+  const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
   const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool is_math = warp < kBwdMath / 32;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
@@ -509,18 +499,11 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     ptx::fence_mbar_init();
   }
   pdl_entry();
-  const int Np = packed_rows(seg, n_seg, capacity);
-  int r_end = r0 + 128 < Np ? r0 + 128 : Np;  // rows from r_end on are not this tile's
-  if (tiles != nullptr) {
-    if ((int)blockIdx.y >= __ldg(tiles)) return;
-    r0 = __ldg(tiles + 2 + 2 * blockIdx.y);
-    r_end = __ldg(tiles + 3 + 2 * blockIdx.y);
-  } else if (r0 >= Np) {
-    return;
-  }
   const bool staged = n_seg < kSegStage;
   if (staged)
     for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  if (r0 >= Np) return;
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
   if (tid == kBwdMath) {  // the own tiles depend only on r0: fetch them under the segment search
     ptx::mbar_expect_tx(bar_x, 2 * kTile);
@@ -543,9 +526,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const int row = r0 + rl;
   RowSeg mine{0, 0};
   if (is_math) {
-    if (row < r_end) mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+    mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
     if (half == 0) {
-      const int last = r_end - 1;
+      const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
       if (row == r0) range[0] = mine.lo;
       if (row == last) range[1] = mine.hi;
     }
@@ -584,7 +567,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next streamed query tile, row rl < 64
   if (is_math) {
     if (kDQ) {
-      if (row < r_end) my_lse = lse[(long long)h * capacity + row] * kLog2e;
+      if (row < Np) my_lse = lse[(long long)h * capacity + row] * kLog2e;
     } else if (half == 0 && rl < kBwdY) {
       const int i = o_lo + rl;
       if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
@@ -693,7 +676,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     }
   } else if (!failed_early) {
     // ---------------------------------------------------------------- arithmetic: two threads per row
-    if (kDQ && row < r_end) {
+    if (kDQ && row < Np) {
       // D_i = dO_i . O_i from the two staged tiles (their load has completed: prep(0) waited for it).  Both
       // carry the same swizzle, so equal positions hold equal columns and the order of the chunks is free:
       // each row starts at a different chunk to keep 8 neighbouring rows off one bank.
@@ -815,15 +798,15 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     if (kDQ) {
       if (is_math) stage_acc(kColAcc1, smem_al, scale);
       __syncthreads();
-      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, r_end, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
     } else {
       if (is_math) {
         stage_acc(kColAcc1, smem_al, 1.f);             // dV
         stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
       }
       __syncthreads();
-      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, r_end, tid);
-      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, r_end, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
     }
   }
   if (failed && tid == kBwdMath) {  // let outstanding loads land before shared memory is released
@@ -856,15 +839,14 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
-                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, const int32_t* __restrict__ tiles,
-                   int32_t* d_status) {
+                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr bool kDQ = false;  // this kernel is the dK / dV pass only
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
   constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
   constexpr float kLog2e = 1.4426950408889634f;
-  int r0 = blockIdx.y * 128;  // grid = (heads, tiles); rows of tile y: [128 y, 128 y + 128), or what the tile map says
+  const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
   const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
   const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
@@ -903,18 +885,11 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
     ptx::fence_mbar_init();
   }
   pdl_entry();
-  const int Np = packed_rows(seg, n_seg, capacity);
-  int r_end = r0 + 128 < Np ? r0 + 128 : Np;  // rows from r_end on are not this tile's
-  if (tiles != nullptr) {
-    if ((int)blockIdx.y >= __ldg(tiles)) return;
-    r0 = __ldg(tiles + 2 + 2 * blockIdx.y);
-    r_end = __ldg(tiles + 3 + 2 * blockIdx.y);
-  } else if (r0 >= Np) {
-    return;
-  }
   const bool staged = n_seg < kSegStage;
   if (staged)
     for (int i = tid; i <= n_seg; i += kAliasedThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  if (r0 >= Np) return;
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
   if (tid == 0) {  // the own tiles depend only on r0: fetch them under the segment search
     ptx::mbar_expect_tx(bar_x, kOwn * kTile);
@@ -934,10 +909,9 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
 
   const int row = r0 + rl;
-  RowSeg mine{0, 0};
-  if (row < r_end) mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+  const RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
   if (half == 0) {
-    const int last = r_end - 1;
+    const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
     if (row == r0) range[0] = mine.lo;
     if (row == last) range[1] = mine.hi;
   }
@@ -1138,13 +1112,13 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
     if (kDQ) {
       stage_acc(kColAcc1, smem_al, scale);
       __syncthreads();
-      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + h * D, ld, r0, r_end, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
     } else {
       stage_acc(kColAcc1, smem_al, 1.f);             // dV
       stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
       __syncthreads();
-      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, r_end, tid);
-      copy_tile_out<D, kAliasedThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, r_end, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
     }
   }
   if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
@@ -1175,8 +1149,7 @@ template <> struct kv_pass<64> {
 
 template <int D>
 int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
-               const int32_t* seg, int n_seg, const int32_t* tiles, void* dqkv, void* workspace, int32_t* d_status,
-               cudaStream_t st) {
+               const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st) {
   CUtensorMap tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o;  // own tiles: 128-row boxes; streamed tiles: 64-row boxes
   if (!make_tmap_bf16_2d(&tm_qkv, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2) ||
       !make_tmap_bf16_2d(&tm_do, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2) ||
@@ -1193,30 +1166,30 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
   });
   if (ea != cudaSuccess) { set_cuda_error(ea, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
-  dim3 grid(p.H, tiles != nullptr ? attention_max_tiles(p, n_seg) : (p.capacity + 127) / 128);
+  dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
   launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D, true>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, tiles, d_status);
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
   launch_pdl(kkv, grid, kv_pass<D>::kThreads, kv_pass<D>::kSmem, st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, tiles, d_status);
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
   return SPA_OK;
 }
 
 template <int D>
-int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, const int32_t* tiles, void* ao,
-               float* lse, int32_t* d_status, cudaStream_t st) {
+int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
+               int32_t* d_status, cudaStream_t st) {
   CUtensorMap tm;
   if (!make_tmap_bf16_2d(&tm, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2)) return SPA_ERR_UNSUPPORTED;
   auto kern = attn_fwd_tc_kernel<D>;
   static DeviceOnce attr;
   cudaError_t ea = attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem_bytes<D>()); });
   if (ea != cudaSuccess) { set_cuda_error(ea, "attn_fwd_tc_kernel"); return SPA_ERR_CUDA; }
-  dim3 grid(p.H, tiles != nullptr ? attention_max_tiles(p, n_seg) : (p.capacity + kQ - 1) / kQ);
+  dim3 grid(p.H, (p.capacity + kQ - 1) / kQ);
   launch_pdl(kern, grid, kFwdThreads, fwd_smem_bytes<D>(), st, tm, seg, n_seg, p.capacity, p.C,
                                                       softmax_scale_of(p) * 1.4426950408889634f,
-                                                      (__nv_bfloat16*)ao, lse, tiles, d_status);
+                                                      (__nv_bfloat16*)ao, lse, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_fwd_tc_kernel");
   return SPA_OK;
 }
@@ -1237,15 +1210,15 @@ size_t tc_attention_workspace_bytes(const spa_params& p) {
 
 int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                             const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
-                            cudaStream_t st, const int32_t* tiles) {
-  return p.C / p.H == 64 ? bwd_launch<64>(p, qkv, ao, lse, dao, seg, n_seg, tiles, dqkv, workspace, d_status, st)
-                         : bwd_launch<32>(p, qkv, ao, lse, dao, seg, n_seg, tiles, dqkv, workspace, d_status, st);
+                            cudaStream_t st) {
+  return p.C / p.H == 64 ? bwd_launch<64>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st)
+                         : bwd_launch<32>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st);
 }
 
 int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
-                            int32_t* d_status, cudaStream_t st, const int32_t* tiles) {
-  return p.C / p.H == 64 ? fwd_launch<64>(p, qkv, seg, n_seg, tiles, ao, lse, d_status, st)
-                         : fwd_launch<32>(p, qkv, seg, n_seg, tiles, ao, lse, d_status, st);
+                            int32_t* d_status, cudaStream_t st) {
+  return p.C / p.H == 64 ? fwd_launch<64>(p, qkv, seg, n_seg, ao, lse, d_status, st)
+                         : fwd_launch<32>(p, qkv, seg, n_seg, ao, lse, d_status, st);
 }
 
 }  // namespace spa

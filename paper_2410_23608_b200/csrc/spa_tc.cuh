@@ -26,18 +26,12 @@ int launch_linear_dgrad_pair(const spa_params& p, const void* W, const void* dou
                              void* da, int32_t* d_status, cudaStream_t st, const int32_t* row_map, bool accumulate);
 
 bool tc_attention_fwd_supported(const spa_params& p);
-// tiles (optional): a row-tile map built by launch_attention_tile_map for the same segments
 int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
-                            int32_t* d_status, cudaStream_t st, const int32_t* tiles = nullptr);
+                            int32_t* d_status, cudaStream_t st);
 bool tc_attention_bwd_supported(const spa_params& p);
 int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                             const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
-                            cudaStream_t st, const int32_t* tiles = nullptr);
-// row tiles that follow the segment boundaries (attn_tiles.cu)
-int attention_max_tiles(const spa_params& p, int n_seg);
-bool attention_tiles_supported(const spa_params& p, int n_seg);
-size_t attention_tiles_bytes(const spa_params& p, int n_seg);
-int launch_attention_tile_map(const spa_params& p, const int32_t* seg, int n_seg, int32_t* tiles, cudaStream_t st);
+                            cudaStream_t st);
 // Device address, on the current device, of the SPA_STATIC_SCRATCH_BYTES array built into the library.
 int static_attention_scratch(void** out);
 

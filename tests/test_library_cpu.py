@@ -89,9 +89,6 @@ def test_later_entry_points_validate_on_the_host(lib):
     assert L.spa_gate_select_pack_supported(pp) == 1
     wide = lib.make_params(2, 16, 2048, 32, "bf16")                 # 256 chunks per row: two-kernel path only
     assert L.spa_gate_select_pack_supported(ctypes.byref(wide)) == 0
-    assert L.spa_attention_tile_map(pp, None, 2, None, None) == inv
-    assert L.spa_packed_attention_fwd_tiled(pp, None, None, 2, None, None, None, None, None) == inv
-    assert L.spa_packed_attention_bwd_tiled(pp, None, None, None, None, None, 2, None, None, None, None, None) == inv
     empty = lib.SpaBlockBuffers()
     assert L.spa_block_fwd(pp, None, None) == inv and L.spa_block_bwd(pp, None, None) == inv
     assert L.spa_block_fwd(pp, ctypes.byref(empty), None) == inv      # no inputs: refused by the first call
