@@ -91,14 +91,12 @@ struct TileCoord { int m0, n0, z, n_t; };
 // overlap the main loop of the next, and the TMA ring runs ahead across tile boundaries.
 // row_map (optional): output row i goes to row row_map[i] of `out` (the unpack scatter fused into the
 // epilogue); with `accumulate` the bf16 result is added to what that row holds.
-// kColSum (wgrad only): while the MMAs run, the epilogue warps add up the columns of the dout tiles
-// that stream through shared memory, which gives the bias gradient at no extra HBM traffic.
-template <int BN, bool kAMn, bool kBMn, typename OutT, bool kColSum>
+template <int BN, bool kAMn, bool kBMn, typename OutT>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
                long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
-               int dyn_which, int k_per_split, float* __restrict__ colsum_part, const int32_t* __restrict__ row_map,
+               int dyn_which, int k_per_split, const int32_t* __restrict__ row_map,
                int accumulate, int32_t* d_status) {
   constexpr int kStage = stage_bytes<BN>();
   constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
@@ -121,7 +119,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::prefetch_tensormap(&tmB);
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full_bar(s), 1);
-      ptx::mbar_init(empty_bar(s), kColSum ? 2 : 1);
+      ptx::mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(tmem_full_bar(a), 1); ptx::mbar_init(tmem_empty_bar(a), 4); }
     *abort_flag = 0;
@@ -258,37 +256,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int q = warp & 3;          // TMEM lane quarter this warp may read
-    const int et = threadIdx.x - 64; // 0..127 over the four epilogue warps, any order of quarters
     uint8_t* stage = smem_al + kStages * kStage + 128 + (warp - 2) * 2048;  // this warp's transposition buffer
-    int it = 0, tl = 0;
+    int tl = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++tl) {
       if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
       const TileCoord c = coord(tile);
-      int k_begin, k_end;
-      k_range(c.z, k_begin, k_end);
-      if (kColSum) {
-        // column sums of the dout tiles (A operand, MN-major: K row k of 64-wide box j is the 128-byte line
-        // at j*8192 + k*128, 16-byte chunks XOR-swizzled by k mod 8); thread et owns column m0 + et
-        float sum = 0.f;
-        for (int k0 = k_begin; k0 < k_end; k0 += BK, ++it) {
-          const int s = it % kStages;
-          bool ok = true;
-          if (c.n_t == 0 || et == 0) ok = ptx::mbar_wait(full_bar(s), (it / kStages) & 1);
-          if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-          if (c.n_t == 0) {
-            const int k_valid = (k_end - k0) < BK ? (k_end - k0) : BK;
-            const uint8_t* box = smem_al + s * kStage + (et >> 6) * (BK * 128);
-            const int ml = et & 63;
-            for (int k = 0; k < k_valid; ++k) {
-              const uint16_t raw = *reinterpret_cast<const uint16_t*>(box + k * 128 + (((ml >> 3) ^ (k & 7)) << 4) + (ml & 7) * 2);
-              sum += __uint_as_float((uint32_t)raw << 16);
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");  // all four warps are done with this stage
-          }
-          if (et == 0) ptx::mbar_arrive(empty_bar(s));
-        }
-        if (c.n_t == 0 && c.m0 + et < M) colsum_part[(long long)c.z * M + c.m0 + et] = sum;
-      }
       const int acc = tl & 1;
       const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(tmem_full_bar(acc), (tl >> 1) & 1) && !*abort_flag);
       if (!ok) {
@@ -375,26 +347,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ---- wgrad helpers --------------------------------------------------------------------------------
-// Partial column sums of dout over the rows of one K split: part[z][col].
+// Partial column sums of dout over one chunk of rows: part[chunk][col].  A streaming reduction: CTA (x, y) owns 64
+// columns and the rows of chunk y, eight threads across the columns (16 bytes each) and 32 down the rows with four
+// loads in flight per thread; the 32 row lanes are added up in shared memory in a fixed order.
+constexpr int kColsumChunks = 64;  // row chunks over the allocated rows (rows per chunk: a multiple of 8)
+inline int colsum_rows_per_chunk(int capacity) { return (((capacity + kColsumChunks - 1) / kColsumChunks) + 7) & ~7; }
+
 __global__ void __launch_bounds__(256)
 colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const int32_t* __restrict__ cu, int n_seg,
-                      int capacity, int k_per_split, float* __restrict__ part) {
+                      int capacity, int rows_per_chunk, float* __restrict__ part) {
   pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
-  const int r_begin = blockIdx.y * k_per_split;
-  int r_end = r_begin + k_per_split;
+  const int r_begin = blockIdx.y * rows_per_chunk;
+  if (r_begin >= rows) return;  // chunks past the valid rows are not read by the reduction
+  int r_end = r_begin + rows_per_chunk;
   if (r_end > rows) r_end = rows;
   __shared__ float red[32][65];
   const int cg = threadIdx.x & 7, rl = threadIdx.x >> 3;  // 8 column groups of 8, 32 row lanes
   const int col = blockIdx.x * 64 + cg * 8;
   float acc[8] = {};
-  if (col < n_out)
-    for (int i = r_begin + rl; i < r_end; i += 32) {
-      float f[8];
-      Vec16<__nv_bfloat16>::to_float(ld_nc16(dout + (long long)i * n_out + col), f);
+  if (col < n_out) {
+    for (int i0 = r_begin + rl; i0 < r_end; i0 += 128) {
+      uint4 v[4];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      for (int u = 0; u < 4; ++u)
+        if (i0 + 32 * u < r_end) v[u] = ld_nc16(dout + (long long)(i0 + 32 * u) * n_out + col);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (i0 + 32 * u < r_end) {
+          float f[8];
+          Vec16<__nv_bfloat16>::to_float(v[u], f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] += f[e];
+        }
+      }
     }
+  }
 #pragma unroll
   for (int e = 0; e < 8; ++e) red[rl][cg * 8 + e] = acc[e];
   __syncthreads();
@@ -410,14 +398,16 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const i
 }
 
 // out[e] = sum over the splits that hold rows (in split order) of part[s][e]; zero if there are none.
-// Two arrays (the weight-gradient partials and, optionally, the bias-gradient partials) in one launch.
+// Two arrays (the weight-gradient partials and, optionally, the bias-gradient partials, which have their own row
+// chunks) in one launch.
 __global__ void __launch_bounds__(256)
 split_reduce_kernel(const float* __restrict__ part, long long n, const float* __restrict__ part2, long long n2,
-                    int k_per_split, const int32_t* __restrict__ cu, int n_seg, int capacity, float* __restrict__ out,
-                    float* __restrict__ out2) {
+                    int k_per_split, int rows_per_chunk2, const int32_t* __restrict__ cu, int n_seg, int capacity,
+                    float* __restrict__ out, float* __restrict__ out2) {
   pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
-  const int valid = (rows + k_per_split - 1) / k_per_split;
+  const int valid1 = (rows + k_per_split - 1) / k_per_split;
+  const int valid2 = (rows + rows_per_chunk2 - 1) / rows_per_chunk2;
   const long long n4 = n >> 2, m4 = n2 >> 2;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4 + m4;
        i += (long long)gridDim.x * blockDim.x) {
@@ -425,6 +415,7 @@ split_reduce_kernel(const float* __restrict__ part, long long n, const float* __
     const float* src = second ? part2 : part;
     const long long stride = second ? n2 : n, j = second ? i - n4 : i;
     float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int valid = second ? valid2 : valid1;
     for (int z = 0; z < valid; ++z) {
       const float4 v = __ldg(reinterpret_cast<const float4*>(src + (long long)z * stride) + j);
       s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w;
@@ -453,15 +444,15 @@ size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
   const SplitPlan sp = plan_splits(capacity, n_in, n_out);
   size_t w = (size_t)sp.splits * n_out * n_in * sizeof(float);
   w = (w + 255) & ~(size_t)255;
-  return w + (size_t)sp.splits * n_out * sizeof(float) + 256;
+  return w + (size_t)kColsumChunks * n_out * sizeof(float) + 256;
 }
 
-template <int BN, bool kAMn, bool kBMn, typename OutT, bool kColSum>
+template <int BN, bool kAMn, bool kBMn, typename OutT>
 int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloat16* bias, OutT* out, long long ldo,
                 long long split_stride, int M, int N, int K, const int32_t* cu, int n_seg, int capacity, int dyn_which,
-                int k_per_split, int splits, float* colsum_part, const int32_t* row_map, int accumulate,
+                int k_per_split, int splits, const int32_t* row_map, int accumulate,
                 int32_t* d_status, cudaStream_t st, const char* what) {
-  auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT, kColSum>;
+  auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT>;
   static DeviceOnce attr;  // per instantiation and device
   cudaError_t ea = attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes<BN>()); });
   if (ea != cudaSuccess) { set_cuda_error(ea, what); return SPA_ERR_CUDA; }
@@ -470,7 +461,7 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
   long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * splits;
   const int grid = (int)(tiles < 2 * kNumSMs ? (tiles < 1 ? 1 : tiles) : 2 * kNumSMs);
   launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu,
-             n_seg, capacity, dyn_which, k_per_split, colsum_part, row_map, accumulate, d_status);
+             n_seg, capacity, dyn_which, k_per_split, row_map, accumulate, d_status);
   SPA_CUDA_CHECK_LAUNCH(what);
   return SPA_OK;
 }
@@ -497,9 +488,9 @@ int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, cons
   if (!make_tmap_bf16_2d(&tmA, a, n_in, p.capacity, (uint64_t)n_in * 2, BK, BM) ||
       !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, BK, 128))
     return SPA_ERR_UNSUPPORTED;
-  return launch_gemm<128, false, false, __nv_bfloat16, false>(tmA, tmB, (const __nv_bfloat16*)bias,
+  return launch_gemm<128, false, false, __nv_bfloat16>(tmA, tmB, (const __nv_bfloat16*)bias,
                                                               (__nv_bfloat16*)out, n_out, 0, p.capacity, n_out, n_in,
-                                                              cu, p.B, p.capacity, 1, n_in, 1, nullptr, row_map,
+                                                              cu, p.B, p.capacity, 1, n_in, 1, row_map,
                                                               accumulate ? 1 : 0, d_status, st, "gemm_tc_kernel(fwd)");
 }
 
@@ -522,9 +513,9 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
     int rc = launch_linear_dgrad_pair(p, W, dout, n_in, n_out, cu, da, d_status, st, row_map, accumulate);
     if (rc != SPA_OK) return rc;
   } else if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
-    int rc = launch_gemm<128, false, true, __nv_bfloat16, false>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
+    int rc = launch_gemm<128, false, true, __nv_bfloat16>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
                                                                  p.capacity, n_in, n_out, cu, p.B, p.capacity, 1, n_out,
-                                                                 1, nullptr, row_map, accumulate ? 1 : 0, d_status, st,
+                                                                 1, row_map, accumulate ? 1 : 0, d_status, st,
                                                                  "gemm_tc_kernel(dgrad)");
     if (rc != SPA_OK) return rc;
   }
@@ -534,30 +525,26 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   size_t off = ((size_t)sp.splits * n_out * n_in * sizeof(float) + 255) & ~(size_t)255;
   float* part_b = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + off);
   const long long n_w = (long long)n_out * n_in;
-  if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]; db rides along as column sums of dout
-    int rc;
-    if (db != nullptr)
-      rc = launch_gemm<128, true, true, float, true>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity, cu,
-                                                     p.B, p.capacity, 2, sp.k_per_split, sp.splits, part_b, nullptr, 0, d_status,
-                                                     st, "gemm_tc_kernel(wgrad+colsum)");
-    else
-      rc = launch_gemm<128, true, true, float, false>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity,
-                                                      cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr, nullptr,
-                                                      0, d_status, st, "gemm_tc_kernel(wgrad)");
+  const int rpc = colsum_rows_per_chunk(p.capacity);
+  if (db != nullptr) {  // db[j] = sum_i dout[i][j]: partial sums per row chunk, added up by the reduction below
+    dim3 grid((n_out + 63) / 64, (p.capacity + rpc - 1) / rpc);
+    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity, rpc, part_b);
+    SPA_CUDA_CHECK_LAUNCH("colsum_partial_kernel");
+  }
+  if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]
+    int rc = launch_gemm<128, true, true, float>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity,
+                                                        cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr,
+                                                        0, d_status, st, "gemm_tc_kernel(wgrad)");
     if (rc != SPA_OK) return rc;
     const long long n_b = db != nullptr ? n_out : 0;
     int grid = (int)(((n_w + n_b) / 4 + 255) / 256);
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
-    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.k_per_split, cu, p.B, p.capacity, dW,
+    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.k_per_split, rpc, cu, p.B, p.capacity, dW,
                db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel");
   } else {  // db alone
-    dim3 grid((n_out + 63) / 64, sp.splits);
-    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity,
-               sp.k_per_split, part_b);
-    SPA_CUDA_CHECK_LAUNCH("colsum_partial_kernel");
     launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, part_b, (long long)n_out, (const float*)nullptr,
-               0LL, sp.k_per_split, cu, p.B, p.capacity, db, (float*)nullptr);
+               0LL, rpc, rpc, cu, p.B, p.capacity, db, (float*)nullptr);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
   }
   return SPA_OK;
