@@ -84,8 +84,8 @@ def work_model(cfg, cu):
     w["attn_bwd"] = dict(bytes=(3 + 1 + 1 + 3) * Np * C * es + 4 * H * Np, flops=10 * C * S2, exps=H * S2)
     for name, n_out in (("proj_bwd", C), ("qkv_bwd", 3 * C)):
         w[name + ".da"] = dict(bytes=(Np * n_out + n_out * C + Np * C) * es, flops=2 * Np * C * n_out)
-        w[name + ".dW"] = dict(bytes=(Np * n_out + Np * C) * es + 4 * n_out * C, flops=2 * Np * C * n_out)
-        w[name + ".db"] = dict(bytes=Np * n_out * es + 4 * n_out, flops=Np * n_out)
+        w[name + ".dW"] = dict(bytes=(Np * n_out + Np * C) * es + 4 * n_out * C + 4 * n_out,
+                               flops=2 * Np * C * n_out + Np * n_out)   # dW and db
     w["pack_bwd"] = dict(bytes=2 * Np * C * es + 4 * Np, flops=0)
     # fused unpack: the gate also writes y = x; the projection writes to the tokens (idx read per row)
     w["gate_prefill"] = dict(bytes=2 * BN * C * es + 5 * BN, flops=2 * BN * C)
@@ -96,9 +96,8 @@ def work_model(cfg, cu):
 
 def timing_units(L, blk, d, b_g):
     """The block's calls as (name, thunk) pairs with the linear-layer gradients split the way the step issues them:
-    the input gradient; the weight gradient (split-K product plus its fixed-order reduction), which for the projection
-    also carries the bias gradient; the bias gradient of the QKV layer (a streaming column sum, issued on the main
-    stream while the weight gradient runs on the second one)."""
+    the input gradient, and the weight gradient together with the bias gradient (column sums taken from the tiles
+    that stream through the weight-gradient product; split-K product plus its fixed-order reduction)."""
     p, C = blk.p, blk.C
     fused = blk.fused
     units = []
@@ -136,8 +135,7 @@ def timing_units(L, blk, d, b_g):
         ("qkv_bwd.da", (lambda: L.spa_packed_linear_bwd_scatter(p, blk.xp, d["W_qkv"], blk.dqkv, C, 3 * C, blk.idx, blk.cu,
                                                                  blk.dX, None, None, None, blk.status))
          if fused else lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, blk.dxp, None, None)),
-        ("qkv_bwd.dW", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, blk.dW_qkv, None)),
-        ("qkv_bwd.db", lin(None, None, blk.dqkv, 3 * C, None, None, blk.db_qkv)),
+        ("qkv_bwd.dW", lin(blk.xp, d["W_qkv"], blk.dqkv, 3 * C, None, blk.dW_qkv, blk.db_qkv)),
     ]
     if not fused:
         units.append(("pack_bwd", lambda: L.spa_select_pack_bwd(p, blk.dxp, d["dY"], blk.idx, blk.cu, blk.dX)))
@@ -664,7 +662,7 @@ def main():
         cpu = cpu_baseline(cfg, wl.inps[0], make_inputs, scaled_config)
 
     flop_units = ("gate_pack" if wl.sets[0][2].one_pass else "gate", "qkv", "attn_fwd", "proj", "attn_bwd", "proj_bwd.da", "proj_bwd.dW",
-                  "qkv_bwd.da", "qkv_bwd.dW", "qkv_bwd.db")
+                  "qkv_bwd.da", "qkv_bwd.dW")
     useful_flops = sum(work[k]["flops"] for k in flop_units)
     Np_head = wl.Np_sets[0]
     fused_head = wl.sets[0][2].fused

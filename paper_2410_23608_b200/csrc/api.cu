@@ -547,14 +547,9 @@ int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream)
     if (ov != nullptr) {
       // the second stream's next call reads dqkv: it waits for the attention backward
       rc_side = fork_side(ov, main);
-      // the weight gradient is the longer of the two branches that follow: the bias gradient (a streaming column sum)
-      // goes to the main stream, ahead of the input gradient
       if (rc_side == SPA_OK)
         rc_side = spa_packed_linear_bwd(p, b->x_packed, b->W_qkv, b->dqkv, C, 3 * C, b->cu_seqlens, nullptr, b->dW_qkv,
-                                        nullptr, b->workspace_side, b->d_status, side);
-      if (rc_side == SPA_OK)
-        rc_side = spa_packed_linear_bwd(p, nullptr, nullptr, b->dqkv, C, 3 * C, b->cu_seqlens, nullptr, nullptr, b->db_qkv,
-                                        b->workspace, b->d_status, stream);
+                                        b->db_qkv, b->workspace_side, b->d_status, side);
     }
     float* dW = ov != nullptr ? nullptr : b->dW_qkv;
     float* db = ov != nullptr ? nullptr : b->db_qkv;
