@@ -193,10 +193,9 @@ int spa_packed_attention_fwd(const spa_params* p, const void* qkv, const int32_t
   return launch_attention_fwd_simt(*p, qkv, seg_offsets, n_seg, attn_out, lse, (cudaStream_t)stream);
 }
 
-// spa_packed_attention_bwd; after_kv (optional) is recorded once the key and value thirds of dqkv are complete
-static int attention_bwd(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
-                         const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg, void* dqkv, void* workspace,
-                         int32_t* d_status, void* stream, cudaEvent_t after_kv) {
+int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
+                             const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg, void* dqkv,
+                             void* workspace, int32_t* d_status, void* stream) {
   int rc = check_params(p);
   if (rc != SPA_OK) return rc;
   rc = check_heads(p);
@@ -206,21 +205,11 @@ static int attention_bwd(const spa_params* p, const void* qkv, const void* attn_
   SPA_REQUIRE(n_seg >= 0, SPA_ERR_INVALID_ARG);
   if (use_tc(p) && tc_attention_bwd_supported(*p) && workspace != nullptr) {
     rc = launch_attention_bwd_tc(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace, d_status,
-                                 (cudaStream_t)stream, after_kv);
+                                 (cudaStream_t)stream);
     if (rc != SPA_ERR_UNSUPPORTED) return rc;
   }
-  rc = launch_attention_bwd_simt(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, (cudaStream_t)stream);
-  if (rc == SPA_OK && after_kv != nullptr) {  // one kernel computes all of dqkv here: the event marks its end
-    cudaError_t e = cudaEventRecord(after_kv, (cudaStream_t)stream);
-    if (e != cudaSuccess) { set_cuda_error(e, "attention backward: event"); return SPA_ERR_CUDA; }
-  }
-  return rc;
-}
-
-int spa_packed_attention_bwd(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
-                             const void* d_attn_out, const int32_t* seg_offsets, int32_t n_seg, void* dqkv,
-                             void* workspace, int32_t* d_status, void* stream) {
-  return attention_bwd(p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv, workspace, d_status, stream, nullptr);
+  return launch_attention_bwd_simt(*p, qkv, attn_out, lse, d_attn_out, seg_offsets, n_seg, dqkv,
+                                   (cudaStream_t)stream);
 }
 
 int spa_packed_attention_bwd_static(const spa_params* p, const void* qkv, const void* attn_out, const float* lse,
@@ -433,17 +422,16 @@ int spa_gelu_bwd(const spa_params* p, const void* dh, const void* u, int32_t n_c
 // ---- the block as one unit: sequencing only ------------------------------------------------------------------
 struct spa_overlap {
   cudaStream_t side;
-  cudaEvent_t fork, join, mid;
+  cudaEvent_t fork, join;
 };
 
 int spa_overlap_create(spa_overlap** out) {
   if (out == nullptr) return SPA_ERR_INVALID_ARG;
-  spa_overlap* ov = new (std::nothrow) spa_overlap{nullptr, nullptr, nullptr, nullptr};
+  spa_overlap* ov = new (std::nothrow) spa_overlap{nullptr, nullptr, nullptr};
   if (ov == nullptr) return SPA_ERR_INVALID_ARG;
   cudaError_t e = cudaStreamCreateWithFlags(&ov->side, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ov->fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ov->join, cudaEventDisableTiming);
-  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ov->mid, cudaEventDisableTiming);
   if (e != cudaSuccess) {
     set_cuda_error(e, "spa_overlap_create");
     spa_overlap_destroy(ov);
@@ -455,7 +443,6 @@ int spa_overlap_create(spa_overlap** out) {
 
 int spa_overlap_destroy(spa_overlap* ov) {
   if (ov == nullptr) return SPA_OK;
-  if (ov->mid != nullptr) cudaEventDestroy(ov->mid);
   if (ov->join != nullptr) cudaEventDestroy(ov->join);
   if (ov->fork != nullptr) cudaEventDestroy(ov->fork);
   if (ov->side != nullptr) cudaStreamDestroy(ov->side);
@@ -553,29 +540,11 @@ int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream)
     rc = spa_packed_linear_bwd(p, b->attn_out, b->W_o, b->dz, C, C, b->cu_seqlens, b->d_attn_out, nullptr, nullptr,
                                b->workspace, b->d_status, stream);
   }
-  // With the second stream and tensor-core sizes, the weight gradient of the QKV layer is cut by thirds: the key and
-  // value thirds of dqkv are complete when the first attention pass ends, so their weight and bias gradients run
-  // under the dQ pass; only the query third is left for the end, beside the input gradient.
-  const bool sliced = ov != nullptr && use_tc(p) && b->workspace_side != nullptr && tc_linear_supported(C, C) &&
-                      tc_linear_supported(C, 2 * C) && tc_attention_bwd_supported(*p) && b->dW_qkv != nullptr &&
-                      b->db_qkv != nullptr;
   if (rc == SPA_OK && rc_side == SPA_OK)
-    rc = attention_bwd(p, b->qkv, b->attn_out, b->lse, b->d_attn_out, seg, n_seg, b->dqkv, b->workspace, b->d_status,
-                       stream, sliced ? ov->mid : nullptr);
+    rc = spa_packed_attention_bwd(p, b->qkv, b->attn_out, b->lse, b->d_attn_out, seg, n_seg, b->dqkv, b->workspace,
+                                  b->d_status, stream);
   if (rc == SPA_OK && rc_side == SPA_OK) {
-    if (sliced) {
-      const __nv_bfloat16* dq = reinterpret_cast<const __nv_bfloat16*>(b->dqkv);
-      cudaError_t e = cudaStreamWaitEvent(ov->side, ov->mid, 0);
-      if (e != cudaSuccess) { set_cuda_error(e, "spa_block_bwd: wait"); rc_side = SPA_ERR_CUDA; }
-      if (rc_side == SPA_OK)   // dW, db of the key and value thirds (rows C .. 3C of dW_qkv)
-        rc_side = launch_linear_bwd_tc(*p, b->x_packed, nullptr, dq + C, C, 2 * C, b->cu_seqlens, nullptr,
-                                       b->dW_qkv + (size_t)C * C, b->db_qkv + C, b->workspace_side, b->d_status, ov->side,
-                                       nullptr, false, 3 * C);
-      if (rc_side == SPA_OK) rc_side = fork_side(ov, main);
-      if (rc_side == SPA_OK)   // the query third, once the dQ pass has finished
-        rc_side = launch_linear_bwd_tc(*p, b->x_packed, nullptr, dq, C, C, b->cu_seqlens, nullptr, b->dW_qkv, b->db_qkv,
-                                       b->workspace_side, b->d_status, ov->side, nullptr, false, 3 * C);
-    } else if (ov != nullptr) {
+    if (ov != nullptr) {
       // the second stream's next call reads dqkv: it waits for the attention backward
       rc_side = fork_side(ov, main);
       if (rc_side == SPA_OK)

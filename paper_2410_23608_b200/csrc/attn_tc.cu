@@ -692,6 +692,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
 #pragma unroll
         for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
       }
+      if (half == 0) delta[(long long)h * capacity + row] = my_D;
     }
 
     constexpr int kPc = kBwdY / 2;  // fp32 columns of each tile owned by this thread
@@ -1134,35 +1135,6 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
 }
 
 
-// D_i = dO_i . O_i per head for every valid packed row (the row term of the softmax gradient), ahead of both passes:
-// one warp per packed row, 16-byte loads of the two rows, the lanes that share a head add up through shuffles.
-template <int D>
-__global__ void __launch_bounds__(256)
-attn_delta_kernel(const uint4* __restrict__ o16, const uint4* __restrict__ do16, const int32_t* __restrict__ seg, int n_seg,
-                  int capacity, int C, float* __restrict__ delta) {
-  pdl_entry();
-  const int Np = packed_rows(seg, n_seg, capacity);
-  const int lane = threadIdx.x & 31;
-  const int Q = C / 8;               // 16-byte chunks per row
-  constexpr int kLanesPerHead = D / 8;
-  for (int row = blockIdx.x * 8 + (threadIdx.x >> 5); row < Np; row += gridDim.x * 8) {
-    for (int c0 = 0; c0 < Q; c0 += 32) {
-      const int c = c0 + lane;
-      float acc = 0.f;
-      if (c < Q) {
-        float a[8], b[8];
-        Vec16<__nv_bfloat16>::to_float(ld_nc16(o16 + (size_t)row * Q + c), a);
-        Vec16<__nv_bfloat16>::to_float(ld_nc16(do16 + (size_t)row * Q + c), b);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc = fmaf(a[e], b[e], acc);
-      }
-#pragma unroll
-      for (int o = 1; o < kLanesPerHead; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (c < Q && (lane & (kLanesPerHead - 1)) == 0) delta[(long long)(c / kLanesPerHead) * capacity + row] = acc;
-    }
-  }
-}
-
 // Which kernel runs the dK / dV pass for head dimension D.
 template <int D> struct kv_pass {
   static constexpr int kThreads = kBwdThreads;
@@ -1177,8 +1149,7 @@ template <> struct kv_pass<64> {
 
 template <int D>
 int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
-               const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st,
-               cudaEvent_t after_kv) {
+               const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status, cudaStream_t st) {
   CUtensorMap tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o;  // own tiles: 128-row boxes; streamed tiles: 64-row boxes
   if (!make_tmap_bf16_2d(&tm_qkv, qkv, 3ull * p.C, p.capacity, 6ull * p.C, D, 128, D * 2) ||
       !make_tmap_bf16_2d(&tm_do, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2) ||
@@ -1197,22 +1168,12 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
   dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
-  // D_i first, then the dK / dV pass (which reads it), then the dQ pass: the key and value thirds of dqkv are
-  // complete while the dQ pass still runs, so their weight gradient can start under it
-  int dgrid = (p.capacity + 7) / 8;
-  if (dgrid > kNumSMs * 8) dgrid = kNumSMs * 8;
-  launch_pdl(attn_delta_kernel<D>, dgrid, 256, 0, st, (const uint4*)ao, (const uint4*)dao, seg, n_seg, p.capacity, p.C, delta);
-  SPA_CUDA_CHECK_LAUNCH("attn_delta_kernel");
-  launch_pdl(kkv, grid, kv_pass<D>::kThreads, kv_pass<D>::kSmem, st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
-  SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
-  if (after_kv != nullptr) {
-    cudaError_t e = cudaEventRecord(after_kv, st);
-    if (e != cudaSuccess) { set_cuda_error(e, "attention backward: event"); return SPA_ERR_CUDA; }
-  }
   launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D, true>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
              n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
+  launch_pdl(kkv, grid, kv_pass<D>::kThreads, kv_pass<D>::kSmem, st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
+  SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
   return SPA_OK;
 }
 
@@ -1249,9 +1210,9 @@ size_t tc_attention_workspace_bytes(const spa_params& p) {
 
 int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                             const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
-                            cudaStream_t st, cudaEvent_t after_kv) {
-  return p.C / p.H == 64 ? bwd_launch<64>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st, after_kv)
-                         : bwd_launch<32>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st, after_kv);
+                            cudaStream_t st) {
+  return p.C / p.H == 64 ? bwd_launch<64>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st)
+                         : bwd_launch<32>(p, qkv, ao, lse, dao, seg, n_seg, dqkv, workspace, d_status, st);
 }
 
 int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,

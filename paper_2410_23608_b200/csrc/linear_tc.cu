@@ -354,8 +354,8 @@ constexpr int kColsumChunks = 64;  // row chunks over the allocated rows (rows p
 inline int colsum_rows_per_chunk(int capacity) { return (((capacity + kColsumChunks - 1) / kColsumChunks) + 7) & ~7; }
 
 __global__ void __launch_bounds__(256)
-colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, long long ld, int n_out, const int32_t* __restrict__ cu,
-                      int n_seg, int capacity, int rows_per_chunk, float* __restrict__ part) {
+colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const int32_t* __restrict__ cu, int n_seg,
+                      int capacity, int rows_per_chunk, float* __restrict__ part) {
   pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
   const int r_begin = blockIdx.y * rows_per_chunk;
@@ -371,7 +371,7 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, long long ld, int 
       uint4 v[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        if (i0 + 32 * u < r_end) v[u] = ld_nc16(dout + (long long)(i0 + 32 * u) * ld + col);
+        if (i0 + 32 * u < r_end) v[u] = ld_nc16(dout + (long long)(i0 + 32 * u) * n_out + col);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         if (i0 + 32 * u < r_end) {
@@ -474,13 +474,9 @@ bool tc_linear_supported(int n_in, int n_out) {
 
 size_t tc_linear_workspace_bytes(const spa_params& p) {
   if (p.dtype != SPA_BF16 || !tc_linear_supported(p.C, 3 * p.C)) return 0;
-  // the largest of the shapes the block issues: the whole QKV layer, two thirds of it, one third (= the projection)
-  size_t w = 0;
-  for (int k = 1; k <= 3; ++k) {
-    const size_t v = wgrad_workspace_bytes(p.capacity, p.C, k * p.C);
-    if (v > w) w = v;
-  }
-  return w;
+  const size_t a = wgrad_workspace_bytes(p.capacity, p.C, 3 * p.C);
+  const size_t b = wgrad_workspace_bytes(p.capacity, p.C, p.C);
+  return a > b ? a : b;
 }
 
 int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, const void* bias, int n_in, int n_out,
@@ -500,16 +496,12 @@ int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, cons
 
 int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
                          const int32_t* cu, void* da, float* dW, float* db, void* workspace, int32_t* d_status,
-                         cudaStream_t st, const int32_t* row_map, bool accumulate, int dout_ld) {
+                         cudaStream_t st, const int32_t* row_map, bool accumulate) {
   CUtensorMap tmA, tmB, tmA2, tmB2;
-  // dout may be a column slice of a wider matrix (the weight gradient of one third of the QKV layer): rows of n_out
-  // values, dout_ld elements apart; the input gradient sums over all columns and takes the whole matrix only
-  if (dout_ld <= 0) dout_ld = n_out;
-  if (da != nullptr && dout_ld != n_out) return SPA_ERR_INVALID_ARG;
   if (da != nullptr && (!make_tmap_bf16_2d(&tmA, dout, n_out, p.capacity, (uint64_t)n_out * 2, BK, BM) ||
                         !make_tmap_bf16_2d(&tmB, W, n_in, n_out, (uint64_t)n_in * 2, 64, BK)))
     return SPA_ERR_UNSUPPORTED;
-  if (dW != nullptr && (!make_tmap_bf16_2d(&tmA2, dout, n_out, p.capacity, (uint64_t)dout_ld * 2, 64, BK) ||
+  if (dW != nullptr && (!make_tmap_bf16_2d(&tmA2, dout, n_out, p.capacity, (uint64_t)n_out * 2, 64, BK) ||
                         !make_tmap_bf16_2d(&tmB2, a, n_in, p.capacity, (uint64_t)n_in * 2, 64, BK)))
     return SPA_ERR_UNSUPPORTED;
   // A pair CTA owns its SM (all 512 TMEM columns, 175 KB of shared memory).  A call that asks for da alone is
@@ -536,8 +528,7 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   const int rpc = colsum_rows_per_chunk(p.capacity);
   if (db != nullptr) {  // db[j] = sum_i dout[i][j]: partial sums per row chunk, added up by the reduction below
     dim3 grid((n_out + 63) / 64, (p.capacity + rpc - 1) / rpc);
-    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, (long long)dout_ld, n_out, cu, p.B,
-               p.capacity, rpc, part_b);
+    launch_pdl(colsum_partial_kernel, grid, 256, 0, st, (const __nv_bfloat16*)dout, n_out, cu, p.B, p.capacity, rpc, part_b);
     SPA_CUDA_CHECK_LAUNCH("colsum_partial_kernel");
   }
   if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]

@@ -15,7 +15,7 @@ int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, cons
                          const int32_t* row_map = nullptr, bool accumulate = false);
 int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, const void* dout, int n_in, int n_out,
                          const int32_t* cu, void* da, float* dW, float* db, void* workspace, int32_t* d_status,
-                         cudaStream_t st, const int32_t* row_map = nullptr, bool accumulate = false, int dout_ld = 0);
+                         cudaStream_t st, const int32_t* row_map = nullptr, bool accumulate = false);
 
 // CTA-pair variants (cta_group::2, 256 x 256 tiles) of the forward product and the input gradient
 bool tc_pair_linear_supported(const spa_params& p, int n_in, int n_out);
@@ -29,11 +29,9 @@ bool tc_attention_fwd_supported(const spa_params& p);
 int launch_attention_fwd_tc(const spa_params& p, const void* qkv, const int32_t* seg, int n_seg, void* ao, float* lse,
                             int32_t* d_status, cudaStream_t st);
 bool tc_attention_bwd_supported(const spa_params& p);
-// The dK / dV pass runs first, the dQ pass second; `after_kv` (optional) is recorded on `st` between them, when the
-// key and value thirds of dqkv are complete.
 int launch_attention_bwd_tc(const spa_params& p, const void* qkv, const void* ao, const float* lse, const void* dao,
                             const int32_t* seg, int n_seg, void* dqkv, void* workspace, int32_t* d_status,
-                            cudaStream_t st, cudaEvent_t after_kv = nullptr);
+                            cudaStream_t st);
 // Device address, on the current device, of the SPA_STATIC_SCRATCH_BYTES array built into the library.
 int static_attention_scratch(void** out);
 
