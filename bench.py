@@ -272,10 +272,10 @@ def run_reference(args):
 class Workload:
     """Rotating buffer sets of one workload, its whole-step graphs and its per-unit timings."""
 
-    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=False):
+    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=False, overlap=True):
         from paper_2410_23608_b200.block import SpaBlock
         from spa_workloads import make_inputs, scaled_config
-        self.torch, self.L, self.cfg = torch, L, cfg
+        self.torch, self.L, self.cfg, self.overlap = torch, L, cfg, overlap
         x_bytes = cfg.B * cfg.N * cfg.C * cfg.elem_size
         # enough sets that even the smallest single tensor a call streams (x) exceeds L2 over one rotation
         self.n_sets = sets if sets > 0 else min(24, max(3, int(np.ceil(1.3 * L2_BYTES / x_bytes))))
@@ -298,8 +298,9 @@ class Workload:
             self.step_graphs.append(g)
             self.launches_per_step = n
 
-    def step_fn(self, s, backward, overlap=True, container_len=0):
+    def step_fn(self, s, backward, container_len=0):
         inp, d, blk = self.sets[s]
+        overlap = self.overlap
 
         def run():
             blk.forward(d["x"], d["w_g"], inp.b_g, d["W_qkv"], d["b_qkv"], d["W_o"], d["b_o"], container_len=container_len)
@@ -459,6 +460,7 @@ def main():
     ap.add_argument("--no-per-config", action="store_true", help="time the headline workload only")
     ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
     ap.add_argument("--one-pass-pack", action="store_true", help="gate, selection and packing as one kernel (spa_gate_select_pack) instead of two")
+    ap.add_argument("--no-overlap", action="store_true", help="weight gradients on the main stream too (no second stream)")
     ap.add_argument("--train", action="store_true", help="also time the trainable-selection calls (loss, gated pack backward, gate backward)")
     ap.add_argument("--layer", action="store_true", help="also time the whole pre-norm block (LayerNorm, SPA, feed-forward) and its new calls")
     args = ap.parse_args()
@@ -487,7 +489,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     cfg = get_config(args.config)
-    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=args.one_pass_pack)
+    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=args.one_pass_pack, overlap=not args.no_overlap)
     stream = wl.stream
     n_sets = wl.n_sets
     wl.warm(args.warmup)
@@ -684,7 +686,7 @@ def main():
             if ci == args.config:
                 continue
             c2 = get_config(ci)
-            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=args.one_pass_pack)
+            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=args.one_pass_pack, overlap=not args.no_overlap)
             w2.warm(20)
             steps2 = 200
             ms2 = w2.time_steps(steps2) / steps2
