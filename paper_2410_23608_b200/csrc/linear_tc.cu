@@ -85,26 +85,6 @@ template <int BN> __host__ __device__ constexpr int gemm_smem_bytes() { return k
 // Tile bookkeeping shared by the three roles of the persistent kernel.
 struct TileCoord { int m0, n0, z, n_t; };
 
-// Split-K plan of a weight gradient, made on the device from the packed row count (K = rows): rows per split, a
-// multiple of BK.  `tiles` output tiles times s splits are work items for `slots` resident CTAs; an item costs its
-// k-blocks plus a fixed part (accumulator drain, fp32 stores), and every split adds a pass of the reduction that
-// follows.  The count with the lowest cost wins, the smaller one on a tie; the same inputs give the same plan in every
-// CTA and in the reduction kernel, so results stay reproducible for a given selection.
-constexpr int kMaxSplits = 8;
-__host__ __device__ inline int wgrad_rows_per_split(int rows, int tiles, int max_splits, int slots) {
-  const int kb = (rows + BK - 1) / BK;
-  if (kb <= 1 || tiles <= 0 || slots <= 0) return BK * (kb > 0 ? kb : 1);
-  int best_len = kb, best_cost = 0x7fffffff;
-  for (int s = 1; s <= max_splits && s <= kb; ++s) {
-    const int len = (kb + s - 1) / s;          // k-blocks per item
-    const int used = (kb + len - 1) / len;     // splits that hold rows
-    const int rounds = (tiles * used + slots - 1) / slots;
-    const int cost = rounds * (len + 3) + used;
-    if (cost < best_cost) { best_cost = cost; best_len = len; }
-  }
-  return best_len * BK;
-}
-
 // dyn_which: 1 = M is the device-side packed row count, 2 = K is.
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... of the (m, n, split) space
 // that the device-side row count leaves; two accumulator stages in TMEM let the epilogue of one tile
@@ -116,7 +96,7 @@ __global__ void __launch_bounds__(kGemmThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
                long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
-               int dyn_which, int k_per_split, int max_splits, const int32_t* __restrict__ row_map,
+               int dyn_which, int k_per_split, const int32_t* __restrict__ row_map,
                int accumulate, int32_t* d_status) {
   constexpr int kStage = stage_bytes<BN>();
   constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
@@ -158,8 +138,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   const int tiles_n = (N + BN - 1) / BN;
   const int tiles_m = (M + BM - 1) / BM;
-  // weight gradient: the split of K = packed rows is planned here, from the row count the selection produced
-  if (dyn_which == 2 && max_splits > 0) k_per_split = wgrad_rows_per_split(K, tiles_m * tiles_n, max_splits, gridDim.x);
   const int n_splits = K > 0 ? (K + k_per_split - 1) / k_per_split : 0;
   const int total = tiles_m * tiles_n * n_splits;
   auto coord = [&](int tile) {
@@ -424,13 +402,10 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const i
 // chunks) in one launch.
 __global__ void __launch_bounds__(256)
 split_reduce_kernel(const float* __restrict__ part, long long n, const float* __restrict__ part2, long long n2,
-                    int k_per_split, int plan_tiles, int plan_max_splits, int plan_slots, int rows_per_chunk2,
-                    const int32_t* __restrict__ cu, int n_seg, int capacity, float* __restrict__ out,
-                    float* __restrict__ out2) {
+                    int k_per_split, int rows_per_chunk2, const int32_t* __restrict__ cu, int n_seg, int capacity,
+                    float* __restrict__ out, float* __restrict__ out2) {
   pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
-  // the plan the weight-gradient kernel made for these rows (plan_tiles > 0), else the caller's rows per split
-  if (plan_tiles > 0) k_per_split = wgrad_rows_per_split(rows, plan_tiles, plan_max_splits, plan_slots);
   const int valid1 = (rows + k_per_split - 1) / k_per_split;
   const int valid2 = (rows + rows_per_chunk2 - 1) / rows_per_chunk2;
   const long long n4 = n >> 2, m4 = n2 >> 2;
@@ -449,22 +424,25 @@ split_reduce_kernel(const float* __restrict__ part, long long n, const float* __
   }
 }
 
-// Splits the device-side plan may use: up to kMaxSplits, fewer where the fp32 partials of one split are large.
-int wgrad_max_splits(int n_in, int n_out) {
-  const size_t one = (size_t)n_out * n_in * sizeof(float);
-  size_t s = ((size_t)256 << 20) / (one > 0 ? one : 1);
-  if (s > (size_t)kMaxSplits) s = kMaxSplits;
-  return s < 1 ? 1 : (int)s;
-}
+struct SplitPlan { int splits, k_per_split; };
 
-inline int wgrad_tiles(int n_in, int n_out) { return ((n_out + BM - 1) / BM) * ((n_in + 127) / 128); }
-inline int wgrad_grid(int n_in, int n_out) {
-  const long long items = (long long)wgrad_tiles(n_in, n_out) * wgrad_max_splits(n_in, n_out);
-  return (int)(items < 2 * kNumSMs ? items : 2 * kNumSMs);
+// K = packed rows is cut into equal spans (multiples of BK) so that tiles x splits fills the GPU.
+SplitPlan plan_splits(int capacity, int n_in, int n_out) {
+  const int tiles = ((n_out + BM - 1) / BM) * ((n_in + 127) / 128);
+  int splits = (2 * kNumSMs + tiles - 1) / tiles;
+  const int max_by_rows = (capacity + BK - 1) / BK;
+  if (splits > max_by_rows) splits = max_by_rows;
+  if (splits > 32) splits = 32;
+  if (splits < 1) splits = 1;
+  int kps = (capacity + splits - 1) / splits;
+  kps = ((kps + BK - 1) / BK) * BK;
+  splits = (capacity + kps - 1) / kps;
+  return {splits, kps};
 }
 
 size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
-  size_t w = (size_t)wgrad_max_splits(n_in, n_out) * n_out * n_in * sizeof(float);
+  const SplitPlan sp = plan_splits(capacity, n_in, n_out);
+  size_t w = (size_t)sp.splits * n_out * n_in * sizeof(float);
   w = (w + 255) & ~(size_t)255;
   return w + (size_t)kColsumChunks * n_out * sizeof(float) + 256;
 }
@@ -472,7 +450,7 @@ size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
 template <int BN, bool kAMn, bool kBMn, typename OutT>
 int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloat16* bias, OutT* out, long long ldo,
                 long long split_stride, int M, int N, int K, const int32_t* cu, int n_seg, int capacity, int dyn_which,
-                int k_per_split, int splits, int max_splits, const int32_t* row_map, int accumulate,
+                int k_per_split, int splits, const int32_t* row_map, int accumulate,
                 int32_t* d_status, cudaStream_t st, const char* what) {
   auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT>;
   static DeviceOnce attr;  // per instantiation and device
@@ -480,10 +458,10 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
   if (ea != cudaSuccess) { set_cuda_error(ea, what); return SPA_ERR_CUDA; }
   // persistent grid: two CTAs per SM (99 KB of shared memory and 256 TMEM columns each), never more
   // CTAs than there are tiles when every allocated row is in use
-  long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * (max_splits > 0 ? max_splits : splits);
+  long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * splits;
   const int grid = (int)(tiles < 2 * kNumSMs ? (tiles < 1 ? 1 : tiles) : 2 * kNumSMs);
   launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu,
-             n_seg, capacity, dyn_which, k_per_split, max_splits, row_map, accumulate, d_status);
+             n_seg, capacity, dyn_which, k_per_split, row_map, accumulate, d_status);
   SPA_CUDA_CHECK_LAUNCH(what);
   return SPA_OK;
 }
@@ -512,7 +490,7 @@ int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, cons
     return SPA_ERR_UNSUPPORTED;
   return launch_gemm<128, false, false, __nv_bfloat16>(tmA, tmB, (const __nv_bfloat16*)bias,
                                                               (__nv_bfloat16*)out, n_out, 0, p.capacity, n_out, n_in,
-                                                              cu, p.B, p.capacity, 1, n_in, 1, 0, row_map,
+                                                              cu, p.B, p.capacity, 1, n_in, 1, row_map,
                                                               accumulate ? 1 : 0, d_status, st, "gemm_tc_kernel(fwd)");
 }
 
@@ -537,14 +515,14 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   } else if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
     int rc = launch_gemm<128, false, true, __nv_bfloat16>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
                                                                  p.capacity, n_in, n_out, cu, p.B, p.capacity, 1, n_out,
-                                                                 1, 0, row_map, accumulate ? 1 : 0, d_status, st,
+                                                                 1, row_map, accumulate ? 1 : 0, d_status, st,
                                                                  "gemm_tc_kernel(dgrad)");
     if (rc != SPA_OK) return rc;
   }
   if (dW == nullptr && db == nullptr) return SPA_OK;
-  const int max_splits = wgrad_max_splits(n_in, n_out);
+  const SplitPlan sp = plan_splits(p.capacity, n_in, n_out);
   float* part_w = reinterpret_cast<float*>(workspace);
-  size_t off = ((size_t)max_splits * n_out * n_in * sizeof(float) + 255) & ~(size_t)255;
+  size_t off = ((size_t)sp.splits * n_out * n_in * sizeof(float) + 255) & ~(size_t)255;
   float* part_b = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + off);
   const long long n_w = (long long)n_out * n_in;
   const int rpc = colsum_rows_per_chunk(p.capacity);
@@ -555,18 +533,18 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   }
   if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]
     int rc = launch_gemm<128, true, true, float>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity,
-                                                        cu, p.B, p.capacity, 2, BK, 1, max_splits, nullptr,
+                                                        cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr,
                                                         0, d_status, st, "gemm_tc_kernel(wgrad)");
     if (rc != SPA_OK) return rc;
     const long long n_b = db != nullptr ? n_out : 0;
     int grid = (int)(((n_w + n_b) / 4 + 255) / 256);
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
-    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, BK, wgrad_tiles(n_in, n_out), max_splits,
-               wgrad_grid(n_in, n_out), rpc, cu, p.B, p.capacity, dW, db);
+    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.k_per_split, rpc, cu, p.B, p.capacity, dW,
+               db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel");
   } else {  // db alone
     launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, part_b, (long long)n_out, (const float*)nullptr,
-               0LL, rpc, 0, 0, 0, rpc, cu, p.B, p.capacity, db, (float*)nullptr);
+               0LL, rpc, rpc, cu, p.B, p.capacity, db, (float*)nullptr);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
   }
   return SPA_OK;
