@@ -5,13 +5,14 @@
 // walks the key range spanned by the segments of those rows in tiles of 128 keys; cu_seqlens alone
 // decides the range, so no padding token is ever loaded or multiplied.  Per key tile:
 //   S = Q K^T        tcgen05.mma, Q and K tiles staged by TMA (K two tiles ahead, V one), S in TMEM (fp32)
-//   P = exp2(S - m)  one thread per query row pulls its S row into registers in one TMEM pass, masks keys
-//                    outside the row's own segment, updates the running max / sum, writes P back as bf16
-//   O_t = P V        tcgen05.mma with P read from TMEM and V from shared memory
-//   O = alpha O + O_t in registers (fp32), so TMEM never needs a rescaling pass.
-// The next tile's S product is issued as soon as every thread holds the current S row, so the tensor
-// core works under the softmax; the O tile is folded in one iteration late for the same reason.
-// K/V rows past the last valid packed row are unspecified memory: K columns are masked after the
+//   P = exp2(S - m)  two threads per query row pull their halves of the S row into registers in one TMEM pass, mask
+//                    keys outside the row's own segment, update the running sum, write P back to TMEM as bf16
+//   O += P V         tcgen05.mma with P read from TMEM and V from shared memory; O accumulates in TMEM over all tiles
+// m is the maximum that the stored P and O refer to.  It is raised - and O rescaled, TMEM -> registers -> TMEM - only
+// when a row's true maximum has outgrown it by more than 2^8, so most tiles cost no pass over O; sums and outputs are
+// exact for any reference value.  The first lane of a ninth warp issues every copy and every product: the next tile's
+// S product is issued as soon as every softmax warp holds the current S row, so the tensor core works under the
+// softmax.  K/V rows past the last valid packed row are unspecified memory: K columns are masked after the
 // product and V lines are zeroed in shared memory before the product.
 #include <math_constants.h>
 

@@ -54,6 +54,9 @@ def assert_close(got, ref, dtype, what, scale_max_abs=False):
     bound = tol["max_abs"]
     if scale_max_abs and np.asarray(ref).size:
         bound *= max(1.0, float(np.abs(ref).max()))
+        # shown with `pytest -s`: which tensors need the scaled bound, and by how much
+        print(f"{what}: max-abs {max_abs:.3e} (flat bound {tol['max_abs']:.1e}, scaled bound {bound:.3e}, "
+              f"max |ref| {float(np.abs(ref).max()):.3e}), rel-rms {rel_rms:.3e}")
     assert max_abs <= bound, f"{what}: max-abs {max_abs:.3e} > {bound:.3e} (rel-rms {rel_rms:.3e})"
     if tol["rel_rms"] is not None:
         assert rel_rms <= tol["rel_rms"], f"{what}: rel-rms {rel_rms:.3e} > {tol['rel_rms']:.1e}"
