@@ -272,7 +272,7 @@ def run_reference(args):
 class Workload:
     """Rotating buffer sets of one workload, its whole-step graphs and its per-unit timings."""
 
-    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=False, overlap=True):
+    def __init__(self, torch, L, cfg, no_fuse=False, sets=0, one_pass=False, overlap=True, flags=0):
         from paper_2410_23608_b200.block import SpaBlock
         from spa_workloads import make_inputs, scaled_config
         self.torch, self.L, self.cfg, self.overlap = torch, L, cfg, overlap
@@ -286,7 +286,7 @@ class Workload:
             inp = make_inputs(scaled_config(cfg, seed=cfg.seed + 1000 * s)) if s < 2 else self.inps[s % 2]
             self.inps.append(inp)
             d = {n: inp.torch(n, "cuda") for n in names}
-            blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau, fused=False if no_fuse else None, one_pass=one_pass)
+            blk = SpaBlock(cfg.B, cfg.N, cfg.C, cfg.H, cfg.dtype, tau=cfg.tau, flags=flags, fused=False if no_fuse else None, one_pass=one_pass)
             self.sets.append((inp, d, blk))
         self.stream = torch.cuda.current_stream()
         for s in range(self.n_sets):     # eager pass: first-use set-up (attributes, tensor maps) outside capture
@@ -460,6 +460,7 @@ def main():
     ap.add_argument("--no-per-config", action="store_true", help="time the headline workload only")
     ap.add_argument("--no-fuse", action="store_true", help="separate projection / scatter kernels instead of the fused calls")
     ap.add_argument("--one-pass-pack", action="store_true", help="gate, selection and packing as one kernel (spa_gate_select_pack) instead of two")
+    ap.add_argument("--one-pass-bwd", action="store_true", help="attention backward: one-pass kernel for segments of at most 128 rows (SPA_FLAG_ONE_PASS_BWD)")
     ap.add_argument("--no-overlap", action="store_true", help="weight gradients on the main stream too (no second stream)")
     ap.add_argument("--train", action="store_true", help="also time the trainable-selection calls (loss, gated pack backward, gate backward)")
     ap.add_argument("--layer", action="store_true", help="also time the whole pre-norm block (LayerNorm, SPA, feed-forward) and its new calls")
@@ -489,7 +490,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     cfg = get_config(args.config)
-    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=args.one_pass_pack, overlap=not args.no_overlap)
+    wl = Workload(torch, L, cfg, no_fuse=args.no_fuse, sets=args.sets, one_pass=args.one_pass_pack, overlap=not args.no_overlap, flags=64 if args.one_pass_bwd else 0)
     stream = wl.stream
     n_sets = wl.n_sets
     wl.warm(args.warmup)
@@ -686,7 +687,7 @@ def main():
             if ci == args.config:
                 continue
             c2 = get_config(ci)
-            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=args.one_pass_pack, overlap=not args.no_overlap)
+            w2 = Workload(torch, L, c2, no_fuse=args.no_fuse, one_pass=args.one_pass_pack, overlap=not args.no_overlap, flags=64 if args.one_pass_bwd else 0)
             w2.warm(20)
             steps2 = 200
             ms2 = w2.time_steps(steps2) / steps2

@@ -55,8 +55,11 @@ enum {
   SPA_FLAG_GATE_SCALE = 4,/* Eq. 5: packed rows are scaled by sigmoid(score)               */
   SPA_FLAG_SIMT_ONLY = 8, /* bf16 only: run the fp32-FMA kernels instead of the tensor-core ones */
   SPA_FLAG_NO_CTA_PAIRS = 16,/* wide linear layers: keep the one-CTA tensor-core kernels (no CTA pairs) */
-  SPA_FLAG_UNFUSED = 32   /* spa_block_fwd / spa_block_bwd: separate projection, scatter and gather kernels even
+  SPA_FLAG_UNFUSED = 32,  /* spa_block_fwd / spa_block_bwd: separate projection, scatter and gather kernels even
                              where the fused calls apply                                                      */
+  SPA_FLAG_ONE_PASS_BWD = 64 /* attention backward (tensor-core problems): segments of at most 128 rows are handled by
+                             a kernel that owns a whole segment and evaluates S, P, dP, dS once; the two-pass kernels
+                             take the longer segments only.  Same results within the stated tolerances               */
 };
 
 typedef struct spa_params {

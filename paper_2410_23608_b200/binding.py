@@ -22,6 +22,7 @@ SPA_STATIC_SCRATCH_BYTES = 4 << 20
 SPA_F32, SPA_BF16 = 0, 1
 SPA_FLAG_RESIDUAL, SPA_FLAG_INPLACE, SPA_FLAG_GATE_SCALE, SPA_FLAG_SIMT_ONLY, SPA_FLAG_NO_CTA_PAIRS = 1, 2, 4, 8, 16
 SPA_FLAG_UNFUSED = 32
+SPA_FLAG_ONE_PASS_BWD = 64
 
 EXPORTS = (
     "spa_workspace_bytes", "spa_gate", "spa_select_pack", "spa_packed_qkv", "spa_packed_attention_fwd",

@@ -65,6 +65,20 @@ __device__ __forceinline__ RowSeg row_segment_staged(const int32_t* s_off, int n
   return r;
 }
 
+constexpr int kShortMax = 128;  // segments of at most this many rows are taken by the one-pass backward kernel
+
+// Does the tile of packed rows [r0, r0 + 128) hold a row of a segment longer than kShortMax?  Such a segment covers
+// the tile's first or its last valid row (one that lies strictly inside the tile has fewer rows than the tile), so two
+// searches decide.  Every thread of a CTA gets the same answer.
+__device__ __forceinline__ bool tile_has_long_rows(const int32_t* s_off, const int32_t* g_off, bool staged, int n_seg, int Np,
+                                                   int r0) {
+  const int last = r0 + 127 < Np - 1 ? r0 + 127 : Np - 1;
+  const RowSeg a = staged ? row_segment_staged(s_off, n_seg, Np, r0) : row_segment(g_off, n_seg, Np, r0);
+  if (a.hi - a.lo > kShortMax) return true;
+  const RowSeg b = staged ? row_segment_staged(s_off, n_seg, Np, last) : row_segment(g_off, n_seg, Np, last);
+  return b.hi - b.lo > kShortMax;
+}
+
 // Rotation of the 16-byte chunks of row r of a [128][D] bf16 tile in shared memory that makes the
 // accesses of 8 neighbouring rows to one chunk index fall into different banks.
 template <int D> __device__ __forceinline__ int chunk_rot(int r) { return D == 64 ? (r & 7) : ((r >> 1) & 3); }
@@ -73,12 +87,13 @@ template <int D> __device__ __forceinline__ int chunk_rot(int r) { return D == 6
 // c ^ chunk_rot(r)) to rows r0.. of a matrix with `ld` elements per row: a warp covers whole rows, so the
 // stores are full 64- or 128-byte lines.  Rows from Np on are not written.
 template <int D, int kThreads>
-__device__ __forceinline__ void copy_tile_out(const uint8_t* tile, __nv_bfloat16* dst, long long ld, int r0, int Np, int tid) {
+__device__ __forceinline__ void copy_tile_out(const uint8_t* tile, __nv_bfloat16* dst, long long ld, int r0, int Np, int tid,
+                                              const volatile uint8_t* row_ok = nullptr) {
   constexpr int kChunks = D * 2 / 16;
 #pragma unroll
   for (int i = tid; i < 128 * kChunks; i += kThreads) {
     const int r = i / kChunks, c = i % kChunks;
-    if (r0 + r < Np)
+    if (r0 + r < Np && (row_ok == nullptr || row_ok[r]))
       *reinterpret_cast<uint4*>(dst + (long long)(r0 + r) * ld + c * 8) =
           *reinterpret_cast<const uint4*>(tile + r * (D * 2) + ((c ^ chunk_rot<D>(r)) << 4));
   }
@@ -430,8 +445,8 @@ constexpr int kBwdStatBytes = 3 * 2 * kBwdY * 4;  // three tiles' worth of lse_i
 // needed for D_i before the loop starts.  A stage is as large as an own tile (two 64-row tiles).
 template <int D, bool kDQ> __host__ __device__ constexpr int bwd_stages() { return D == 32 ? 6 : (kDQ ? 4 : 3); }
 template <int D, bool kDQ> __host__ __device__ constexpr int bwd_smem_bytes() {
-  // two own tiles, streamed stages, alignment slack, statistics, barriers, segment offsets
-  return (2 + bwd_stages<D, kDQ>()) * 128 * D * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64;
+  // two own tiles, streamed stages, alignment slack, statistics, barriers, segment offsets, row flags
+  return (2 + bwd_stages<D, kDQ>()) * 128 * D * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64 + 128;
 }
 
 template <int D, bool kDQ>
@@ -440,7 +455,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
-                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
+                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
@@ -481,10 +496,14 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + kBarBase + 92);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + kBarBase + 96);
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kBarBase + 128);  // [kSegStage + 1]
+  // rows of this tile whose results this kernel writes (all valid rows, or those of the long segments only)
+  volatile uint8_t* row_ok = reinterpret_cast<volatile uint8_t*>(smem_al + kBarBase + 128 + kSegStage * 4 + 64);
 
   // everything up to the wait touches no global memory, so it runs under the previous kernel's tail.  The thread
   // that sets the barriers up is the one that later issues the copies counted on them.
   if (tid == kBwdMath) {
+    range[0] = 0x7fffffff;
+    range[1] = 0;
     ptx::prefetch_tensormap(&tm_qkv);
     ptx::prefetch_tensormap(&tm_do);
     ptx::prefetch_tensormap(&tm_qkv_y);
@@ -505,6 +524,11 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
   if (r0 >= Np) return;
+  if (skip_short) {
+    // tiles whose rows all belong to the one-pass kernel leave before they fetch anything
+    __syncthreads();  // the staged offsets are visible
+    if (!tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) return;
+  }
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
   if (tid == kBwdMath) {  // the own tiles depend only on r0: fetch them under the segment search
     ptx::mbar_expect_tx(bar_x, 2 * kTile);
@@ -528,14 +552,19 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   RowSeg mine{0, 0};
   if (is_math) {
     mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+    // segments that fit one tile belong to the one-pass kernel: their rows are no rows of this one
+    if (skip_short && mine.hi - mine.lo <= kShortMax) mine = RowSeg{0, 0};
     if (half == 0) {
-      const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
-      if (row == r0) range[0] = mine.lo;
-      if (row == last) range[1] = mine.hi;
+      row_ok[rl] = mine.hi > mine.lo ? 1 : 0;
+      if (mine.hi > mine.lo) {  // the rows of the other side to visit: the union of the segments of this tile's rows
+        atomicMin(const_cast<int*>(range), mine.lo);
+        atomicMax(const_cast<int*>(range) + 1, mine.hi);
+      }
     }
   }
   __syncthreads();
-  const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
+  const bool any_row = range[1] > range[0];  // false: every row of the tile belongs to the one-pass kernel
+  const int o_lo = any_row ? range[0] : 0, o_hi = any_row ? range[1] : 0;
   const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
 
   const int y1_col = (kDQ ? C : 0) + h * D;           // streamed operand inside qkv: K | Q
@@ -568,7 +597,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next streamed query tile, row rl < 64
   if (is_math) {
     if (kDQ) {
-      if (row < Np) my_lse = lse[(long long)h * capacity + row] * kLog2e;
+      if (mine.hi > mine.lo) my_lse = lse[(long long)h * capacity + row] * kLog2e;
     } else if (half == 0 && rl < kBwdY) {
       const int i = o_lo + rl;
       if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
@@ -614,10 +643,10 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     return ok;
   };
 
-  if (is_math && !prep(0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
+  if (is_math && n_tiles > 0 && !prep(0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
   ptx::tc_fence_before_sync();
   __syncthreads();  // tile 0 is ready; a failure so far is seen by all threads or by none
-  const bool failed_early = *abort_any != 0;
+  const bool failed_early = *abort_any != 0 || n_tiles == 0;
 
   if (!is_math) {
     // ---------------------------------------------------------------- copies and products: one thread
@@ -677,7 +706,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     }
   } else if (!failed_early) {
     // ---------------------------------------------------------------- arithmetic: two threads per row
-    if (kDQ && row < Np) {
+    if (kDQ && mine.hi > mine.lo) {
       // D_i = dO_i . O_i from the two staged tiles (their load has completed: prep(0) waited for it).  Both
       // carry the same swizzle, so equal positions hold equal columns and the order of the chunks is free:
       // each row starts at a different chunk to keep 8 neighbouring rows off one bank.
@@ -799,18 +828,18 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     if (kDQ) {
       if (is_math) stage_acc(kColAcc1, smem_al, scale);
       __syncthreads();
-      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid, row_ok);
     } else {
       if (is_math) {
         stage_acc(kColAcc1, smem_al, 1.f);             // dV
         stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
       }
       __syncthreads();
-      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
-      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid, row_ok);
+      copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid, row_ok);
     }
   }
-  if (failed && tid == kBwdMath) {  // let outstanding loads land before shared memory is released
+  if ((failed || n_tiles == 0) && tid == kBwdMath) {  // let outstanding loads land before shared memory is released
     for (int t = issued > kStages ? issued - kStages : 0; t < issued; ++t) ptx::mbar_wait(bar_y(stage_of(t)), use_of(t));
     if (kDQ && issued < kStages) ptx::mbar_wait(bar_y(0), 0);  // the O tile, if no streamed tile followed it there
     ptx::mbar_wait(bar_x, 0);
@@ -830,8 +859,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
 // warp: with nothing to run under the arithmetic, thread 0 issues the copies and products between the barriers.
 constexpr int kAliasedThreads = 256;   // two threads per TMEM lane (row): each owns 32 of the 64 streamed columns
 template <int D> __host__ __device__ constexpr int aliased_smem_bytes() {
-  // own tiles, streamed tiles, alignment slack, statistics, barriers, segment offsets
-  return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64;
+  // own tiles, streamed tiles, alignment slack, statistics, barriers, segment offsets, row flags
+  return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64 + 128;
 }
 
 template <int D>
@@ -840,7 +869,7 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
-                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
+                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr bool kDQ = false;  // this kernel is the dK / dV pass only
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
@@ -870,9 +899,13 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 68);
   volatile int* range = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 72);
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kStatBase + 1024 + 128);  // [kSegStage + 1]
+  // rows of this tile whose results this kernel writes (all valid rows, or those of the long segments only)
+  volatile uint8_t* row_ok = reinterpret_cast<volatile uint8_t*>(smem_al + kStatBase + 1024 + 128 + kSegStage * 4 + 64);
 
   // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
   if (tid == 0) {
+    range[0] = 0x7fffffff;
+    range[1] = 0;
     ptx::prefetch_tensormap(&tm_qkv);
     ptx::prefetch_tensormap(&tm_do);
     ptx::prefetch_tensormap(&tm_qkv_y);
@@ -891,6 +924,11 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
     for (int i = tid; i <= n_seg; i += kAliasedThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
   if (r0 >= Np) return;
+  if (skip_short) {
+    // tiles whose rows all belong to the one-pass kernel leave before they fetch anything
+    __syncthreads();  // the staged offsets are visible
+    if (!tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) return;
+  }
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
   if (tid == 0) {  // the own tiles depend only on r0: fetch them under the segment search
     ptx::mbar_expect_tx(bar_x, kOwn * kTile);
@@ -910,14 +948,19 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
 
   const int row = r0 + rl;
-  const RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+  RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+  // segments that fit one tile belong to the one-pass kernel: their rows are no rows of this one
+  if (skip_short && mine.hi - mine.lo <= kShortMax) mine = RowSeg{0, 0};
   if (half == 0) {
-    const int last = (r0 + 127 < Np - 1) ? r0 + 127 : Np - 1;
-    if (row == r0) range[0] = mine.lo;
-    if (row == last) range[1] = mine.hi;
+    row_ok[rl] = mine.hi > mine.lo ? 1 : 0;
+    if (mine.hi > mine.lo) {  // the query rows to visit: the union of the segments of this tile's rows
+      atomicMin(const_cast<int*>(range), mine.lo);
+      atomicMax(const_cast<int*>(range) + 1, mine.hi);
+    }
   }
   __syncthreads();
-  const int o_lo = range[0], o_hi = range[1];  // rows of the other side this CTA must visit
+  const bool any_row = range[1] > range[0];  // false: every row of the tile belongs to the one-pass kernel
+  const int o_lo = any_row ? range[0] : 0, o_hi = any_row ? range[1] : 0;
   const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
 
   const int y1_col = (kDQ ? C : 0) + h * D;           // streamed operand inside qkv: K | Q
@@ -984,10 +1027,10 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
     ptx::mma_commit(bar_s);
   };
 
-  prep(0);
+  if (n_tiles > 0) prep(0);
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if (tid == 0 && !*abort_flag) { ptx::tc_fence_after_sync(); issue_s(0); }
+  if (tid == 0 && !*abort_flag && n_tiles > 0) { ptx::tc_fence_after_sync(); issue_s(0); }
   if (kDQ && row < Np) {
     // D_i = dO_i . O_i from the two staged tiles (their load has completed: prep(0) waited for it).  Both
     // carry the same swizzle, so equal positions hold equal columns and the order of the chunks is free:
@@ -1118,11 +1161,11 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
       stage_acc(kColAcc1, smem_al, 1.f);             // dV
       stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
       __syncthreads();
-      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid);
-      copy_tile_out<D, kAliasedThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid);
+      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid, row_ok);
+      copy_tile_out<D, kAliasedThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid, row_ok);
     }
   }
-  if (*abort_flag && tid == 0) {  // let outstanding loads land before shared memory is released
+  if ((*abort_flag || n_tiles == 0) && tid == 0) {  // let outstanding loads land before shared memory is released
     for (int t = issued > kBwdStages ? issued - kBwdStages : 0; t < issued; ++t)
       ptx::mbar_wait(bar_y(t % kBwdStages), (t / kBwdStages) & 1);
     ptx::mbar_wait(bar_x, 0);
@@ -1135,6 +1178,237 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Backward for segments of at most 128 rows, in one pass: a CTA owns one segment and one head, holds its queries
+// and its keys at once, and evaluates S, P, dP and dS exactly once.
+//   loads    Q, K, V, dO, O rows of the segment (one TMA tile each, 128 rows from the segment's first row)
+//   MMA      S = Q K^T and dP = dO V^T, 128 x 128 fp32 each, TMEM columns [0,128) and [128,256)
+//   threads  two per query row: D_i = dO_i . O_i, P = 2^(S - lse), dS = P (dP - D); P and dS go to shared memory
+//            as bf16 in one layout that the tensor core can read both ways (rows = queries of 128 bytes per 64 keys,
+//            16-byte chunks XOR-swizzled by the row): K-major for dQ = dS K, MN-major for dV = P^T dO, dK = dS^T Q
+//   MMA      dV, dK, dQ into TMEM columns [0, 3d), over the fp32 tiles that the threads have taken into registers
+//   stores   the three tiles leave through shared memory as whole lines, rows of the segment only.
+// Nothing is recomputed and q, k, v, dO are read once.  Rows of the tiles beyond the segment belong to other
+// segments (finite data, multiplied by zeros) or lie past the last valid packed row (unspecified memory: zeroed in
+// shared memory before any product sums over them).  256 TMEM columns and under 113 KB: two CTAs per SM.
+constexpr int kShortThreads = 256;
+template <int D> __host__ __device__ constexpr int short_smem_bytes() {
+  // Q, K, dO tiles; P buffer (V tile first lives there); dS buffer (O tile first lives there); barriers.  No slack
+  // for aligning the base: with it two CTAs would not fit an SM at d = 64; the kernel checks the alignment instead.
+  return 3 * 128 * D * 2 + 2 * 128 * 128 * 2 + 64;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kShortThreads, 2)
+attn_bwd_short_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
+                      const __grid_constant__ CUtensorMap tm_o, const float* __restrict__ lse,
+                      const int32_t* __restrict__ seg, int n_seg, int capacity, int C, float scale,
+                      __nv_bfloat16* __restrict__ dqkv, int32_t* d_status) {
+  using HT = HeadTile<D>;
+  constexpr int kTile = HT::kTileBytes;
+  constexpr int kOp = 128 * 128 * 2;  // a P or dS buffer: two panels of 64 keys, 128 query rows of 128 bytes each
+  constexpr float kLog2e = 1.4426950408889634f;
+  const int h = blockIdx.x, s_idx = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + lane;
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = ptx::smem_u32(smem_raw);
+  uint8_t* smem_al = smem_raw;
+  if ((smem_base & 1023u) != 0u) {  // the swizzled tiles need a 1024-byte aligned base: refuse rather than misread
+    if (threadIdx.x == 0) record_status(d_status, SPA_ERR_UNSUPPORTED);
+    return;
+  }
+  const uint32_t q_s = smem_base, k_s = smem_base + kTile, do_s = smem_base + 2 * kTile;
+  const uint32_t p_s = smem_base + 3 * kTile, ds_s = p_s + kOp;
+  const uint32_t v_s = p_s, o_s = ds_s;  // needed only until the first products / D_i are done
+  constexpr int kBarOff = 3 * kTile + 2 * kOp;
+  const uint32_t bar_ld = smem_base + kBarOff, bar_s = bar_ld + 8, bar_acc = bar_ld + 16;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kBarOff + 24);
+  volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + kBarOff + 28);
+
+  if (tid == 0) {
+    ptx::prefetch_tensormap(&tm_qkv);
+    ptx::prefetch_tensormap(&tm_do);
+    ptx::prefetch_tensormap(&tm_o);
+    ptx::mbar_init(bar_ld, 1);
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_acc, 1);
+    *abort_any = 0;
+    ptx::fence_mbar_init();
+  }
+  pdl_entry();
+  const int Np = packed_rows(seg, n_seg, capacity);
+  const int lo = __ldg(seg + s_idx);
+  int hi = __ldg(seg + s_idx + 1);
+  hi = hi < Np ? hi : Np;
+  const int n = hi - lo;  // rows of this segment
+  if (n <= 0 || n > kShortMax) return;  // empty, or one for the two-pass kernels
+  if (tid == 0) {
+    ptx::mbar_expect_tx(bar_ld, 5 * kTile);
+    ptx::tma_load_2d(q_s, &tm_qkv, bar_ld, h * D, lo);
+    ptx::tma_load_2d(k_s, &tm_qkv, bar_ld, C + h * D, lo);
+    ptx::tma_load_2d(v_s, &tm_qkv, bar_ld, 2 * C + h * D, lo);
+    ptx::tma_load_2d(do_s, &tm_do, bar_ld, h * D, lo);
+    ptx::tma_load_2d(o_s, &tm_o, bar_ld, h * D, lo);
+  }
+  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), 256);
+  const bool valid = rl < n;
+  const float my_lse = valid ? lse[(long long)h * capacity + lo + rl] * kLog2e : 0.f;
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // barriers and the TMEM address are visible
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+  const float scale_log2e = scale * kLog2e;
+
+  bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_ld, 0)) != 0;
+  // D_i = dO_i . O_i (both tiles carry the same swizzle: equal positions hold equal columns)
+  float my_D = 0.f;
+  if (valid) {
+    constexpr int kChunks = HT::kRowBytes / 16;
+    const uint8_t* po = smem_al + (o_s - smem_base) + rl * HT::kRowBytes;
+    const uint8_t* pg = smem_al + 2 * kTile + rl * HT::kRowBytes;
+    const int rot = chunk_rot<D>(rl);
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      float a[8], b[8];
+      Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(po + ((c ^ rot) << 4)), a);
+      Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(pg + ((c ^ rot) << 4)), b);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
+    }
+  }
+  // lines past the last valid packed row are unspecified memory: the second products sum over the rows of Q, K and dO
+  if (lo + 128 > Np) {
+    const int first = Np - lo;  // >= n >= 1
+    constexpr int kChunks = HT::kRowBytes / 16;
+    for (int c = tid; c < (128 - first) * kChunks; c += kShortThreads) {
+      const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
+      *reinterpret_cast<uint4*>(smem_al + off) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(smem_al + kTile + off) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(smem_al + 2 * kTile + off) = make_uint4(0, 0, 0, 0);
+    }
+    ptx::fence_proxy_async_smem();
+  }
+  if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // tiles are ready (and everybody has read the O tile, whose memory becomes the dS buffer)
+  if (tid == 0 && !*abort_any) {
+    ptx::tc_fence_after_sync();
+    constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, 128, false, false);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem, HT::kmajor(q_s, k), HT::kmajor(k_s, k), kIdescS, k != 0 ? 1u : 0u);          // S = Q K^T
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)
+      ptx::mma_bf16(tmem + 128, HT::kmajor(do_s, k), HT::kmajor(v_s, k), kIdescS, k != 0 ? 1u : 0u);   // dP = dO V^T
+    ptx::mma_commit(bar_s);
+  }
+  if (!*abort_any) {
+    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_s, 0)) != 0;
+    if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
+  }
+  ptx::tc_fence_after_sync();
+  // ---- P and dS of this thread's 64 key columns, 32 at a time, into the operand buffers (the V tile has been read:
+  // the products above have completed)
+  if (ok) {
+    uint8_t* prow = smem_al + (p_s - smem_base) + half * (kOp / 2) + rl * 128;
+    uint8_t* dsrow = prow + kOp;
+    const int rsw = rl & 7;
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+      const int col0 = half * 64 + part * 32;  // first key column of this group
+      uint32_t rs[32], rp[32];
+      ptx::tmem_ld_32x32(tmem + lane_base + col0, rs);
+      ptx::tmem_ld_32x32(tmem + lane_base + 128 + col0, rp);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {  // 16-byte chunk: 8 keys
+        uint32_t wp[4], wd[4];
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+          float pv[2], dsv[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int col = col0 + c * 8 + j + u;
+            const bool in = valid && col < n;
+            const float pe = ptx::ex2_approx(fmaf(__uint_as_float(rs[c * 8 + j + u]), scale_log2e, -my_lse));
+            pv[u] = in ? pe : 0.f;
+            dsv[u] = in ? pe * (__uint_as_float(rp[c * 8 + j + u]) - my_D) : 0.f;
+          }
+          __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
+          __nv_bfloat162 bd = __floats2bfloat162_rn(dsv[0], dsv[1]);
+          wp[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+          wd[j >> 1] = *reinterpret_cast<uint32_t*>(&bd);
+        }
+        const int chunk = (part * 4 + c) ^ rsw;
+        *reinterpret_cast<uint4*>(prow + (chunk << 4)) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+        *reinterpret_cast<uint4*>(dsrow + (chunk << 4)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+      }
+    }
+    ptx::fence_proxy_async_smem();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // operands complete; every thread holds its fp32 values: their TMEM columns take the results
+  if (tid == 0 && !*abort_any) {
+    ptx::tc_fence_after_sync();
+    constexpr uint32_t kIdescT = ptx::idesc_bf16_f32(128, D, true, true);    // A = P^T or dS^T (MN-major), B MN-major
+    constexpr uint32_t kIdescQ = ptx::idesc_bf16_f32(128, D, false, true);   // A = dS (K-major), B = K (MN-major)
+#pragma unroll
+    for (int k = 0; k < 8; ++k)   // dV = P^T dO: 16 query rows per step
+      ptx::mma_bf16(tmem, ptx::smem_desc_sw128(p_s + k * 2048, kOp / 2, 1024), HT::mnmajor(do_s, k), kIdescT, k != 0 ? 1u : 0u);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)   // dK = dS^T Q
+      ptx::mma_bf16(tmem + D, ptx::smem_desc_sw128(ds_s + k * 2048, kOp / 2, 1024), HT::mnmajor(q_s, k), kIdescT, k != 0 ? 1u : 0u);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)   // dQ = dS K: 16 keys per step, 64 keys per panel
+      ptx::mma_bf16(tmem + 2 * D, ptx::smem_desc_sw128(ds_s + (k >> 2) * (kOp / 2) + (k & 3) * 32, 16, 1024),
+                    HT::mnmajor(k_s, k), kIdescQ, k != 0 ? 1u : 0u);
+    ptx::mma_commit(bar_acc);
+  }
+  if (!*abort_any) {
+    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_acc, 0)) != 0;
+    if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // nobody reports a failure from here on
+  ptx::tc_fence_after_sync();
+  if (!*abort_any) {
+    // dV, dK, dQ rows as bf16 into the Q, K, dO tiles' memory (idle now), from where whole lines go out
+    constexpr int kDh = D / 2;
+    const float mul[3] = {1.f, scale, scale};
+#pragma unroll
+    for (int a = 0; a < 3; ++a) {
+      uint32_t r[kDh];
+      if (kDh == 32) ptx::tmem_ld_32x32(tmem + lane_base + a * D + half * kDh, r);
+      else ptx::tmem_ld_32x16(tmem + lane_base + a * D + half * kDh, r);
+      ptx::tmem_ld_wait();
+      const int rot = chunk_rot<D>(rl);
+#pragma unroll
+      for (int g = 0; g < kDh / 8; ++g) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]) * mul[a];
+        *reinterpret_cast<uint4*>(smem_al + a * kTile + rl * HT::kRowBytes + (((half * (kDh / 8) + g) ^ rot) << 4)) =
+            Vec16<__nv_bfloat16>::from_float(v);
+      }
+    }
+    __syncthreads();
+    const long long ld = 3LL * C;
+    copy_tile_out<D, kShortThreads>(smem_al, dqkv + 2 * C + h * D, ld, lo, hi, tid);               // dV
+    copy_tile_out<D, kShortThreads>(smem_al + kTile, dqkv + C + h * D, ld, lo, hi, tid);           // dK
+    copy_tile_out<D, kShortThreads>(smem_al + 2 * kTile, dqkv + h * D, ld, lo, hi, tid);           // dQ
+  } else if (tid == 0) {
+    ptx::mbar_wait(bar_ld, 0);  // let the loads land before shared memory is released
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem, 256);
+  }
+}
 
 // Which kernel runs the dK / dV pass for head dimension D.
 template <int D> struct kv_pass {
@@ -1163,17 +1437,28 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
   static DeviceOnce attr;
   cudaError_t ea = attr.run([&] {
     cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, true>());
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attn_bwd_short_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, short_smem_bytes<D>());
     return e != cudaSuccess ? e : cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_pass<D>::kSmem);
   });
   if (ea != cudaSuccess) { set_cuda_error(ea, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
   dim3 grid(p.H, (p.capacity + 127) / 128);
   const float scale = softmax_scale_of(p);
+  // Under SPA_FLAG_ONE_PASS_BWD segments of at most 128 rows go to the one-pass kernel (one CTA per segment and
+  // head) and the two passes take the longer ones; otherwise, or with more segments than a grid dimension holds, the
+  // two passes take everything.
+  const int skip_short = ((p.flags & SPA_FLAG_ONE_PASS_BWD) && n_seg >= 1 && n_seg <= 65535) ? 1 : 0;
+  if (skip_short) {
+    launch_pdl(attn_bwd_short_kernel<D>, dim3(p.H, n_seg), kShortThreads, short_smem_bytes<D>(), st, tm_qkv, tm_do, tm_o, lse,
+               seg, n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
+    SPA_CUDA_CHECK_LAUNCH("attn_bwd_short_kernel");
+  }
   launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D, true>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, skip_short, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
   launch_pdl(kkv, grid, kv_pass<D>::kThreads, kv_pass<D>::kSmem, st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, d_status);
+             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, skip_short, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
   return SPA_OK;
 }

@@ -36,8 +36,9 @@ def random_problem(B, N, C, H, dtype, counts, seed=0):
     return x, mask, W_qkv, b_qkv, W_o, b_o, dY
 
 
+# xflags 8: fp32-FMA kernels; 64: segments of at most 128 rows through the one-pass backward kernel
 @pytest.mark.parametrize("dtype,C,H,xflags", [("f32", 96, 3, 0), ("bf16", 128, 2, 0), ("bf16", 128, 4, 0),
-                                               ("bf16", 128, 2, 8)])
+                                               ("bf16", 128, 2, 8), ("bf16", 128, 2, 64), ("bf16", 128, 4, 64)])
 def test_ragged_segments_from_a_given_mask(dtype, C, H, xflags):
     counts = [0, 1, 2, 63, 64, 65, 130, 0, 197, 7, 0]
     B, N = len(counts), 197
@@ -199,8 +200,9 @@ def test_invalid_arguments_are_rejected_on_the_host():
         assert e.value.status == lib.SPA_ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("xflags", [0, 64])             # 64: the one-pass backward kernel takes every segment here
 @pytest.mark.parametrize("C,H", [(128, 2), (128, 4)])   # head dimension 64 and 32
-def test_attention_with_more_segments_than_the_kernels_stage(C, H):
+def test_attention_with_more_segments_than_the_kernels_stage(C, H, xflags):
     """600 segments of 1-40 rows: above 512 segments the attention kernels search the offsets in global memory
     instead of their shared-memory copy.  Forward and backward against the oracle fed the same rounded bits."""
     lib = L()
@@ -213,7 +215,7 @@ def test_attention_with_more_segments_than_the_kernels_stage(C, H):
     n_seg, Np = len(counts), int(cu_np[-1])
     B, N = 24, 1024                     # capacity B*N >= Np; the segments are not images here
     assert Np <= B * N
-    blk = block(B, N, C, H, dt)
+    blk = block(B, N, C, H, dt, flags=xflags)
     p, cap = blk.p, blk.cap
 
     def padded(a, cols):

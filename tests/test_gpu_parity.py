@@ -44,8 +44,9 @@ def check_indices(blk, fwd):
     return Np
 
 
-# (config, extra flags); 8 = fp32-FMA kernels, 16 = one-CTA GEMMs where CTA pairs would be used (configs 4, 5)
-VARIANTS = [(1, 0), (2, 0), (2, 8), (3, 0), (3, 8), (4, 0), (4, 16), (5, 0), (5, 8)]
+# (config, extra flags); 8 = fp32-FMA kernels, 16 = one-CTA GEMMs where CTA pairs would be used (configs 4, 5),
+# 64 = one-pass attention backward for segments of at most 128 rows (all of config 5, most of 2, half of 4)
+VARIANTS = [(1, 0), (2, 0), (2, 8), (2, 64), (3, 0), (3, 8), (4, 0), (4, 16), (4, 64), (5, 0), (5, 8), (5, 64)]
 # the same with the unpack scatter either fused into the matrix products (tensor-core problems) or as kernels of its own
 E2E_VARIANTS = [(ci, fl, False) for ci, fl in VARIANTS] + [(ci, 0, True) for ci in (2, 3, 4, 5)]
 
