@@ -107,12 +107,14 @@ template <int D> __host__ __device__ constexpr int fwd_smem_bytes() {
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __restrict__ seg, int n_seg, int capacity,
-                   int C, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
+                   int C, int H, float scale_log2e, __nv_bfloat16* __restrict__ ao, float* __restrict__ lse,
                    int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;
-  const int q0 = blockIdx.y * kQ;  // grid = (heads, tiles): CTAs past the last valid tile are dispatched last
-  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // A CTA takes the work items blockIdx.x, blockIdx.x + gridDim.x, ... of the (tile, head) pairs that the device-side
+  // row count leaves (heads fastest, so that CTAs running side by side share their K / V tiles in L2): no CTA is
+  // launched for rows that do not exist, and TMEM and the staged segment offsets are set up once per CTA.
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool is_softmax = warp < kSoftmaxThreads / 32;  // warps 0-7; warp 8 issues the copies and the products
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 query rows and split
   // the work of each row (key columns of S and P, head dimensions of O) in two halves
@@ -138,11 +140,29 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   float* xch = reinterpret_cast<float*>(smem_al + 5 * kTile + 128);  // [2 tile parities][2 halves][128 rows]
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + 5 * kTile + 128 + 2048);  // [kSegStage + 1]
 
-  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail.  The thread
-  // that sets the barriers up is the one that later issues the copies counted on them (program order: no copy
-  // can meet a barrier that is not initialised yet).
+  if (tid == kSoftmaxThreads) ptx::prefetch_tensormap(&tm);
+  pdl_entry();
+  const bool staged = n_seg < kSegStage;
+  if (staged)
+    for (int i = tid; i <= n_seg; i += kFwdThreads) seg_s[i] = __ldg(seg + i);
+  const int Np = packed_rows(seg, n_seg, capacity);
+  const int n_items = ((Np + kQ - 1) / kQ) * H;
+  if ((int)blockIdx.x >= n_items) return;
+  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  bool cta_failed = false;
+  for (int item = blockIdx.x; item < n_items && !cta_failed; item += gridDim.x) {
+  const int h = item % H, q0 = (item / H) * kQ;
+  // The thread that sets the barriers up is the one that later issues the copies counted on them (program order: no
+  // copy can meet a barrier that is not initialised yet).  Every phase of the previous item has completed.
   if (tid == kSoftmaxThreads) {
-    ptx::prefetch_tensormap(&tm);
+    if (item != (int)blockIdx.x) {
+      ptx::mbar_inval(bar_q);
+      for (int s = 0; s < 2; ++s) { ptx::mbar_inval(bar_k(s)); ptx::mbar_inval(bar_v(s)); }
+      ptx::mbar_inval(bar_s);
+      ptx::mbar_inval(bar_o);
+      ptx::mbar_inval(bar_sfree);
+      ptx::mbar_inval(bar_pready);
+    }
     ptx::mbar_init(bar_q, 1);
     for (int s = 0; s < 2; ++s) { ptx::mbar_init(bar_k(s), 1); ptx::mbar_init(bar_v(s), 1); }
     ptx::mbar_init(bar_s, 1);
@@ -152,18 +172,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     *abort_any = 0;
     for (int i = 0; i < 8; ++i) abort_pair[i] = 0;
     ptx::fence_mbar_init();
-  }
-  pdl_entry();
-  const bool staged = n_seg < kSegStage;
-  if (staged)
-    for (int i = tid; i <= n_seg; i += kFwdThreads) seg_s[i] = __ldg(seg + i);
-  const int Np = packed_rows(seg, n_seg, capacity);
-  if (q0 >= Np) return;
-  if (tid == kSoftmaxThreads) {  // the Q tile depends only on q0: fetch it under the segment search
+    // the Q tile depends only on q0: fetch it under the segment search
     ptx::mbar_expect_tx(bar_q, kTile);
     ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
   }
-  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
   ptx::tc_fence_before_sync();
   __syncthreads();  // barriers, TMEM address and staged offsets are visible
   ptx::tc_fence_after_sync();
@@ -410,11 +422,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   }
   __syncthreads();
   if (!failed) copy_tile_out<D, kFwdThreads>(smem_al, ao + h * D, C, q0, Np, tid);
+  cta_failed = failed;
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  __syncthreads();  // the tile's memory and the barriers are free for the next item
+  }
   if (warp == 0) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem, kTmemCols);
+    ptx::tmem_dealloc(*tmem_slot, kTmemCols);
   }
 }
 
@@ -1472,8 +1486,10 @@ int fwd_launch(const spa_params& p, const void* qkv, const int32_t* seg, int n_s
   static DeviceOnce attr;
   cudaError_t ea = attr.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem_bytes<D>()); });
   if (ea != cudaSuccess) { set_cuda_error(ea, "attn_fwd_tc_kernel"); return SPA_ERR_CUDA; }
-  dim3 grid(p.H, (p.capacity + kQ - 1) / kQ);
-  launch_pdl(kern, grid, kFwdThreads, fwd_smem_bytes<D>(), st, tm, seg, n_seg, p.capacity, p.C,
+  // a persistent grid: two CTAs per SM (87 KB of shared memory, 256 TMEM columns each), never more than work items
+  const long long items = (long long)p.H * ((p.capacity + kQ - 1) / kQ);
+  const int grid = (int)(items < 2 * kNumSMs ? items : 2 * kNumSMs);
+  launch_pdl(kern, grid, kFwdThreads, fwd_smem_bytes<D>(), st, tm, seg, n_seg, p.capacity, p.C, p.H,
                                                       softmax_scale_of(p) * 1.4426950408889634f,
                                                       (__nv_bfloat16*)ao, lse, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_fwd_tc_kernel");
