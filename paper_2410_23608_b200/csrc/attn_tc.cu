@@ -140,7 +140,24 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   float* xch = reinterpret_cast<float*>(smem_al + 5 * kTile + 128);  // [2 tile parities][2 halves][128 rows]
   int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + 5 * kTile + 128 + 2048);  // [kSegStage + 1]
 
-  if (tid == kSoftmaxThreads) ptx::prefetch_tensormap(&tm);
+  // The thread that sets the barriers up is the one that later issues the copies counted on them (program order: no
+  // copy can meet a barrier that is not initialised yet).
+  auto init_barriers = [&]() {
+    ptx::mbar_init(bar_q, 1);
+    for (int s = 0; s < 2; ++s) { ptx::mbar_init(bar_k(s), 1); ptx::mbar_init(bar_v(s), 1); }
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_o, 1);
+    ptx::mbar_init(bar_sfree, kSoftmaxThreads / 32);
+    ptx::mbar_init(bar_pready, kSoftmaxThreads / 32);
+    *abort_any = 0;
+    for (int i = 0; i < 8; ++i) abort_pair[i] = 0;
+    ptx::fence_mbar_init();
+  };
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
+  if (tid == kSoftmaxThreads) {
+    ptx::prefetch_tensormap(&tm);
+    init_barriers();
+  }
   pdl_entry();
   const bool staged = n_seg < kSegStage;
   if (staged)
@@ -152,26 +169,16 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
   bool cta_failed = false;
   for (int item = blockIdx.x; item < n_items && !cta_failed; item += gridDim.x) {
   const int h = item % H, q0 = (item / H) * kQ;
-  // The thread that sets the barriers up is the one that later issues the copies counted on them (program order: no
-  // copy can meet a barrier that is not initialised yet).  Every phase of the previous item has completed.
   if (tid == kSoftmaxThreads) {
-    if (item != (int)blockIdx.x) {
+    if (item != (int)blockIdx.x) {  // every phase of the previous item has completed: the barriers start over
       ptx::mbar_inval(bar_q);
       for (int s = 0; s < 2; ++s) { ptx::mbar_inval(bar_k(s)); ptx::mbar_inval(bar_v(s)); }
       ptx::mbar_inval(bar_s);
       ptx::mbar_inval(bar_o);
       ptx::mbar_inval(bar_sfree);
       ptx::mbar_inval(bar_pready);
+      init_barriers();
     }
-    ptx::mbar_init(bar_q, 1);
-    for (int s = 0; s < 2; ++s) { ptx::mbar_init(bar_k(s), 1); ptx::mbar_init(bar_v(s), 1); }
-    ptx::mbar_init(bar_s, 1);
-    ptx::mbar_init(bar_o, 1);
-    ptx::mbar_init(bar_sfree, kSoftmaxThreads / 32);
-    ptx::mbar_init(bar_pready, kSoftmaxThreads / 32);
-    *abort_any = 0;
-    for (int i = 0; i < 8; ++i) abort_pair[i] = 0;
-    ptx::fence_mbar_init();
     // the Q tile depends only on q0: fetch it under the segment search
     ptx::mbar_expect_tx(bar_q, kTile);
     ptx::tma_load_2d(q_s, &tm, bar_q, h * D, q0);
@@ -463,13 +470,13 @@ template <int D, bool kDQ> __host__ __device__ constexpr int bwd_smem_bytes() {
   return (2 + bwd_stages<D, kDQ>()) * 128 * D * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64 + 128;
 }
 
-template <int D, bool kDQ>
+template <int D, bool kDQ, bool kLoop>
 __global__ void __launch_bounds__(kBwdThreads, 2)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
-                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
+                   int capacity, int C, int H, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
@@ -481,8 +488,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_aliased_kernel");
   constexpr uint32_t kColOpP = 160u;                // P^T (dK/dV pass only)
   constexpr uint32_t kColOpDS = kDQ ? 192u : 224u;  // dS or dS^T
-  const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
-  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // A CTA takes the work items blockIdx.x, blockIdx.x + gridDim.x, ... of the (tile, head) pairs that the device-side
+  // row count leaves (heads fastest); TMEM and the staged segment offsets are set up once per CTA.
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool is_math = warp < kBwdMath / 32;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
   const int quarter = warp & 3, half = (warp >> 2) & 1, rl = quarter * 32 + lane;
@@ -513,16 +521,10 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   // rows of this tile whose results this kernel writes (all valid rows, or those of the long segments only)
   volatile uint8_t* row_ok = reinterpret_cast<volatile uint8_t*>(smem_al + kBarBase + 128 + kSegStage * 4 + 64);
 
-  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail.  The thread
-  // that sets the barriers up is the one that later issues the copies counted on them.
-  if (tid == kBwdMath) {
+  // The thread that sets the barriers up is the one that later issues the copies counted on them.
+  auto init_barriers = [&]() {
     range[0] = 0x7fffffff;
     range[1] = 0;
-    ptx::prefetch_tensormap(&tm_qkv);
-    ptx::prefetch_tensormap(&tm_do);
-    ptx::prefetch_tensormap(&tm_qkv_y);
-    ptx::prefetch_tensormap(&tm_do_y);
-    if (kDQ) ptx::prefetch_tensormap(&tm_o);
     ptx::mbar_init(bar_x, 1);
     for (int s3 = 0; s3 < kStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
@@ -531,20 +533,42 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     ptx::mbar_init(bar_opready, kBwdMath / 32);
     *abort_any = 0;
     ptx::fence_mbar_init();
+  };
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
+  if (tid == kBwdMath) {
+    ptx::prefetch_tensormap(&tm_qkv);
+    ptx::prefetch_tensormap(&tm_do);
+    ptx::prefetch_tensormap(&tm_qkv_y);
+    ptx::prefetch_tensormap(&tm_do_y);
+    if (kDQ) ptx::prefetch_tensormap(&tm_o);
+    init_barriers();
   }
   pdl_entry();
   const bool staged = n_seg < kSegStage;
   if (staged)
     for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
-  if (r0 >= Np) return;
-  if (skip_short) {
-    // tiles whose rows all belong to the one-pass kernel leave before they fetch anything
-    __syncthreads();  // the staged offsets are visible
-    if (!tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) return;
-  }
+  const int n_items = ((Np + 127) / 128) * H;
+  if ((int)blockIdx.x >= n_items) return;
+  if (skip_short) __syncthreads();  // the staged offsets are visible to the tile test
+  bool cta_failed = false, first_item = true;
+  int item = blockIdx.x;
+  do {  // kLoop: this CTA strides over the items; otherwise the grid holds one CTA per item and this is no loop
+  const int h = item % H, r0 = (item / H) * 128;
+  // tiles whose rows all belong to the one-pass kernel are passed over before anything is fetched
+  if (skip_short && !tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) continue;
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
-  if (tid == kBwdMath) {  // the own tiles depend only on r0: fetch them under the segment search
+  if (tid == kBwdMath) {
+    if (!first_item) {  // every phase of the previous item has completed: the barriers start over
+      ptx::mbar_inval(bar_x);
+      for (int s3 = 0; s3 < kStages; ++s3) ptx::mbar_inval(bar_y(s3));
+      ptx::mbar_inval(bar_s);
+      ptx::mbar_inval(bar_acc);
+      ptx::mbar_inval(bar_sfree);
+      ptx::mbar_inval(bar_opready);
+      init_barriers();
+    }
+    // the own tiles depend only on r0: fetch them under the segment search
     ptx::mbar_expect_tx(bar_x, 2 * kTile);
     ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
     if (kDQ) {
@@ -555,9 +579,10 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
       ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
     }
   }
-  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
+  if (first_item && warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
+  first_item = false;
   ptx::tc_fence_before_sync();
-  __syncthreads();  // barriers, TMEM address and staged offsets are visible
+  __syncthreads();  // barriers, (first item) the TMEM address and the staged offsets are visible
   ptx::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
@@ -858,11 +883,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
     if (kDQ && issued < kStages) ptx::mbar_wait(bar_y(0), 0);  // the O tile, if no streamed tile followed it there
     ptx::mbar_wait(bar_x, 0);
   }
+  cta_failed = failed;
   ptx::tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 0) {
+  __syncthreads();  // the tiles' memory and the barriers are free for the next item
+  } while (kLoop && (item += gridDim.x) < n_items && !cta_failed);
+  if (!first_item && warp == 0) {  // TMEM was taken with the first item that this CTA worked on
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem, kBwdTmemCols);
+    ptx::tmem_dealloc(*tmem_slot, kBwdTmemCols);
   }
 }
 
@@ -877,21 +904,22 @@ template <int D> __host__ __device__ constexpr int aliased_smem_bytes() {
   return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64 + 128;
 }
 
-template <int D>
+template <int D, bool kLoop>
 __global__ void __launch_bounds__(kAliasedThreads)
 attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
-                   int capacity, int C, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
+                   int capacity, int C, int H, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
   using HT = HeadTile<D>;
   constexpr bool kDQ = false;  // this kernel is the dK / dV pass only
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
   constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
   constexpr float kLog2e = 1.4426950408889634f;
-  const int r0 = blockIdx.y * 128;  // grid = (heads, tiles)
-  const int h = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
+  // A CTA takes the work items blockIdx.x, blockIdx.x + gridDim.x, ... of the (tile, head) pairs that the device-side
+  // row count leaves (heads fastest); TMEM and the staged segment offsets are set up once per CTA.
+  const int tid = threadIdx.x, warp = tid >> 5;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
   const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
   const float scale_log2e = scale * kLog2e;
@@ -899,7 +927,7 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const uint32_t x1_s = smem_base, x2_s = smem_base + kTile, x3_s = smem_base + 2 * kTile;
+  const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
   constexpr int kYBase = kOwn * kTile;
   auto y1_off = [&](int st) { return kYBase + kYTile * (2 * st); };
   auto y2_off = [&](int st) { return kYBase + kYTile * (2 * st + 1); };
@@ -916,47 +944,56 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   // rows of this tile whose results this kernel writes (all valid rows, or those of the long segments only)
   volatile uint8_t* row_ok = reinterpret_cast<volatile uint8_t*>(smem_al + kStatBase + 1024 + 128 + kSegStage * 4 + 64);
 
-  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
-  if (tid == 0) {
+  auto init_barriers = [&]() {
     range[0] = 0x7fffffff;
     range[1] = 0;
-    ptx::prefetch_tensormap(&tm_qkv);
-    ptx::prefetch_tensormap(&tm_do);
-    ptx::prefetch_tensormap(&tm_qkv_y);
-    ptx::prefetch_tensormap(&tm_do_y);
-    if (kDQ) ptx::prefetch_tensormap(&tm_o);
     ptx::mbar_init(bar_x, 1);
     for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_o, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
+  };
+  // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
+  if (tid == 0) {
+    ptx::prefetch_tensormap(&tm_qkv);
+    ptx::prefetch_tensormap(&tm_do);
+    ptx::prefetch_tensormap(&tm_qkv_y);
+    ptx::prefetch_tensormap(&tm_do_y);
+    init_barriers();
   }
   pdl_entry();
   const bool staged = n_seg < kSegStage;
   if (staged)
     for (int i = tid; i <= n_seg; i += kAliasedThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
-  if (r0 >= Np) return;
-  if (skip_short) {
-    // tiles whose rows all belong to the one-pass kernel leave before they fetch anything
-    __syncthreads();  // the staged offsets are visible
-    if (!tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) return;
-  }
+  const int n_items = ((Np + 127) / 128) * H;
+  if ((int)blockIdx.x >= n_items) return;
+  if (skip_short) __syncthreads();  // the staged offsets are visible to the tile test
+  bool cta_failed = false, first_item = true;
+  int item = blockIdx.x;
+  do {  // kLoop: this CTA strides over the items; otherwise the grid holds one CTA per item and this is no loop
+  const int h = item % H, r0 = (item / H) * 128;
+  // tiles whose rows all belong to the one-pass kernel are passed over before anything is fetched
+  if (skip_short && !tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) continue;
   const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
-  if (tid == 0) {  // the own tiles depend only on r0: fetch them under the segment search
+  if (tid == 0) {
+    if (!first_item) {  // every phase of the previous item has completed: the barriers start over
+      ptx::mbar_inval(bar_x);
+      for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_inval(bar_y(s3));
+      ptx::mbar_inval(bar_s);
+      ptx::mbar_inval(bar_o);
+      init_barriers();
+    }
+    // the own tiles depend only on r0: fetch them under the segment search
     ptx::mbar_expect_tx(bar_x, kOwn * kTile);
     ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
-    if (kDQ) {
-      ptx::tma_load_2d(x2_s, &tm_do, bar_x, h * D, r0);                  // dO
-      ptx::tma_load_2d(x3_s, &tm_o, bar_x, h * D, r0);                   // O, for D_i = dO_i . O_i
-    } else {
-      ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
-    }
+    ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
   }
-  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
+  if (first_item && warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
+  first_item = false;
   ptx::tc_fence_before_sync();
-  __syncthreads();  // barriers, TMEM address and staged offsets are visible
+  __syncthreads();  // barriers, (first item) the TMEM address and the staged offsets are visible
   ptx::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
@@ -1184,11 +1221,13 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
       ptx::mbar_wait(bar_y(t % kBwdStages), (t / kBwdStages) & 1);
     ptx::mbar_wait(bar_x, 0);
   }
+  cta_failed = *abort_flag != 0;
   ptx::tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 0) {
+  __syncthreads();  // the tiles' memory and the barriers are free for the next item
+  } while (kLoop && (item += gridDim.x) < n_items && !cta_failed);
+  if (!first_item && warp == 0) {  // TMEM was taken with the first item that this CTA worked on
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem, kBwdTmemCols);
+    ptx::tmem_dealloc(*tmem_slot, kBwdTmemCols);
   }
 }
 
@@ -1428,12 +1467,12 @@ attn_bwd_short_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_c
 template <int D> struct kv_pass {
   static constexpr int kThreads = kBwdThreads;
   static constexpr int kSmem = bwd_smem_bytes<D, false>();
-  static auto kernel() { return attn_bwd_tc_kernel<D, false>; }
+  template <bool kLoop> static auto kernel() { return attn_bwd_tc_kernel<D, false, kLoop>; }
 };
 template <> struct kv_pass<64> {
   static constexpr int kThreads = kAliasedThreads;
   static constexpr int kSmem = aliased_smem_bytes<64>();
-  static auto kernel() { return attn_bwd_kv_aliased_kernel<64>; }
+  template <bool kLoop> static auto kernel() { return attn_bwd_kv_aliased_kernel<64, kLoop>; }
 };
 
 template <int D>
@@ -1446,18 +1485,29 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
       !make_tmap_bf16_2d(&tm_do_y, dao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, kBwdY, D * 2) ||
       !make_tmap_bf16_2d(&tm_o, ao, (uint64_t)p.C, p.capacity, 2ull * p.C, D, 128, D * 2))
     return SPA_ERR_UNSUPPORTED;
-  auto kq = attn_bwd_tc_kernel<D, true>;
-  auto kkv = kv_pass<D>::kernel();
   static DeviceOnce attr;
   cudaError_t ea = attr.run([&] {
-    cudaError_t e = cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem_bytes<D, true>());
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_bwd_short_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, short_smem_bytes<D>());
-    return e != cudaSuccess ? e : cudaFuncSetAttribute(kkv, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_pass<D>::kSmem);
+    const auto smem_attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_tc_kernel<D, true, false>, smem_attr, bwd_smem_bytes<D, true>());
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_tc_kernel<D, true, true>, smem_attr, bwd_smem_bytes<D, true>());
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_short_kernel<D>, smem_attr, short_smem_bytes<D>());
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kv_pass<D>::template kernel<false>(), smem_attr, kv_pass<D>::kSmem);
+    return e != cudaSuccess ? e : cudaFuncSetAttribute(kv_pass<D>::template kernel<true>(), smem_attr, kv_pass<D>::kSmem);
   });
   if (ea != cudaSuccess) { set_cuda_error(ea, "attn_bwd_tc_kernel"); return SPA_ERR_CUDA; }
   float* delta = reinterpret_cast<float*>(workspace);  // [H][capacity]
-  dim3 grid(p.H, (p.capacity + 127) / 128);
+  // One CTA per (tile, head) item, or a persistent grid of two CTAs per SM that strides over the items.  The stride
+  // is a static assignment: it pays (one prologue per CTA instead of one per item) where the items cost about the
+  // same, i.e. short segments that span a key tile or two, and where a CTA gets several of them; with long segments
+  // the key ranges differ widely from item to item and the hardware's own block scheduling balances them better.
+  // The host knows the item slots of the capacity, not the rows that the selection kept (typically about half):
+  // three grids' worth of slots stands for one and a half items per CTA or more.
+  const long long items = (long long)p.H * ((p.capacity + 127) / 128);
+  const bool even_items = (long long)p.capacity <= 256ll * (n_seg > 0 ? n_seg : 1);
+  const bool loop = even_items && items >= 3ll * 2 * kNumSMs;
+  const int grid = (int)(loop ? 2 * kNumSMs : items);
+  auto kq = loop ? attn_bwd_tc_kernel<D, true, true> : attn_bwd_tc_kernel<D, true, false>;
+  auto kkv = loop ? kv_pass<D>::template kernel<true>() : kv_pass<D>::template kernel<false>();
   const float scale = softmax_scale_of(p);
   // Under SPA_FLAG_ONE_PASS_BWD segments of at most 128 rows go to the one-pass kernel (one CTA per segment and
   // head) and the two passes take the longer ones; otherwise, or with more segments than a grid dimension holds, the
@@ -1469,10 +1519,10 @@ int bwd_launch(const spa_params& p, const void* qkv, const void* ao, const float
     SPA_CUDA_CHECK_LAUNCH("attn_bwd_short_kernel");
   }
   launch_pdl(kq, grid, kBwdThreads, bwd_smem_bytes<D, true>(), st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, skip_short, d_status);
+             n_seg, p.capacity, p.C, p.H, scale, (__nv_bfloat16*)dqkv, skip_short, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dQ)");
   launch_pdl(kkv, grid, kv_pass<D>::kThreads, kv_pass<D>::kSmem, st, tm_qkv, tm_do, tm_qkv_y, tm_do_y, tm_o, lse, delta, seg,
-             n_seg, p.capacity, p.C, scale, (__nv_bfloat16*)dqkv, skip_short, d_status);
+             n_seg, p.capacity, p.C, p.H, scale, (__nv_bfloat16*)dqkv, skip_short, d_status);
   SPA_CUDA_CHECK_LAUNCH("attn_bwd_tc_kernel(dKV)");
   return SPA_OK;
 }
