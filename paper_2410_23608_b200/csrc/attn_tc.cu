@@ -688,17 +688,22 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   const bool failed_early = *abort_any != 0 || n_tiles == 0;
 
   if (!is_math) {
-    // ---------------------------------------------------------------- copies and products: one thread
-    if (lane == 0 && !failed_early) {
+    // ---------------------------------------------------------------- copies and products: one warp, whose lanes
+    // all follow the tiles and take every wait together; one elected lane issues (see ptx::elect_one)
+    if (!failed_early) {
       auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
         const int st = stage_of(t_);
+        const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
+        if (ptx::elect_one()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(smem_base + y1_off(st), k), kIdescS, k != 0 ? 1u : 0u);
+          for (int k = 0; k < D / 16; ++k)
+            ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1a, k), kIdescS, k != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(smem_base + y2_off(st), k), kIdescS, k != 0 ? 1u : 0u);
-        ptx::mma_commit(bar_s);
+          for (int k = 0; k < D / 16; ++k)
+            ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2a, k), kIdescS, k != 0 ? 1u : 0u);
+          ptx::mma_commit(bar_s);
+        }
+        __syncwarp();
       };
       bool ok = true;
       ptx::tc_fence_after_sync();
@@ -707,8 +712,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
         const int st = stage_of(t);
         if (t + 1 < n_tiles) {
           // the fp32 values of tile t are in registers and tile t + 1 is ready: its products run under the arithmetic
-          if (!(ok = wait(bar_sfree, t & 1))) break;
-          if (!(ok = wait(bar_y(stage_of(t + 1)), use_of(t + 1)))) break;
+          if (!(ok = wait_w(bar_sfree, t & 1))) break;
+          if (!(ok = wait_w(bar_y(stage_of(t + 1)), use_of(t + 1)))) break;
           ptx::tc_fence_after_sync();
           issue_s(t + 1);
         }
@@ -716,29 +721,33 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
         // is filled is the last one, or in the dQ pass the O tile's memory, which the arithmetic warps have finished
         // with before they announce tile 0 (waited for above: a tile to prefetch implies a tile t + 1)
         if (t + kStages - 1 < n_tiles) {
-          if (t > 0 && !(ok = wait(bar_acc, (t - 1) & 1))) break;
-          load_other(t + kStages - 1);
+          if (t > 0 && !(ok = wait_w(bar_acc, (t - 1) & 1))) break;
+          if (ptx::elect_one()) load_other(t + kStages - 1);
+          __syncwarp();
           issued = t + kStages;
         }
-        if (!(ok = wait(bar_opready, t & 1))) break;
+        if (!(ok = wait_w(bar_opready, t & 1))) break;
         ptx::tc_fence_after_sync();
         const uint32_t acc = (t != 0) ? 1u : 0u;
         const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
-        if (kDQ) {
+        if (ptx::elect_one()) {
+          if (kDQ) {
 #pragma unroll
-          for (int k = 0; k < kBwdY / 16; ++k)   // dQ += dS K
-            ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpDS + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
-        } else {
+            for (int k = 0; k < kBwdY / 16; ++k)   // dQ += dS K
+              ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpDS + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+          } else {
 #pragma unroll
-          for (int k = 0; k < kBwdY / 16; ++k)   // dV += P^T dO
-            ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpP + k * 8, HT::mnmajor(y2a, k), kIdescAcc, acc | (k != 0));
+            for (int k = 0; k < kBwdY / 16; ++k)   // dV += P^T dO
+              ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColOpP + k * 8, HT::mnmajor(y2a, k), kIdescAcc, acc | (k != 0));
 #pragma unroll
-          for (int k = 0; k < kBwdY / 16; ++k)   // dK += dS^T Q
-            ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColOpDS + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+            for (int k = 0; k < kBwdY / 16; ++k)   // dK += dS^T Q
+              ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColOpDS + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+          }
+          ptx::mma_commit(bar_acc);
         }
-        ptx::mma_commit(bar_acc);
+        __syncwarp();
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         record_status(d_status, SPA_ERR_TIMEOUT);
         *abort_any = 1;
       }

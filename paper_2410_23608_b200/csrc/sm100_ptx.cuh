@@ -49,6 +49,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   return false;
 }
 
+// True in exactly one lane of a converged warp (all 32 lanes must execute it together).  Work that one thread has to
+// issue (tensor-core products, bulk copies) is written as `if (elect_one()) ...` inside code that the whole warp
+// runs: the operands computed outside the branch are then known to be the same in every lane and can be held in the
+// uniform registers that those instructions read, instead of being moved there one by one for each instruction.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // Barrier `id` (1-15; 0 is __syncthreads) among `threads` threads (a multiple of 32) of the CTA.
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
