@@ -453,11 +453,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
 // fp32 values in registers and when its bf16 operands are in TMEM.
 // The bf16 operands have TMEM columns of their own, so the next tile's fp32 products are issued as soon as
 // the current ones are in registers and run under the arithmetic.  That needs room in TMEM: this kernel serves
-// the dQ pass and the dK/dV pass at d = 32; the dK/dV pass at d = 64 is attn_bwd_kv_aliased_kernel below.
+// the dQ pass and the dK/dV pass at d = 32; the dK/dV pass at d = 64 is attn_bwd_kv_split_kernel below.
 constexpr int kBwdMath = 256;      // arithmetic threads: two per TMEM lane (row)
 constexpr int kBwdThreads = kBwdMath + 32;
 constexpr int kBwdY = 64;          // rows of a streamed tile
-constexpr int kBwdStages = 4;      // streamed tiles in shared memory of the aliased dK / dV kernel
 constexpr uint32_t kBwdTmemCols = 256;
 constexpr uint32_t kColS1 = 0, kColS2 = 64, kColAcc1 = 128, kColAcc2 = 192;
 constexpr int kBwdStatBytes = 3 * 2 * kBwdY * 4;  // three tiles' worth of lse_i and D_i of the streamed queries
@@ -485,7 +484,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   static_assert(2 * kYTile == kTile, "a stage is as large as an own tile");
   constexpr float kLog2e = 1.4426950408889634f;
   // the bf16 operands have TMEM columns of their own, so the next fp32 products need not wait for the accumulating ones
-  static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_aliased_kernel");
+  static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_split_kernel");
   constexpr uint32_t kColOpP = 160u;                // P^T (dK/dV pass only)
   constexpr uint32_t kColOpDS = kDQ ? 192u : 224u;  // dS or dS^T
   // A CTA takes the work items blockIdx.x, blockIdx.x + gridDim.x, ... of the (tile, head) pairs that the device-side
@@ -902,69 +901,87 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   }
 }
 
-// The dK / dV pass where TMEM has no room for the bf16 operands beside the fp32 tiles (d = 64: S^T, dP^T, dV and dK
-// fill all 256 columns).  P^T and dS^T are written over the first half of the fp32 tiles they were computed from -
-// after a barrier, once every thread holds its fp32 columns in registers - and the next tile's fp32 products are
-// queued behind the accumulating products that read them (MMAs execute in issue order).  Eight warps, no issuing
-// warp: with nothing to run under the arithmetic, thread 0 issues the copies and products between the barriers.
-constexpr int kAliasedThreads = 256;   // two threads per TMEM lane (row): each owns 32 of the 64 streamed columns
-template <int D> __host__ __device__ constexpr int aliased_smem_bytes() {
-  // own tiles, streamed tiles, alignment slack, statistics, barriers, segment offsets, row flags
-  return 2 * 128 * D * 2 + kBwdStages * 2 * kBwdY * D * 2 + 1024 + 1024 + 128 + kSegStage * 4 + 64 + 128;
+// The dK / dV pass at d = 64 with the products running under the arithmetic.  S^T, dP^T, dV and dK fill the 256 TMEM
+// columns of a CTA, so the bf16 operands live elsewhere: P^T in shared memory (the A operand of dV += P^T dO, K-major,
+// written by the threads that computed it) and dS^T over the dP^T columns it was computed from.  The arithmetic of a
+// tile splits the same way: P^T = 2^(S^T - lse) needs S^T only - it holds the exponentials, the expensive part - and
+// runs while dP^T of the same tile is still being computed; dS^T = P^T (dP^T - D) follows.  Per tile the issuing warp
+// queues S^T(t+1) (once every arithmetic warp holds S^T(t) in registers), dV(t) (P^T(t) written), dK(t) (dS^T(t)
+// stored) and dP^T(t+1), the last behind dK(t), which reads the columns it overwrites.
+constexpr int kSplitStages = 3;  // streamed stages of a 64-row Q tile and a 64-row dO tile
+template <int D> __host__ __device__ constexpr int split_smem_bytes() {
+  // own K and V, streamed stages, P^T, alignment slack, statistics, barriers, segment offsets, row flags
+  return (2 + kSplitStages) * 128 * D * 2 + 128 * kBwdY * 2 + 1024 + kBwdStatBytes + 128 + kSegStage * 4 + 64 + 128;
 }
 
 template <int D, bool kLoop>
-__global__ void __launch_bounds__(kAliasedThreads)
-attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
+__global__ void __launch_bounds__(kBwdThreads, 2)
+attn_bwd_kv_split_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_constant__ CUtensorMap tm_do,
                    const __grid_constant__ CUtensorMap tm_qkv_y, const __grid_constant__ CUtensorMap tm_do_y,
                    const __grid_constant__ CUtensorMap tm_o,
                    const float* __restrict__ lse, float* __restrict__ delta, const int32_t* __restrict__ seg, int n_seg,
                    int capacity, int C, int H, float scale, __nv_bfloat16* __restrict__ dqkv, int skip_short, int32_t* d_status) {
   using HT = HeadTile<D>;
-  constexpr bool kDQ = false;  // this kernel is the dK / dV pass only
   constexpr int kTile = HT::kTileBytes;             // own tiles: 128 rows
   constexpr int kYTile = kBwdY * HT::kRowBytes;     // streamed tiles: 64 rows
-  constexpr int kOwn = kDQ ? 3 : 2;                 // own tiles in shared memory
+  constexpr int kStages = kSplitStages;             // streamed stages (a Q and a dO tile each): tile t lives in stage t mod kStages
+  constexpr int kShift = 0;
+  static_assert(2 * kYTile == kTile, "a stage is as large as an own tile");
   constexpr float kLog2e = 1.4426950408889634f;
+  static_assert(D == 64, "d = 32 leaves TMEM columns for the operands: attn_bwd_tc_kernel");
   // A CTA takes the work items blockIdx.x, blockIdx.x + gridDim.x, ... of the (tile, head) pairs that the device-side
   // row count leaves (heads fastest); TMEM and the staged segment offsets are set up once per CTA.
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool is_math = warp < kBwdMath / 32;
   // warps w and w + 4 may touch the same quarter of the TMEM lanes: they share 32 rows and split the columns
-  const int quarter = warp & 3, half = warp >> 2, rl = quarter * 32 + (tid & 31);
+  const int quarter = warp & 3, half = (warp >> 2) & 1, rl = quarter * 32 + lane;
   const float scale_log2e = scale * kLog2e;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   const uint32_t x1_s = smem_base, x2_s = smem_base + kTile;
-  constexpr int kYBase = kOwn * kTile;
+  constexpr int kYBase = 2 * kTile;
   auto y1_off = [&](int st) { return kYBase + kYTile * (2 * st); };
   auto y2_off = [&](int st) { return kYBase + kYTile * (2 * st + 1); };
-  constexpr int kStatBase = kYBase + kBwdStages * 2 * kYTile;
-  float* stat_lse = reinterpret_cast<float*>(smem_al + kStatBase);  // [2][64] lse_i * log2e of the staged query tile
-  float* stat_D = stat_lse + 2 * kBwdY;                              // [2][64] D_i
-  const uint32_t bar_base = smem_base + kStatBase + 1024;
-  const uint32_t bar_x = bar_base, bar_s = bar_base + 40, bar_o = bar_base + 48;
-  auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kStatBase + 1024 + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 68);
-  volatile int* range = reinterpret_cast<volatile int*>(smem_al + kStatBase + 1024 + 72);
-  int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kStatBase + 1024 + 128);  // [kSegStage + 1]
+  auto stage_of = [&](int t_) { return (t_ + kShift) % kStages; };
+  auto use_of = [&](int t_) { return (uint32_t)(((t_ + kShift) / kStages) & 1); };  // parity of that stage's barrier
+  constexpr int kPBase = kYBase + kStages * 2 * kYTile;   // P^T of the current tile: [128 keys][64 queries] bf16, K-major
+  const uint32_t p_s = smem_base + kPBase;
+  constexpr int kStatBase = kPBase + kTile;
+  float* stat_lse = reinterpret_cast<float*>(smem_al + kStatBase);  // [3][64] lse_i * log2e of the staged query tile
+  float* stat_D = stat_lse + 3 * kBwdY;                              // [3][64] D_i
+  constexpr int kBarBase = kStatBase + kBwdStatBytes;
+  const uint32_t bar_base = smem_base + kBarBase;
+  const uint32_t bar_x = bar_base, bar_s = bar_base + 32, bar_dp = bar_base + 40, bar_acc = bar_base + 48;
+  const uint32_t bar_sfree = bar_base + 56;    // 8 arrivals: every arithmetic warp holds S^T of tile t in registers
+  const uint32_t bar_pready = bar_base + 64;   // 8 arrivals: every arithmetic warp has written its part of P^T of tile t
+  const uint32_t bar_dsready = bar_base + 72;  // 8 arrivals: every arithmetic warp has stored its part of dS^T of tile t
+  auto bar_y = [&](int st) { return bar_base + 8 + 8 * st; };  // three stages
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_al + kBarBase + 88);
+  volatile int* abort_any = reinterpret_cast<volatile int*>(smem_al + kBarBase + 92);
+  volatile int* range = reinterpret_cast<volatile int*>(smem_al + kBarBase + 96);
+  int32_t* seg_s = reinterpret_cast<int32_t*>(smem_al + kBarBase + 128);  // [kSegStage + 1]
   // rows of this tile whose results this kernel writes (all valid rows, or those of the long segments only)
-  volatile uint8_t* row_ok = reinterpret_cast<volatile uint8_t*>(smem_al + kStatBase + 1024 + 128 + kSegStage * 4 + 64);
+  volatile uint8_t* row_ok = reinterpret_cast<volatile uint8_t*>(smem_al + kBarBase + 128 + kSegStage * 4 + 64);
 
+  // The thread that sets the barriers up is the one that later issues the copies counted on them.
   auto init_barriers = [&]() {
     range[0] = 0x7fffffff;
     range[1] = 0;
     ptx::mbar_init(bar_x, 1);
-    for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
+    for (int s3 = 0; s3 < kStages; ++s3) ptx::mbar_init(bar_y(s3), 1);
     ptx::mbar_init(bar_s, 1);
-    ptx::mbar_init(bar_o, 1);
-    *abort_flag = 0;
+    ptx::mbar_init(bar_dp, 1);
+    ptx::mbar_init(bar_acc, 1);
+    ptx::mbar_init(bar_sfree, kBwdMath / 32);
+    ptx::mbar_init(bar_pready, kBwdMath / 32);
+    ptx::mbar_init(bar_dsready, kBwdMath / 32);
+    *abort_any = 0;
     ptx::fence_mbar_init();
   };
   // everything up to the wait touches no global memory, so it runs under the previous kernel's tail
-  if (tid == 0) {
+  if (tid == kBwdMath) {
     ptx::prefetch_tensormap(&tm_qkv);
     ptx::prefetch_tensormap(&tm_do);
     ptx::prefetch_tensormap(&tm_qkv_y);
@@ -974,7 +991,7 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   pdl_entry();
   const bool staged = n_seg < kSegStage;
   if (staged)
-    for (int i = tid; i <= n_seg; i += kAliasedThreads) seg_s[i] = __ldg(seg + i);
+    for (int i = tid; i <= n_seg; i += kBwdThreads) seg_s[i] = __ldg(seg + i);
   const int Np = packed_rows(seg, n_seg, capacity);
   const int n_items = ((Np + 127) / 128) * H;
   if ((int)blockIdx.x >= n_items) return;
@@ -985,19 +1002,23 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   const int h = item % H, r0 = (item / H) * 128;
   // tiles whose rows all belong to the one-pass kernel are passed over before anything is fetched
   if (skip_short && !tile_has_long_rows(seg_s, seg, staged, n_seg, Np, r0)) continue;
-  const int x1_col = (kDQ ? 0 : C) + h * D;           // own operand inside qkv: Q | K
-  if (tid == 0) {
+  const int x1_col = C + h * D;                       // own operand inside qkv: K
+  if (tid == kBwdMath) {
     if (!first_item) {  // every phase of the previous item has completed: the barriers start over
       ptx::mbar_inval(bar_x);
-      for (int s3 = 0; s3 < kBwdStages; ++s3) ptx::mbar_inval(bar_y(s3));
+      for (int s3 = 0; s3 < kStages; ++s3) ptx::mbar_inval(bar_y(s3));
       ptx::mbar_inval(bar_s);
-      ptx::mbar_inval(bar_o);
+      ptx::mbar_inval(bar_dp);
+      ptx::mbar_inval(bar_acc);
+      ptx::mbar_inval(bar_sfree);
+      ptx::mbar_inval(bar_pready);
+      ptx::mbar_inval(bar_dsready);
       init_barriers();
     }
     // the own tiles depend only on r0: fetch them under the segment search
-    ptx::mbar_expect_tx(bar_x, kOwn * kTile);
+    ptx::mbar_expect_tx(bar_x, 2 * kTile);
     ptx::tma_load_2d(x1_s, &tm_qkv, bar_x, x1_col, r0);
-    ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);         // V
+    ptx::tma_load_2d(x2_s, &tm_qkv, bar_x, 2 * C + h * D, r0);           // V
   }
   if (first_item && warp == 0) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
   first_item = false;
@@ -1008,14 +1029,17 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
 
   const int row = r0 + rl;
-  RowSeg mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
-  // segments that fit one tile belong to the one-pass kernel: their rows are no rows of this one
-  if (skip_short && mine.hi - mine.lo <= kShortMax) mine = RowSeg{0, 0};
-  if (half == 0) {
-    row_ok[rl] = mine.hi > mine.lo ? 1 : 0;
-    if (mine.hi > mine.lo) {  // the query rows to visit: the union of the segments of this tile's rows
-      atomicMin(const_cast<int*>(range), mine.lo);
-      atomicMax(const_cast<int*>(range) + 1, mine.hi);
+  RowSeg mine{0, 0};
+  if (is_math) {
+    mine = staged ? row_segment_staged(seg_s, n_seg, Np, row) : row_segment(seg, n_seg, Np, row);
+    // segments that fit one tile belong to the one-pass kernel: their rows are no rows of this one
+    if (skip_short && mine.hi - mine.lo <= kShortMax) mine = RowSeg{0, 0};
+    if (half == 0) {
+      row_ok[rl] = mine.hi > mine.lo ? 1 : 0;
+      if (mine.hi > mine.lo) {  // the rows of the other side to visit: the union of the segments of this tile's rows
+        atomicMin(const_cast<int*>(range), mine.lo);
+        atomicMax(const_cast<int*>(range) + 1, mine.hi);
+      }
     }
   }
   __syncthreads();
@@ -1023,177 +1047,252 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
   const int o_lo = any_row ? range[0] : 0, o_hi = any_row ? range[1] : 0;
   const int n_tiles = (o_hi - o_lo + kBwdY - 1) / kBwdY;
 
-  const int y1_col = (kDQ ? C : 0) + h * D;           // streamed operand inside qkv: K | Q
-  auto load_other = [&](int t_) {  // streamed tile t_ into stage t_ mod kBwdStages
-    const int st = t_ % kBwdStages, y0 = o_lo + t_ * kBwdY;
+  const int y1_col = h * D;                           // streamed operand inside qkv: Q
+  auto load_other = [&](int t_) {  // streamed tile t_ into its stage
+    const int st = stage_of(t_), y0 = o_lo + t_ * kBwdY;
     ptx::mbar_expect_tx(bar_y(st), 2 * kYTile);
     ptx::tma_load_2d(smem_base + y1_off(st), &tm_qkv_y, bar_y(st), y1_col, y0);
-    if (kDQ) ptx::tma_load_2d(smem_base + y2_off(st), &tm_qkv_y, bar_y(st), 2 * C + h * D, y0);   // V
-    else ptx::tma_load_2d(smem_base + y2_off(st), &tm_do_y, bar_y(st), h * D, y0);                // dO
+    ptx::tma_load_2d(smem_base + y2_off(st), &tm_do_y, bar_y(st), h * D, y0);                     // dO
   };
-  int issued = 0;  // streamed tiles whose loads thread 0 has issued
-  if (tid == 0) {
-    for (int t_ = 0; t_ < n_tiles && t_ < kBwdStages - 1; ++t_) load_other(t_);
-    issued = n_tiles < kBwdStages - 1 ? n_tiles : kBwdStages - 1;
+  int issued = 0;  // streamed tiles whose loads have been issued (kept by the issuing thread)
+  if (tid == kBwdMath) {
+    for (int t_ = 0; t_ < n_tiles && t_ < kStages; ++t_) load_other(t_);  // every stage is free at the start
+    issued = n_tiles < kStages ? n_tiles : kStages;
   }
+
+  // Bounded wait that also gives up as soon as any thread of the CTA has reported a failure.
+  auto wait = [&](uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < ptx::kWaitLimit; ++i) {
+      if (ptx::mbar_try_wait(bar, parity)) return true;
+      if ((i & 255u) == 255u && *abort_any) return false;
+    }
+    return false;
+  };
+  // every lane polls; the warp takes one answer, so that a whole warp gives up or none of it
+  auto wait_w = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, wait(bar, parity)) != 0; };
+
   // per-row statistics of the query side
-  float my_lse = 0.f, my_D = 0.f;   // kDQ: this thread's query row
-  float nxt_lse = 0.f, nxt_D = 0.f; // !kDQ: prefetched values of the next streamed query tile, row rl < 64
-  if (kDQ) {
-    if (row < Np) my_lse = lse[(long long)h * capacity + row] * kLog2e;
-  } else if (half == 0 && rl < kBwdY) {
+  float nxt_lse = 0.f, nxt_D = 0.f;  // prefetched values of the next streamed query tile, row rl < 64
+  if (is_math && half == 0 && rl < kBwdY) {
     const int i = o_lo + rl;
     if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
   }
 
   constexpr uint32_t kIdescS = ptx::idesc_bf16_f32(128, kBwdY, false, false);
-  constexpr uint32_t kIdescAcc = ptx::idesc_bf16_f32(128, D, false, true);
   const unsigned span = (unsigned)(mine.hi - mine.lo);
 
-  // Make streamed tile t_ ready for the products: its load has landed, lines past the last valid packed row
-  // are zeroed (they are unspecified memory and would be summed over), its query statistics are staged.
+  // Make streamed tile t_ ready for the products (arithmetic warps): its load has landed, lines past the last
+  // valid packed row are zeroed (they are unspecified memory and would be summed over), its query statistics
+  // are staged.  Returns false when the wait for the load gave up.
   auto prep = [&](int t_) {
-    const int st = t_ % kBwdStages;
-    bool ok = ptx::mbar_wait(bar_y(st), (t_ / kBwdStages) & 1);
-    if (t_ == 0) ok = ptx::mbar_wait(bar_x, 0) && ok;
-    if (!ok) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
+    const int st = stage_of(t_);
+    bool ok = true;
     const int y0 = o_lo + t_ * kBwdY;
+    // the issuing thread waits for the load itself; the arithmetic warps need it only where they touch the tile
+    if (t_ == 0) {
+      ok = wait_w(bar_y(st), use_of(t_));
+      ok = wait_w(bar_x, 0) && ok;
+    } else if (y0 + kBwdY > Np) {
+      ok = wait_w(bar_y(st), use_of(t_));
+    }
     if (y0 + kBwdY > Np) {
       const int first = Np - y0;
       constexpr int kChunks = HT::kRowBytes / 16;
-      for (int c = tid; c < (kBwdY - first) * kChunks; c += kAliasedThreads) {
+      for (int c = tid; c < (kBwdY - first) * kChunks; c += kBwdMath) {
         const int off = (first + c / kChunks) * HT::kRowBytes + (c % kChunks) * 16;
         *reinterpret_cast<uint4*>(smem_al + y1_off(st) + off) = make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4*>(smem_al + y2_off(st) + off) = make_uint4(0, 0, 0, 0);
       }
       ptx::fence_proxy_async_smem();
     }
-    if (!kDQ && half == 0 && rl < kBwdY) {
-      stat_lse[(t_ & 1) * kBwdY + rl] = nxt_lse;
-      stat_D[(t_ & 1) * kBwdY + rl] = nxt_D;
+    if (half == 0 && rl < kBwdY) {
+      stat_lse[(t_ % 3) * kBwdY + rl] = nxt_lse;
+      stat_D[(t_ % 3) * kBwdY + rl] = nxt_D;
       const int i = y0 + kBwdY + rl;
       nxt_lse = 0.f; nxt_D = 0.f;
       if (i < o_hi) { nxt_lse = lse[(long long)h * capacity + i] * kLog2e; nxt_D = delta[(long long)h * capacity + i]; }
     }
-  };
-  auto issue_s = [&](int t_) {  // the two fp32 tiles of streamed tile t_ (S and dP, or their transposes)
-    const int st = t_ % kBwdStages;
-#pragma unroll
-    for (int k = 0; k < D / 16; ++k)
-      ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(smem_base + y1_off(st), k), kIdescS, k != 0 ? 1u : 0u);
-#pragma unroll
-    for (int k = 0; k < D / 16; ++k)
-      ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(smem_base + y2_off(st), k), kIdescS, k != 0 ? 1u : 0u);
-    ptx::mma_commit(bar_s);
+    return ok;
   };
 
-  if (n_tiles > 0) prep(0);
+  if (is_math && n_tiles > 0 && !prep(0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
   ptx::tc_fence_before_sync();
-  __syncthreads();
-  if (tid == 0 && !*abort_flag && n_tiles > 0) { ptx::tc_fence_after_sync(); issue_s(0); }
-  if (kDQ && row < Np) {
-    // D_i = dO_i . O_i from the two staged tiles (their load has completed: prep(0) waited for it).  Both
-    // carry the same swizzle, so equal positions hold equal columns and the order of the chunks is free:
-    // each row starts at a different chunk to keep 8 neighbouring rows off one bank.
-    constexpr int kChunks = HT::kRowBytes / 16;
-    const uint8_t* po = smem_al + 2 * kTile + rl * HT::kRowBytes;
-    const uint8_t* pg = smem_al + kTile + rl * HT::kRowBytes;
-    const int rot = chunk_rot<D>(rl);
-#pragma unroll
-    for (int c = 0; c < kChunks; ++c) {
-      float a[8], b[8];
-      Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(po + ((c ^ rot) << 4)), a);
-      Vec16<__nv_bfloat16>::to_float(*reinterpret_cast<const uint4*>(pg + ((c ^ rot) << 4)), b);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) my_D = fmaf(a[e], b[e], my_D);
-    }
-    if (half == 0) delta[(long long)h * capacity + row] = my_D;
-  }
+  __syncthreads();  // tile 0 is ready; a failure so far is seen by all threads or by none
+  const bool failed_early = *abort_any != 0 || n_tiles == 0;
 
-  constexpr int kPc = kBwdY / 2;  // fp32 columns of each tile owned by this thread
-  const int col0 = half * kPc;
-  bool dead = false;
-  for (int t = 0; t < n_tiles; ++t) {
-    const int st = t % kBwdStages;
-    const int y0 = o_lo + t * kBwdY;
-    // ---- this thread's columns of both fp32 tiles into registers.  bar_s also covers the accumulating
-    // products of tile t-1 (commits are in issue order), so its streamed stage is free again.
-    if (!ptx::mbar_wait(bar_s, t & 1)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-    ptx::tc_fence_after_sync();
-    if (tid == 0 && t + kBwdStages - 1 < n_tiles) { load_other(t + kBwdStages - 1); issued = t + kBwdStages; }  // stage of tile t - 1
-    uint32_t rs[kPc], rp[kPc];
-    ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0, rs);
-    ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0, rp);
-    ptx::tmem_ld_wait();
-    ptx::tc_fence_before_sync();
-    __syncthreads();  // A: every thread holds its fp32 columns; their TMEM columns may now take the bf16 operands
-    if (*abort_flag) { dead = true; break; }
-
-    // ---- P = 2^(S - lse), dS = P (dP - D).  A thread whose 32 columns lie wholly outside its row's segment
-    // writes zeros without doing the arithmetic; the mask costs something only where a boundary crosses.
-    const int yc0 = y0 + col0;
-    uint32_t pk_p[kPc / 2], pk_ds[kPc / 2];
-    if (yc0 < mine.hi && yc0 + kPc > mine.lo) {
-      if (!(yc0 >= mine.lo && yc0 + kPc <= mine.hi)) {
+  if (!is_math) {
+    // ---------------------------------------------------------------- copies and products: one warp, whose lanes
+    // all follow the tiles and take every wait together; one elected lane issues (the same one each time, so its
+    // commits cover all its products)
+    if (!failed_early) {
+      constexpr uint32_t kIdescV = ptx::idesc_bf16_f32(128, D, false, true);  // A K-major (P^T in shared memory or dS^T in TMEM)
+      auto issue_st = [&](int t_) {  // S^T of streamed tile t_
+        const uint32_t y1a = smem_base + y1_off(stage_of(t_));
+        if (ptx::elect_one()) {
 #pragma unroll
-        for (int j = 0; j < kPc; ++j)
-          if ((unsigned)(yc0 + j - mine.lo) >= span) { rs[j] = 0xff800000u; rp[j] = 0u; }  // p = 2^-inf = 0, dP = 0
-      }
-      const float* sl = stat_lse + (t & 1) * kBwdY + col0;
-      const float* sd = stat_D + (t & 1) * kBwdY + col0;
-#pragma unroll
-      for (int j = 0; j < kPc; j += 2) {
-        float pv[2], dsv[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const float l2 = kDQ ? my_lse : sl[j + u];
-          const float Dv = kDQ ? my_D : sd[j + u];
-          pv[u] = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + u]), scale_log2e, -l2));
-          dsv[u] = pv[u] * (__uint_as_float(rp[j + u]) - Dv);
+          for (int k = 0; k < D / 16; ++k)
+            ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1a, k), kIdescS, k != 0 ? 1u : 0u);
+          ptx::mma_commit(bar_s);
         }
-        __nv_bfloat162 bds = __floats2bfloat162_rn(dsv[0], dsv[1]);
-        pk_ds[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
-        __nv_bfloat162 bp = __floats2bfloat162_rn(pv[0], pv[1]);
-        pk_p[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
-      }
-    } else {
+        __syncwarp();
+      };
+      auto issue_dpt = [&](int t_) {  // dP^T of streamed tile t_
+        const uint32_t y2a = smem_base + y2_off(stage_of(t_));
 #pragma unroll
-      for (int j = 0; j < kPc / 2; ++j) { pk_p[j] = 0u; pk_ds[j] = 0u; }
-    }
-    if (!kDQ) ptx::tmem_st_32x16(tmem + lane_base + kColS1 + (col0 >> 1), pk_p);   // P^T over the consumed S^T
-    ptx::tmem_st_32x16(tmem + lane_base + kColS2 + (col0 >> 1), pk_ds);            // dS (or dS^T) over the consumed dP
-    ptx::tmem_st_wait();
-    if (t + 1 < n_tiles) prep(t + 1);
-    ptx::tc_fence_before_sync();
-    __syncthreads();  // B: the bf16 operands of tile t are complete, tile t+1 is ready
-    if (*abort_flag) { dead = true; break; }
-    if (tid == 0) {
+        for (int k = 0; k < D / 16; ++k)
+          ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2a, k), kIdescS, k != 0 ? 1u : 0u);
+        ptx::mma_commit(bar_dp);
+      };
+      bool ok = true;
       ptx::tc_fence_after_sync();
-      const uint32_t acc = (t != 0) ? 1u : 0u;
-      const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
-      if (kDQ) {
+      issue_st(0);
+      if (ptx::elect_one()) issue_dpt(0);
+      __syncwarp();
+      for (int t = 0; ok && t < n_tiles; ++t) {
+        const int st = stage_of(t);
+        if (t + 1 < n_tiles) {
+          // S^T of tile t is in registers and tile t + 1 has landed: its S^T runs under the arithmetic of tile t
+          if (!(ok = wait_w(bar_sfree, t & 1))) break;
+          if (!(ok = wait_w(bar_y(stage_of(t + 1)), use_of(t + 1)))) break;
+          ptx::tc_fence_after_sync();
+          issue_st(t + 1);
+        }
+        // the stage of tile t - 1 is free once its accumulating products have completed
+        if (t > 0 && t - 1 + kStages < n_tiles) {
+          if (!(ok = wait_w(bar_acc, (t - 1) & 1))) break;
+          if (ptx::elect_one()) load_other(t - 1 + kStages);
+          __syncwarp();
+          issued = t + kStages;
+        }
+        const uint32_t acc = (t != 0) ? 1u : 0u;
+        const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
+        if (!(ok = wait_w(bar_pready, t & 1))) break;     // P^T of tile t is in shared memory
+        ptx::tc_fence_after_sync();
+        if (ptx::elect_one()) {
 #pragma unroll
-        for (int k = 0; k < kBwdY / 16; ++k)   // dQ += dS K
-          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS2 + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+          for (int k = 0; k < kBwdY / 16; ++k)   // dV += P^T dO
+            ptx::mma_bf16(tmem + kColAcc1, HT::kmajor(p_s, k), HT::mnmajor(y2a, k), kIdescV, acc | (k != 0));
+        }
+        __syncwarp();
+        if (!(ok = wait_w(bar_dsready, t & 1))) break;    // dS^T of tile t is in TMEM, over the dP^T columns
+        ptx::tc_fence_after_sync();
+        if (ptx::elect_one()) {
+#pragma unroll
+          for (int k = 0; k < kBwdY / 16; ++k)   // dK += dS^T Q: queries 16k.. of the tile, stored by the warps of half k / 2
+            ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColS2 + (k >> 1) * 32 + (k & 1) * 8, HT::mnmajor(y1a, k), kIdescV,
+                             acc | (k != 0));
+          ptx::mma_commit(bar_acc);
+          // queued behind dK, which reads the columns that it overwrites (products of one thread execute in issue order)
+          if (t + 1 < n_tiles) issue_dpt(t + 1);
+        }
+        __syncwarp();
+      }
+      if (!ok && lane == 0) {
+        record_status(d_status, SPA_ERR_TIMEOUT);
+        *abort_any = 1;
+      }
+    }
+  } else if (!failed_early) {
+    // ---------------------------------------------------------------- arithmetic: two threads per key row
+    constexpr int kPc = kBwdY / 2;  // fp32 columns of each tile owned by this thread
+    const int col0 = half * kPc;
+    // no barrier joins the arithmetic warps inside the loop, so a warp whose wait gave up may leave it alone: the
+    // others see the flag in their own waits
+    auto fail = [&]() {
+      record_status(d_status, SPA_ERR_TIMEOUT);
+      *abort_any = 1;
+    };
+    // this thread's 64 bytes of its row of P^T: chunks 4 * half .. of a 128-byte line, under the 128-byte swizzle
+    uint8_t* p_row = smem_al + kPBase + rl * 128;
+    const int p_rot = rl & 7;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int y0 = o_lo + t * kBwdY;
+      // ---- S^T: this thread's columns into registers
+      bool ok = wait_w(bar_s, t & 1);
+      ptx::tc_fence_after_sync();
+      uint32_t rs[kPc];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS1 + col0, rs);
+      ptx::tmem_ld_wait();
+      if (ok && t + 1 < n_tiles) ok = prep(t + 1);
+      // the statistics of tile t were staged by other warps before they announced tile t - 1 (that phase has
+      // completed; it is waited for, before this warp's own arrival for tile t, to order the reads below)
+      if (ok && t > 0) ok = wait_w(bar_sfree, (t - 1) & 1);
+      if (!ok) { fail(); break; }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_sfree);
+
+      // ---- P^T = 2^(S^T - lse): needs S^T only, and holds the exponentials.  A thread whose 32 columns lie wholly
+      // outside its row's segment writes zeros without doing the arithmetic; the mask costs something only where a
+      // boundary crosses.
+      const int yc0 = y0 + col0;
+      const bool some = yc0 < mine.hi && yc0 + kPc > mine.lo;
+      const bool partial = some && !(yc0 >= mine.lo && yc0 + kPc <= mine.hi);
+      uint32_t pk[kPc / 2];
+      if (some) {
+        if (partial) {
+#pragma unroll
+          for (int j = 0; j < kPc; ++j)
+            if ((unsigned)(yc0 + j - mine.lo) >= span) rs[j] = 0xff800000u;  // p = 2^-inf = 0
+        }
+        const float* sl = stat_lse + (t % 3) * kBwdY + col0;
+#pragma unroll
+        for (int j = 0; j < kPc; j += 2) {
+          const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(rs[j]), scale_log2e, -sl[j]));
+          const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(rs[j + 1]), scale_log2e, -sl[j + 1]));
+          rs[j] = __float_as_uint(p0);
+          rs[j + 1] = __float_as_uint(p1);
+          __nv_bfloat162 bp = __floats2bfloat162_rn(p0, p1);
+          pk[j >> 1] = *reinterpret_cast<uint32_t*>(&bp);
+        }
       } else {
 #pragma unroll
-        for (int k = 0; k < kBwdY / 16; ++k)   // dV += P^T dO
-          ptx::mma_bf16_ts(tmem + kColAcc1, tmem + kColS1 + k * 8, HT::mnmajor(y2a, k), kIdescAcc, acc | (k != 0));
-#pragma unroll
-        for (int k = 0; k < kBwdY / 16; ++k)   // dK += dS^T Q
-          ptx::mma_bf16_ts(tmem + kColAcc2, tmem + kColS2 + k * 8, HT::mnmajor(y1a, k), kIdescAcc, acc | (k != 0));
+        for (int j = 0; j < kPc / 2; ++j) pk[j] = 0u;
       }
-      if (t + 1 < n_tiles) issue_s(t + 1);  // queued behind the products above, which read the columns it overwrites
-      else ptx::mma_commit(bar_o);
-    }
-  }
-  if (!dead && n_tiles > 0) {
-    if (!ptx::mbar_wait(bar_o, 0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
-    ptx::tc_fence_after_sync();
-  }
-  __syncthreads();  // nobody sets the flag from here on: the branch below is taken by all threads or by none
+      // dV of tile t - 1 must have read P^T (its completion is announced together with dK's)
+      if (t > 0) {
+        if (!wait_w(bar_acc, (t - 1) & 1)) { fail(); break; }
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<uint4*>(p_row + (((half * 4 + c) ^ p_rot) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_pready);
 
-  if (!*abort_flag && n_tiles > 0) {
+      // ---- dS^T = P^T (dP^T - D), stored over this thread's own dP^T columns (the first 16 of its 32)
+      if (!wait_w(bar_dp, t & 1)) { fail(); break; }
+      ptx::tc_fence_after_sync();
+      uint32_t rp[kPc];
+      ptx::tmem_ld_32x32(tmem + lane_base + kColS2 + col0, rp);  // by the whole warp: the load is a collective
+      ptx::tmem_ld_wait();
+      if (some) {
+        const float* sd = stat_D + (t % 3) * kBwdY + col0;
+#pragma unroll
+        for (int j = 0; j < kPc; j += 2) {
+          // a masked column has p = 0 exactly and a finite dP^T (rows past the last valid one are zeroed): dS^T = 0
+          const float d0 = __uint_as_float(rs[j]) * (__uint_as_float(rp[j]) - sd[j]);
+          const float d1 = __uint_as_float(rs[j + 1]) * (__uint_as_float(rp[j + 1]) - sd[j + 1]);
+          __nv_bfloat162 bds = __floats2bfloat162_rn(d0, d1);
+          pk[j >> 1] = *reinterpret_cast<uint32_t*>(&bds);
+        }
+      }
+      ptx::tmem_st_32x16(tmem + lane_base + kColS2 + col0, pk);
+      ptx::tmem_st_wait();
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_dsready);
+    }
+    // the last accumulating products complete the outputs
+    const bool gave_up = __shfl_sync(0xffffffffu, *abort_any, 0) != 0;  // one answer per warp
+    if (n_tiles > 0 && !gave_up && !wait_w(bar_acc, (n_tiles - 1) & 1)) fail();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();  // nobody reports a failure from here on: the branches below are taken by all threads or by none
+  ptx::tc_fence_after_sync();
+  const bool failed = *abort_any != 0;
+
+  if (!failed && n_tiles > 0) {
     // Each thread drains d/2 columns of its row of the accumulators into the own tiles' shared memory (idle
     // now: every product has completed), from where whole rows go out as full lines.
     constexpr int kDh = D / 2;
@@ -1213,24 +1312,19 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
       }
     };
     const long long ld = 3LL * C;
-    if (kDQ) {
-      stage_acc(kColAcc1, smem_al, scale);
-      __syncthreads();
-      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + h * D, ld, r0, Np, tid);
-    } else {
+    if (is_math) {
       stage_acc(kColAcc1, smem_al, 1.f);             // dV
       stage_acc(kColAcc2, smem_al + kTile, scale);   // dK
-      __syncthreads();
-      copy_tile_out<D, kAliasedThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid, row_ok);
-      copy_tile_out<D, kAliasedThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid, row_ok);
     }
+    __syncthreads();
+    copy_tile_out<D, kBwdThreads>(smem_al, dqkv + 2 * C + h * D, ld, r0, Np, tid, row_ok);
+    copy_tile_out<D, kBwdThreads>(smem_al + kTile, dqkv + C + h * D, ld, r0, Np, tid, row_ok);
   }
-  if ((*abort_flag || n_tiles == 0) && tid == 0) {  // let outstanding loads land before shared memory is released
-    for (int t = issued > kBwdStages ? issued - kBwdStages : 0; t < issued; ++t)
-      ptx::mbar_wait(bar_y(t % kBwdStages), (t / kBwdStages) & 1);
+  if ((failed || n_tiles == 0) && tid == kBwdMath) {  // let outstanding loads land before shared memory is released
+    for (int t = issued > kStages ? issued - kStages : 0; t < issued; ++t) ptx::mbar_wait(bar_y(stage_of(t)), use_of(t));
     ptx::mbar_wait(bar_x, 0);
   }
-  cta_failed = *abort_flag != 0;
+  cta_failed = failed;
   ptx::tc_fence_before_sync();
   __syncthreads();  // the tiles' memory and the barriers are free for the next item
   } while (kLoop && (item += gridDim.x) < n_items && !cta_failed);
@@ -1239,7 +1333,6 @@ attn_bwd_kv_aliased_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __g
     ptx::tmem_dealloc(*tmem_slot, kBwdTmemCols);
   }
 }
-
 
 // ------------------------------------------------------------------------------------------------
 // Backward for segments of at most 128 rows, in one pass: a CTA owns one segment and one head, holds its queries
@@ -1479,9 +1572,9 @@ template <int D> struct kv_pass {
   template <bool kLoop> static auto kernel() { return attn_bwd_tc_kernel<D, false, kLoop>; }
 };
 template <> struct kv_pass<64> {
-  static constexpr int kThreads = kAliasedThreads;
-  static constexpr int kSmem = aliased_smem_bytes<64>();
-  template <bool kLoop> static auto kernel() { return attn_bwd_kv_aliased_kernel<64, kLoop>; }
+  static constexpr int kThreads = kBwdThreads;
+  static constexpr int kSmem = split_smem_bytes<64>();
+  template <bool kLoop> static auto kernel() { return attn_bwd_kv_split_kernel<64, kLoop>; }
 };
 
 template <int D>
