@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(kGemmThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, long long ldo,
                long long split_stride, int M, int N, int K, const int32_t* __restrict__ cu, int n_seg, int capacity,
-               int dyn_which, int k_per_split, const int32_t* __restrict__ row_map,
+               int dyn_which, int k_per_split, int k_interleave, const int32_t* __restrict__ row_map,
                int accumulate, int32_t* d_status) {
   constexpr int kStage = stage_bytes<BN>();
   constexpr uint32_t kIdesc = ptx::idesc_bf16_f32(BM, BN, kAMn, kBMn);
@@ -138,7 +138,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   const int tiles_n = (N + BN - 1) / BN;
   const int tiles_m = (M + BM - 1) / BM;
-  const int n_splits = K > 0 ? (K + k_per_split - 1) / k_per_split : 0;
+  // Split-K: contiguous spans of k_per_split, or (k_interleave > 0) that many splits dealt the BK-blocks of K in
+  // turn - split z takes blocks z, z + splits, ... - so that the splits get equal work whatever K turns out to be.
+  const int k_blocks = (K + BK - 1) / BK;
+  const int n_splits = k_interleave > 0 ? (k_blocks < k_interleave ? k_blocks : k_interleave)
+                                        : (K > 0 ? (K + k_per_split - 1) / k_per_split : 0);
   const int total = tiles_m * tiles_n * n_splits;
   auto coord = [&](int tile) {
     TileCoord c;
@@ -149,10 +153,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     c.n0 = c.n_t * BN;
     return c;
   };
-  auto k_range = [&](int z, int& k_begin, int& k_end) {
-    k_begin = z * k_per_split;
-    k_end = k_begin + k_per_split;
-    if (k_end > K) k_end = K;
+  auto k_range = [&](int z, int& k_begin, int& k_end, int& k_step) {
+    if (k_interleave > 0) {
+      k_begin = z * BK;
+      k_end = K;
+      k_step = n_splits * BK;
+    } else {
+      k_begin = z * k_per_split;
+      k_end = k_begin + k_per_split;
+      if (k_end > K) k_end = K;
+      k_step = BK;
+    }
   };
 
   if (warp == 0) {
@@ -161,9 +172,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int it = 0;  // k-block counter over all tiles of this CTA: ring position and phase
       for (int tile = blockIdx.x; tile < total && !*abort_flag; tile += gridDim.x) {
         const TileCoord c = coord(tile);
-        int k_begin, k_end;
-        k_range(c.z, k_begin, k_end);
-        for (int k0 = k_begin; k0 < k_end; k0 += BK, ++it) {
+        int k_begin, k_end, k_step;
+        k_range(c.z, k_begin, k_end, k_step);
+        for (int k0 = k_begin; k0 < k_end; k0 += k_step, ++it) {
           const int s = it % kStages;
           if (it >= kStages && !ptx::mbar_wait(empty_bar(s), ((it / kStages) - 1) & 1)) {
             record_status(d_status, SPA_ERR_TIMEOUT);
@@ -200,8 +211,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int tile = blockIdx.x; tile < total && !dead; tile += gridDim.x, ++tl) {
       if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
       const TileCoord c = coord(tile);
-      int k_begin, k_end;
-      k_range(c.z, k_begin, k_end);
+      int k_begin, k_end, k_step;
+      k_range(c.z, k_begin, k_end, k_step);
       const int acc = tl & 1;
       if (tl >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(tmem_empty_bar(acc), ((tl >> 1) - 1) & 1))) {
         if (lane == 0) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_flag = 1; }
@@ -210,7 +221,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ptx::tc_fence_after_sync();
       const uint32_t tmem_d = tmem_base + acc * BN;
       bool first = true;
-      for (int k0 = k_begin; k0 < k_end; k0 += BK, ++it) {
+      for (int k0 = k_begin; k0 < k_end; k0 += k_step, ++it) {
         const int s = it % kStages;
         if (__any_sync(0xffffffffu, *abort_flag != 0)) { dead = true; break; }
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(full_bar(s), (it / kStages) & 1))) {
@@ -237,7 +248,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           __syncwarp();
         }
         ptx::tc_fence_after_sync();
-        if (lane == 0) {
+        if (ptx::elect_one()) {  // one lane of the converged warp issues: the descriptors stay in uniform registers
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t adesc = kAMn ? ptx::smem_desc_sw128(a_src + k * 2048, BK * 128, 1024)
@@ -251,7 +262,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         first = false;
         __syncwarp();
       }
-      if (lane == 0 && !first) ptx::mma_commit(tmem_full_bar(acc));
+      if (!first && ptx::elect_one()) ptx::mma_commit(tmem_full_bar(acc));  // the same lane as above: it covers its products
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
@@ -402,11 +413,12 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const i
 // chunks) in one launch.
 __global__ void __launch_bounds__(256)
 split_reduce_kernel(const float* __restrict__ part, long long n, const float* __restrict__ part2, long long n2,
-                    int k_per_split, int rows_per_chunk2, const int32_t* __restrict__ cu, int n_seg, int capacity,
+                    int splits, int rows_per_chunk2, const int32_t* __restrict__ cu, int n_seg, int capacity,
                     float* __restrict__ out, float* __restrict__ out2) {
   pdl_entry();
   const int rows = packed_rows(cu, n_seg, capacity);
-  const int valid1 = (rows + k_per_split - 1) / k_per_split;
+  const int k_blocks = (rows + BK - 1) / BK;  // the splits were dealt the BK-blocks of the rows in turn
+  const int valid1 = k_blocks < splits ? k_blocks : splits;
   const int valid2 = (rows + rows_per_chunk2 - 1) / rows_per_chunk2;
   const long long n4 = n >> 2, m4 = n2 >> 2;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4 + m4;
@@ -426,10 +438,12 @@ split_reduce_kernel(const float* __restrict__ part, long long n, const float* __
 
 struct SplitPlan { int splits, k_per_split; };
 
-// K = packed rows is cut into equal spans (multiples of BK) so that tiles x splits fills the GPU.
+// The BK-blocks of K = packed rows are dealt to the splits in turn, so every split is in use whatever the row count;
+// as many splits as keep tiles x splits within the CTAs that are resident at once (a second tile for some of the CTAs
+// would double the longest path).
 SplitPlan plan_splits(int capacity, int n_in, int n_out) {
   const int tiles = ((n_out + BM - 1) / BM) * ((n_in + 127) / 128);
-  int splits = (2 * kNumSMs + tiles - 1) / tiles;
+  int splits = (2 * kNumSMs) / tiles;
   const int max_by_rows = (capacity + BK - 1) / BK;
   if (splits > max_by_rows) splits = max_by_rows;
   if (splits > 32) splits = 32;
@@ -450,7 +464,7 @@ size_t wgrad_workspace_bytes(int capacity, int n_in, int n_out) {
 template <int BN, bool kAMn, bool kBMn, typename OutT>
 int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloat16* bias, OutT* out, long long ldo,
                 long long split_stride, int M, int N, int K, const int32_t* cu, int n_seg, int capacity, int dyn_which,
-                int k_per_split, int splits, const int32_t* row_map, int accumulate,
+                int k_per_split, int splits, int k_interleave, const int32_t* row_map, int accumulate,
                 int32_t* d_status, cudaStream_t st, const char* what) {
   auto kern = gemm_tc_kernel<BN, kAMn, kBMn, OutT>;
   static DeviceOnce attr;  // per instantiation and device
@@ -461,7 +475,7 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const __nv_bfloa
   long long tiles = (long long)((N + BN - 1) / BN) * ((M + BM - 1) / BM) * splits;
   const int grid = (int)(tiles < 2 * kNumSMs ? (tiles < 1 ? 1 : tiles) : 2 * kNumSMs);
   launch_pdl(kern, grid, kGemmThreads, gemm_smem_bytes<BN>(), st, tmA, tmB, bias, out, ldo, split_stride, M, N, K, cu,
-             n_seg, capacity, dyn_which, k_per_split, row_map, accumulate, d_status);
+             n_seg, capacity, dyn_which, k_per_split, k_interleave, row_map, accumulate, d_status);
   SPA_CUDA_CHECK_LAUNCH(what);
   return SPA_OK;
 }
@@ -490,7 +504,7 @@ int launch_linear_fwd_tc(const spa_params& p, const void* a, const void* W, cons
     return SPA_ERR_UNSUPPORTED;
   return launch_gemm<128, false, false, __nv_bfloat16>(tmA, tmB, (const __nv_bfloat16*)bias,
                                                               (__nv_bfloat16*)out, n_out, 0, p.capacity, n_out, n_in,
-                                                              cu, p.B, p.capacity, 1, n_in, 1, row_map,
+                                                              cu, p.B, p.capacity, 1, n_in, 1, 0, row_map,
                                                               accumulate ? 1 : 0, d_status, st, "gemm_tc_kernel(fwd)");
 }
 
@@ -515,7 +529,7 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   } else if (da != nullptr) {  // da[M][n_in] = dout[M][n_out] W[n_out][n_in]
     int rc = launch_gemm<128, false, true, __nv_bfloat16>(tmA, tmB, nullptr, (__nv_bfloat16*)da, n_in, 0,
                                                                  p.capacity, n_in, n_out, cu, p.B, p.capacity, 1, n_out,
-                                                                 1, row_map, accumulate ? 1 : 0, d_status, st,
+                                                                 1, 0, row_map, accumulate ? 1 : 0, d_status, st,
                                                                  "gemm_tc_kernel(dgrad)");
     if (rc != SPA_OK) return rc;
   }
@@ -533,18 +547,18 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
   }
   if (dW != nullptr) {  // dW[n_out][n_in] = sum_i dout[i][:]^T a[i][:]
     int rc = launch_gemm<128, true, true, float>(tmA2, tmB2, nullptr, part_w, n_in, n_w, n_out, n_in, p.capacity,
-                                                        cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, nullptr,
-                                                        0, d_status, st, "gemm_tc_kernel(wgrad)");
+                                                        cu, p.B, p.capacity, 2, sp.k_per_split, sp.splits, sp.splits,
+                                                        nullptr, 0, d_status, st, "gemm_tc_kernel(wgrad)");
     if (rc != SPA_OK) return rc;
     const long long n_b = db != nullptr ? n_out : 0;
     int grid = (int)(((n_w + n_b) / 4 + 255) / 256);
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
-    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.k_per_split, rpc, cu, p.B, p.capacity, dW,
+    launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.splits, rpc, cu, p.B, p.capacity, dW,
                db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel");
   } else {  // db alone
-    launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, part_b, (long long)n_out, (const float*)nullptr,
-               0LL, rpc, rpc, cu, p.B, p.capacity, db, (float*)nullptr);
+    launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, (const float*)nullptr, 0LL, (const float*)part_b,
+               (long long)n_out, 0, rpc, cu, p.B, p.capacity, (float*)nullptr, db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
   }
   return SPA_OK;
