@@ -10,7 +10,7 @@
 //   O += P V         tcgen05.mma with P read from TMEM and V from shared memory; O accumulates in TMEM over all tiles
 // m is the maximum that the stored P and O refer to.  It is raised - and O rescaled, TMEM -> registers -> TMEM - only
 // when a row's true maximum has outgrown it by more than 2^8, so most tiles cost no pass over O; sums and outputs are
-// exact for any reference value.  The first lane of a ninth warp issues every copy and every product: the next tile's
+// exact for any reference value.  One elected lane of a ninth warp issues every copy and every product: the next tile's
 // S product is issued as soon as every softmax warp holds the current S row, so the tensor core works under the
 // softmax.  K/V rows past the last valid packed row are unspecified memory: K columns are masked after the
 // product and V lines are zeroed in shared memory before the product.
@@ -27,7 +27,7 @@ namespace {
 constexpr int kQ = 128;        // query rows per CTA = TMEM lanes
 constexpr int kKV = 128;       // keys per tile
 constexpr int kSoftmaxThreads = 256;  // two threads per query row: each owns half of the key columns and half of d
-constexpr int kFwdThreads = kSoftmaxThreads + 32;  // and one warp whose first lane issues every copy and product
+constexpr int kFwdThreads = kSoftmaxThreads + 32;  // and one warp, one lane of which issues every copy and product
 constexpr float kRescaleGap = 8.f;  // log2 units by which a row's maximum may outgrow the one its P and O refer to
 constexpr uint32_t kTmemCols = 256;  // S: 128 fp32 columns, P: 64 (bf16 pairs), O tile: up to 64
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
@@ -219,61 +219,75 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
     return false;
   };
 
+  // every lane polls (measured faster than one lane polling for the warp); the warp takes one answer
+  auto wait_w = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, wait(bar, parity)) != 0; };
   if (!is_softmax) {
-    // ---------------------------------------------------------------- copies and products: one thread
-    if (lane == 0) {
-      auto load_k = [&](int t) {
+    // ---------------------------------------------------------------- copies and products: one warp, whose lanes
+    // all follow the tiles and take every wait together; one elected lane issues (see ptx::elect_one)
+    auto load_k = [&](int t) {
+      if (ptx::elect_one()) {
         ptx::mbar_expect_tx(bar_k(t & 1), kTile);
         ptx::tma_load_2d(k_s(t & 1), &tm, bar_k(t & 1), C + h * D, kv_lo + t * kKV);
-      };
-      auto load_v = [&](int t) {
+      }
+      __syncwarp();
+    };
+    auto load_v = [&](int t) {
+      if (ptx::elect_one()) {
         ptx::mbar_expect_tx(bar_v(t & 1), kTile);
         ptx::tma_load_2d(v_s(t & 1), &tm, bar_v(t & 1), 2 * C + h * D, kv_lo + t * kKV);
-      };
-      auto issue_qk = [&](int t) {  // S = Q K_t^T into TMEM; bar_s completes when it is done
-        if (!wait(bar_k(t & 1), (t >> 1) & 1)) return false;
-        ptx::tc_fence_after_sync();
+      }
+      __syncwarp();
+    };
+    auto issue_qk = [&](int t) {  // S = Q K_t^T into TMEM; bar_s completes when it is done
+      if (!wait_w(bar_k(t & 1), (t >> 1) & 1)) return false;
+      ptx::tc_fence_after_sync();
+      const uint32_t ka = k_s(t & 1);
+      if (ptx::elect_one()) {
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(k_s(t & 1), k), kIdescS, k != 0 ? 1u : 0u);
+          ptx::mma_bf16(tmem + kColS, HT::kmajor(q_s, k), HT::kmajor(ka, k), kIdescS, k != 0 ? 1u : 0u);
         ptx::mma_commit(bar_s);
-        return true;
-      };
-      int loads_k = 0, loads_v = 0;  // tiles whose loads have been issued
-      bool ok = true;
-      if (n_tiles > 0) {
-        load_k(0);
-        load_v(0);
-        loads_k = loads_v = 1;
-        if (n_tiles > 1) { load_k(1); loads_k = 2; }
-        ok = wait(bar_q, 0) && issue_qk(0);
       }
-      for (int t = 0; ok && t < n_tiles; ++t) {
-        // every softmax thread holds its S_t columns: the S columns and K stage t & 1 are free
-        if (!(ok = wait(bar_sfree, t & 1))) break;
-        if (t + 1 < n_tiles) {
-          if (!(ok = issue_qk(t + 1))) break;  // runs on the tensor core under the softmax of tile t
-          if (t + 2 < n_tiles) { load_k(t + 2); loads_k = t + 3; }
-        }
-        // P_t is in TMEM, O has been rescaled where needed, and the previous P V product has completed
-        if (!(ok = wait(bar_pready, t & 1))) break;
-        if (!(ok = wait(bar_v(t & 1), (t >> 1) & 1))) break;
-        ptx::tc_fence_after_sync();
+      __syncwarp();
+      return true;
+    };
+    int loads_k = 0, loads_v = 0;  // tiles whose loads have been issued
+    bool ok = true;
+    if (n_tiles > 0) {
+      load_k(0);
+      load_v(0);
+      loads_k = loads_v = 1;
+      if (n_tiles > 1) { load_k(1); loads_k = 2; }
+      ok = wait_w(bar_q, 0) && issue_qk(0);
+    }
+    for (int t = 0; ok && t < n_tiles; ++t) {
+      // every softmax thread holds its S_t columns: the S columns and K stage t & 1 are free
+      if (!(ok = wait_w(bar_sfree, t & 1))) break;
+      if (t + 1 < n_tiles) {
+        if (!(ok = issue_qk(t + 1))) break;  // runs on the tensor core under the softmax of tile t
+        if (t + 2 < n_tiles) { load_k(t + 2); loads_k = t + 3; }
+      }
+      // P_t is in TMEM, O has been rescaled where needed, and the previous P V product has completed
+      if (!(ok = wait_w(bar_pready, t & 1))) break;
+      if (!(ok = wait_w(bar_v(t & 1), (t >> 1) & 1))) break;
+      ptx::tc_fence_after_sync();
+      const uint32_t va = v_s(t & 1);
+      if (ptx::elect_one()) {
 #pragma unroll
         for (int k = 0; k < kKV / 16; ++k)
-          ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(v_s(t & 1), k), kIdescO,
-                           (k != 0 || t > 0) ? 1u : 0u);
+          ptx::mma_bf16_ts(tmem + kColO, tmem + kColP + k * 8, HT::mnmajor(va, k), kIdescO, (k != 0 || t > 0) ? 1u : 0u);
         ptx::mma_commit(bar_o);
-        if (t + 1 < n_tiles) { load_v(t + 1); loads_v = t + 2; }  // its stage held V of tile t - 1
       }
-      if (!ok) {
-        record_status(d_status, SPA_ERR_TIMEOUT);
-        *abort_any = 1;
-        // let outstanding loads land before shared memory is released
-        for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
-        for (int t = loads_v > 2 ? loads_v - 2 : 0; t < loads_v; ++t) ptx::mbar_wait(bar_v(t & 1), (t >> 1) & 1);
-        ptx::mbar_wait(bar_q, 0);
-      }
+      __syncwarp();
+      if (t + 1 < n_tiles) { load_v(t + 1); loads_v = t + 2; }  // its stage held V of tile t - 1
+    }
+    if (!ok && lane == 0) {
+      record_status(d_status, SPA_ERR_TIMEOUT);
+      *abort_any = 1;
+      // let outstanding loads land before shared memory is released
+      for (int t = loads_k > 2 ? loads_k - 2 : 0; t < loads_k; ++t) ptx::mbar_wait(bar_k(t & 1), (t >> 1) & 1);
+      for (int t = loads_v > 2 ? loads_v - 2 : 0; t < loads_v; ++t) ptx::mbar_wait(bar_v(t & 1), (t >> 1) & 1);
+      ptx::mbar_wait(bar_q, 0);
     }
   } else {
     // ---------------------------------------------------------------- online softmax: two threads per query row
@@ -284,8 +298,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm, const int32_t* __rest
       abort_pair[slot * 4 + quarter] = 1;
       *abort_any = 1;
     };
-    // every lane polls (measured faster than one lane polling for the warp); the warp takes one answer
-    auto wait_w = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, wait(bar, parity)) != 0; };
     for (int t = 0; t < n_tiles; ++t) {
       const int st = t & 1;
       const int kv0 = kv_lo + t * kKV;
