@@ -428,10 +428,20 @@ split_reduce_kernel(const float* __restrict__ part, long long n, const float* __
     const long long stride = second ? n2 : n, j = second ? i - n4 : i;
     float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
     const int valid = second ? valid2 : valid1;
-    for (int z = 0; z < valid; ++z) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(src + (long long)z * stride) + j);
-      s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w;
+    // loads four splits at a time in flight; the additions stay in split order
+    auto add = [&](const float4& v) { s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w; };
+    auto at = [&](int z) { return __ldcs(reinterpret_cast<const float4*>(src + (long long)z * stride) + j); };
+    int z = 0;
+    for (; z + 4 <= valid; z += 4) {
+      const float4 v0 = at(z), v1 = at(z + 1), v2 = at(z + 2), v3 = at(z + 3);
+      add(v0); add(v1); add(v2); add(v3);
     }
+    if (z + 2 <= valid) {
+      const float4 v0 = at(z), v1 = at(z + 1);
+      add(v0); add(v1);
+      z += 2;
+    }
+    if (z < valid) add(at(z));
     reinterpret_cast<float4*>(second ? out2 : out)[j] = s4;
   }
 }
