@@ -413,9 +413,17 @@ int spa_block_bwd(const spa_params* p, const spa_block_buffers* b, void* stream)
  * 4d flops).  sink: float[n_ctas], never written in practice.
  * spa_probe_wait_expiry: one warp waits on a barrier that nobody arrives at and gives up after `limit` polls
  * (<= 2^20): d_status receives SPA_ERR_TIMEOUT and *polls_done (device int32, may be NULL) the polls made.  Shows,
- * without any fault or hang, what every bounded wait of the kernels does when it runs out. */
+ * without any fault or hang, what every bounded wait of the kernels does when it runs out.
+ * spa_probe_mma_issue: one CTA issues 32 back-to-back tensor-core products of a shape the attention kernels use
+ * (M = 128, K = 16, bf16, zeroed operands; variant 0: both operands in shared memory, N = 64; 1: A in TMEM, N = 64;
+ * 2, 3: shared memory, N = 128, 256) and commits them to a barrier; elected = 0: lane 0 of a warp issues alone,
+ * 1: all lanes of the warp run the loop and one elected lane issues.  cycles (device uint32[2]) receives the fastest
+ * of 20 repetitions: [0] SM clocks from the first product to the commit, [1] until the barrier completes.  The probe
+ * takes all 512 TMEM columns of its SM while it runs: call it with nothing else in flight.  Its wait is bounded
+ * (SPA_ERR_TIMEOUT in d_status). */
 int spa_probe_exp2(int32_t n_ctas, int32_t iters, float* sink, unsigned long long* n_exp, void* stream);
 int spa_probe_wait_expiry(int32_t limit, int32_t* d_status, int32_t* polls_done, void* stream);
+int spa_probe_mma_issue(int32_t variant, int32_t elected, uint32_t* cycles, int32_t* d_status, void* stream);
 
 /* Blocking read of the device status word: synchronises `stream` and returns its value. */
 int spa_read_status(const int32_t* d_status, void* stream);

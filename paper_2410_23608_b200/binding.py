@@ -33,7 +33,7 @@ EXPORTS = (
     "spa_select_pack_ordered", "spa_train_workspace_bytes", "spa_score_pool", "spa_select_loss", "spa_select_pack_bwd_gated", "spa_gate_bwd",
     "spa_packed_linear", "spa_layer_norm", "spa_layer_norm_bwd", "spa_gelu", "spa_gelu_bwd",
     "spa_overlap_create", "spa_overlap_destroy", "spa_block_fwd", "spa_block_bwd",
-    "spa_probe_exp2", "spa_probe_wait_expiry", "spa_pack_state_bytes", "spa_gate_select_pack_supported",
+    "spa_probe_exp2", "spa_probe_wait_expiry", "spa_probe_mma_issue", "spa_pack_state_bytes", "spa_gate_select_pack_supported",
     "spa_gate_select_pack", "spa_container_max_segments", "spa_container_offsets",
 )
 
@@ -128,6 +128,7 @@ def lib() -> C.CDLL:
         L.spa_container_offsets.argtypes = [pp, vp, i32, vp, vp]
         L.spa_probe_exp2.argtypes = [i32, i32, vp, C.POINTER(C.c_ulonglong), vp]
         L.spa_probe_wait_expiry.argtypes = [i32, vp, vp, vp]
+        L.spa_probe_mma_issue.argtypes = [i32, i32, vp, vp, vp]
         L.spa_read_status.argtypes = [vp, vp]
         for name in EXPORTS:
             if name not in ("spa_workspace_bytes", "spa_train_workspace_bytes", "spa_pack_state_bytes", "spa_status_string", "spa_last_cuda_error",
@@ -375,6 +376,13 @@ def spa_probe_exp2(n_ctas, iters, sink, stream=None) -> int:
 def spa_probe_wait_expiry(limit, d_status, polls_done=None, stream=None):
     _check(lib().spa_probe_wait_expiry(int(limit), _ptr(d_status), _ptr(polls_done), _stream(stream)),
            "spa_probe_wait_expiry")
+
+
+def spa_probe_mma_issue(variant, elected, cycles, d_status, stream=None):
+    """Enqueue the product-issue probe: cycles (device int32[2]) receives the SM clocks to issue 32 products and until
+    they complete (variant 0-3: operands in shared memory N = 64, A in TMEM N = 64, shared memory N = 128, N = 256)."""
+    _check(lib().spa_probe_mma_issue(int(variant), int(bool(elected)), _ptr(cycles), _ptr(d_status), _stream(stream)),
+           "spa_probe_mma_issue")
 
 
 def spa_read_status(d_status, stream=None) -> int:

@@ -241,6 +241,46 @@ def test_attention_with_more_segments_than_the_kernels_stage(C, H, xflags):
     assert blk.read_status() == 0
 
 
+@pytest.mark.parametrize("C,H", [(256, 8), (512, 8)])   # head dimension 32 and 64
+def test_attention_kernels_striding_over_items(C, H):
+    """200 short segments in a capacity of 128 row tiles and 8 heads: the forward kernel and (many short, even segments,
+    more than three grids' worth of item slots) both backward passes run as persistent grids in which a CTA works on
+    two or three (tile, head) items one after the other.  Against the oracle fed the same rounded bits."""
+    lib = L()
+    dt = "bf16"
+    rng = np.random.default_rng(500 + C)
+    counts = rng.integers(20, 101, size=200)
+    counts[[0, 99]] = [128, 1]
+    cu_np = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    n_seg, Np = len(counts), int(cu_np[-1])
+    B, N = 16, 1024
+    assert Np <= B * N and H * ((Np + 127) // 128) > 2 * 296
+    blk = block(B, N, C, H, dt)
+    p, cap = blk.p, blk.cap
+
+    def padded(a, cols):
+        buf = np.zeros((cap, cols))
+        buf[:Np] = a
+        return buf
+
+    qkv_r = round_to(rng.normal(size=(Np, 3 * C)), dt)
+    ao_ref, lse_ref = O.attention_fwd(qkv_r, cu_np, H)
+    seg = torch.from_numpy(cu_np).cuda()
+    qkv = dev(padded(qkv_r, 3 * C), dt)
+    lib.spa_packed_attention_fwd(p, qkv, seg, n_seg, blk.ao, blk.lse, blk.status)
+    assert_close(host(blk.ao)[:Np], ao_ref, dt, "attn_out")
+    assert np.abs(host(blk.lse)[:, :Np] - lse_ref).max() <= TOL[dt]["lse"]
+    ao_r = round_to(ao_ref, dt)
+    dao_r = round_to(rng.normal(size=(Np, C)), dt)
+    lse_t = torch.zeros(H, cap, dtype=torch.float32, device="cuda")
+    lse_t[:, :Np] = torch.from_numpy(lse_ref).float().cuda()
+    ref = O.attention_bwd(qkv_r, ao_r, lse_t[:, :Np].double().cpu().numpy(), dao_r, cu_np, H)
+    lib.spa_packed_attention_bwd(p, qkv, dev(padded(ao_r, C), dt), lse_t, dev(padded(dao_r, C), dt), seg, n_seg,
+                                 blk.dqkv, blk.workspace, blk.status)
+    assert_close(host(blk.dqkv)[:Np], ref, dt, "dqkv", scale_max_abs=True)
+    assert blk.read_status() == 0
+
+
 # device_cuts: the library builds the container cuts itself inside the block call (nothing comes from the host)
 @pytest.mark.parametrize("ci,fused,device_cuts", [(1, False, False), (2, False, False), (2, True, False),
                                                   (1, False, True), (2, True, True), (4, True, True)])
@@ -361,6 +401,28 @@ def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
     fwd = O.block_fwd(inp.x, inp.w_g, inp.b_g, inp.tau, inp.W_qkv, inp.b_qkv, inp.W_o, inp.b_o, cfg.H)
     assert_close(host(y), fwd["y"], cfg.dtype, "y after an expired wait")
     assert blk.read_status() == 0 and lib.spa_read_status(status) == 0
+
+
+def test_product_issue_probe_runs_and_reports_plausible_cycles():
+    """spa_probe_mma_issue: 32 products of each shape, issued by lane 0 and by an elected lane; the status word stays
+    clean, a product costs between its arithmetic (N / 2 clocks) and a few hundred clocks, and an accumulating product
+    whose A operand is in TMEM is issued faster by the elected lane (the reason the kernels issue that way)."""
+    lib = L()
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    cyc = torch.zeros(2, dtype=torch.int32, device="cuda")
+    got = {}
+    for variant, n in ((0, 64), (1, 64), (2, 128), (3, 256)):
+        for elected in (0, 1):
+            lib.spa_probe_mma_issue(variant, elected, cyc, status)
+            torch.cuda.synchronize()
+            issue, total = (int(v) for v in cyc.tolist())
+            assert lib.spa_read_status(status) == 0
+            assert 0 < issue <= total
+            assert n / 2 * 0.9 <= total / 32 <= 400, (variant, elected, issue, total)
+            got[(variant, elected)] = (issue / 32, total / 32)
+            print(f"product issue probe: variant {variant} (N = {n}) elected {elected}: issue {issue / 32:.1f}, "
+                  f"until complete {total / 32:.1f} clocks per product")
+    assert got[(1, 1)][0] < got[(1, 0)][0]
 
 
 @pytest.mark.parametrize("L_c,counts", [(49, [0, 1, 49, 48, 50, 98, 0, 0, 147, 5]), (16, [3, 16, 0, 31, 33, 1]),

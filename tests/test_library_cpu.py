@@ -85,6 +85,7 @@ def test_later_entry_points_validate_on_the_host(lib):
     assert L.spa_gelu(pp, None, 256, None, None) == inv
     assert L.spa_gelu_bwd(pp, None, None, 256, None, None) == inv
     assert L.spa_gate_select_pack(pp, None, None, 0.0, None, None, None, None, None, None, None, None, None, None, None) == inv
+    assert L.spa_probe_mma_issue(0, 0, None, None, None) == inv and L.spa_probe_mma_issue(7, 0, None, None, None) == inv
     assert L.spa_pack_state_bytes(pp) >= 16 + 4 and L.spa_pack_state_bytes(None) == 0
     assert L.spa_gate_select_pack_supported(pp) == 1
     wide = lib.make_params(2, 16, 2048, 32, "bf16")                 # 256 chunks per row: two-kernel path only
