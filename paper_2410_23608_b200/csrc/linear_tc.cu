@@ -409,8 +409,10 @@ colsum_partial_kernel(const __nv_bfloat16* __restrict__ dout, int n_out, const i
 }
 
 // out[e] = sum over the splits that hold rows (in split order) of part[s][e]; zero if there are none.
-// Two arrays (the weight-gradient partials and, optionally, the bias-gradient partials, which have their own row
-// chunks) in one launch.
+// Two arrays in one launch: the weight-gradient partials (a few splits: a thread adds them in split order) and,
+// optionally, the bias-gradient partials, which have row chunks of their own - up to hundreds of them for a few
+// thousand outputs, so there a warp owns four outputs: lane l adds chunks l, l + 32, ... in order and a fixed shuffle
+// tree adds the lanes.  The first ceil(n2 / 32) blocks take the second array.
 __global__ void __launch_bounds__(256)
 split_reduce_kernel(const float* __restrict__ part, long long n, const float* __restrict__ part2, long long n2,
                     int splits, int rows_per_chunk2, const int32_t* __restrict__ cu, int n_seg, int capacity,
@@ -419,30 +421,41 @@ split_reduce_kernel(const float* __restrict__ part, long long n, const float* __
   const int rows = packed_rows(cu, n_seg, capacity);
   const int k_blocks = (rows + BK - 1) / BK;  // the splits were dealt the BK-blocks of the rows in turn
   const int valid1 = k_blocks < splits ? k_blocks : splits;
-  const int valid2 = (rows + rows_per_chunk2 - 1) / rows_per_chunk2;
   const long long n4 = n >> 2, m4 = n2 >> 2;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4 + m4;
-       i += (long long)gridDim.x * blockDim.x) {
-    const bool second = i >= n4;
-    const float* src = second ? part2 : part;
-    const long long stride = second ? n2 : n, j = second ? i - n4 : i;
+  const int nb2 = (int)((m4 + 7) / 8);
+  if ((int)blockIdx.x < nb2) {
+    const int valid2 = (rows + rows_per_chunk2 - 1) / rows_per_chunk2;
+    const long long j = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (j >= m4) return;
+    const int lane = threadIdx.x & 31;
     float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int valid = second ? valid2 : valid1;
-    // loads four splits at a time in flight; the additions stay in split order
+    for (int z = lane; z < valid2; z += 32) {
+      const float4 v = __ldcs(reinterpret_cast<const float4*>(part2 + (long long)z * n2) + j);
+      s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w;
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+      s4.x += __shfl_xor_sync(0xffffffffu, s4.x, off);
+      s4.y += __shfl_xor_sync(0xffffffffu, s4.y, off);
+      s4.z += __shfl_xor_sync(0xffffffffu, s4.z, off);
+      s4.w += __shfl_xor_sync(0xffffffffu, s4.w, off);
+    }
+    if (lane == 0) reinterpret_cast<float4*>(out2)[j] = s4;
+    return;
+  }
+  const long long first = (long long)(blockIdx.x - nb2) * blockDim.x + threadIdx.x;
+  for (long long j = first; j < n4; j += (long long)(gridDim.x - nb2) * blockDim.x) {
+    float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    // four splits' loads in flight at a time; the additions stay in split order
     auto add = [&](const float4& v) { s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w; };
-    auto at = [&](int z) { return __ldcs(reinterpret_cast<const float4*>(src + (long long)z * stride) + j); };
+    auto at = [&](int z) { return __ldcs(reinterpret_cast<const float4*>(part + (long long)z * n) + j); };
     int z = 0;
-    for (; z + 4 <= valid; z += 4) {
+    for (; z + 4 <= valid1; z += 4) {
       const float4 v0 = at(z), v1 = at(z + 1), v2 = at(z + 2), v3 = at(z + 3);
       add(v0); add(v1); add(v2); add(v3);
     }
-    if (z + 2 <= valid) {
-      const float4 v0 = at(z), v1 = at(z + 1);
-      add(v0); add(v1);
-      z += 2;
-    }
-    if (z < valid) add(at(z));
-    reinterpret_cast<float4*>(second ? out2 : out)[j] = s4;
+    for (; z < valid1; ++z) add(at(z));
+    reinterpret_cast<float4*>(out)[j] = s4;
   }
 }
 
@@ -561,13 +574,14 @@ int launch_linear_bwd_tc(const spa_params& p, const void* a, const void* W, cons
                                                         nullptr, 0, d_status, st, "gemm_tc_kernel(wgrad)");
     if (rc != SPA_OK) return rc;
     const long long n_b = db != nullptr ? n_out : 0;
-    int grid = (int)(((n_w + n_b) / 4 + 255) / 256);
+    int grid = (int)((n_w / 4 + 255) / 256);
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
+    grid += (int)((n_b / 4 + 7) / 8);  // the blocks of the bias gradient come first
     launch_pdl(split_reduce_kernel, grid, 256, 0, st, part_w, n_w, part_b, n_b, sp.splits, rpc, cu, p.B, p.capacity, dW,
                db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel");
   } else {  // db alone
-    launch_pdl(split_reduce_kernel, (n_out / 4 + 255) / 256, 256, 0, st, (const float*)nullptr, 0LL, (const float*)part_b,
+    launch_pdl(split_reduce_kernel, (n_out / 4 + 7) / 8, 256, 0, st, (const float*)nullptr, 0LL, (const float*)part_b,
                (long long)n_out, 0, rpc, cu, p.B, p.capacity, (float*)nullptr, db);
     SPA_CUDA_CHECK_LAUNCH("split_reduce_kernel(db)");
   }
