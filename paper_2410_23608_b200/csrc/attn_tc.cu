@@ -499,6 +499,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   static_assert(kDQ || D == 32, "the dK / dV pass at d = 64 fills TMEM: attn_bwd_kv_split_kernel");
   constexpr uint32_t kColOpP = 160u;                // P^T (dK/dV pass only)
   constexpr uint32_t kColOpDS = kDQ ? 192u : 224u;  // dS or dS^T
+  // dQ pass: the last 32 columns hold the Q tile (d = 64) or the Q and the dO tile (d = 32, 16 columns each) as bf16
+  // operands, so that S = Q K^T (and dP = dO V^T) reads only the streamed tile from shared memory (a product with both
+  // operands there is bound by the operand read: 52 clocks against 36)
+  constexpr bool kQTmem = kDQ;
+  constexpr bool kDoTmem = kDQ && D == 32;
+  constexpr uint32_t kColQ = 224u, kColDO = 240u;
   // A CTA takes the work items blockIdx.x, blockIdx.x + gridDim.x, ... of the (tile, head) pairs that the device-side
   // row count leaves (heads fastest); TMEM and the staged segment offsets are set up once per CTA.
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -694,6 +700,20 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
   };
 
   if (is_math && n_tiles > 0 && !prep(0)) { record_status(d_status, SPA_ERR_TIMEOUT); *abort_any = 1; }
+  if (kQTmem && is_math && n_tiles > 0) {
+    // the own tiles have landed (prep(0) waited for them).  d = 64: each of a row's two threads moves its half of the
+    // Q row; d = 32: one moves the Q row, the other the dO row (16 columns either way).
+    uint32_t q[16];
+    const uint8_t* src = smem_al + (D == 32 && half == 1 ? kTile : 0) + rl * HT::kRowBytes;
+    const int c0 = D == 64 ? half * 4 : 0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint4 v = *reinterpret_cast<const uint4*>(src + (((c0 + c) ^ chunk_rot<D>(rl)) << 4));
+      q[4 * c] = v.x; q[4 * c + 1] = v.y; q[4 * c + 2] = v.z; q[4 * c + 3] = v.w;
+    }
+    ptx::tmem_st_32x16(tmem + lane_base + (D == 64 ? kColQ + half * 16 : (half == 0 ? kColQ : kColDO)), q);
+    ptx::tmem_st_wait();
+  }
   ptx::tc_fence_before_sync();
   __syncthreads();  // tile 0 is ready; a failure so far is seen by all threads or by none
   const bool failed_early = *abort_any != 0 || n_tiles == 0;
@@ -707,11 +727,15 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv, const __grid_cons
         const uint32_t y1a = smem_base + y1_off(st), y2a = smem_base + y2_off(st);
         if (ptx::elect_one()) {
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k)
-            ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1a, k), kIdescS, k != 0 ? 1u : 0u);
+          for (int k = 0; k < D / 16; ++k) {
+            if (kQTmem) ptx::mma_bf16_ts(tmem + kColS1, tmem + kColQ + k * 8, HT::kmajor(y1a, k), kIdescS, k != 0 ? 1u : 0u);
+            else ptx::mma_bf16(tmem + kColS1, HT::kmajor(x1_s, k), HT::kmajor(y1a, k), kIdescS, k != 0 ? 1u : 0u);
+          }
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k)
-            ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2a, k), kIdescS, k != 0 ? 1u : 0u);
+          for (int k = 0; k < D / 16; ++k) {
+            if (kDoTmem) ptx::mma_bf16_ts(tmem + kColS2, tmem + kColDO + k * 8, HT::kmajor(y2a, k), kIdescS, k != 0 ? 1u : 0u);
+            else ptx::mma_bf16(tmem + kColS2, HT::kmajor(x2_s, k), HT::kmajor(y2a, k), kIdescS, k != 0 ? 1u : 0u);
+          }
           ptx::mma_commit(bar_s);
         }
         __syncwarp();
